@@ -1,0 +1,191 @@
+/* hq.h -- C ABI of the in-hindsight int8 quantized-layer library for NVIDIA B200 (sm_100a).
+ *
+ * Method: "In-Hindsight Quantization Range Estimation for Quantized Training",
+ * arxiv 2105.04246.  Section/equation numbers below refer to that paper.
+ *
+ * What the calls compute, in the paper's terms:
+ *   - a layer call is the MAC of 8-bit operands into 32-bit accumulators (Sec. 3.1) whose
+ *     output is quantized "directly", with a range known in advance (static quantization,
+ *     Sec. 3.2) -- here the range estimated on earlier iterations (Sec. 4, step 1) -- while
+ *     min/max of the unquantized output are taken at the accumulator (Sec. 4, step 2);
+ *   - hq_range_update applies the moving average of Eq. 2-3 (Sec. 4.1) once the whole
+ *     output tensor exists, giving the range of the next iteration;
+ *   - hq_dynamic_quant is the comparison path of Sec. 3.2 / Eq. 1 / Eq. 5: the 32-bit
+ *     output goes to memory, the range is taken from the current tensor, the output is
+ *     read back and quantized.
+ *
+ * General rules of the boundary
+ *   - Plain C: no C++ types, no exceptions.  Every call returns an hq_status.
+ *   - Unless marked HOST, every pointer argument is a DEVICE pointer owned by the caller.
+ *     The library never allocates, frees or keeps caller tensors; it owns only the
+ *     context, prepared weights and their internal tables.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Layer,
+ *     update and dynamic calls only enqueue work: they do not synchronise and read every
+ *     quantization parameter from device memory.
+ *   - Arguments are validated before anything is launched; a rejected call launches
+ *     nothing and hq_last_error() holds a HOST string describing the reason.
+ *   - Every device-side wait is bounded.  If one expires the kernel records a code in the
+ *     context's device status word and ends normally; hq_get_async_error() reads it.
+ *   - Tensors are dense int8: activations and gradients NHWC, linear operands row-major
+ *     [rows][K], convolution weights [K_out][R][S][C_in] (depthwise: [C][R][S]).
+ *     Base pointers must be 16-byte aligned.
+ */
+#ifndef HQ_H_
+#define HQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  HQ_OK = 0,
+  HQ_ERR_INVALID_ARG = 1,     /* null pointer, non-positive size, inconsistent descriptor      */
+  HQ_ERR_UNSUPPORTED = 2,     /* a shape this build has no kernel for                          */
+  HQ_ERR_ALIGNMENT = 3,       /* pointer or leading dimension breaks a 16-byte rule            */
+  HQ_ERR_CUDA = 4,            /* a CUDA runtime/driver call failed (see hq_last_error)         */
+  HQ_ERR_NOT_INITIALIZED = 5, /* library built without / running without its device code       */
+  HQ_ERR_TIMEOUT = 6          /* a bounded device-side wait expired (hq_get_async_error)       */
+} hq_status;
+
+/* Per-tensor quantizer state, device resident, 48 bytes, 16-byte aligned, plain data:
+ * a checkpoint of the method's whole state is a copy of the array of these.
+ *   acc_min/acc_max  statistics slot (Sec. 4 step 2): min and max of the zero-point-corrected
+ *                    int32 accumulator of the tensor, merged by the layer kernels with atomics.
+ *                    Empty slot = {INT32_MAX, INT32_MIN}.
+ *   acc_scale        real value of one accumulator unit, fl(s_x * s_w), written by the layer call.
+ *   step             number of range updates applied so far; 0 = no range yet (t = 0, Sec. 4.1).
+ *   q_min/q_max      running range of Eq. 2-3.
+ *   scale, inv_scale, zero_point   the 2^8-level grid derived from the running range:
+ *                    lo = min(q_min,0), hi = max(q_max,0), scale = (hi-lo)/255 (1 if not > 0),
+ *                    inv_scale = 1/scale, zero_point = clamp(-128 - rint(lo/scale), -128, 127).
+ * For a layer INPUT only scale and zero_point are read.                                      */
+typedef struct {
+  int32_t acc_min, acc_max;
+  float acc_scale;
+  uint32_t step;
+  float q_min, q_max;
+  float scale, inv_scale;
+  int32_t zero_point;
+  uint32_t reserved[3];
+} hq_range_state;
+
+/* Forward-convolution geometry.  Input N x H x W x C, output N x Ho x Wo x K with
+ * Ho = (H + 2*pad_h - R)/stride_h + 1 (Wo alike).  groups is 1, or C (== K) for depthwise. */
+typedef struct {
+  int32_t N, H, W, C;
+  int32_t K;
+  int32_t R, S;
+  int32_t stride_h, stride_w;
+  int32_t pad_h, pad_w;
+  int32_t groups;
+} hq_conv_desc;
+
+typedef enum { HQ_DIR_FWD = 0, HQ_DIR_BWD_DATA = 1 } hq_direction;
+typedef enum { HQ_OP_LINEAR = 0, HQ_OP_CONV_FWD = 1, HQ_OP_CONV_BWD_DATA = 2 } hq_op_kind;
+
+typedef struct hq_ctx hq_ctx;                           /* HOST handle */
+typedef struct hq_prepared_weights hq_prepared_weights; /* HOST handle to device-side tables */
+
+/* Operation descriptor for hq_dynamic_quant and hq_debug_accumulate: the operands of the layer
+ * call it mirrors.  kind = HQ_OP_LINEAR uses M, N, K, w, bias; the conv kinds use conv, pw. */
+typedef struct {
+  int32_t kind;                  /* hq_op_kind */
+  int32_t M, N, K;               /* linear only */
+  const hq_conv_desc* conv;      /* HOST; conv kinds only */
+  const int8_t* x;               /* input (linear X, conv X, or dY for backward data) */
+  const hq_range_state* xq;      /* its scale / zero_point */
+  const int8_t* w;               /* linear only: W[N][K] */
+  const int32_t* bias;           /* linear only, may be NULL */
+  const hq_prepared_weights* pw; /* conv kinds only */
+  const float* w_scale;          /* one float: the weights' scale s_w (zero point 0) */
+} hq_op_desc;
+
+/* ---- context ------------------------------------------------------------------------------ */
+
+/* Creates a context on CUDA device `device` (HOST out-pointer).  Allocates a small device
+ * status word and scratch for weight column sums.  HQ_ERR_CUDA if the device cannot be used,
+ * HQ_ERR_UNSUPPORTED if it is not compute capability 10.0. */
+hq_status hq_create(hq_ctx** ctx, int device);
+hq_status hq_destroy(hq_ctx* ctx);
+const char* hq_status_string(hq_status s);       /* HOST string, static storage */
+const char* hq_last_error(const hq_ctx* ctx);    /* HOST string of the last rejected call */
+/* Synchronises `stream`, copies the device status word to *code (HOST) and clears it.
+ * Returns HQ_ERR_TIMEOUT if a bounded wait expired since the last call, else HQ_OK. */
+hq_status hq_get_async_error(hq_ctx* ctx, void* stream, int32_t* code);
+/* Number of kernel launches this context has enqueued so far (HOST counter). */
+uint64_t hq_launch_count(const hq_ctx* ctx);
+
+/* ---- weights ------------------------------------------------------------------------------ */
+
+/* Once per weight update (Sec. 3.1: the weights are quantized before they are loaded into the
+ * MAC array; their range can be pre-computed, Sec. 3.1 last paragraph).  Copies W (int8,
+ * [K][R][S][C], depthwise [C][R][S]) into library-owned device memory in the operand order the
+ * direction needs (backward data: the transposed, spatially reversed filter, split by output
+ * parity for strided layers) and builds the integer tables that remove the input zero point
+ * at padded borders.  W may be released after the call's work on `stream` completes.
+ * The handle is valid for this geometry (including N, H, W) only. */
+hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir,
+                             const int8_t* W, hq_prepared_weights** out);
+hq_status hq_weights_release(hq_ctx* ctx, hq_prepared_weights* pw);
+
+/* ---- the hot path --------------------------------------------------------------------------- */
+
+/* Y[M][N] = Q_Y( sum_k (X[m][k] - z_x) * W[n][k] + bias[n] ), Sec. 3.1 + Sec. 4 step 1, with
+ * z_x = xq->zero_point, s_acc = xq->scale * *w_scale, and (inv_scale, zero_point) taken from *yq
+ * as left by the previous hq_range_update / hq_dynamic_quant.  Per element:
+ *   y = float(acc) * s_acc;  q = clamp(rint(y * inv_scale) + zero_point, -128, 127)
+ * (round half to even, one binary32 rounding per operation).  Merges min/max of acc into
+ * yq->acc_min/acc_max (Sec. 4 step 2) and writes yq->acc_scale.  bias may be NULL.
+ * Requires K % 16 == 0.  Backward data of a linear layer is this call with W transposed. */
+hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K,
+                        const int8_t* X, const hq_range_state* xq,
+                        const int8_t* W, const float* w_scale, const int32_t* bias,
+                        int8_t* Y, hq_range_state* yq);
+
+/* Forward convolution as an implicit GEMM (Sec. 3.1), same epilogue as hq_linear_fwd.
+ * Padding is zero in the real domain.  pw must come from hq_weights_prepare(.., HQ_DIR_FWD, ..)
+ * with the same descriptor.  groups == C selects the depthwise kernel. */
+hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
+                      const int8_t* X, const hq_range_state* xq,
+                      const hq_prepared_weights* pw, const float* w_scale,
+                      int8_t* Y, hq_range_state* yq);
+
+/* Input gradient of the convolution described by desc (Sec. 3.1, backward pass: G_X from the
+ * quantized output gradient and the weights, always quantized by Q_G):
+ *   dX[n][hi][wi][c] = Q_G( sum over (r,s,k) with ho*stride_h - pad_h + r == hi (wo alike)
+ *                           of (dY[n][ho][wo][k] - z_dy) * W[k][r][s][c] ).
+ * dY is N x Ho x Wo x K, dX is N x H x W x C.  pw from hq_weights_prepare(.., HQ_DIR_BWD_DATA, ..). */
+hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
+                           const int8_t* dY, const hq_range_state* dyq,
+                           const hq_prepared_weights* pw, const float* w_scale,
+                           int8_t* dX, hq_range_state* dxq);
+
+/* Eq. 2-3 for `count` consecutive states, to be enqueued after the layer calls of the iteration:
+ *   m_lo = float(acc_min) * acc_scale, m_hi alike;
+ *   step == 0:  q_min = m_lo, q_max = m_hi                      (initialisation, Sec. 4.1)
+ *   else:       q_min = (1-eta)*m_lo + eta*q_min, q_max alike    (Eq. 2-3)
+ * then derives scale / inv_scale / zero_point, increments step and empties the statistics slot.
+ * A state whose slot is empty is left untouched. */
+hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, float eta);
+
+/* Dynamic quantization of the same layer (Sec. 3.2, Eq. 1; traffic of Eq. 5): kernel 1 runs the
+ * layer's MAC loop and writes y = float(acc) * s_acc as binary32 to `workspace` (caller-owned,
+ * one float per output element) while reducing min/max; kernel 2 sets q_min/q_max of *yq to the
+ * CURRENT tensor's extremes, derives the grid, increments step and empties the slot; kernel 3
+ * reads the workspace back and writes the int8 output.  Also serves as iteration 0 of the
+ * in-hindsight scheme (q^0 = min/max of the first tensor, Sec. 4.1). */
+hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op,
+                           float* workspace, int8_t* Y, hq_range_state* yq);
+
+/* Test hook: writes the zero-point-corrected int32 accumulator (+bias) of the layer to `acc`
+ * (one int32 per output element) and merges its min/max into *yq.  The hot path never
+ * materialises this tensor. */
+hq_status hq_debug_accumulate(hq_ctx* ctx, void* stream, const hq_op_desc* op, int32_t* acc, hq_range_state* yq);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HQ_H_ */

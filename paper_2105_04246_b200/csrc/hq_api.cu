@@ -1,0 +1,626 @@
+// C ABI of libhq: argument validation, launch planning, TMA descriptor encoding.
+// No arithmetic of the method lives here; every step runs in the kernels of hq_gemm.cu / hq_aux.cu.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdarg.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "hq.h"
+#include "hq_internal.h"
+
+using namespace hq;
+
+namespace {
+
+hq_status fail(hq_ctx* ctx, hq_status s, const char* fmt, ...) {
+  if (ctx) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    ctx->err = buf;
+  }
+  return s;
+}
+
+#define HQ_CUDA(ctx, expr)                                                                                   \
+  do {                                                                                                       \
+    cudaError_t e__ = (expr);                                                                                \
+    if (e__ != cudaSuccess) return fail(ctx, HQ_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
+  } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
+
+int out_dim(int in, int pad, int k, int stride) { return (in + 2 * pad - k) / stride + 1; }
+
+hq_status check_desc(hq_ctx* ctx, const hq_conv_desc* d) {
+  if (!d) return fail(ctx, HQ_ERR_INVALID_ARG, "conv descriptor is null");
+  if (d->N <= 0 || d->H <= 0 || d->W <= 0 || d->C <= 0 || d->K <= 0 || d->R <= 0 || d->S <= 0 || d->stride_h <= 0 || d->stride_w <= 0 ||
+      d->pad_h < 0 || d->pad_w < 0)
+    return fail(ctx, HQ_ERR_INVALID_ARG, "conv descriptor has a non-positive size");
+  if (d->groups != 1 && !(d->groups == d->C && d->K == d->C)) return fail(ctx, HQ_ERR_UNSUPPORTED, "groups must be 1 or C (depthwise, K == C)");
+  if (d->H + 2 * d->pad_h < d->R || d->W + 2 * d->pad_w < d->S) return fail(ctx, HQ_ERR_INVALID_ARG, "filter larger than padded input");
+  if (d->R > 7 || d->S > 7) return fail(ctx, HQ_ERR_UNSUPPORTED, "filters larger than 7x7 are not supported");
+  if (d->pad_h >= d->R || d->pad_w >= d->S) return fail(ctx, HQ_ERR_UNSUPPORTED, "padding must be smaller than the filter");
+  return HQ_OK;
+}
+
+bool same_desc(const hq_conv_desc& a, const hq_conv_desc& b) {
+  return a.N == b.N && a.H == b.H && a.W == b.W && a.C == b.C && a.K == b.K && a.R == b.R && a.S == b.S && a.stride_h == b.stride_h &&
+         a.stride_w == b.stride_w && a.pad_h == b.pad_h && a.pad_w == b.pad_w && a.groups == b.groups;
+}
+
+// border classes of one tile-space axis: which taps of `d` fall inside [0, a_dim) at position i
+void border_classes(int T, int in_mul, const std::vector<int>& d, int a_dim, std::vector<uint8_t>& cls, std::vector<uint32_t>& masks) {
+  cls.assign(T, 0);
+  masks.clear();
+  for (int i = 0; i < T; ++i) {
+    uint32_t m = 0;
+    for (size_t t = 0; t < d.size(); ++t) {
+      const int x = i * in_mul + d[t];
+      if (x >= 0 && x < a_dim) m |= 1u << t;
+    }
+    size_t k = 0;
+    while (k < masks.size() && masks[k] != m) ++k;
+    if (k == masks.size()) masks.push_back(m);
+    cls[i] = (uint8_t)k;
+  }
+  if (masks.empty()) masks.push_back(0);
+}
+
+// 128 = Nt*Ht*Wt with powers of two; the split that covers the tile space with least waste
+void pick_tile(int n_img, int TH, int TW, int in_mul_h, int in_mul_w, int& Nt, int& Ht, int& Wt) {
+  double best = -1.0;
+  for (int a = 7; a >= 0; --a)
+    for (int b = 7 - a; b >= 0; --b) {
+      const int wt = 1 << a, ht = 1 << b, nt = kTileM / (wt * ht);
+      if (wt * in_mul_w > 256 || ht * in_mul_h > 256) continue;
+      const double covered = (double)round_up(TW, wt) * round_up(TH, ht) * round_up(n_img, nt);
+      const double util = (double)TW * TH * n_img / covered;
+      if (util > best + 1e-12) {
+        best = util;
+        Nt = nt;
+        Ht = ht;
+        Wt = wt;
+      }
+    }
+}
+
+struct SubSpec {            // geometry of one launch, before tiling
+  int n_img, TH, TW;
+  int in_mul_h, in_mul_w;
+  std::vector<int> dh, dw;  // tap offsets per axis (taps = product, row-major)
+  int a_H, a_W;             // image size of operand A (for border classes)
+  int Cin;                  // reduction length per tap
+  int Nout;
+  int out_H, out_W, os_h, os_w, oa_h, oa_w;
+  int64_t ldY;
+  bool flat;
+};
+
+// fills everything in sub.p that does not depend on per-call pointers
+hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
+                   std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks) {
+  GemmParams& p = sub.p;
+  p.n_img = sp.n_img;
+  p.TH = sp.TH;
+  p.TW = sp.TW;
+  p.in_mul_h = sp.in_mul_h;
+  p.in_mul_w = sp.in_mul_w;
+  pick_tile(sp.n_img, sp.TH, sp.TW, sp.in_mul_h, sp.in_mul_w, p.Nt, p.Ht, p.Wt);
+  p.tiles_n = ceil_div(sp.n_img, p.Nt);
+  p.tiles_h = ceil_div(sp.TH, p.Ht);
+  p.tiles_w = ceil_div(sp.TW, p.Wt);
+  p.ntaps = (int)(sp.dh.size() * sp.dw.size());
+  if (p.ntaps > kMaxTaps) return fail(ctx, HQ_ERR_UNSUPPORTED, "too many filter taps");
+  for (size_t a = 0; a < sp.dh.size(); ++a)
+    for (size_t b = 0; b < sp.dw.size(); ++b) {
+      p.tap_dh[a * sp.dw.size() + b] = (int8_t)sp.dh[a];
+      p.tap_dw[a * sp.dw.size() + b] = (int8_t)sp.dw[b];
+    }
+  if (sp.Cin % 16 != 0) return fail(ctx, HQ_ERR_UNSUPPORTED, "reduction length per tap (%d) must be a multiple of 16", sp.Cin);
+  p.BK = (sp.Cin % 128 == 0) ? 128 : 64;
+  p.swizzle64 = p.BK == 64;
+  p.Cpad = round_up(sp.Cin, p.BK);
+  p.chunks_per_tap = p.Cpad / p.BK;
+  p.Nout = sp.Nout;
+  const int ncol = ceil_div(sp.Nout, 256);
+  p.BN = round_up(ceil_div(sp.Nout, ncol), 16);
+  p.tiles_col = ceil_div(sp.Nout, p.BN);
+  const int64_t nt = (int64_t)p.tiles_n * p.tiles_h * p.tiles_w * p.tiles_col;
+  if (nt > INT32_MAX) return fail(ctx, HQ_ERR_UNSUPPORTED, "too many tiles");
+  p.num_tiles = (int)nt;
+  p.out_H = sp.out_H;
+  p.out_W = sp.out_W;
+  p.os_h = sp.os_h;
+  p.os_w = sp.os_w;
+  p.oa_h = sp.oa_h;
+  p.oa_w = sp.oa_w;
+  p.ldY = sp.ldY;
+  p.corr_ld = p.tiles_col * p.BN;
+  // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = BN, M = 128
+  p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+  if (p.BN > 128) {
+    p.tmem_buf_stride = 256;
+    p.tmem_cols = 512;
+  } else {
+    uint32_t s = 32;
+    while ((int)s < p.BN) s <<= 1;
+    p.tmem_buf_stride = s;
+    p.tmem_cols = 2 * s;
+  }
+  p.stage_bytes_a = (uint32_t)kTileM * p.BK;
+  p.stage_bytes_b = (uint32_t)p.BN * p.BK;
+  p.stages = (int)std::min<uint32_t>(12, kSmemBudget / (p.stage_bytes_a + p.stage_bytes_b));
+  if (p.stages < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
+  sub.smem_bytes = kSmemBudget + 1024;
+  p.small_acc = 0;
+  sub.a_flat = sp.flat;
+  sub.a_stride_h = sp.in_mul_h;
+  sub.a_stride_w = sp.in_mul_w;
+  p.status = ctx->d_status;
+  if (sp.flat) {
+    rowcls.clear();
+    colcls.clear();
+    rowmasks.assign(1, 1u);
+    colmasks.assign(1, 1u);
+  } else {
+    border_classes(sp.TH, sp.in_mul_h, sp.dh, sp.a_H, rowcls, rowmasks);
+    border_classes(sp.TW, sp.in_mul_w, sp.dw, sp.a_W, colcls, colmasks);
+    if (rowmasks.size() > 16 || colmasks.size() > 16) return fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes");
+  }
+  p.ncolcls = (int)colmasks.size();
+  return HQ_OK;
+}
+
+hq_status encode_map(hq_ctx* ctx, CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                     const uint32_t* box, const uint32_t* estr, bool sw64, bool weights) {
+  CUresult r = ctx->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), dims, strides_bytes, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, sw64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                           weights ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(ctx, HQ_ERR_CUDA, "tensor map encoding failed (CUresult %d)", (int)r);
+  return HQ_OK;
+}
+
+hq_status encode_b(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* wmat, int64_t row_bytes, CUtensorMap* m) {
+  const GemmParams& p = sub.p;
+  uint64_t dims[2] = {(uint64_t)row_bytes, (uint64_t)p.Nout};
+  uint64_t strides[1] = {(uint64_t)row_bytes};
+  uint32_t box[2] = {(uint32_t)p.BK, (uint32_t)p.BN};
+  uint32_t es[2] = {1, 1};
+  return encode_map(ctx, m, wmat, 2, dims, strides, box, es, p.swizzle64, true);
+}
+
+// operand A: flat [rows][C] view, or NHWC image with one box per tile (traversal strides for strided layers)
+hq_status encode_a(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* base, int C, int W, int H, int N, CUtensorMap* m) {
+  const GemmParams& p = sub.p;
+  uint64_t dims[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
+  uint64_t strides[3] = {(uint64_t)C, (uint64_t)C * W, (uint64_t)C * W * H};
+  uint32_t box[4] = {(uint32_t)p.BK, (uint32_t)(p.Wt * sub.a_stride_w), (uint32_t)(p.Ht * sub.a_stride_h), (uint32_t)p.Nt};
+  uint32_t es[4] = {1, (uint32_t)sub.a_stride_w, (uint32_t)sub.a_stride_h, 1};
+  return encode_map(ctx, m, base, 4, dims, strides, box, es, p.swizzle64, false);
+}
+
+hq_status dev_alloc(hq_ctx* ctx, hq_prepared_weights* pw, void** p, size_t bytes) {
+  HQ_CUDA(ctx, cudaMalloc(p, bytes ? bytes : 16));
+  pw->allocs.push_back(*p);
+  return HQ_OK;
+}
+
+hq_status upload(hq_ctx* ctx, hq_prepared_weights* pw, const std::vector<uint8_t>& v, uint8_t** out, cudaStream_t s) {
+  if (v.empty()) {
+    *out = nullptr;
+    return HQ_OK;
+  }
+  void* d = nullptr;
+  hq_status st = dev_alloc(ctx, pw, &d, v.size());
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, cudaMemcpyAsync(d, v.data(), v.size(), cudaMemcpyHostToDevice, s));
+  HQ_CUDA(ctx, cudaStreamSynchronize(s));  // v is a temporary on the host
+  *out = (uint8_t*)d;
+  return HQ_OK;
+}
+
+// builds weight matrix, correction table and class maps of one sub-problem
+hq_status build_sub(hq_ctx* ctx, hq_prepared_weights* pw, cudaStream_t s, const SubSpec& sp, const hq_conv_desc& d, const int8_t* W,
+                    const std::vector<int>& tap_r, const std::vector<int>& tap_s, bool transposed, int gfold) {
+  pw->subs.emplace_back();
+  hq_sub_problem& sub = pw->subs.back();
+  sub.gfold = gfold;
+  std::vector<uint8_t> rowcls, colcls;
+  std::vector<uint32_t> rowmasks, colmasks;
+  hq_status st = plan_sub(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks);
+  if (st != HQ_OK) return st;
+  GemmParams& p = sub.p;
+  if (p.ntaps == 0) return HQ_OK;  // nothing to multiply: the epilogue stores the code of real zero
+  const size_t wbytes = (size_t)p.Nout * p.ntaps * p.Cpad;
+  st = dev_alloc(ctx, pw, (void**)&sub.wmat, wbytes);
+  if (st != HQ_OK) return st;
+  st = dev_alloc(ctx, pw, (void**)&sub.corr, (size_t)rowmasks.size() * colmasks.size() * p.corr_ld * sizeof(int32_t));
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, cudaMemsetAsync(sub.corr, 0, (size_t)rowmasks.size() * colmasks.size() * p.corr_ld * sizeof(int32_t), s));
+  int8_t tr[kMaxTaps], ts[kMaxTaps];
+  for (int t = 0; t < p.ntaps; ++t) {
+    tr[t] = (int8_t)tap_r[t / (int)sp.dw.size()];
+    ts[t] = (int8_t)tap_s[t % (int)sp.dw.size()];
+  }
+  HQ_CUDA(ctx, launch_prep_weights(W, sub.wmat, p.Nout, p.ntaps, p.Cpad, d.K, d.R, d.S, d.C, tr, ts, transposed ? 1 : 0, gfold, s));
+  HQ_CUDA(ctx, launch_corr(sub.wmat, sub.corr, p.Nout, p.ntaps, p.Cpad, (int)sp.dh.size(), (int)sp.dw.size(), rowmasks.data(),
+                           (int)rowmasks.size(), colmasks.data(), (int)colmasks.size(), p.corr_ld, s));
+  ctx->launches += 2;
+  st = upload(ctx, pw, rowcls, &sub.rowcls, s);
+  if (st != HQ_OK) return st;
+  st = upload(ctx, pw, colcls, &sub.colcls, s);
+  if (st != HQ_OK) return st;
+  p.corr = sub.corr;
+  p.rowcls = sub.rowcls;
+  p.colcls = sub.colcls;
+  return encode_b(ctx, sub, sub.wmat, (int64_t)p.ntaps * p.Cpad, &sub.tmap_b);
+}
+
+int fold_factor(int channels, int64_t pixels) {
+  for (int g = 1; g <= 16; g *= 2)
+    if ((g * channels) % 16 == 0 && pixels % g == 0) return g;
+  return 0;
+}
+
+hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, const CUtensorMap& ta, const CUtensorMap& tb, const hq_range_state* xq,
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode) {
+  GemmParams p = sub.p;
+  p.xq = xq;
+  p.w_scale = w_scale;
+  p.bias = bias;
+  p.out = out;
+  p.yq = yq;
+  const int grid = std::min(p.num_tiles, ctx->num_sms);
+  HQ_CUDA(ctx, launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s));
+  ctx->launches += 1;
+  return HQ_OK;
+}
+
+hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_direction dir, const int8_t* in, const hq_range_state* inq,
+                   const hq_prepared_weights* pw, const float* w_scale, void* out, hq_range_state* outq, int out_mode) {
+  hq_status st = check_desc(ctx, desc);
+  if (st != HQ_OK) return st;
+  if (!in || !inq || !pw || !w_scale || !out || !outq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (!aligned16(in) || !aligned16(out) || !aligned16(inq) || !aligned16(outq))
+    return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
+  if (pw->dir != dir || !same_desc(pw->desc, *desc)) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights were built for another layer");
+  const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
+  if (pw->depthwise) {
+    DwParams p{};
+    p.N = desc->N; p.H = desc->H; p.W = desc->W; p.C = desc->C; p.Ho = Ho; p.Wo = Wo; p.R = desc->R; p.S = desc->S;
+    p.stride_h = desc->stride_h; p.stride_w = desc->stride_w; p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
+    p.x = in; p.w = pw->dw_w; p.corr = pw->dw_corr; p.rowcls = pw->dw_rowcls; p.colcls = pw->dw_colcls; p.ncolcls = pw->dw_ncolcls;
+    p.xq = inq; p.w_scale = w_scale; p.yq = outq; p.out = out;
+    HQ_CUDA(ctx, launch_depthwise(p, out_mode, ctx->num_sms, s));
+    ctx->launches += 1;
+    return HQ_OK;
+  }
+  // operand A is the forward input (fwd) or the output gradient (bwd data)
+  const int aC = dir == HQ_DIR_FWD ? desc->C : desc->K;
+  const int aH = dir == HQ_DIR_FWD ? desc->H : Ho;
+  const int aW = dir == HQ_DIR_FWD ? desc->W : Wo;
+  for (const hq_sub_problem& sub : pw->subs) {
+    CUtensorMap ta;
+    if (sub.p.ntaps == 0) {
+      ta = CUtensorMap{};
+    } else if (sub.a_flat) {
+      const int64_t rows = (int64_t)desc->N * aH * aW / sub.gfold;
+      st = encode_a(ctx, sub, in, aC * sub.gfold, (int)rows, 1, 1, &ta);
+    } else {
+      st = encode_a(ctx, sub, in, aC, aW, aH, desc->N, &ta);
+    }
+    if (st != HQ_OK) return st;
+    st = launch_sub(ctx, s, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode);
+    if (st != HQ_OK) return st;
+  }
+  return HQ_OK;
+}
+
+hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode) {
+  if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
+  if (!X || !xq || !W || !w_scale || !out || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (K % 16 != 0) return fail(ctx, HQ_ERR_ALIGNMENT, "K (%d) must be a multiple of 16", K);
+  if (!aligned16(X) || !aligned16(W) || !aligned16(out) || !aligned16(xq) || !aligned16(yq))
+    return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
+  SubSpec sp{};
+  sp.n_img = 1; sp.TH = 1; sp.TW = M; sp.in_mul_h = 1; sp.in_mul_w = 1;
+  sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = M; sp.Cin = K; sp.Nout = N;
+  sp.out_H = 1; sp.out_W = M; sp.os_h = 1; sp.os_w = 1; sp.oa_h = 0; sp.oa_w = 0; sp.ldY = N; sp.flat = true;
+  hq_sub_problem sub;
+  std::vector<uint8_t> rc, cc;
+  std::vector<uint32_t> rm, cm;
+  hq_status st = plan_sub(ctx, sp, sub, rc, cc, rm, cm);
+  if (st != HQ_OK) return st;
+  if ((size_t)sub.p.corr_ld > ctx->scratch_elems) {
+    if (ctx->d_scratch) HQ_CUDA(ctx, cudaFree(ctx->d_scratch));
+    ctx->d_scratch = nullptr;
+    ctx->scratch_elems = 0;
+    HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_scratch, (size_t)sub.p.corr_ld * sizeof(int32_t)));
+    ctx->scratch_elems = sub.p.corr_ld;
+  }
+  // column sums of W for the input zero point (weights may change between calls, so per call)
+  const uint32_t one = 1u;
+  HQ_CUDA(ctx, launch_corr(W, ctx->d_scratch, N, 1, K, 1, 1, &one, 1, &one, 1, sub.p.corr_ld, s));
+  ctx->launches += 1;
+  sub.p.corr = ctx->d_scratch;
+  sub.p.Cpad = K;  // the caller's matrix is used as is; the K tail is zero-filled by the copy engine
+  CUtensorMap ta, tb;
+  st = encode_a(ctx, sub, X, K, M, 1, 1, &ta);
+  if (st != HQ_OK) return st;
+  st = encode_b(ctx, sub, W, K, &tb);
+  if (st != HQ_OK) return st;
+  return launch_sub(ctx, s, sub, ta, tb, xq, w_scale, bias, out, yq, out_mode);
+}
+
+hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, hq_range_state* yq, int out_mode) {
+  if (!op) return fail(ctx, HQ_ERR_INVALID_ARG, "operation descriptor is null");
+  switch (op->kind) {
+    case HQ_OP_LINEAR: return run_linear(ctx, s, op->M, op->N, op->K, op->x, op->xq, op->w, op->w_scale, op->bias, out, yq, out_mode);
+    case HQ_OP_CONV_FWD: return run_conv(ctx, s, op->conv, HQ_DIR_FWD, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
+    case HQ_OP_CONV_BWD_DATA: return run_conv(ctx, s, op->conv, HQ_DIR_BWD_DATA, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
+    default: return fail(ctx, HQ_ERR_INVALID_ARG, "unknown operation kind %d", op->kind);
+  }
+}
+
+int64_t op_out_elems(const hq_op_desc* op) {
+  if (op->kind == HQ_OP_LINEAR) return (int64_t)op->M * op->N;
+  const hq_conv_desc* d = op->conv;
+  if (op->kind == HQ_OP_CONV_FWD)
+    return (int64_t)d->N * out_dim(d->H, d->pad_h, d->R, d->stride_h) * out_dim(d->W, d->pad_w, d->S, d->stride_w) * d->K;
+  return (int64_t)d->N * d->H * d->W * d->C;
+}
+
+}  // namespace
+
+extern "C" {
+
+__attribute__((visibility("default"))) const char* hq_status_string(hq_status s) {
+  switch (s) {
+    case HQ_OK: return "ok";
+    case HQ_ERR_INVALID_ARG: return "invalid argument";
+    case HQ_ERR_UNSUPPORTED: return "unsupported shape";
+    case HQ_ERR_ALIGNMENT: return "alignment rule violated";
+    case HQ_ERR_CUDA: return "CUDA call failed";
+    case HQ_ERR_NOT_INITIALIZED: return "not initialised";
+    case HQ_ERR_TIMEOUT: return "a bounded device-side wait expired";
+  }
+  return "unknown status";
+}
+
+__attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int device) {
+  if (!out) return HQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  hq_ctx* ctx = new (std::nothrow) hq_ctx();
+  if (!ctx) return HQ_ERR_CUDA;
+  ctx->device = device;
+  cudaDeviceProp prop{};
+  if (cudaSetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+    delete ctx;
+    return HQ_ERR_CUDA;
+  }
+  if (prop.major != 10) {
+    delete ctx;
+    return HQ_ERR_UNSUPPORTED;
+  }
+  ctx->num_sms = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess ||
+      !fn) {
+    delete ctx;
+    return HQ_ERR_NOT_INITIALIZED;
+  }
+  ctx->encode = (EncodeTiledFn)fn;
+  ctx->scratch_elems = 4096;
+  if (cudaMalloc((void**)&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
+      cudaMalloc((void**)&ctx->d_scratch, ctx->scratch_elems * sizeof(int32_t)) != cudaSuccess ||
+      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess) {
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->d_scratch) cudaFree(ctx->d_scratch);
+    delete ctx;
+    return HQ_ERR_CUDA;
+  }
+  *out = ctx;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  cudaFree(ctx->d_status);
+  cudaFree(ctx->d_scratch);
+  delete ctx;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) const char* hq_last_error(const hq_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+__attribute__((visibility("default"))) uint64_t hq_launch_count(const hq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+__attribute__((visibility("default"))) hq_status hq_get_async_error(hq_ctx* ctx, void* stream, int32_t* code) {
+  if (!ctx || !code) return HQ_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  HQ_CUDA(ctx, cudaStreamSynchronize(s));
+  HQ_CUDA(ctx, cudaMemcpy(code, ctx->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  if (*code != 0) {
+    HQ_CUDA(ctx, cudaMemset(ctx->d_status, 0, sizeof(int32_t)));
+    return fail(ctx, HQ_ERR_TIMEOUT, "device-side wait %d expired", *code);
+  }
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W, hq_prepared_weights** out) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (!out) return fail(ctx, HQ_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  hq_status st = check_desc(ctx, desc);
+  if (st != HQ_OK) return st;
+  if (!W) return fail(ctx, HQ_ERR_INVALID_ARG, "W is null");
+  if (dir != HQ_DIR_FWD && dir != HQ_DIR_BWD_DATA) return fail(ctx, HQ_ERR_INVALID_ARG, "unknown direction");
+  cudaStream_t s = (cudaStream_t)stream;
+  const hq_conv_desc& d = *desc;
+  const int Ho = out_dim(d.H, d.pad_h, d.R, d.stride_h), Wo = out_dim(d.W, d.pad_w, d.S, d.stride_w);
+  hq_prepared_weights* pw = new (std::nothrow) hq_prepared_weights();
+  if (!pw) return fail(ctx, HQ_ERR_CUDA, "out of host memory");
+  pw->desc = d;
+  pw->dir = dir;
+  auto bail = [&](hq_status e) {
+    for (void* p : pw->allocs) cudaFree(p);
+    delete pw;
+    return e;
+  };
+
+  if (d.groups != 1) {
+    if (dir != HQ_DIR_FWD) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data is not implemented"));
+    if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise needs C %% 16 == 0"));
+    pw->depthwise = true;
+    std::vector<int> dh, dw;
+    for (int r = 0; r < d.R; ++r) dh.push_back(r - d.pad_h);
+    for (int q = 0; q < d.S; ++q) dw.push_back(q - d.pad_w);
+    std::vector<uint8_t> rowcls, colcls;
+    std::vector<uint32_t> rm, cm;
+    border_classes(Ho, d.stride_h, dh, d.H, rowcls, rm);
+    border_classes(Wo, d.stride_w, dw, d.W, colcls, cm);
+    if (rm.size() > 16 || cm.size() > 16) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes"));
+    pw->dw_ncolcls = (int)cm.size();
+    if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_w, (size_t)d.C * d.R * d.S)) != HQ_OK) return bail(st);
+    if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_corr, rm.size() * cm.size() * d.C * sizeof(int32_t))) != HQ_OK) return bail(st);
+    cudaError_t e = launch_dw_prep(W, pw->dw_w, pw->dw_corr, d.C, d.R, d.S, rm.data(), (int)rm.size(), cm.data(), (int)cm.size(), s);
+    if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "depthwise weight preparation failed: %s", cudaGetErrorString(e)));
+    ctx->launches += 1;
+    if ((st = upload(ctx, pw, rowcls, &pw->dw_rowcls, s)) != HQ_OK) return bail(st);
+    if ((st = upload(ctx, pw, colcls, &pw->dw_colcls, s)) != HQ_OK) return bail(st);
+    *out = pw;
+    return HQ_OK;
+  }
+
+  const bool pointwise = d.R == 1 && d.S == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_h == 0 && d.pad_w == 0;
+  if (dir == HQ_DIR_FWD) {
+    SubSpec sp{};
+    std::vector<int> tr, ts;
+    int g = 1;
+    if (pointwise) {
+      g = fold_factor(d.C, (int64_t)d.N * d.H * d.W);
+      if (g == 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "C = %d cannot be folded to a 16-byte multiple", d.C));
+      const int64_t rows = (int64_t)d.N * d.H * d.W / g;
+      if (rows > INT32_MAX) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many pixels"));
+      sp.n_img = 1; sp.TH = 1; sp.TW = (int)rows; sp.in_mul_h = sp.in_mul_w = 1; sp.dh = {0}; sp.dw = {0};
+      sp.a_H = 1; sp.a_W = (int)rows; sp.Cin = g * d.C; sp.Nout = g * d.K;
+      sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = (int64_t)g * d.K; sp.flat = true;
+      tr = {0}; ts = {0};
+    } else {
+      if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "C = %d: spatial filters need C %% 16 == 0", d.C));
+      sp.n_img = d.N; sp.TH = Ho; sp.TW = Wo; sp.in_mul_h = d.stride_h; sp.in_mul_w = d.stride_w;
+      for (int r = 0; r < d.R; ++r) { sp.dh.push_back(r - d.pad_h); tr.push_back(r); }
+      for (int q = 0; q < d.S; ++q) { sp.dw.push_back(q - d.pad_w); ts.push_back(q); }
+      sp.a_H = d.H; sp.a_W = d.W; sp.Cin = d.C; sp.Nout = d.K;
+      sp.out_H = Ho; sp.out_W = Wo; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.K; sp.flat = false;
+    }
+    if ((st = build_sub(ctx, pw, s, sp, d, W, tr, ts, false, g)) != HQ_OK) return bail(st);
+  } else {
+    if (pointwise) {
+      const int g = fold_factor(d.K, (int64_t)d.N * d.H * d.W);
+      if (g == 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "K = %d cannot be folded to a 16-byte multiple", d.K));
+      const int64_t rows = (int64_t)d.N * d.H * d.W / g;
+      if (rows > INT32_MAX) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many pixels"));
+      SubSpec sp{};
+      sp.n_img = 1; sp.TH = 1; sp.TW = (int)rows; sp.in_mul_h = sp.in_mul_w = 1; sp.dh = {0}; sp.dw = {0};
+      sp.a_H = 1; sp.a_W = (int)rows; sp.Cin = g * d.K; sp.Nout = g * d.C;
+      sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = (int64_t)g * d.C; sp.flat = true;
+      if ((st = build_sub(ctx, pw, s, sp, d, W, {0}, {0}, true, g)) != HQ_OK) return bail(st);
+    } else {
+      if (d.K % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "K = %d: backward data needs K %% 16 == 0", d.K));
+      // one dense stride-1 problem per output parity class (a, b): hi = i*stride_h + a, wi = j*stride_w + b
+      for (int a = 0; a < d.stride_h; ++a)
+        for (int b = 0; b < d.stride_w; ++b) {
+          SubSpec sp{};
+          sp.n_img = d.N;
+          sp.TH = (d.H - a + d.stride_h - 1) / d.stride_h;
+          sp.TW = (d.W - b + d.stride_w - 1) / d.stride_w;
+          if (sp.TH <= 0 || sp.TW <= 0) continue;
+          sp.in_mul_h = sp.in_mul_w = 1;
+          std::vector<int> tr, ts;
+          for (int r = 0; r < d.R; ++r) {
+            const int x = a + d.pad_h - r;
+            if (((x % d.stride_h) + d.stride_h) % d.stride_h == 0) { sp.dh.push_back(x / d.stride_h); tr.push_back(r); }
+          }
+          for (int q = 0; q < d.S; ++q) {
+            const int x = b + d.pad_w - q;
+            if (((x % d.stride_w) + d.stride_w) % d.stride_w == 0) { sp.dw.push_back(x / d.stride_w); ts.push_back(q); }
+          }
+          sp.a_H = Ho; sp.a_W = Wo; sp.Cin = d.K; sp.Nout = d.C;
+          sp.out_H = d.H; sp.out_W = d.W; sp.os_h = d.stride_h; sp.os_w = d.stride_w; sp.oa_h = a; sp.oa_w = b; sp.ldY = d.C; sp.flat = false;
+          if ((st = build_sub(ctx, pw, s, sp, d, W, tr, ts, true, 1)) != HQ_OK) return bail(st);
+        }
+    }
+  }
+  *out = pw;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_weights_release(hq_ctx* ctx, hq_prepared_weights* pw) {
+  if (!ctx || !pw) return HQ_ERR_INVALID_ARG;
+  for (void* p : pw->allocs) cudaFree(p);
+  delete pw;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
+                        const float* w_scale, const int32_t* bias, int8_t* Y, hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  return run_linear(ctx, (cudaStream_t)stream, M, N, K, X, xq, W, w_scale, bias, Y, yq, kOutInt8);
+}
+
+__attribute__((visibility("default"))) hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* X, const hq_range_state* xq,
+                      const hq_prepared_weights* pw, const float* w_scale, int8_t* Y, hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  return run_conv(ctx, (cudaStream_t)stream, desc, HQ_DIR_FWD, X, xq, pw, w_scale, Y, yq, kOutInt8);
+}
+
+__attribute__((visibility("default"))) hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* dY, const hq_range_state* dyq,
+                           const hq_prepared_weights* pw, const float* w_scale, int8_t* dX, hq_range_state* dxq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  return run_conv(ctx, (cudaStream_t)stream, desc, HQ_DIR_BWD_DATA, dY, dyq, pw, w_scale, dX, dxq, kOutInt8);
+}
+
+__attribute__((visibility("default"))) hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, float eta) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (!states || count <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "states is null or count is not positive");
+  if (!aligned16(states)) return fail(ctx, HQ_ERR_ALIGNMENT, "range states must be 16-byte aligned");
+  if (!(eta >= 0.0f && eta <= 1.0f)) return fail(ctx, HQ_ERR_INVALID_ARG, "eta must lie in [0, 1]");
+  HQ_CUDA(ctx, launch_range_update(states, count, eta, (cudaStream_t)stream));
+  ctx->launches += 1;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op, float* workspace, int8_t* Y, hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (!op || !workspace || !Y || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (!aligned16(workspace) || !aligned16(Y)) return fail(ctx, HQ_ERR_ALIGNMENT, "workspace and Y must be 16-byte aligned");
+  cudaStream_t s = (cudaStream_t)stream;
+  hq_status st = run_op(ctx, s, op, workspace, yq, kOutF32);
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, launch_dynamic_derive(yq, s));
+  HQ_CUDA(ctx, launch_quantize_pass(workspace, Y, op_out_elems(op), yq, ctx->num_sms, s));
+  ctx->launches += 2;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_debug_accumulate(hq_ctx* ctx, void* stream, const hq_op_desc* op, int32_t* acc, hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (!op || !acc || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  return run_op(ctx, (cudaStream_t)stream, op, acc, yq, kOutAcc);
+}
+
+}  // extern "C"

@@ -1,0 +1,331 @@
+// Small kernels around the layer kernels: range update (Eq. 2-3), the dynamic path's derive and
+// quantize passes (Eq. 1), weight preparation, and the depthwise convolution on CUDA cores.
+// arxiv 2105.04246; equation numbers refer to that paper.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hq_internal.h"
+
+namespace hq {
+namespace {
+
+// Grid derived from the running range: the range is widened to contain 0, split into 255 steps.
+__device__ __forceinline__ void derive_grid(hq_range_state* s) {
+  const float lo = s->q_min < 0.0f ? s->q_min : 0.0f;
+  const float hi = s->q_max > 0.0f ? s->q_max : 0.0f;
+  float scale = __fdiv_rn(__fsub_rn(hi, lo), 255.0f);
+  if (!(scale > 0.0f)) scale = 1.0f;
+  s->scale = scale;
+  s->inv_scale = __fdiv_rn(1.0f, scale);
+  const long long r = (long long)__float2int_rn(__fdiv_rn(lo, scale));
+  long long z = -128ll - r;
+  z = z < -128 ? -128 : (z > 127 ? 127 : z);
+  s->zero_point = (int32_t)z;
+}
+
+__global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  hq_range_state* s = st + i;
+  const int mn = s->acc_min, mx = s->acc_max;
+  if (mn > mx) return;  // no layer wrote statistics: leave the state alone
+  const float m_lo = __fmul_rn(__int2float_rn(mn), s->acc_scale);
+  const float m_hi = __fmul_rn(__int2float_rn(mx), s->acc_scale);
+  if (s->step == 0) {  // t = 0: the range is the first tensor's min/max
+    s->q_min = m_lo;
+    s->q_max = m_hi;
+  } else {  // Eq. 2-3
+    const float ome = __fsub_rn(1.0f, eta);
+    s->q_min = __fadd_rn(__fmul_rn(ome, m_lo), __fmul_rn(eta, s->q_min));
+    s->q_max = __fadd_rn(__fmul_rn(ome, m_hi), __fmul_rn(eta, s->q_max));
+  }
+  s->step += 1;
+  derive_grid(s);
+  s->acc_min = INT32_MAX;
+  s->acc_max = INT32_MIN;
+}
+
+// Eq. 1: the range is the min/max of the tensor that was just written.
+__global__ void dynamic_derive_kernel(hq_range_state* s) {
+  const int mn = s->acc_min, mx = s->acc_max;
+  if (mn > mx) return;
+  s->q_min = __fmul_rn(__int2float_rn(mn), s->acc_scale);
+  s->q_max = __fmul_rn(__int2float_rn(mx), s->acc_scale);
+  s->step += 1;
+  derive_grid(s);
+  s->acc_min = INT32_MAX;
+  s->acc_max = INT32_MIN;
+}
+
+__device__ __forceinline__ int quantize_real(float y, float inv_scale, int zp) {
+  const float u = __fmul_rn(y, inv_scale);
+  const int r = __float2int_rn(u);
+  int s;
+  asm("add.sat.s32 %0, %1, %2;" : "=r"(s) : "r"(r), "r"(zp));
+  return min(max(s, -128), 127);
+}
+
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+  return ((uint32_t)a & 0xffu) | (((uint32_t)b & 0xffu) << 8) | (((uint32_t)c & 0xffu) << 16) | (((uint32_t)d & 0xffu) << 24);
+}
+
+// second pass of the dynamic path: read the binary32 output back and quantize it
+__global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __restrict__ out, int64_t count, const hq_range_state* st) {
+  const float inv_scale = st->inv_scale;
+  const int zp = st->zero_point;
+  const int64_t groups = count / 16;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) {
+    const float4* src = reinterpret_cast<const float4*>(y) + 4 * g;
+    uint32_t w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float4 f = __ldcs(src + e);
+      w[e] = pack4(quantize_real(f.x, inv_scale, zp), quantize_real(f.y, inv_scale, zp), quantize_real(f.z, inv_scale, zp),
+                   quantize_real(f.w, inv_scale, zp));
+    }
+    reinterpret_cast<uint4*>(out)[g] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  if (blockIdx.x == 0) {
+    for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x) out[i] = (int8_t)quantize_real(y[i], inv_scale, zp);
+  }
+}
+
+// ---- weight preparation -----------------------------------------------------------------------
+struct TapList {
+  int8_t r[kMaxTaps], s[kMaxTaps];
+};
+struct ClassMasks {
+  uint32_t row[16], col[16];
+};
+
+// Wmat[n][t][c] (row length ntaps*Cpad, zero padded) from the forward filter W[Ksrc][R][S][Csrc]:
+//   plain      : W[n][r_t][s_t][c]
+//   transposed : W[c][r_t][s_t][n]                       (backward data: rows are input channels)
+//   g > 1      : g copies of that matrix on the block diagonal (g pixels folded into one GEMM row)
+__global__ void prep_weights_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S,
+                                    int Csrc, TapList taps, int transposed, int g) {
+  const int64_t total = (int64_t)Nout * ntaps * Cpad;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(idx % Cpad);
+    const int t = (int)((idx / Cpad) % ntaps);
+    const int n = (int)(idx / ((int64_t)Cpad * ntaps));
+    int8_t v = 0;
+    const int r = taps.r[t], s = taps.s[t];
+    const int rows_per = transposed ? Csrc : Ksrc;   // GEMM rows of one block
+    const int cols_per = transposed ? Ksrc : Csrc;   // GEMM columns (reduction) of one block
+    int nn = n, cc = c;
+    if (g > 1) {
+      const int j = n / rows_per;
+      nn = n % rows_per;
+      cc = c - j * cols_per;
+    }
+    if (cc >= 0 && cc < cols_per)
+      v = transposed ? W[(((int64_t)cc * R + r) * S + s) * Csrc + nn] : W[(((int64_t)nn * R + r) * S + s) * Csrc + cc];
+    Wmat[idx] = v;
+  }
+}
+
+// corr[(rc*ncolcls + cc)*corr_ld + n] = sum of Wmat[n][t][:] over the taps t = (ri, si) that are inside
+// the image for border class (rc, cc).  Multiplied by the input zero point in the epilogue, this is
+// what the zero-filled padding taps did NOT contribute.
+__global__ void corr_kernel(const int8_t* __restrict__ Wmat, int32_t* __restrict__ corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps,
+                            ClassMasks m, int nrowcls, int ncolcls, int corr_ld) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= nrowcls * ncolcls * Nout) return;
+  const int n = idx % Nout;
+  const int cls = idx / Nout;
+  const int rc = cls / ncolcls, cc = cls % ncolcls;
+  int32_t sum = 0;
+  for (int ri = 0; ri < nrowtaps; ++ri) {
+    if (!((m.row[rc] >> ri) & 1u)) continue;
+    for (int si = 0; si < ncoltaps; ++si) {
+      if (!((m.col[cc] >> si) & 1u)) continue;
+      const int8_t* w = Wmat + ((int64_t)n * ntaps + (ri * ncoltaps + si)) * Cpad;
+      for (int c = 0; c < Cpad; ++c) sum += w[c];
+    }
+  }
+  corr[(int64_t)cls * corr_ld + n] = sum;
+}
+
+// depthwise: weights to tap-major [R*S][C]; corr[cls][c] = sum of valid taps
+__global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wt, int32_t* __restrict__ corr, int C, int R, int S, ClassMasks m,
+                               int nrowcls, int ncolcls) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < C * R * S) {
+    const int c = idx % C, t = idx / C;
+    Wt[idx] = W[c * R * S + t];
+  }
+  if (idx < nrowcls * ncolcls * C) {
+    const int c = idx % C, cls = idx / C;
+    const int rc = cls / ncolcls, cc = cls % ncolcls;
+    int32_t sum = 0;
+    for (int r = 0; r < R; ++r)
+      for (int s = 0; s < S; ++s)
+        if (((m.row[rc] >> r) & 1u) && ((m.col[cc] >> s) & 1u)) sum += W[c * R * S + r * S + s];
+    corr[idx] = sum;
+  }
+}
+
+// ---- depthwise convolution on CUDA cores --------------------------------------------------------
+// One thread: one output pixel x 16 consecutive channels.  Same epilogue as the tensor-core kernel.
+__device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xffu); }
+
+template <int kOut>
+__global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
+  __shared__ int red_min[8], red_max[8];
+  const float s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
+  const int zx = p.xq->zero_point;
+  const float inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 0.0f;
+  const int zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = s_acc;
+  const int cgs = p.C / 16;
+  const int64_t total = (int64_t)p.N * p.Ho * p.Wo * cgs;
+  int mn = INT32_MAX, mx = INT32_MIN;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int cg = (int)(idx % cgs);
+    int64_t t = idx / cgs;
+    const int wo = (int)(t % p.Wo);
+    t /= p.Wo;
+    const int ho = (int)(t % p.Ho);
+    const int n = (int)(t / p.Ho);
+    int acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0;
+    for (int r = 0; r < p.R; ++r) {
+      const int hi = ho * p.stride_h - p.pad_h + r;
+      if (hi < 0 || hi >= p.H) continue;
+      for (int s = 0; s < p.S; ++s) {
+        const int wi = wo * p.stride_w - p.pad_w + s;
+        if (wi < 0 || wi >= p.W) continue;
+        const uint4 xv = *reinterpret_cast<const uint4*>(p.x + (((int64_t)n * p.H + hi) * p.W + wi) * p.C + cg * 16);
+        const uint4 wv = *reinterpret_cast<const uint4*>(p.w + (int64_t)(r * p.S + s) * p.C + cg * 16);
+        const uint32_t xa[4] = {xv.x, xv.y, xv.z, xv.w};
+        const uint32_t wa[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] += sx8(xa[e >> 2], e & 3) * sx8(wa[e >> 2], e & 3);
+      }
+    }
+    if (zx != 0) {
+      const int cls = p.rowcls[ho] * p.ncolcls + p.colcls[wo];
+      const int32_t* cr = p.corr + (int64_t)cls * p.C + cg * 16;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[e] -= zx * cr[e];
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      mn = min(mn, acc[e]);
+      mx = max(mx, acc[e]);
+    }
+    const int64_t o = (((int64_t)n * p.Ho + ho) * p.Wo + wo) * p.C + cg * 16;
+    if constexpr (kOut == kOutInt8) {
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        int q[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) q[k] = quantize_real(__fmul_rn(__int2float_rn(acc[4 * e + k]), s_acc), inv_scale, zp);
+        w[e] = pack4(q[0], q[1], q[2], q[3]);
+      }
+      *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + o;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(acc[4 * e + k]), s_acc)) : (uint32_t)acc[4 * e + k];
+        *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+  mn = __reduce_min_sync(0xffffffffu, mn);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    red_min[warp] = mn;
+    red_max[warp] = mx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int e = 1; e < (int)(blockDim.x >> 5); ++e) {
+      mn = min(mn, red_min[e]);
+      mx = max(mx, red_max[e]);
+    }
+    if (mn <= mx) {
+      atomicMin(&p.yq->acc_min, mn);
+      atomicMax(&p.yq->acc_max, mx);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s) {
+  range_update_kernel<<<(count + 127) / 128, 128, 0, s>>>(st, count, eta);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s) {
+  dynamic_derive_kernel<<<1, 1, 0, s>>>(st);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s) {
+  const int threads = 256;
+  int64_t want = (count / 16 + threads - 1) / threads;
+  int blocks = (int)(want < 1 ? 1 : (want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want));
+  quantize_pass_kernel<<<blocks, threads, 0, s>>>(y, out, count, st);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
+                                const int8_t* tap_r, const int8_t* tap_s, int transposed, int blockdiag_g, cudaStream_t s) {
+  TapList tl{};
+  for (int t = 0; t < ntaps; ++t) {
+    tl.r[t] = tap_r[t];
+    tl.s[t] = tap_s[t];
+  }
+  const int64_t total = (int64_t)Nout * ntaps * Cpad;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 4096) blocks = 4096;
+  prep_weights_kernel<<<blocks, 256, 0, s>>>(W, Wmat, Nout, ntaps, Cpad, Ksrc, R, S, Csrc, tl, transposed, blockdiag_g);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps, const uint32_t* rowmasks,
+                        int nrowcls, const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s) {
+  ClassMasks m{};
+  for (int i = 0; i < nrowcls; ++i) m.row[i] = rowmasks[i];
+  for (int i = 0; i < ncolcls; ++i) m.col[i] = colmasks[i];
+  const int total = nrowcls * ncolcls * Nout;
+  corr_kernel<<<(total + 127) / 128, 128, 0, s>>>(Wmat, corr, Nout, ntaps, Cpad, nrowtaps, ncoltaps, m, nrowcls, ncolcls, corr_ld);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
+                           const uint32_t* colmasks, int ncolcls, cudaStream_t s) {
+  ClassMasks m{};
+  for (int i = 0; i < nrowcls; ++i) m.row[i] = rowmasks[i];
+  for (int i = 0; i < ncolcls; ++i) m.col[i] = colmasks[i];
+  int total = nrowcls * ncolcls * C;
+  if (C * R * S > total) total = C * R * S;
+  dw_prep_kernel<<<(total + 127) / 128, 128, 0, s>>>(W, Wt, corr, C, R, S, m, nrowcls, ncolcls);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s) {
+  const int64_t total = (int64_t)p.N * p.Ho * p.Wo * (p.C / 16);
+  int64_t want = (total + 255) / 256;
+  int blocks = (int)(want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want);
+  if (blocks < 1) blocks = 1;
+  switch (out_mode) {
+    case kOutInt8: depthwise_kernel<kOutInt8><<<blocks, 256, 0, s>>>(p); break;
+    case kOutF32: depthwise_kernel<kOutF32><<<blocks, 256, 0, s>>>(p); break;
+    default: depthwise_kernel<kOutAcc><<<blocks, 256, 0, s>>>(p); break;
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace hq

@@ -1,0 +1,139 @@
+// Internal declarations shared by the translation units of libhq (host side + kernel params).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "hq.h"
+
+namespace hq {
+
+constexpr int kMaxTaps = 49;          // 7x7
+constexpr int kTileM = 128;           // rows of one accumulator tile = TMEM lanes
+constexpr int kEpilogueWarps = 4;
+constexpr int kGemmThreads = 32 * (2 + kEpilogueWarps);   // producer warp, MMA warp, epilogue warps
+constexpr uint32_t kSmemBudget = 200 * 1024;              // operand ring; barriers and tables sit on top
+constexpr uint64_t kWaitLimitNs = 2000000000ull;          // bound of every device-side wait
+
+// status-word codes written by kernels when a bounded wait expires
+enum AsyncCode : int32_t {
+  kAsyncOk = 0,
+  kAsyncProducerEmptyWait = 1,
+  kAsyncMmaFullWait = 2,
+  kAsyncMmaTmemEmptyWait = 3,
+  kAsyncEpilogueTmemFullWait = 4,
+  kAsyncDrainWait = 5,
+};
+
+enum OutMode : int { kOutInt8 = 0, kOutF32 = 1, kOutAcc = 2 };
+
+// One launch of the tensor-core kernel: an implicit GEMM over a "tile space" of output pixels.
+//   tile-space pixel (n, i, j), i in [0,TH), j in [0,TW)
+//   output pixel     (n, i*os_h + oa_h, j*os_w + oa_w) in an out_H x out_W image of ldY bytes/elements per pixel
+//   operand A, tap t (n, i*in_mul_h + tap_dh[t], j*in_mul_w + tap_dw[t], c)   -- fetched by a 4-D TMA box,
+//                    out-of-image coordinates are filled with zeros by the copy engine
+//   operand B        weight matrix [Nout][ntaps][Cpad], K-major
+struct GemmParams {
+  int32_t n_img, TH, TW;
+  int32_t Nt, Ht, Wt;                 // Nt*Ht*Wt == kTileM
+  int32_t tiles_n, tiles_h, tiles_w, tiles_col, num_tiles;
+  int32_t in_mul_h, in_mul_w;
+  int32_t ntaps, chunks_per_tap, BK, Cpad;
+  int8_t tap_dh[kMaxTaps], tap_dw[kMaxTaps];
+  int32_t Nout, BN;
+  int32_t out_H, out_W, os_h, os_w, oa_h, oa_w;
+  int64_t ldY;
+  const int32_t* corr;                // [ncls][corr_ld]: sum of the weights of the taps valid in that border class
+  int32_t corr_ld, ncolcls;
+  const uint8_t* rowcls;              // [TH] or null (single class)
+  const uint8_t* colcls;              // [TW] or null
+  const int32_t* bias;                // [Nout] or null
+  const hq_range_state* xq;
+  const float* w_scale;
+  hq_range_state* yq;
+  void* out;
+  int32_t* status;
+  uint32_t idesc;
+  uint32_t tmem_cols, tmem_buf_stride;
+  int32_t stages;
+  uint32_t stage_bytes_a, stage_bytes_b;
+  int32_t swizzle64;                  // 1: 64-byte swizzle (BK = 64), 0: 128-byte swizzle (BK = 128)
+  int32_t small_acc;                  // |acc| provably < 2^22: conversions may use the exact magic-number form
+};
+
+struct DwParams {                     // depthwise 3x3 (CUDA cores)
+  int32_t N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w;
+  const int8_t* x;
+  const int8_t* w;                    // [R*S][C] tap-major
+  const int32_t* corr;                // [ncls][C]
+  const uint8_t* rowcls;
+  const uint8_t* colcls;
+  int32_t ncolcls;
+  const hq_range_state* xq;
+  const float* w_scale;
+  hq_range_state* yq;
+  void* out;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// kernel launchers (defined in the .cu files)
+cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int out_mode, int grid, uint32_t smem_bytes,
+                        cudaStream_t s);
+cudaError_t gemm_set_smem_attr(uint32_t smem_bytes);
+cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s);
+cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s);
+cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s);
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s);
+cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
+                                const int8_t* tap_r, const int8_t* tap_s, int transposed, int blockdiag_g, cudaStream_t s);
+cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps, const uint32_t* rowmasks,
+                        int nrowcls, const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s);
+cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
+                           const uint32_t* colmasks, int ncolcls, cudaStream_t s);
+
+}  // namespace hq
+
+struct hq_ctx {
+  int device = 0;
+  int num_sms = 0;
+  int32_t* d_status = nullptr;
+  int32_t* d_scratch = nullptr;       // column sums of linear weights
+  size_t scratch_elems = 0;
+  hq::EncodeTiledFn encode = nullptr;
+  uint64_t launches = 0;
+  std::string err;
+};
+
+struct hq_sub_problem {               // one kernel launch of a prepared convolution
+  hq::GemmParams p{};                 // everything except per-call pointers
+  CUtensorMap tmap_b{};
+  int8_t* wmat = nullptr;
+  int32_t* corr = nullptr;
+  uint8_t* rowcls = nullptr;
+  uint8_t* colcls = nullptr;
+  uint32_t smem_bytes = 0;
+  int a_stride_h = 1, a_stride_w = 1; // traversal strides of the A tensor map
+  int a_flat = 0;                     // 1: A is viewed as [pixels][C] (1x1 stride-1 layers and linear)
+  int gfold = 1;                      // pixels folded into one GEMM row (channel counts that are not multiples of 16)
+};
+
+struct hq_prepared_weights {
+  hq_conv_desc desc{};
+  hq_direction dir = HQ_DIR_FWD;
+  bool depthwise = false;
+  std::vector<hq_sub_problem> subs;
+  // depthwise tables
+  int8_t* dw_w = nullptr;
+  int32_t* dw_corr = nullptr;
+  uint8_t* dw_rowcls = nullptr;
+  uint8_t* dw_colcls = nullptr;
+  int dw_ncolcls = 1;
+  std::vector<void*> allocs;          // everything to cudaFree on release
+};

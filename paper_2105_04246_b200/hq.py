@@ -1,0 +1,219 @@
+"""Python face of the C-ABI library libhq.so: the same call names as include/hq.h.
+
+Argument marshalling only.  Tensors are passed as objects with a ``data_ptr()`` (torch
+tensors) or as raw integer device addresses; streams as ``torch.cuda.Stream`` objects, raw
+handles or None.  There is no fallback: if the compiled library is missing, the first call
+raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhq.so")
+
+HQ_OK = 0
+STATUS_NAMES = {0: "HQ_OK", 1: "HQ_ERR_INVALID_ARG", 2: "HQ_ERR_UNSUPPORTED", 3: "HQ_ERR_ALIGNMENT", 4: "HQ_ERR_CUDA",
+                5: "HQ_ERR_NOT_INITIALIZED", 6: "HQ_ERR_TIMEOUT"}
+DIR_FWD, DIR_BWD_DATA = 0, 1
+OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
+
+# every extern "C" symbol include/hq.h declares
+EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count",
+           "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
+           "hq_dynamic_quant", "hq_debug_accumulate"]
+
+# numpy view of hq_range_state (48 bytes)
+RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
+                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("reserved", "<u4", (3,))])
+assert RANGE_STATE_DTYPE.itemsize == 48
+INT32_MAX, INT32_MIN = 2**31 - 1, -2**31
+
+
+class ConvDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("N", "H", "W", "C", "K", "R", "S", "stride_h", "stride_w", "pad_h", "pad_w", "groups")]
+
+
+class OpDesc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32), ("conv", C.POINTER(ConvDesc)),
+                ("x", C.c_void_p), ("xq", C.c_void_p), ("w", C.c_void_p), ("bias", C.c_void_p), ("pw", C.c_void_p),
+                ("w_scale", C.c_void_p)]
+
+
+class HqError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{STATUS_NAMES.get(status, status)}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Loads libhq.so; raises if it has not been built (there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2105_04246_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i32 = C.c_void_p, C.c_int32
+        L.hq_create.argtypes = [C.POINTER(vp), C.c_int]
+        L.hq_destroy.argtypes = [vp]
+        L.hq_status_string.argtypes = [C.c_int]; L.hq_status_string.restype = C.c_char_p
+        L.hq_last_error.argtypes = [vp]; L.hq_last_error.restype = C.c_char_p
+        L.hq_get_async_error.argtypes = [vp, vp, C.POINTER(i32)]
+        L.hq_launch_count.argtypes = [vp]; L.hq_launch_count.restype = C.c_uint64
+        L.hq_weights_prepare.argtypes = [vp, vp, C.POINTER(ConvDesc), C.c_int, vp, C.POINTER(vp)]
+        L.hq_weights_release.argtypes = [vp, vp]
+        L.hq_linear_fwd.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.hq_conv_fwd.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp, vp]
+        L.hq_conv_bwd_data.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp, vp]
+        L.hq_range_update.argtypes = [vp, vp, vp, i32, C.c_float]
+        L.hq_dynamic_quant.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp, vp]
+        L.hq_debug_accumulate.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
+        for name in EXPORTS:
+            if name not in ("hq_status_string", "hq_last_error", "hq_launch_count"):
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    return int(x)
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if hasattr(s, "cuda_stream"):
+        return s.cuda_stream
+    return int(s)
+
+
+def conv_desc(N, H, W, Cin, K, R=1, S=1, stride=1, pad=0, groups=1) -> ConvDesc:
+    sh, sw = (stride, stride) if np.isscalar(stride) else stride
+    ph, pw = (pad, pad) if np.isscalar(pad) else pad
+    return ConvDesc(N, H, W, Cin, K, R, S, sh, sw, ph, pw, groups)
+
+
+class PreparedWeights:
+    def __init__(self, ctx: "Context", handle: int, desc: ConvDesc, direction: int):
+        self.ctx, self.handle, self.desc, self.direction = ctx, handle, desc, direction
+
+    def release(self):
+        if self.handle:
+            lib().hq_weights_release(self.ctx.handle, self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.release()
+        except Exception:
+            pass
+
+
+class Context:
+    """hq_ctx: one per device."""
+
+    def __init__(self, device: int = 0):
+        h = C.c_void_p()
+        st = lib().hq_create(C.byref(h), int(device))
+        if st != HQ_OK:
+            raise HqError(st, lib().hq_status_string(st).decode())
+        self.handle = h.value
+        self.device = int(device)
+
+    def close(self):
+        if self.handle:
+            lib().hq_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st != HQ_OK:
+            raise HqError(st, lib().hq_last_error(self.handle).decode())
+
+    # ---- calls, named as in include/hq.h ------------------------------------------------------
+    def weights_prepare(self, stream, desc: ConvDesc, direction: int, W) -> PreparedWeights:
+        out = C.c_void_p()
+        self._check(lib().hq_weights_prepare(self.handle, _stream(stream), C.byref(desc), int(direction), _ptr(W), C.byref(out)))
+        return PreparedWeights(self, out.value, desc, int(direction))
+
+    def linear_fwd(self, stream, M, N, K, X, xq, W, w_scale, bias, Y, yq):
+        self._check(lib().hq_linear_fwd(self.handle, _stream(stream), M, N, K, _ptr(X), _ptr(xq), _ptr(W), _ptr(w_scale), _ptr(bias),
+                                        _ptr(Y), _ptr(yq)))
+
+    def conv_fwd(self, stream, desc, X, xq, pw: PreparedWeights, w_scale, Y, yq):
+        self._check(lib().hq_conv_fwd(self.handle, _stream(stream), C.byref(desc), _ptr(X), _ptr(xq), pw.handle, _ptr(w_scale), _ptr(Y),
+                                      _ptr(yq)))
+
+    def conv_bwd_data(self, stream, desc, dY, dyq, pw: PreparedWeights, w_scale, dX, dxq):
+        self._check(lib().hq_conv_bwd_data(self.handle, _stream(stream), C.byref(desc), _ptr(dY), _ptr(dyq), pw.handle, _ptr(w_scale),
+                                           _ptr(dX), _ptr(dxq)))
+
+    def range_update(self, stream, states, count: int, eta: float):
+        self._check(lib().hq_range_update(self.handle, _stream(stream), _ptr(states), int(count), float(eta)))
+
+    def dynamic_quant(self, stream, op: OpDesc, workspace, Y, yq):
+        self._check(lib().hq_dynamic_quant(self.handle, _stream(stream), C.byref(op), _ptr(workspace), _ptr(Y), _ptr(yq)))
+
+    def debug_accumulate(self, stream, op: OpDesc, acc, yq):
+        self._check(lib().hq_debug_accumulate(self.handle, _stream(stream), C.byref(op), _ptr(acc), _ptr(yq)))
+
+    def get_async_error(self, stream=None) -> int:
+        code = C.c_int32(0)
+        st = lib().hq_get_async_error(self.handle, _stream(stream), C.byref(code))
+        if st not in (HQ_OK, 6):
+            self._check(st)
+        return code.value
+
+    def launch_count(self) -> int:
+        return int(lib().hq_launch_count(self.handle))
+
+
+def linear_op(M, N, K, X, xq, W, w_scale, bias=None) -> OpDesc:
+    return OpDesc(OP_LINEAR, M, N, K, None, _ptr(X), _ptr(xq), _ptr(W), _ptr(bias), None, _ptr(w_scale))
+
+
+def conv_op(kind: int, desc: ConvDesc, X, xq, pw: PreparedWeights, w_scale) -> OpDesc:
+    op = OpDesc(kind, 0, 0, 0, C.pointer(desc), _ptr(X), _ptr(xq), None, None, pw.handle, _ptr(w_scale))
+    op._keep = (desc, pw)
+    return op
+
+
+# ---- range-state helpers (host-side packing of the plain-data struct) -------------------------------
+def new_states(count: int) -> np.ndarray:
+    """`count` empty states: no range yet (step 0), empty statistics slot."""
+    s = np.zeros(count, RANGE_STATE_DTYPE)
+    s["acc_min"] = INT32_MAX
+    s["acc_max"] = INT32_MIN
+    return s
+
+
+def input_state(scale: float, zero_point: int) -> np.ndarray:
+    """State describing a layer INPUT: only scale and zero_point are read."""
+    s = new_states(1)
+    s["scale"] = np.float32(scale)
+    s["zero_point"] = int(zero_point)
+    return s
+
+
+def states_to_device(states: np.ndarray, device="cuda"):
+    import torch
+    return torch.from_numpy(states.view(np.uint8).reshape(-1).copy()).to(device)
+
+
+def states_from_device(t) -> np.ndarray:
+    return t.detach().cpu().numpy().view(RANGE_STATE_DTYPE).copy()

@@ -1,0 +1,131 @@
+"""Test-side drivers: one layer run on the GPU through the C-ABI binding, and the same layer on
+the CPU oracle.  Only tests (and the smoke check) use this module."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle as O
+from paper_2105_04246_b200 import hq
+from paper_2105_04246_b200.synth import QTensor
+
+
+class GpuLayer:
+    """kind: 'linear' | 'conv_fwd' | 'conv_bwd'.  For conv kinds `shape` is a dict of conv_desc arguments."""
+
+    def __init__(self, ctx: hq.Context, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9):
+        self.ctx, self.kind, self.eta = ctx, kind, eta
+        self.dev = torch.device("cuda", ctx.device)
+        self.W = torch.from_numpy(np.ascontiguousarray(W.q)).to(self.dev)
+        self.w_scale = torch.tensor([W.scale], dtype=torch.float32, device=self.dev)
+        self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias, dtype=np.int32)).to(self.dev)
+        self.yq = hq.states_to_device(hq.new_states(1), self.dev)
+        self.stream = torch.cuda.current_stream(self.dev)
+        if kind == "linear":
+            self.N, self.K = W.q.shape
+            self.pw = None
+        else:
+            self.desc = hq.conv_desc(**shape)
+            self.pw = ctx.weights_prepare(self.stream, self.desc, hq.DIR_FWD if kind == "conv_fwd" else hq.DIR_BWD_DATA, self.W)
+            d = self.desc
+            Ho = (d.H + 2 * d.pad_h - d.R) // d.stride_h + 1
+            Wo = (d.W + 2 * d.pad_w - d.S) // d.stride_w + 1
+            self.in_shape = (d.N, d.H, d.W, d.C) if kind == "conv_fwd" else (d.N, Ho, Wo, d.K)
+            self.out_shape = (d.N, Ho, Wo, d.K) if kind == "conv_fwd" else (d.N, d.H, d.W, d.C)
+
+    def _put(self, x: QTensor):
+        xd = torch.from_numpy(np.ascontiguousarray(x.q)).to(self.dev)
+        xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), self.dev)
+        if self.kind == "linear":
+            assert x.q.shape[1] == self.K
+            out_shape = (x.q.shape[0], self.N)
+        else:
+            assert tuple(x.q.shape) == self.in_shape, (x.q.shape, self.in_shape)
+            out_shape = self.out_shape
+        return xd, xq, out_shape
+
+    def _op(self, xd, xq):
+        if self.kind == "linear":
+            return hq.linear_op(xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias)
+        return hq.conv_op(hq.OP_CONV_FWD if self.kind == "conv_fwd" else hq.OP_CONV_BWD_DATA, self.desc, xd, xq, self.pw, self.w_scale)
+
+    def state(self) -> np.ndarray:
+        return hq.states_from_device(self.yq)[0]
+
+    def set_state(self, st: np.ndarray):
+        arr = np.array([st], dtype=hq.RANGE_STATE_DTYPE)
+        self.yq.copy_(torch.from_numpy(arr.view(np.uint8).reshape(-1).copy()))
+
+    def accumulate(self, x: QTensor):
+        """Debug hook: int32 accumulator and its min/max (does not disturb the layer's own state)."""
+        xd, xq, out_shape = self._put(x)
+        acc = torch.empty(out_shape, dtype=torch.int32, device=self.dev)
+        tmp = hq.states_to_device(hq.new_states(1), self.dev)
+        self.ctx.debug_accumulate(self.stream, self._op(xd, xq), acc, tmp)
+        torch.cuda.synchronize(self.dev)
+        st = hq.states_from_device(tmp)[0]
+        return acc.cpu().numpy(), int(st["acc_min"]), int(st["acc_max"]), float(st["acc_scale"])
+
+    def dynamic(self, x: QTensor):
+        xd, xq, out_shape = self._put(x)
+        ws = torch.empty(out_shape, dtype=torch.float32, device=self.dev)
+        y = torch.full(out_shape, 99, dtype=torch.int8, device=self.dev)
+        self.ctx.dynamic_quant(self.stream, self._op(xd, xq), ws, y, self.yq)
+        torch.cuda.synchronize(self.dev)
+        return y.cpu().numpy(), ws.cpu().numpy()
+
+    def hindsight(self, x: QTensor, update: bool = True):
+        xd, xq, out_shape = self._put(x)
+        y = torch.full(out_shape, 99, dtype=torch.int8, device=self.dev)
+        if self.kind == "linear":
+            self.ctx.linear_fwd(self.stream, xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias, y, self.yq)
+        elif self.kind == "conv_fwd":
+            self.ctx.conv_fwd(self.stream, self.desc, xd, xq, self.pw, self.w_scale, y, self.yq)
+        else:
+            self.ctx.conv_bwd_data(self.stream, self.desc, xd, xq, self.pw, self.w_scale, y, self.yq)
+        torch.cuda.synchronize(self.dev)
+        stats = self.state()
+        if update:
+            self.ctx.range_update(self.stream, self.yq, 1, self.eta)
+            torch.cuda.synchronize(self.dev)
+        return y.cpu().numpy(), (int(stats["acc_min"]), int(stats["acc_max"]), float(stats["acc_scale"]))
+
+    def step(self, x: QTensor):
+        """Iteration 0: dynamic path; afterwards: in-hindsight layer call + range update."""
+        if int(self.state()["step"]) == 0:
+            return self.dynamic(x)[0]
+        return self.hindsight(x)[0]
+
+
+class OracleLayer:
+    def __init__(self, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9):
+        self.kind, self.W, self.bias = kind, W, bias
+        self.layer = O.Layer(eta)
+        self.desc = None if kind == "linear" else O.conv_desc(shape["N"], shape["H"], shape["W"], shape["Cin"], shape["K"], shape.get("R", 1),
+                                                              shape.get("S", 1), shape.get("stride", 1), shape.get("pad", 0),
+                                                              shape.get("groups", 1))
+
+    def accumulate(self, x: QTensor) -> np.ndarray:
+        if self.kind == "linear":
+            return O.linear_acc(x.q, x.zero_point, self.W.q, 0, self.bias)
+        if self.kind == "conv_fwd":
+            return O.conv_fwd_acc(self.desc, x.q, x.zero_point, self.W.q, 0)
+        return O.conv_bwd_data_acc(self.desc, x.q, x.zero_point, self.W.q, 0)
+
+    def s_acc(self, x: QTensor) -> float:
+        return O.acc_scale(x.scale, self.W.scale)
+
+    def step(self, x: QTensor, force_state: O.Range | None = None) -> O.StepResult:
+        return self.layer.step(self.accumulate(x), self.s_acc(x), force_state)
+
+
+def oracle_range_from_gpu(st: np.ndarray) -> O.Range:
+    return O.Range(float(st["q_min"]), float(st["q_max"]), float(st["scale"]), float(st["inv_scale"]), int(st["zero_point"]), int(st["step"]))
+
+
+def assert_state_close(gpu_st: np.ndarray, orc: O.Range, rel: float = 1e-6):
+    for name in ("q_min", "q_max", "scale", "inv_scale"):
+        a, b = float(gpu_st[name]), float(getattr(orc, name))
+        assert abs(a - b) <= rel * max(abs(a), abs(b), 1e-30), (name, a, b)
+    assert int(gpu_st["zero_point"]) == orc.zero_point, (int(gpu_st["zero_point"]), orc.zero_point)
+    assert int(gpu_st["step"]) == orc.step

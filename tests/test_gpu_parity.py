@@ -1,0 +1,217 @@
+"""GPU path vs CPU oracle, element by element, through the C-ABI binding.
+
+Bar: bit-exact for the int32 accumulator, its min/max, the binary32 output of the dynamic path
+and every int8 code; 1e-6 relative for the binary32 running range (it is expected to be equal).
+Shapes are small enough for the oracle to finish in seconds and still span several 128-row
+tiles, ragged tails in M, N and K, every border class of the padding, strides and channel
+counts that are not multiples of 16.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2105_04246_b200 import hq, synth
+from tests.harness import GpuLayer, OracleLayer, assert_state_close, oracle_range_from_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = hq.Context(0)
+    yield c
+    assert c.get_async_error() == 0
+    c.close()
+
+
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9):
+    g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
+    o = OracleLayer(kind, W, shape, bias=bias, eta=eta)
+    for t in range(iters):
+        x = make_x(t)
+        if t == 0:
+            acc, mn, mx, s_acc = g.accumulate(x)
+            ref = o.accumulate(x)
+            assert np.array_equal(acc, ref), f"accumulator mismatch: {np.argwhere(acc != ref)[:5]}"
+            assert (mn, mx) == O.minmax(ref)
+            assert s_acc == o.s_acc(x)
+            yq, ws = g.dynamic(x)
+            res = o.step(x)
+            assert res.mode == "dynamic"
+            assert np.array_equal(ws, ref.astype(np.float32) * np.float32(s_acc))
+        else:
+            yq, stats = g.hindsight(x)
+            res = o.step(x)
+            assert res.mode == "hindsight"
+            assert stats[:2] == (res.mn, res.mx), (t, stats, res.mn, res.mx)
+        bad = np.argwhere(yq != res.q)
+        assert bad.size == 0, f"iteration {t}: {len(bad)} int8 mismatches, first {bad[:5]}, gpu {yq[tuple(bad[0])]} oracle {res.q[tuple(bad[0])]}"
+        st = g.state()
+        assert_state_close(st, o.layer.state)
+        assert (int(st["acc_min"]), int(st["acc_max"])) == (hq.INT32_MAX, hq.INT32_MIN)   # slot emptied by the update
+    assert ctx.get_async_error() == 0
+    return g, o
+
+
+# ---- linear ---------------------------------------------------------------------------------
+def test_cfg1_linear_ten_iterations_with_scale_drift(ctx):
+    r = synth.rng(101)
+    W = synth.uniform_int8(r, (128, 256), scale=0.01)
+    scale = [0.02]
+
+    def make_x(t):
+        scale[0] *= float(r.uniform(0.8, 1.25))
+        return synth.uniform_int8(r, (256, 256), scale=scale[0], zero_point=0)
+
+    _run_iterations(ctx, "linear", W, None, make_x, 10)
+
+
+@pytest.mark.parametrize("M,N,K,zx,use_bias", [
+    (200, 1000, 512, -7, True),     # ragged M, four column tiles with a ragged last one, bias
+    (130, 24, 144, 5, False),       # N below one MMA tile, K tail zero-filled
+    (1, 16, 16, -128, False),       # smallest
+    (515, 272, 80, 127, True),      # two column tiles of 144 (second ragged), K = 64 + 16
+    (384, 8, 64, 3, False),         # N not a multiple of 16
+])
+def test_linear_ragged(ctx, M, N, K, zx, use_bias):
+    r = synth.rng(102, M, N, K)
+    W = synth.uniform_int8(r, (N, K), scale=0.003)
+    bias = r.integers(-5000, 5000, size=N).astype(np.int32) if use_bias else None
+    _run_iterations(ctx, "linear", W, None, lambda t: synth.uniform_int8(r, (M, K), scale=0.05 * (1 + 0.3 * t), zero_point=zx), 3, bias=bias)
+
+
+# ---- convolutions -----------------------------------------------------------------------------
+FWD_CASES = {
+    "3x3_c64_k64": dict(N=3, H=12, W=20, Cin=64, K=64, R=3, S=3, stride=1, pad=1),
+    "3x3_c128_k256": dict(N=2, H=9, W=9, Cin=128, K=256, R=3, S=3, stride=1, pad=1),
+    "3x3_c256_k512_7x7": dict(N=5, H=7, W=7, Cin=256, K=512, R=3, S=3, stride=1, pad=1),
+    "3x3_s2_c64_k128": dict(N=2, H=14, W=14, Cin=64, K=128, R=3, S=3, stride=2, pad=1),
+    "3x3_s2_odd": dict(N=2, H=15, W=13, Cin=64, K=32, R=3, S=3, stride=2, pad=1),
+    "1x1_s2": dict(N=2, H=14, W=14, Cin=64, K=128, R=1, S=1, stride=2, pad=0),
+    "1x1_c24_k144_fold": dict(N=2, H=10, W=13, Cin=24, K=144, R=1, S=1),
+    "1x1_c144_k24": dict(N=2, H=10, W=13, Cin=144, K=24, R=1, S=1),
+    "5x5_c16": dict(N=1, H=11, W=11, Cin=16, K=48, R=5, S=5, stride=1, pad=2),
+    "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
+    "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
+    "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
+}
+
+
+def _weights(r, shape):
+    if shape.get("groups", 1) != 1:
+        return synth.weights(r, (shape["K"], shape["R"], shape["S"]))
+    return synth.weights(r, (shape["K"], shape["R"], shape["S"], shape["Cin"]))
+
+
+@pytest.mark.parametrize("name", list(FWD_CASES))
+def test_conv_fwd(ctx, name):
+    shape = dict(FWD_CASES[name])
+    shape.setdefault("R", 1); shape.setdefault("S", 1)
+    r = synth.rng(103, len(name), shape["H"], shape["Cin"])
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3)
+
+
+BWD_CASES = {
+    "3x3_c64_k64": dict(N=3, H=12, W=20, Cin=64, K=64, R=3, S=3, stride=1, pad=1),
+    "3x3_c256_k256_14x14": dict(N=3, H=14, W=14, Cin=256, K=256, R=3, S=3, stride=1, pad=1),
+    "3x3_s2_c64_k128": dict(N=2, H=14, W=14, Cin=64, K=128, R=3, S=3, stride=2, pad=1),
+    "3x3_s2_odd": dict(N=2, H=15, W=13, Cin=48, K=64, R=3, S=3, stride=2, pad=1),
+    "1x1_s2": dict(N=2, H=14, W=14, Cin=64, K=128, R=1, S=1, stride=2, pad=0),
+    "1x1_k24_fold": dict(N=2, H=10, W=13, Cin=144, K=24, R=1, S=1),
+    "1x1_k144_c24": dict(N=2, H=10, W=13, Cin=24, K=144, R=1, S=1),
+}
+
+
+@pytest.mark.parametrize("name", list(BWD_CASES))
+def test_conv_bwd_data(ctx, name):
+    shape = dict(BWD_CASES[name])
+    r = synth.rng(104, len(name), shape["H"], shape["Cin"])
+    W = _weights(r, shape)
+    Ho = (shape["H"] + 2 * shape.get("pad", 0) - shape["R"]) // shape.get("stride", 1) + 1
+    Wo = (shape["W"] + 2 * shape.get("pad", 0) - shape["S"]) // shape.get("stride", 1) + 1
+    in_shape = (shape["N"], Ho, Wo, shape["K"])
+    _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3)
+
+
+# ---- protocol and edge cases ---------------------------------------------------------------------
+def test_teacher_forced_state_and_saturation(ctx):
+    """The oracle is fed the GPU's own state before each step: isolates the layer kernel from the
+    update kernel.  The input scale jumps up so that most codes saturate, then down."""
+    r = synth.rng(105)
+    shape = dict(N=2, H=8, W=8, Cin=64, K=64, R=3, S=3, stride=1, pad=1)
+    W = _weights(r, shape)
+    g = GpuLayer(ctx, "conv_fwd", W, shape)
+    o = OracleLayer("conv_fwd", W, shape)
+    mult = [1.0, 1.0, 8.0, 8.0, 0.05, 0.05]
+    for t, m in enumerate(mult):
+        x = synth.relu_activations(r, (2, 8, 8, 64))
+        x.scale *= m
+        forced = oracle_range_from_gpu(g.state())
+        yq = g.step(x)
+        res = o.step(x, force_state=forced)
+        assert np.array_equal(yq, res.q), t
+        assert_state_close(g.state(), o.layer.state)
+        if t == 2:
+            assert ((yq == 127) | (yq == -128)).mean() > 0.3
+
+
+def test_eta_extremes_and_skipped_update(ctx):
+    r = synth.rng(106)
+    W = synth.uniform_int8(r, (32, 64), scale=0.01)
+    for eta in (0.0, 1.0):
+        _run_iterations(ctx, "linear", W, None, lambda t: synth.uniform_int8(r, (64, 64), scale=0.1 * (t + 1)), 4, eta=eta)
+    g = GpuLayer(ctx, "linear", W)
+    g.step(synth.uniform_int8(r, (64, 64), scale=0.1))
+    before = g.state().copy()
+    ctx.range_update(g.stream, g.yq, 1, 0.9)          # empty statistics slot: nothing may change
+    torch.cuda.synchronize()
+    assert g.state().tobytes() == before.tobytes()
+
+
+def test_checkpoint_resume_is_identical(ctx):
+    r = synth.rng(107)
+    W = synth.uniform_int8(r, (48, 64), scale=0.01)
+    xs = [synth.uniform_int8(r, (96, 64), scale=0.1 * (1 + t % 3)) for t in range(6)]
+    a = GpuLayer(ctx, "linear", W)
+    outs = [a.step(x) for x in xs]
+    b = GpuLayer(ctx, "linear", W)
+    for x in xs[:3]:
+        b.step(x)
+    saved = b.state().copy()                           # the whole state of the method is this struct
+    c = GpuLayer(ctx, "linear", W)
+    c.set_state(saved)
+    for t in range(3, 6):
+        assert np.array_equal(c.step(xs[t]), outs[t])
+    assert c.state().tobytes() == a.state().tobytes()
+
+
+def test_rejected_calls_launch_nothing(ctx):
+    dev = torch.device("cuda", 0)
+    x = torch.zeros(64 * 64 + 16, dtype=torch.int8, device=dev)
+    st = hq.states_to_device(hq.new_states(2), dev)
+    ws = torch.ones(1, dtype=torch.float32, device=dev)
+    n0 = ctx.launch_count()
+    with pytest.raises(hq.HqError) as e:
+        ctx.linear_fwd(None, 64, 64, 40, x, st, x, ws, None, x, st[48:])          # K not a multiple of 16
+    assert e.value.status == 3
+    with pytest.raises(hq.HqError) as e:
+        ctx.linear_fwd(None, 64, 64, 64, x[1:], st, x, ws, None, x, st[48:])      # misaligned X
+    assert e.value.status == 3
+    with pytest.raises(hq.HqError) as e:
+        ctx.linear_fwd(None, 0, 64, 64, x, st, x, ws, None, x, st[48:])
+    assert e.value.status == 1
+    with pytest.raises(hq.HqError) as e:
+        ctx.linear_fwd(None, 64, 64, 64, x, None, x, ws, None, x, st[48:])
+    assert e.value.status == 1
+    with pytest.raises(hq.HqError) as e:
+        ctx.weights_prepare(None, hq.conv_desc(1, 8, 8, 3, 16, 3, 3, 1, 1), hq.DIR_FWD, x)   # C = 3 with a spatial filter
+    assert e.value.status == 2
+    with pytest.raises(hq.HqError) as e:
+        ctx.range_update(None, st, 2, 1.5)
+    assert e.value.status == 1
+    assert ctx.launch_count() == n0
+    torch.cuda.synchronize()
