@@ -180,6 +180,31 @@ hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int
 hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op,
                            float* workspace, int8_t* Y, hq_range_state* yq);
 
+/* Largest output, in elements, that hq_dynamic_quant_static accepts (16 MiB of binary32). */
+#define HQ_STATIC_WORKSPACE_ELEMS (4 * 1024 * 1024)
+
+/* hq_dynamic_quant for callers that cannot allocate.  (The paper has no counterpart: this is a
+ * property of the boundary, not of the method.)  Who needs it: code that runs where cudaMalloc is
+ * not allowed or not wanted -- inside an allocator or profiler callback, in a latency-critical loop
+ * that must never enter the allocator (cudaMalloc and cudaFree synchronise the device), or in a
+ * process whose device memory was handed out in full at start-up -- and that therefore cannot
+ * provide the one-float-per-output workspace of hq_dynamic_quant.  Here the workspace is a fixed device array that is part of the library image:
+ * every GPU that loads the library sets aside HQ_STATIC_WORKSPACE_ELEMS floats (16 MiB) for it until
+ * the process exits.  The call itself allocates and frees nothing, neither through CUDA nor through
+ * any other library.
+ *   - Same operands, results and status codes as hq_dynamic_quant; Y and *yq are still the caller's.
+ *   - Outputs of more than HQ_STATIC_WORKSPACE_ELEMS elements are rejected with HQ_ERR_UNSUPPORTED
+ *     before anything is launched; so is a linear layer whose N exceeds the column-sum scratch the
+ *     context allocated when it was created (4096 columns).
+ *   - The context's device must be the current device.  The first call on a device looks up the
+ *     array's device address (a host-side query, no launch); make that first call before starting
+ *     any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing
+ *     in it has to start at zero (the first kernel writes every element the last one reads), but two
+ *     calls that overlap on the GPU -- different streams, or different contexts on the same device --
+ *     race on it.  Serialise them. */
+hq_status hq_dynamic_quant_static(hq_ctx* ctx, void* stream, const hq_op_desc* op, int8_t* Y, hq_range_state* yq);
+
 /* Test hook: writes the zero-point-corrected int32 accumulator (+bias) of the layer to `acc`
  * (one int32 per output element) and merges its min/max into *yq.  The hot path never
  * materialises this tensor. */

@@ -624,3 +624,66 @@ __attribute__((visibility("default"))) hq_status hq_debug_accumulate(hq_ctx* ctx
 }
 
 }  // extern "C"
+
+// ---- dynamic quantization without any allocation ------------------------------------------------
+// Some callers cannot allocate device memory around a call: allocator or profiler callbacks,
+// latency-critical loops that must stay out of the allocator (cudaMalloc / cudaFree synchronise the
+// device), or embedders whose memory budget is fixed at start-up.  For them the binary32 workspace of the dynamic path lives in this file-scope device
+// array.  In host code the array's name is only a stand-in; the device address is looked up once
+// per device with cudaGetSymbolAddress and handed to the kernels.
+static __device__ __align__(256) float hq_static_workspace[HQ_STATIC_WORKSPACE_ELEMS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_ws[kMaxDevices] = {};
+
+hq_status static_workspace(hq_ctx* ctx, float** out) {
+  int cur = -1;
+  HQ_CUDA(ctx, cudaGetDevice(&cur));
+  if (cur != ctx->device) return fail(ctx, HQ_ERR_INVALID_ARG, "device %d must be current (device %d is)", ctx->device, cur);
+  if (cur < 0 || cur >= kMaxDevices) return fail(ctx, HQ_ERR_UNSUPPORTED, "device index %d out of range", cur);
+  if (g_static_ws[cur] == nullptr) {
+    void* p = nullptr;
+    HQ_CUDA(ctx, cudaGetSymbolAddress(&p, hq_static_workspace));
+    g_static_ws[cur] = static_cast<float*>(p);
+  }
+  *out = g_static_ws[cur];
+  return HQ_OK;
+}
+}  // namespace
+
+extern "C" __attribute__((visibility("default"))) hq_status hq_dynamic_quant_static(hq_ctx* ctx, void* stream, const hq_op_desc* op, int8_t* Y,
+                                                                                   hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (!op || !Y || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (op->kind != HQ_OP_LINEAR && op->kind != HQ_OP_CONV_FWD && op->kind != HQ_OP_CONV_BWD_DATA)
+    return fail(ctx, HQ_ERR_INVALID_ARG, "unknown operation kind %d", op->kind);
+  if (op->kind != HQ_OP_LINEAR) {
+    hq_status st = check_desc(ctx, op->conv);
+    if (st != HQ_OK) return st;
+  } else if (op->M <= 0 || op->N <= 0 || op->K <= 0) {
+    return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
+  }
+  const int64_t elems = op_out_elems(op);
+  if (elems > (int64_t)HQ_STATIC_WORKSPACE_ELEMS)
+    return fail(ctx, HQ_ERR_UNSUPPORTED, "output has %lld elements; the built-in workspace holds at most %lld", (long long)elems,
+                (long long)HQ_STATIC_WORKSPACE_ELEMS);
+  if (op->kind == HQ_OP_LINEAR) {
+    // the column-sum scratch of the context is fixed here: it is never grown on this path
+    const int ncol = ceil_div(op->N, 256);
+    const int bn = round_up(ceil_div(op->N, ncol), 16);
+    if ((size_t)(ceil_div(op->N, bn) * bn) > ctx->scratch_elems)
+      return fail(ctx, HQ_ERR_UNSUPPORTED, "N = %d needs more column-sum scratch than the context holds (%zu)", op->N, ctx->scratch_elems);
+  }
+  if (!aligned16(Y)) return fail(ctx, HQ_ERR_ALIGNMENT, "Y must be 16-byte aligned");
+  float* ws = nullptr;
+  hq_status st = static_workspace(ctx, &ws);
+  if (st != HQ_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  st = run_op(ctx, s, op, ws, yq, kOutF32);
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, launch_dynamic_derive(yq, s));
+  HQ_CUDA(ctx, launch_quantize_pass(ws, Y, elems, yq, ctx->num_sms, s));
+  ctx->launches += 2;
+  return HQ_OK;
+}

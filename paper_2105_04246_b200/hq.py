@@ -24,7 +24,7 @@ OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 # every extern "C" symbol include/hq.h declares
 EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count",
            "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
-           "hq_dynamic_quant", "hq_debug_accumulate"]
+           "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate"]
 
 # numpy view of hq_range_state (48 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
@@ -74,6 +74,7 @@ def lib():
         L.hq_range_update.argtypes = [vp, vp, vp, i32, C.c_float]
         L.hq_dynamic_quant.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp, vp]
         L.hq_debug_accumulate.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
+        L.hq_dynamic_quant_static.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
         for name in EXPORTS:
             if name not in ("hq_status_string", "hq_last_error", "hq_launch_count"):
                 getattr(L, name).restype = C.c_int
@@ -168,6 +169,11 @@ class Context:
 
     def dynamic_quant(self, stream, op: OpDesc, workspace, Y, yq):
         self._check(lib().hq_dynamic_quant(self.handle, _stream(stream), C.byref(op), _ptr(workspace), _ptr(Y), _ptr(yq)))
+
+    def dynamic_quant_static(self, stream, op: OpDesc, Y, yq):
+        """hq_dynamic_quant with the library's built-in workspace: for callers that cannot allocate
+        device memory (see include/hq.h).  Shares one array per device; do not overlap calls."""
+        self._check(lib().hq_dynamic_quant_static(self.handle, _stream(stream), C.byref(op), _ptr(Y), _ptr(yq)))
 
     def debug_accumulate(self, stream, op: OpDesc, acc, yq):
         self._check(lib().hq_debug_accumulate(self.handle, _stream(stream), C.byref(op), _ptr(acc), _ptr(yq)))
