@@ -417,6 +417,27 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_profile(args):
+    import torch
+    from paper_2105_04246_b200 import hq
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    ctx = hq.Context(0)
+    wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0)
+    stream = torch.cuda.current_stream(dev)
+    for j in range(2):
+        wk.step(stream, j, dynamic=True)
+    torch.cuda.synchronize()
+    for k in range(args.steps):
+        wk.step(stream, k % 2)
+    torch.cuda.synchronize()
+    for k in range(args.steps):
+        wk.step(stream, k % 2, dynamic=True)
+    torch.cuda.synchronize()
+    assert ctx.get_async_error() == 0
+    print(json.dumps({"profile": args.workload, "steps": args.steps, "launches": ctx.launch_count()}))
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", 0))
     if rank != 0:
@@ -442,9 +463,14 @@ def main():
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
+                         "then --steps in-hindsight steps, then --steps dynamic steps")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.profile:
+        run_profile(args)
     else:
         run_gpu(args)
 

@@ -117,6 +117,11 @@ const char* hq_last_error(const hq_ctx* ctx);    /* HOST string of the last reje
 hq_status hq_get_async_error(hq_ctx* ctx, void* stream, int32_t* code);
 /* Number of kernel launches this context has enqueued so far (HOST counter). */
 uint64_t hq_launch_count(const hq_ctx* ctx);
+/* Tuning knob (HOST key string), for tests and experiments; results are identical for every value.
+ *   "staging": how convolutions prepared AFTER this call bring their input to the MAC array (the
+ *              paper's "loaded into the MAC array", Sec. 3.1): -1 = chosen per layer (default),
+ *              0 = one copy per filter tap, 1 = input rows kept resident wherever the layer allows. */
+hq_status hq_set_option(hq_ctx* ctx, const char* key, int32_t value);
 
 /* ---- weights ------------------------------------------------------------------------------ */
 

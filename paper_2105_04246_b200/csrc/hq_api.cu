@@ -8,6 +8,7 @@
 
 #include <algorithm>
 #include <new>
+#include <string>
 #include <vector>
 
 #include "hq.h"
@@ -157,12 +158,68 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     p.tmem_buf_stride = s;
     p.tmem_cols = 2 * s;
   }
-  p.stage_bytes_a = (uint32_t)kTileM * p.BK;
+  // ---- operand staging: resident input rows (kModeHalo) where the tile space is stride-1, else one box per tap ----
+  p.mode = kModeTap;
   p.stage_bytes_b = (uint32_t)p.BN * p.BK;
-  p.stages = (int)std::min<uint32_t>(12, kSmemBudget / (p.stage_bytes_a + p.stage_bytes_b));
-  if (p.stages < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
+  bool halo = !sp.flat && sp.in_mul_h == 1 && sp.in_mul_w == 1 && p.ntaps >= 2 && ctx->force_mode != kModeTap;
+  if (halo) {
+    const int dh_min = *std::min_element(sp.dh.begin(), sp.dh.end()), dh_max = *std::max_element(sp.dh.begin(), sp.dh.end());
+    const int dw_min = *std::min_element(sp.dw.begin(), sp.dw.end()), dw_max = *std::max_element(sp.dw.begin(), sp.dw.end());
+    const int dh_span = dh_max - dh_min, dw_span = dw_max - dw_min;
+    const int P = sp.TW + dw_span;
+    const int L = sp.TH * P;
+    const int tiles_per_img = ceil_div(L, kTileM);
+    int NR = 0;
+    for (int lt = 0; lt < tiles_per_img; ++lt) NR = std::max(NR, ((lt * kTileM) % P + kTileM - 1 + dh_span * P + dw_span) / P + 1);
+    const uint32_t box = (uint32_t)p.BK * P * NR;
+    const uint32_t stride = (box + 1023u) & ~1023u;
+    const double util = (double)sp.TH * sp.TW / ((double)tiles_per_img * kTileM);
+    const int kiters = p.ntaps * p.chunks_per_tap;
+    halo = (int)sp.dh.size() == dh_span + 1 && (int)sp.dw.size() == dw_span + 1 && P <= 256 && NR <= 256 &&
+           (util >= 0.6 || ctx->force_mode == kModeHalo);
+    int stages_a = 0, stages_b = 0, resident = 0;
+    if (halo) {
+      if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * p.stage_bytes_b + 2ull * stride <= kSmemBudget) {
+        resident = 1;
+        stages_b = kiters;
+        stages_a = (int)std::min<uint64_t>(4, (kSmemBudget - (uint64_t)kiters * p.stage_bytes_b) / stride);
+      } else {
+        stages_a = 2;
+        while (stages_a < 4 && (uint64_t)(stages_a + 1) * stride + 4ull * p.stage_bytes_b <= kSmemBudget) ++stages_a;
+        if ((uint64_t)stages_a * stride < kSmemBudget)
+          stages_b = (int)std::min<uint64_t>(8, (kSmemBudget - (uint64_t)stages_a * stride) / p.stage_bytes_b);
+        if (stages_b < 2) halo = false;
+      }
+    }
+    if (halo) {
+      p.mode = kModeHalo;
+      p.P = P;
+      p.L = L;
+      p.NR = NR;
+      p.tiles_per_img = tiles_per_img;
+      p.dh_min = dh_min;
+      p.dw_min = dw_min;
+      p.patch_box_bytes = box;
+      p.patch_chunk_stride = stride;
+      p.stage_bytes_a = stride;
+      p.stages_a = stages_a;
+      p.stages_b = stages_b;
+      p.b_resident = resident;
+      p.Nt = 1;
+      p.Ht = 1;
+      p.Wt = kTileM;
+      p.num_tiles = sp.n_img * tiles_per_img * p.tiles_col;
+      p.producer_lanes = 1;
+    }
+  }
+  if (p.mode == kModeTap) {
+    p.stage_bytes_a = (uint32_t)kTileM * p.BK;
+    p.stages_a = (int)std::min<uint32_t>(kMaxStagesA, kSmemBudget / (p.stage_bytes_a + p.stage_bytes_b));
+    p.stages_b = 0;
+    if (p.stages_a < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
+    p.producer_lanes = std::min(4, p.stages_a);
+  }
   sub.smem_bytes = kSmemBudget + 1024;
-  p.small_acc = 0;
   sub.a_flat = sp.flat;
   sub.a_stride_h = sp.in_mul_h;
   sub.a_stride_w = sp.in_mul_w;
@@ -207,6 +264,11 @@ hq_status encode_a(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* base, i
   uint64_t strides[3] = {(uint64_t)C, (uint64_t)C * W, (uint64_t)C * W * H};
   uint32_t box[4] = {(uint32_t)p.BK, (uint32_t)(p.Wt * sub.a_stride_w), (uint32_t)(p.Ht * sub.a_stride_h), (uint32_t)p.Nt};
   uint32_t es[4] = {1, (uint32_t)sub.a_stride_w, (uint32_t)sub.a_stride_h, 1};
+  if (p.mode == kModeHalo) {  // NR padded rows of P pixels of one image
+    box[1] = (uint32_t)p.P;
+    box[2] = (uint32_t)p.NR;
+    box[3] = 1;
+  }
   return encode_map(ctx, m, base, 4, dims, strides, box, es, p.swizzle64, false);
 }
 
@@ -447,6 +509,16 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
 __attribute__((visibility("default"))) const char* hq_last_error(const hq_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
 __attribute__((visibility("default"))) uint64_t hq_launch_count(const hq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+__attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, const char* key, int32_t value) {
+  if (!ctx || !key) return HQ_ERR_INVALID_ARG;
+  if (std::string(key) == "staging") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "staging must be -1, 0 or 1");
+    ctx->force_mode = value;
+    return HQ_OK;
+  }
+  return fail(ctx, HQ_ERR_INVALID_ARG, "unknown option '%s'", key);
+}
 
 __attribute__((visibility("default"))) hq_status hq_get_async_error(hq_ctx* ctx, void* stream, int32_t* code) {
   if (!ctx || !code) return HQ_ERR_INVALID_ARG;

@@ -2,10 +2,10 @@
 // operands staged by TMA, with the requantization + min/max epilogue of the in-hindsight
 // scheme (arxiv 2105.04246, Sec. 3.1, Sec. 3.2 "static quantization", Sec. 4 steps 1 and 2).
 //
-// One persistent CTA per SM walks over 128-row output tiles.  Warp 0 feeds a ring of
-// shared-memory stages with TMA box copies (one box of A per filter tap and channel chunk,
-// zero-filled outside the image; one box of the weight matrix), warp 1 issues the MMAs, and
-// four epilogue warps drain a double-buffered TMEM accumulator, so the epilogue of tile i
+// One persistent CTA per SM walks over 128-row output tiles.  Roles: warp 0 feeds operand A
+// (kModeTap: one box of A and one of B per filter tap and channel chunk; kModeHalo: the padded
+// input rows of the tile, once), warp 2 streams the weights in kModeHalo, warp 1 issues the MMAs,
+// eight epilogue warps drain a double-buffered TMEM accumulator, so the epilogue of tile i
 // overlaps the MAC loop of tile i+1.  Every wait is bounded (see mbar_wait).
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -76,8 +76,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// Shared-memory matrix descriptor of a K-major operand tile whose rows are one swizzle span
-// wide (64 or 128 bytes): 8-row groups are `8 * span` bytes apart.
+// Shared-memory matrix descriptor of a K-major operand whose rows are one swizzle span wide
+// (64 or 128 bytes) and contiguous: 8-row groups are 8 spans apart.  The swizzle is applied to the
+// absolute shared-memory address (the same function the TMA write used), so a start that is
+// shifted by whole rows -- a tile that begins at an arbitrary pixel of a resident patch -- reads
+// the right bytes with the base-offset field left at zero.
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, bool sw64) {
   uint64_t d = 0;
   d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
@@ -98,11 +101,14 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int* v) {
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int* v) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
-        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+        "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
       : "r"(taddr)
       : "memory");
 }
@@ -113,32 +119,41 @@ struct QParams {
   int zx, zp;
 };
 
-// y = fl(float(acc) * s_acc); q = clamp(rint(fl(y * inv_scale)) + zero_point): one rounding per step.
-__device__ __forceinline__ int quantize_one(int a, const QParams& q) {
-  float y = __fmul_rn(__int2float_rn(a), q.s_acc);
-  float u = __fmul_rn(y, q.inv_scale);
-  int r = __float2int_rn(u);  // saturating conversion, NaN -> 0
+// y = fl(float(acc) * s_acc); r = rint(fl(y * inv_scale)) + zero_point (saturating add): one rounding per step.
+__device__ __forceinline__ int requant_unclamped(int a, const QParams& q) {
+  const float y = __fmul_rn(__int2float_rn(a), q.s_acc);
+  const float u = __fmul_rn(y, q.inv_scale);
+  const int r = __float2int_rn(u);  // saturating conversion, NaN -> 0
   int s;
   asm("add.sat.s32 %0, %1, %2;" : "=r"(s) : "r"(r), "r"(q.zp));
-  return min(max(s, -128), 127);
+  return s;
+}
+// four values -> four saturated int8 codes in one word, element 0 in the lowest byte
+__device__ __forceinline__ uint32_t pack_sat4(int q0, int q1, int q2, int q3) {
+  uint32_t hi, d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(q1), "r"(q0), "r"(hi));
+  return d;
 }
 
 template <int V>
-__device__ __forceinline__ void store_bytes16(int8_t* p, const uint32_t* w, int nvalid) {
-  // w: 4 words = 16 output bytes; store the first nvalid bytes in pieces of V bytes
+__device__ __forceinline__ void store_bytes32(int8_t* p, const uint32_t* w, int nvalid) {
+  // w: 8 words = 32 output bytes; store the first nvalid bytes in pieces of V bytes
   if constexpr (V == 16) {
-    if (nvalid >= 16) *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
-  } else if constexpr (V == 8) {
 #pragma unroll
     for (int g = 0; g < 2; ++g)
+      if ((g + 1) * 16 <= nvalid) *reinterpret_cast<uint4*>(p + 16 * g) = make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+  } else if constexpr (V == 8) {
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
       if ((g + 1) * 8 <= nvalid) *reinterpret_cast<uint2*>(p + 8 * g) = make_uint2(w[2 * g], w[2 * g + 1]);
   } else if constexpr (V == 4) {
 #pragma unroll
-    for (int g = 0; g < 4; ++g)
+    for (int g = 0; g < 8; ++g)
       if ((g + 1) * 4 <= nvalid) *reinterpret_cast<uint32_t*>(p + 4 * g) = w[g];
   } else {
 #pragma unroll
-    for (int g = 0; g < 16; ++g)
+    for (int g = 0; g < 32; ++g)
       if (g < nvalid) p[g] = (int8_t)((w[g >> 2] >> (8 * (g & 3))) & 0xffu);
   }
 }
@@ -148,7 +163,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int out_vec) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * 16 + 4];   // full[16], empty[16], tmem_full[2], tmem_empty[2]
+  __shared__ __align__(8) uint64_t bars[2 * kMaxStagesA + 2 * kMaxStagesB + 4];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int red_min[kEpilogueWarps], red_max[kEpilogueWarps];
@@ -157,21 +172,30 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   const int lane = threadIdx.x & 31;
   volatile int* abort_flag = &abort_flag_s;
 
-  const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t stage_bytes = p.stage_bytes_a + p.stage_bytes_b;
+  const uint32_t ring_a = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const bool halo = p.mode == kModeHalo;
+  // kModeTap: one ring, stage = [A tile | B tile]; kModeHalo: patch ring, then weight ring
+  const uint32_t a_stride = halo ? p.stage_bytes_a : p.stage_bytes_a + p.stage_bytes_b;
+  const uint32_t ring_b = ring_a + (uint32_t)p.stages_a * a_stride;
   const uint32_t bar0 = smem_u32(bars);
-  auto full_bar = [&](int s) { return bar0 + 8u * s; };
-  auto empty_bar = [&](int s) { return bar0 + 8u * (16 + s); };
-  auto tfull_bar = [&](int b) { return bar0 + 8u * (32 + b); };
-  auto tempty_bar = [&](int b) { return bar0 + 8u * (34 + b); };
+  auto a_full = [&](int s) { return bar0 + 8u * s; };
+  auto a_empty = [&](int s) { return bar0 + 8u * (kMaxStagesA + s); };
+  auto b_full = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + s); };
+  auto b_empty = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + kMaxStagesB + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + 2 + b); };
 
   const int kiters = p.ntaps * p.chunks_per_tap;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int s = 0; s < p.stages; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < p.stages_a; ++s) {
+      mbar_init(a_full(s), 1);
+      mbar_init(a_empty(s), 1);
+    }
+    for (int s = 0; s < p.stages_b; ++s) {
+      mbar_init(b_full(s), 1);
+      mbar_init(b_empty(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
@@ -190,61 +214,106 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
+  // tile index -> origin.  kModeTap: (n0, h0, w0) of the pixel box; kModeHalo: image n0, first linear pixel h0
   auto decode = [&](int tile, int& n0, int& h0, int& w0, int& col0) {
-    int ct = tile % p.tiles_col;
+    const int ct = tile % p.tiles_col;
     int t = tile / p.tiles_col;
-    int wt = t % p.tiles_w;
-    t /= p.tiles_w;
-    int ht = t % p.tiles_h;
-    int nt = t / p.tiles_h;
-    n0 = nt * p.Nt;
-    h0 = ht * p.Ht;
-    w0 = wt * p.Wt;
     col0 = ct * p.BN;
+    if (halo) {
+      const int lt = t % p.tiles_per_img;
+      n0 = t / p.tiles_per_img;
+      h0 = lt * kTileM;
+      w0 = 0;
+    } else {
+      const int wt = t % p.tiles_w;
+      t /= p.tiles_w;
+      const int ht = t % p.tiles_h;
+      n0 = (t / p.tiles_h) * p.Nt;
+      h0 = ht * p.Ht;
+      w0 = wt * p.Wt;
+    }
   };
+  const int my_tiles = (p.num_tiles > (int)blockIdx.x) ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
-    if (lane == 0 && kiters > 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      int issued = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-        int n0, h0, w0, col0;
-        decode(tile, n0, h0, w0, col0);
-        for (int t = 0; t < p.ntaps && ok; ++t) {
-          const int ch = h0 * p.in_mul_h + p.tap_dh[t];
-          const int cw = w0 * p.in_mul_w + p.tap_dw[t];
-          for (int cc = 0; cc < p.chunks_per_tap; ++cc) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait)) {
+    // ------------------------------ operand A producer ------------------------------
+    if (halo) {
+      if (lane == 0 && kiters > 0) {
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+          int n0, o0, w0, col0;
+          decode(tile, n0, o0, w0, col0);
+          const int hp0 = o0 / p.P;
+          bool ok = true;
+          for (int cb = 0; cb < p.chunks_per_tap; ++cb) {   // one ring stage per channel chunk of the patch
+            if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait)) {
               ok = false;
               break;
             }
-            const uint32_t sa = ring + stage * stage_bytes;
-            mbar_expect_tx(full_bar(stage), stage_bytes);
-            tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, full_bar(stage));
-            tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, full_bar(stage));
-            ++issued;
-            if (++stage == p.stages) {
+            mbar_expect_tx(a_full(stage), p.patch_box_bytes);
+            tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
+            if (++stage == p.stages_a) {
               stage = 0;
               phase ^= 1u;
             }
           }
+          if (!ok) break;
         }
       }
-      if (!ok) {
-        // give copies already in flight a bounded time to land before the CTA retires
-        int pending = issued < p.stages ? issued : p.stages;
-        int s = stage;
-        uint32_t ph = phase;
-        for (int i = 0; i < pending; ++i) {
-          if (--s < 0) {
-            s = p.stages - 1;
-            ph ^= 1u;
+    } else if (lane < p.producer_lanes && kiters > 0) {
+      // lane l issues the copies of ring iterations l, l + lanes, ... (each lane tracks its own stage and phase)
+      const int total = my_tiles * kiters;
+      int stage = lane % p.stages_a;
+      uint32_t phase = (uint32_t)(lane / p.stages_a) & 1u;
+      for (int it = lane; it < total; it += p.producer_lanes) {
+        const int lt = it / kiters;
+        const int ki = it - lt * kiters;
+        const int t = ki / p.chunks_per_tap;
+        const int cc = ki - t * p.chunks_per_tap;
+        int n0, h0, w0, col0;
+        decode((int)blockIdx.x + lt * (int)gridDim.x, n0, h0, w0, col0);
+        if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait)) break;
+        const uint32_t sa = ring_a + stage * a_stride;
+        mbar_expect_tx(a_full(stage), a_stride);
+        tma_load_4d(sa, &tmap_a, cc * p.BK, w0 * p.in_mul_w + p.tap_dw[t], h0 * p.in_mul_h + p.tap_dh[t], n0, a_full(stage));
+        tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+        stage += p.producer_lanes;
+        while (stage >= p.stages_a) {
+          stage -= p.stages_a;
+          phase ^= 1u;
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------ weight producer (kModeHalo) ------------------------------
+    if (halo && lane == 0 && kiters > 0) {
+      if (p.b_resident) {
+        if (my_tiles > 0) {
+          for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
+            const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
+            mbar_expect_tx(b_full(ki), p.stage_bytes_b);
+            tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(ki));
           }
-          const uint64_t t0 = global_timer_ns();
-          while (!mbar_try(full_bar(s), ph) && global_timer_ns() - t0 < 100000000ull) {
+        }
+      } else {
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+          const int col0 = (tile % p.tiles_col) * p.BN;
+          for (int ki = 0; ki < kiters; ++ki) {
+            const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
+            if (!mbar_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait)) {
+              ok = false;
+              break;
+            }
+            mbar_expect_tx(b_full(stage), p.stage_bytes_b);
+            tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
+            if (++stage == p.stages_b) {
+              stage = 0;
+              phase ^= 1u;
+            }
           }
         }
       }
@@ -252,8 +321,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
     if (lane == 0 && kiters > 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, bstage = 0;
+      uint32_t phase = 0, bphase = 0;
       int local_tile = 0;
       bool ok = true;
       const bool sw64 = p.swizzle64 != 0;
@@ -261,34 +330,87 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
         const int buf = local_tile & 1;
         const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait)) {
-          ok = false;
-          break;
-        }
+        if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * p.tmem_buf_stride;
-        for (int ki = 0; ki < kiters; ++ki) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, kAsyncMmaFullWait)) {
-            ok = false;
-            break;
+        if (halo) {
+          int n0, o0, w0, col0;
+          decode(tile, n0, o0, w0, col0);
+          const int rel0 = o0 - (o0 / p.P) * p.P;
+          int ki = 0;
+          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
+            if (!mbar_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t patch = ring_a + stage * a_stride;
+            for (int t = 0; t < p.ntaps; ++t, ++ki) {
+              const int shift = rel0 + (p.tap_dh[t] - p.dh_min) * p.P + (p.tap_dw[t] - p.dw_min);
+              uint32_t sb;
+              if (p.b_resident) {
+                sb = ring_b + ki * p.stage_bytes_b;
+                if (local_tile == 0) {
+                  if (!mbar_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait)) {
+                    ok = false;
+                    break;
+                  }
+                  tc_fence_after();
+                }
+              } else {
+                sb = ring_b + bstage * p.stage_bytes_b;
+                if (!mbar_wait(b_full(bstage), bphase, abort_flag, p.status, kAsyncMmaBFullWait)) {
+                  ok = false;
+                  break;
+                }
+                tc_fence_after();
+              }
+              const uint64_t adesc = make_smem_desc(patch + (uint32_t)shift * (uint32_t)p.BK, sw64);
+              const uint64_t bdesc = make_smem_desc(sb, sw64);
+              for (int k = 0; k < kk; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (ki | k) != 0 ? 1u : 0u);
+              if (!p.b_resident) {
+                umma_commit(b_empty(bstage));
+                if (++bstage == p.stages_b) {
+                  bstage = 0;
+                  bphase ^= 1u;
+                }
+              }
+            }
+            if (!ok) break;
+            umma_commit(a_empty(stage));
+            if (++stage == p.stages_a) {
+              stage = 0;
+              phase ^= 1u;
+            }
           }
-          tc_fence_after();
-          const uint32_t sa = ring + stage * stage_bytes;
-          const uint64_t adesc = make_smem_desc(sa, sw64);
-          const uint64_t bdesc = make_smem_desc(sa + p.stage_bytes_a, sw64);
-          for (int k = 0; k < kk; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (ki | k) != 0 ? 1u : 0u);
-          umma_commit(empty_bar(stage));
-          if (++stage == p.stages) {
-            stage = 0;
-            phase ^= 1u;
+          if (!ok) break;
+        } else {
+          for (int ki = 0; ki < kiters; ++ki) {
+            if (!mbar_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sa = ring_a + stage * a_stride;
+            const uint64_t adesc = make_smem_desc(sa, sw64);
+            const uint64_t bdesc = make_smem_desc(sa + p.stage_bytes_a, sw64);
+            for (int k = 0; k < kk; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (ki | k) != 0 ? 1u : 0u);
+            umma_commit(a_empty(stage));
+            if (++stage == p.stages_a) {
+              stage = 0;
+              phase ^= 1u;
+            }
           }
+          if (!ok) break;
         }
-        if (ok) umma_commit(tfull_bar(buf));
+        umma_commit(tfull_bar(buf));
       }
     }
-  } else {
+  } else if (warp >= kFirstEpilogueWarp) {
     // ------------------------------ epilogue ------------------------------
-    const int quarter = warp & 3;  // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int quarter = warp & 3;                         // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int half = (warp - kFirstEpilogueWarp) >> 2;    // the two warps of a quarter split the column chunks
+    const int ew = warp - kFirstEpilogueWarp;
     const int row = quarter * 32 + lane;
     QParams q;
     {
@@ -299,18 +421,32 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 0.0f;
       q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
     }
-    if (blockIdx.x == 0 && warp == 2 && lane == 0) p.yq->acc_scale = q.s_acc;
+    if (blockIdx.x == 0 && ew == 0 && lane == 0) p.yq->acc_scale = q.s_acc;
     int mn = INT32_MAX, mx = INT32_MIN;
     const int rn = row / (p.Ht * p.Wt);
     const int rh = (row / p.Wt) % p.Ht;
     const int rw = row % p.Wt;
+    const int nchunks = (p.BN + 31) / 32;
+    const int c_begin = half == 0 ? 0 : (nchunks + 1) / 2;
+    const int c_end = half == 0 ? (nchunks + 1) / 2 : nchunks;
     int local_tile = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
       int n0, h0, w0, col0;
       decode(tile, n0, h0, w0, col0);
-      const int n = n0 + rn, i = h0 + rh, j = w0 + rw;
-      const bool row_valid = (n < p.n_img) && (i < p.TH) && (j < p.TW);
+      int n, i, j;
+      bool row_valid;
+      if (halo) {
+        const int o = h0 + row;
+        n = n0;
+        i = o / p.P;
+        j = o - i * p.P;
+        row_valid = (o < p.L) && (j < p.TW);
+      } else {
+        n = n0 + rn;
+        i = h0 + rh;
+        j = w0 + rw;
+        row_valid = (n < p.n_img) && (i < p.TH) && (j < p.TW);
+      }
       const int64_t pix = ((int64_t)n * p.out_H + (i * p.os_h + p.oa_h)) * p.out_W + (j * p.os_w + p.oa_w);
       const int32_t* corr_row = nullptr;
       if (p.corr != nullptr && q.zx != 0 && row_valid) {
@@ -323,78 +459,84 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       if (kiters > 0) {
         bool w = mbar_wait(tfull_bar(buf), tph, abort_flag, p.status, kAsyncEpilogueTmemFullWait);
         w = __all_sync(0xffffffffu, w);
-        if (!w) {
-          ok = false;
-          break;
-        }
+        if (!w) break;
         tc_fence_after();
       }
       const uint32_t taddr = tmem_base + buf * p.tmem_buf_stride + ((uint32_t)(quarter * 32) << 16);
-      for (int c0 = 0; c0 < p.BN; c0 += 16) {
-        int v[16];
+      for (int ch = c_begin; ch < c_end; ++ch) {
+        const int c0 = ch * 32;
+        int v[32];
         if (kiters > 0) {
-          tmem_ld16(taddr + c0, v);
+          tmem_ld32(taddr + c0, v);
           tmem_ld_wait();
         } else {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) v[e] = 0;
+          for (int e = 0; e < 32; ++e) v[e] = 0;
         }
         int nvalid = p.Nout - (col0 + c0);
-        nvalid = nvalid < 0 ? 0 : (nvalid > 16 ? 16 : nvalid);
+        nvalid = nvalid < 0 ? 0 : (nvalid > 32 ? 32 : nvalid);
+        if (c0 + nvalid > p.BN) nvalid = p.BN - c0;
         if (!row_valid) nvalid = 0;
         if (corr_row != nullptr) {
+          const int lim = (p.BN - c0 < 32) ? p.BN - c0 : 32;   // the table is padded to whole column tiles
 #pragma unroll
-          for (int e = 0; e < 16; e += 4) {
-            const int4 cr = *reinterpret_cast<const int4*>(corr_row + c0 + e);
-            v[e + 0] -= q.zx * cr.x;
-            v[e + 1] -= q.zx * cr.y;
-            v[e + 2] -= q.zx * cr.z;
-            v[e + 3] -= q.zx * cr.w;
+          for (int e = 0; e < 32; e += 4) {
+            if (e < lim) {
+              const int4 cr = *reinterpret_cast<const int4*>(corr_row + c0 + e);
+              v[e + 0] -= q.zx * cr.x;
+              v[e + 1] -= q.zx * cr.y;
+              v[e + 2] -= q.zx * cr.z;
+              v[e + 3] -= q.zx * cr.w;
+            }
           }
         }
         if (p.bias != nullptr) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e)
+          for (int e = 0; e < 32; ++e)
             if (e < nvalid) v[e] += p.bias[col0 + c0 + e];
         }
+        if (nvalid == 32) {
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          if (e < nvalid) {
-            mn = min(mn, v[e]);
-            mx = max(mx, v[e]);
+          for (int e = 0; e < 32; e += 2) {
+            mn = __vimin3_s32(mn, v[e], v[e + 1]);
+            mx = __vimax3_s32(mx, v[e], v[e + 1]);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            if (e < nvalid) {
+              mn = min(mn, v[e]);
+              mx = max(mx, v[e]);
+            }
           }
         }
         if (nvalid > 0) {
           if constexpr (kOut == kOutInt8) {
-            uint32_t w[4];
+            uint32_t w[8];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              uint32_t b0 = (uint32_t)quantize_one(v[4 * e + 0], q) & 0xffu;
-              uint32_t b1 = (uint32_t)quantize_one(v[4 * e + 1], q) & 0xffu;
-              uint32_t b2 = (uint32_t)quantize_one(v[4 * e + 2], q) & 0xffu;
-              uint32_t b3 = (uint32_t)quantize_one(v[4 * e + 3], q) & 0xffu;
-              w[e] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
-            }
+            for (int e = 0; e < 8; ++e)
+              w[e] = pack_sat4(requant_unclamped(v[4 * e + 0], q), requant_unclamped(v[4 * e + 1], q), requant_unclamped(v[4 * e + 2], q),
+                               requant_unclamped(v[4 * e + 3], q));
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16) store_bytes16<16>(dst, w, nvalid);
-            else if (out_vec == 8) store_bytes16<8>(dst, w, nvalid);
-            else if (out_vec == 4) store_bytes16<4>(dst, w, nvalid);
-            else store_bytes16<1>(dst, w, nvalid);
+            if (out_vec == 16) store_bytes32<16>(dst, w, nvalid);
+            else if (out_vec == 8) store_bytes32<8>(dst, w, nvalid);
+            else if (out_vec == 4) store_bytes32<4>(dst, w, nvalid);
+            else store_bytes32<1>(dst, w, nvalid);
           } else {
-            uint32_t w[16];
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              if constexpr (kOut == kOutF32) w[e] = __float_as_uint(__fmul_rn(__int2float_rn(v[e]), q.s_acc));
-              else w[e] = (uint32_t)v[e];
-            }
             uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16 && nvalid == 16) {
+            if (out_vec == 16 && nvalid == 32) {
 #pragma unroll
-              for (int e = 0; e < 4; ++e) *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[4 * e], w[4 * e + 1], w[4 * e + 2], w[4 * e + 3]);
+              for (int e = 0; e < 8; ++e) {
+                uint32_t w[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[4 * e + k]), q.s_acc)) : (uint32_t)v[4 * e + k];
+                *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[0], w[1], w[2], w[3]);
+              }
             } else {
 #pragma unroll
-              for (int e = 0; e < 16; ++e)
-                if (e < nvalid) dst[e] = w[e];
+              for (int e = 0; e < 32; ++e)
+                if (e < nvalid) dst[e] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[e]), q.s_acc)) : (uint32_t)v[e];
             }
           }
         }
@@ -409,18 +551,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
     if (lane == 0) {
-      red_min[quarter] = mn;
-      red_max[quarter] = mx;
+      red_min[ew] = mn;
+      red_max[ew] = mx;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(kEpilogueWarps * 32) : "memory");
-    if (warp == 2 && lane == 0) {
+    if (ew == 0 && lane == 0) {
       for (int e = 1; e < kEpilogueWarps; ++e) {
-        red_min[0] = min(red_min[0], red_min[e]);
-        red_max[0] = max(red_max[0], red_max[e]);
+        mn = min(mn, red_min[e]);
+        mx = max(mx, red_max[e]);
       }
-      if (red_min[0] <= red_max[0]) {
-        atomicMin(&p.yq->acc_min, red_min[0]);
-        atomicMax(&p.yq->acc_max, red_max[0]);
+      if (mn <= mx) {
+        atomicMin(&p.yq->acc_min, mn);
+        atomicMax(&p.yq->acc_max, mx);
       }
     }
   }

@@ -14,9 +14,12 @@ namespace hq {
 
 constexpr int kMaxTaps = 49;          // 7x7
 constexpr int kTileM = 128;           // rows of one accumulator tile = TMEM lanes
-constexpr int kEpilogueWarps = 4;
-constexpr int kGemmThreads = 32 * (2 + kEpilogueWarps);   // producer warp, MMA warp, epilogue warps
-constexpr uint32_t kSmemBudget = 200 * 1024;              // operand ring; barriers and tables sit on top
+constexpr int kEpilogueWarps = 8;     // two per TMEM lane quarter; they split the columns
+constexpr int kFirstEpilogueWarp = 4; // warps 0..3: A producer, MMA issuer, B producer, spare
+constexpr int kGemmThreads = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
+constexpr int kMaxStagesA = 12;
+constexpr int kMaxStagesB = 32;
+constexpr uint32_t kSmemBudget = 212 * 1024;              // operand rings; barriers sit in static shared memory
 constexpr uint64_t kWaitLimitNs = 2000000000ull;          // bound of every device-side wait
 
 // status-word codes written by kernels when a bounded wait expires
@@ -26,24 +29,39 @@ enum AsyncCode : int32_t {
   kAsyncMmaFullWait = 2,
   kAsyncMmaTmemEmptyWait = 3,
   kAsyncEpilogueTmemFullWait = 4,
-  kAsyncDrainWait = 5,
+  kAsyncProducerBEmptyWait = 5,
+  kAsyncMmaBFullWait = 6,
 };
 
 enum OutMode : int { kOutInt8 = 0, kOutF32 = 1, kOutAcc = 2 };
+enum GemmMode : int { kModeTap = 0, kModeHalo = 1 };
 
 // One launch of the tensor-core kernel: an implicit GEMM over a "tile space" of output pixels.
 //   tile-space pixel (n, i, j), i in [0,TH), j in [0,TW)
-//   output pixel     (n, i*os_h + oa_h, j*os_w + oa_w) in an out_H x out_W image of ldY bytes/elements per pixel
-//   operand A, tap t (n, i*in_mul_h + tap_dh[t], j*in_mul_w + tap_dw[t], c)   -- fetched by a 4-D TMA box,
-//                    out-of-image coordinates are filled with zeros by the copy engine
+//   output pixel     (n, i*os_h + oa_h, j*os_w + oa_w) in an out_H x out_W image of ldY elements per pixel
+//   operand A, tap t (n, i*in_mul_h + tap_dh[t], j*in_mul_w + tap_dw[t], c); out-of-image coordinates read as zero
 //   operand B        weight matrix [Nout][ntaps][Cpad], K-major
+//
+// kModeTap : every (tap, channel chunk) is one ring stage = one TMA box of A (128 pixels x BK bytes) and one of B.
+// kModeHalo: stride-1 tile spaces only.  The output pixels of an image are numbered o = i*P + j with
+//            P = TW + (max tap_dw - min tap_dw) (j >= TW are dead columns); a tile is 128 consecutive o.  One TMA
+//            box per channel chunk brings the NR padded input rows the tile touches into shared memory once, and
+//            tap (dr, ds) reads them through a matrix descriptor whose start is shifted by (dr*P + ds) pixels.
+//            Only the weights stream through the B ring (or stay resident when they fit).
 struct GemmParams {
+  int32_t mode;
   int32_t n_img, TH, TW;
-  int32_t Nt, Ht, Wt;                 // Nt*Ht*Wt == kTileM
+  int32_t Nt, Ht, Wt;                 // kModeTap: Nt*Ht*Wt == kTileM
   int32_t tiles_n, tiles_h, tiles_w, tiles_col, num_tiles;
   int32_t in_mul_h, in_mul_w;
   int32_t ntaps, chunks_per_tap, BK, Cpad;
   int8_t tap_dh[kMaxTaps], tap_dw[kMaxTaps];
+  // kModeHalo
+  int32_t P, L, NR, tiles_per_img, dh_min, dw_min;
+  uint32_t patch_chunk_stride;        // bytes between channel chunks of one patch (1024-aligned)
+  uint32_t patch_box_bytes;           // bytes one patch TMA delivers
+  int32_t b_resident;
+  // common
   int32_t Nout, BN;
   int32_t out_H, out_W, os_h, os_w, oa_h, oa_w;
   int64_t ldY;
@@ -59,13 +77,13 @@ struct GemmParams {
   int32_t* status;
   uint32_t idesc;
   uint32_t tmem_cols, tmem_buf_stride;
-  int32_t stages;
-  uint32_t stage_bytes_a, stage_bytes_b;
+  int32_t stages_a, stages_b;
+  uint32_t stage_bytes_a, stage_bytes_b;   // kModeTap: A and B part of one stage; kModeHalo: patch stage, B stage
   int32_t swizzle64;                  // 1: 64-byte swizzle (BK = 64), 0: 128-byte swizzle (BK = 128)
-  int32_t small_acc;                  // |acc| provably < 2^22: conversions may use the exact magic-number form
+  int32_t producer_lanes;             // kModeTap: lanes of the producer warp that issue copies
 };
 
-struct DwParams {                     // depthwise 3x3 (CUDA cores)
+struct DwParams {                     // depthwise (CUDA cores)
   int32_t N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w;
   const int8_t* x;
   const int8_t* w;                    // [R*S][C] tap-major
@@ -108,6 +126,7 @@ struct hq_ctx {
   size_t scratch_elems = 0;
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
+  int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
   std::string err;
 };
 

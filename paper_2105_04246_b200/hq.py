@@ -22,7 +22,7 @@ DIR_FWD, DIR_BWD_DATA = 0, 1
 OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 
 # every extern "C" symbol include/hq.h declares
-EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count",
+EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_set_option",
            "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
            "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate"]
 
@@ -66,6 +66,7 @@ def lib():
         L.hq_last_error.argtypes = [vp]; L.hq_last_error.restype = C.c_char_p
         L.hq_get_async_error.argtypes = [vp, vp, C.POINTER(i32)]
         L.hq_launch_count.argtypes = [vp]; L.hq_launch_count.restype = C.c_uint64
+        L.hq_set_option.argtypes = [vp, C.c_char_p, i32]
         L.hq_weights_prepare.argtypes = [vp, vp, C.POINTER(ConvDesc), C.c_int, vp, C.POINTER(vp)]
         L.hq_weights_release.argtypes = [vp, vp]
         L.hq_linear_fwd.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
@@ -184,6 +185,9 @@ class Context:
         if st not in (HQ_OK, 6):
             self._check(st)
         return code.value
+
+    def set_option(self, key: str, value: int):
+        self._check(lib().hq_set_option(self.handle, key.encode(), int(value)))
 
     def launch_count(self) -> int:
         return int(lib().hq_launch_count(self.handle))

@@ -25,8 +25,12 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9):
-    g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1):
+    ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
+    try:
+        g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
+    finally:
+        ctx.set_option("staging", -1)
     o = OracleLayer(kind, W, shape, bias=bias, eta=eta)
     for t in range(iters):
         x = make_x(t)
@@ -91,6 +95,10 @@ FWD_CASES = {
     "1x1_s2": dict(N=2, H=14, W=14, Cin=64, K=128, R=1, S=1, stride=2, pad=0),
     "1x1_c24_k144_fold": dict(N=2, H=10, W=13, Cin=24, K=144, R=1, S=1),
     "1x1_c144_k24": dict(N=2, H=10, W=13, Cin=144, K=24, R=1, S=1),
+    "3x3_c64_56x56": dict(N=2, H=56, W=56, Cin=64, K=64, R=3, S=3, stride=1, pad=1),
+    "3x3_c128_28x28": dict(N=3, H=28, W=28, Cin=128, K=128, R=3, S=3, stride=1, pad=1),
+    "3x3_c512_k512_7x7": dict(N=4, H=7, W=7, Cin=512, K=512, R=3, S=3, stride=1, pad=1),
+    "7x7_c16_s1": dict(N=1, H=20, W=23, Cin=16, K=32, R=7, S=7, stride=1, pad=3),
     "5x5_c16": dict(N=1, H=11, W=11, Cin=16, K=48, R=5, S=5, stride=1, pad=2),
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
@@ -104,15 +112,16 @@ def _weights(r, shape):
     return synth.weights(r, (shape["K"], shape["R"], shape["S"], shape["Cin"]))
 
 
+@pytest.mark.parametrize("staging", [-1, 0, 1])
 @pytest.mark.parametrize("name", list(FWD_CASES))
-def test_conv_fwd(ctx, name):
+def test_conv_fwd(ctx, name, staging):
     shape = dict(FWD_CASES[name])
     shape.setdefault("R", 1); shape.setdefault("S", 1)
     r = synth.rng(103, len(name), shape["H"], shape["Cin"])
     W = _weights(r, shape)
     in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
     makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
-    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3)
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, staging=staging)
 
 
 BWD_CASES = {
@@ -126,15 +135,16 @@ BWD_CASES = {
 }
 
 
+@pytest.mark.parametrize("staging", [-1, 0, 1])
 @pytest.mark.parametrize("name", list(BWD_CASES))
-def test_conv_bwd_data(ctx, name):
+def test_conv_bwd_data(ctx, name, staging):
     shape = dict(BWD_CASES[name])
     r = synth.rng(104, len(name), shape["H"], shape["Cin"])
     W = _weights(r, shape)
     Ho = (shape["H"] + 2 * shape.get("pad", 0) - shape["R"]) // shape.get("stride", 1) + 1
     Wo = (shape["W"] + 2 * shape.get("pad", 0) - shape["S"]) // shape.get("stride", 1) + 1
     in_shape = (shape["N"], Ho, Wo, shape["K"])
-    _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3)
+    _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3, staging=staging)
 
 
 # ---- protocol and edge cases ---------------------------------------------------------------------
