@@ -95,6 +95,16 @@ void pick_tile(int n_img, int TH, int TW, int in_mul_h, int in_mul_w, int& Nt, i
     }
 }
 
+FastDiv make_fastdiv(int d) {
+  FastDiv f{1u, 0u};
+  if (d <= 1) return f;
+  uint32_t l = 0;
+  while ((1ull << l) < (uint64_t)d) ++l;
+  f.l = l;
+  f.m = (uint32_t)(((1ull << 32) * ((1ull << l) - (uint64_t)d)) / (uint64_t)d + 1ull);
+  return f;
+}
+
 struct SubSpec {            // geometry of one launch, before tiling
   int n_img, TH, TW;
   int in_mul_h, in_mul_w;
@@ -158,6 +168,23 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     p.tmem_buf_stride = s;
     p.tmem_cols = 2 * s;
   }
+  // border classes first: the size of the correction table decides how much shared memory the rings get
+  if (sp.flat) {
+    rowcls.clear();
+    colcls.clear();
+    rowmasks.assign(1, 1u);
+    colmasks.assign(1, 1u);
+  } else {
+    border_classes(sp.TH, sp.in_mul_h, sp.dh, sp.a_H, rowcls, rowmasks);
+    border_classes(sp.TW, sp.in_mul_w, sp.dw, sp.a_W, colcls, colmasks);
+    if (rowmasks.size() > 16 || colmasks.size() > 16) return fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes");
+  }
+  p.ncolcls = (int)colmasks.size();
+  p.zc_elems = (int)(rowmasks.size() * colmasks.size()) * p.corr_ld;
+  p.zc_in_smem = ((uint32_t)p.zc_elems * 4u <= kMaxZcBytes && p.ntaps > 0) ? 1 : 0;
+  const uint32_t zc_bytes = p.zc_in_smem ? (((uint32_t)p.zc_elems * 4u + 1023u) & ~1023u) : 0u;
+  const uint32_t ring_budget = kSmemBudget - zc_bytes;
+  p.zc_offset = ring_budget;
   // ---- operand staging: resident input rows (kModeHalo) where the tile space is stride-1, else one box per tap ----
   p.mode = kModeTap;
   p.stage_bytes_b = (uint32_t)p.BN * p.BK;
@@ -179,15 +206,15 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
            (util >= 0.6 || ctx->force_mode == kModeHalo);
     int stages_a = 0, stages_b = 0, resident = 0;
     if (halo) {
-      if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * p.stage_bytes_b + 2ull * stride <= kSmemBudget) {
+      if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * p.stage_bytes_b + 2ull * stride <= ring_budget) {
         resident = 1;
         stages_b = kiters;
-        stages_a = (int)std::min<uint64_t>(4, (kSmemBudget - (uint64_t)kiters * p.stage_bytes_b) / stride);
+        stages_a = (int)std::min<uint64_t>(4, (ring_budget - (uint64_t)kiters * p.stage_bytes_b) / stride);
       } else {
         stages_a = 2;
-        while (stages_a < 4 && (uint64_t)(stages_a + 1) * stride + 4ull * p.stage_bytes_b <= kSmemBudget) ++stages_a;
-        if ((uint64_t)stages_a * stride < kSmemBudget)
-          stages_b = (int)std::min<uint64_t>(8, (kSmemBudget - (uint64_t)stages_a * stride) / p.stage_bytes_b);
+        while (stages_a < 4 && (uint64_t)(stages_a + 1) * stride + 4ull * p.stage_bytes_b <= ring_budget) ++stages_a;
+        if ((uint64_t)stages_a * stride < ring_budget)
+          stages_b = (int)std::min<uint64_t>(8, (ring_budget - (uint64_t)stages_a * stride) / p.stage_bytes_b);
         if (stages_b < 2) halo = false;
       }
     }
@@ -214,7 +241,7 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   }
   if (p.mode == kModeTap) {
     p.stage_bytes_a = (uint32_t)kTileM * p.BK;
-    p.stages_a = (int)std::min<uint32_t>(kMaxStagesA, kSmemBudget / (p.stage_bytes_a + p.stage_bytes_b));
+    p.stages_a = (int)std::min<uint32_t>(kMaxStagesA, ring_budget / (p.stage_bytes_a + p.stage_bytes_b));
     p.stages_b = 0;
     if (p.stages_a < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
     p.producer_lanes = std::min(4, p.stages_a);
@@ -224,17 +251,11 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   sub.a_stride_h = sp.in_mul_h;
   sub.a_stride_w = sp.in_mul_w;
   p.status = ctx->d_status;
-  if (sp.flat) {
-    rowcls.clear();
-    colcls.clear();
-    rowmasks.assign(1, 1u);
-    colmasks.assign(1, 1u);
-  } else {
-    border_classes(sp.TH, sp.in_mul_h, sp.dh, sp.a_H, rowcls, rowmasks);
-    border_classes(sp.TW, sp.in_mul_w, sp.dw, sp.a_W, colcls, colmasks);
-    if (rowmasks.size() > 16 || colmasks.size() > 16) return fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes");
-  }
-  p.ncolcls = (int)colmasks.size();
+  p.fd_tiles_col = make_fastdiv(p.tiles_col);
+  p.fd_tiles_per_img = make_fastdiv(p.mode == kModeHalo ? p.tiles_per_img : 1);
+  p.fd_tiles_w = make_fastdiv(p.tiles_w);
+  p.fd_tiles_h = make_fastdiv(p.tiles_h);
+  p.fd_P = make_fastdiv(p.mode == kModeHalo ? p.P : 1);
   return HQ_OK;
 }
 
@@ -326,6 +347,7 @@ hq_status build_sub(hq_ctx* ctx, hq_prepared_weights* pw, cudaStream_t s, const 
   p.corr = sub.corr;
   p.rowcls = sub.rowcls;
   p.colcls = sub.colcls;
+  p.cls_in_smem = (sub.rowcls && sub.colcls && p.TH <= 512 && p.TW <= 512) ? 1 : 0;
   return encode_b(ctx, sub, sub.wmat, (int64_t)p.ntaps * p.Cpad, &sub.tmap_b);
 }
 

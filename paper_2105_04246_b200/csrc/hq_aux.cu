@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "hq_internal.h"
+#include "hq_quant.cuh"
 
 namespace hq {
 namespace {
@@ -57,22 +58,14 @@ __global__ void dynamic_derive_kernel(hq_range_state* s) {
   s->acc_max = INT32_MIN;
 }
 
-__device__ __forceinline__ int quantize_real(float y, float inv_scale, int zp) {
-  const float u = __fmul_rn(y, inv_scale);
-  const int r = __float2int_rn(u);
-  int s;
-  asm("add.sat.s32 %0, %1, %2;" : "=r"(s) : "r"(r), "r"(zp));
-  return min(max(s, -128), 127);
-}
-
-__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
-  return ((uint32_t)a & 0xffu) | (((uint32_t)b & 0xffu) << 8) | (((uint32_t)c & 0xffu) << 16) | (((uint32_t)d & 0xffu) << 24);
-}
-
 // second pass of the dynamic path: read the binary32 output back and quantize it
 __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __restrict__ out, int64_t count, const hq_range_state* st) {
-  const float inv_scale = st->inv_scale;
-  const int zp = st->zero_point;
+  QParams q;
+  q.s_acc = 1.0f;
+  q.zx = 0;
+  q.inv_scale = st->inv_scale;
+  q.zp = st->zero_point;
+  qparams_finish(q);
   const int64_t groups = count / 16;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) {
@@ -81,13 +74,14 @@ __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __rest
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const float4 f = __ldcs(src + e);
-      w[e] = pack4(quantize_real(f.x, inv_scale, zp), quantize_real(f.y, inv_scale, zp), quantize_real(f.z, inv_scale, zp),
-                   quantize_real(f.w, inv_scale, zp));
+      w[e] = q.fast ? pack_sat4(requant_real<true>(f.x, q), requant_real<true>(f.y, q), requant_real<true>(f.z, q), requant_real<true>(f.w, q))
+                    : pack_sat4(requant_real<false>(f.x, q), requant_real<false>(f.y, q), requant_real<false>(f.z, q), requant_real<false>(f.w, q));
     }
     reinterpret_cast<uint4*>(out)[g] = make_uint4(w[0], w[1], w[2], w[3]);
   }
   if (blockIdx.x == 0) {
-    for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x) out[i] = (int8_t)quantize_real(y[i], inv_scale, zp);
+    for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x)
+      out[i] = (int8_t)min(max(requant_real<false>(y[i], q), -128), 127);
   }
 }
 
@@ -174,10 +168,14 @@ __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w 
 template <int kOut>
 __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
   __shared__ int red_min[8], red_max[8];
-  const float s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
-  const int zx = p.xq->zero_point;
-  const float inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 0.0f;
-  const int zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  QParams q;
+  q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
+  q.zx = p.xq->zero_point;
+  q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
+  q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  qparams_finish(q);
+  const float s_acc = q.s_acc;
+  const int zx = q.zx;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = s_acc;
   const int cgs = p.C / 16;
   const int64_t total = (int64_t)p.N * p.Ho * p.Wo * cgs;
@@ -222,10 +220,10 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
       uint32_t w[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        int q[4];
+        int c[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) q[k] = quantize_real(__fmul_rn(__int2float_rn(acc[4 * e + k]), s_acc), inv_scale, zp);
-        w[e] = pack4(q[0], q[1], q[2], q[3]);
+        for (int k = 0; k < 4; ++k) c[k] = q.fast ? requant_acc<true>(acc[4 * e + k], q) : requant_acc<false>(acc[4 * e + k], q);
+        w[e] = pack_sat4(c[0], c[1], c[2], c[3]);
       }
       *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
     } else {

@@ -11,7 +11,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "hq_internal.h"
+#include "hq_quant.cuh"
 
 namespace hq {
 namespace {
@@ -27,12 +30,14 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
+// One try_wait; the hardware may suspend the thread for up to `hint_ns` while the phase is pending, which keeps
+// waiting threads from flooding the memory-instruction queue that the MMA and TMA issue also go through.
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity, uint32_t hint_ns) {
   uint32_t ok;
   asm volatile(
-      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(hint_ns)
       : "memory");
   return ok;
 }
@@ -44,13 +49,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 
 // Bounded wait on an mbarrier phase.  Gives up when another role has already given up or
 // after kWaitLimitNs; the first to give up records `code` in the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code) {
-  if (mbar_try(bar, parity)) return true;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code,
+                                          uint32_t hint_ns = 200u) {
+  if (mbar_try(bar, parity, hint_ns)) return true;
   const uint64_t t0 = global_timer_ns();
   uint32_t spins = 0;
   for (;;) {
-    if (mbar_try(bar, parity)) return true;
-    if ((++spins & 63u) == 0u) {
+    if (mbar_try(bar, parity, hint_ns)) return true;
+    if ((++spins & 15u) == 0u) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
         *abort_flag = 1;
@@ -59,6 +65,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+
+// n / d for 0 <= n < 2^31 with the multiplier and shift prepared on the host (see make_fastdiv)
+__device__ __forceinline__ int fdiv(int n, FastDiv d) { return (int)((__umulhi(d.m, (uint32_t)n) + (uint32_t)n) >> d.l); }
+
+// all 32 lanes wait (warp-uniform result)
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code,
+                                          uint32_t hint_ns) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, status, code, hint_ns);
+  return __all_sync(0xffffffffu, ok);
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
@@ -114,28 +136,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int* v) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-struct QParams {
-  float s_acc, inv_scale;
-  int zx, zp;
-};
-
-// y = fl(float(acc) * s_acc); r = rint(fl(y * inv_scale)) + zero_point (saturating add): one rounding per step.
-__device__ __forceinline__ int requant_unclamped(int a, const QParams& q) {
-  const float y = __fmul_rn(__int2float_rn(a), q.s_acc);
-  const float u = __fmul_rn(y, q.inv_scale);
-  const int r = __float2int_rn(u);  // saturating conversion, NaN -> 0
-  int s;
-  asm("add.sat.s32 %0, %1, %2;" : "=r"(s) : "r"(r), "r"(q.zp));
-  return s;
-}
-// four values -> four saturated int8 codes in one word, element 0 in the lowest byte
-__device__ __forceinline__ uint32_t pack_sat4(int q0, int q1, int q2, int q3) {
-  uint32_t hi, d;
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
-  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(q1), "r"(q0), "r"(hi));
-  return d;
-}
-
 template <int V>
 __device__ __forceinline__ void store_bytes32(int8_t* p, const uint32_t* w, int nvalid) {
   // w: 8 words = 32 output bytes; store the first nvalid bytes in pieces of V bytes
@@ -167,6 +167,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int red_min[kEpilogueWarps], red_max[kEpilogueWarps];
+  __shared__ uint32_t tapoff_s[kMaxTaps];      // kModeHalo: start shift of tap t in 16-byte units
+  __shared__ uint8_t cls_s[1024];              // border classes of rows [0,512) and columns [512,1024) when they fit
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -204,6 +206,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (threadIdx.x < (unsigned)p.ntaps && p.mode == kModeHalo)
+    tapoff_s[threadIdx.x] =
+        (uint32_t)(((p.tap_dh[threadIdx.x] - p.dh_min) * p.P + (p.tap_dw[threadIdx.x] - p.dw_min)) * p.BK) >> 4;
+  int32_t* zc_s = reinterpret_cast<int32_t*>(smem_raw + ((ring_a - smem_u32(smem_raw)) + p.zc_offset));
+  if (p.zc_in_smem) {   // zx * (sum of in-image weights) per border class and output channel
+    const int zx = p.xq->zero_point;
+    for (int i = threadIdx.x; i < p.zc_elems; i += blockDim.x) zc_s[i] = zx * p.corr[i];
+  }
+  if (p.cls_in_smem) {
+    for (int i = threadIdx.x; i < p.TH; i += blockDim.x) cls_s[i] = p.rowcls[i];
+    for (int i = threadIdx.x; i < p.TW; i += blockDim.x) cls_s[512 + i] = p.colcls[i];
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(p.tmem_cols)
                  : "memory");
@@ -216,84 +230,82 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 
   // tile index -> origin.  kModeTap: (n0, h0, w0) of the pixel box; kModeHalo: image n0, first linear pixel h0
   auto decode = [&](int tile, int& n0, int& h0, int& w0, int& col0) {
-    const int ct = tile % p.tiles_col;
-    int t = tile / p.tiles_col;
-    col0 = ct * p.BN;
+    int t = fdiv(tile, p.fd_tiles_col);
+    col0 = (tile - t * p.tiles_col) * p.BN;
     if (halo) {
-      const int lt = t % p.tiles_per_img;
-      n0 = t / p.tiles_per_img;
-      h0 = lt * kTileM;
+      n0 = fdiv(t, p.fd_tiles_per_img);
+      h0 = (t - n0 * p.tiles_per_img) * kTileM;
       w0 = 0;
     } else {
-      const int wt = t % p.tiles_w;
-      t /= p.tiles_w;
-      const int ht = t % p.tiles_h;
-      n0 = (t / p.tiles_h) * p.Nt;
-      h0 = ht * p.Ht;
-      w0 = wt * p.Wt;
+      const int t2 = fdiv(t, p.fd_tiles_w);
+      w0 = (t - t2 * p.tiles_w) * p.Wt;
+      const int t3 = fdiv(t2, p.fd_tiles_h);
+      h0 = (t2 - t3 * p.tiles_h) * p.Ht;
+      n0 = t3 * p.Nt;
     }
   };
   const int my_tiles = (p.num_tiles > (int)blockIdx.x) ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
+  // The three single-issuer roles below are executed by their WHOLE warp with warp-uniform control flow and
+  // values; only the copy / MMA / commit instructions themselves sit under a one-lane predicate (elect.sync).
+  // Uniform values stay in uniform registers, which is what the TMA and MMA instructions take their operands from.
   if (warp == 0) {
     // ------------------------------ operand A producer ------------------------------
-    if (halo) {
-      if (lane == 0 && kiters > 0) {
-        int stage = 0;
-        uint32_t phase = 0;
-        for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-          int n0, o0, w0, col0;
-          decode(tile, n0, o0, w0, col0);
-          const int hp0 = o0 / p.P;
-          bool ok = true;
+    if (kiters > 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        int n0, h0, w0, col0;
+        decode(tile, n0, h0, w0, col0);
+        if (halo) {
+          const int hp0 = fdiv(h0, p.fd_P);   // h0 is the tile's first linear pixel
           for (int cb = 0; cb < p.chunks_per_tap; ++cb) {   // one ring stage per channel chunk of the patch
-            if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait)) {
-              ok = false;
-              break;
+            ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
+            if (!ok) break;
+            if (elect_one()) {
+              mbar_expect_tx(a_full(stage), p.patch_box_bytes);
+              tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
             }
-            mbar_expect_tx(a_full(stage), p.patch_box_bytes);
-            tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
             if (++stage == p.stages_a) {
               stage = 0;
               phase ^= 1u;
             }
           }
-          if (!ok) break;
-        }
-      }
-    } else if (lane < p.producer_lanes && kiters > 0) {
-      // lane l issues the copies of ring iterations l, l + lanes, ... (each lane tracks its own stage and phase)
-      const int total = my_tiles * kiters;
-      int stage = lane % p.stages_a;
-      uint32_t phase = (uint32_t)(lane / p.stages_a) & 1u;
-      for (int it = lane; it < total; it += p.producer_lanes) {
-        const int lt = it / kiters;
-        const int ki = it - lt * kiters;
-        const int t = ki / p.chunks_per_tap;
-        const int cc = ki - t * p.chunks_per_tap;
-        int n0, h0, w0, col0;
-        decode((int)blockIdx.x + lt * (int)gridDim.x, n0, h0, w0, col0);
-        if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait)) break;
-        const uint32_t sa = ring_a + stage * a_stride;
-        mbar_expect_tx(a_full(stage), a_stride);
-        tma_load_4d(sa, &tmap_a, cc * p.BK, w0 * p.in_mul_w + p.tap_dw[t], h0 * p.in_mul_h + p.tap_dh[t], n0, a_full(stage));
-        tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
-        stage += p.producer_lanes;
-        while (stage >= p.stages_a) {
-          stage -= p.stages_a;
-          phase ^= 1u;
+        } else {
+          for (int t = 0; t < p.ntaps && ok; ++t) {
+            const int ch = h0 * p.in_mul_h + p.tap_dh[t];
+            const int cw = w0 * p.in_mul_w + p.tap_dw[t];
+            for (int cc = 0; cc < p.chunks_per_tap; ++cc) {
+              ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
+              if (!ok) break;
+              const uint32_t sa = ring_a + stage * a_stride;
+              if (elect_one()) {
+                mbar_expect_tx(a_full(stage), a_stride);
+                tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
+                tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+              }
+              if (++stage == p.stages_a) {
+                stage = 0;
+                phase ^= 1u;
+              }
+            }
+          }
         }
       }
     }
+    __syncwarp();
   } else if (warp == 2) {
     // ------------------------------ weight producer (kModeHalo) ------------------------------
-    if (halo && lane == 0 && kiters > 0) {
+    if (halo && kiters > 0) {
       if (p.b_resident) {
         if (my_tiles > 0) {
           for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
             const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
-            mbar_expect_tx(b_full(ki), p.stage_bytes_b);
-            tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(ki));
+            if (elect_one()) {
+              mbar_expect_tx(b_full(ki), p.stage_bytes_b);
+              tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(ki));
+            }
           }
         }
       } else {
@@ -302,82 +314,95 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
           const int col0 = (tile % p.tiles_col) * p.BN;
-          for (int ki = 0; ki < kiters; ++ki) {
-            const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
-            if (!mbar_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait)) {
-              ok = false;
-              break;
-            }
-            mbar_expect_tx(b_full(stage), p.stage_bytes_b);
-            tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
-            if (++stage == p.stages_b) {
-              stage = 0;
-              phase ^= 1u;
+          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
+            for (int t = 0; t < p.ntaps; ++t) {
+              ok = warp_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait, 1000u);
+              if (!ok) break;
+              if (elect_one()) {
+                mbar_expect_tx(b_full(stage), p.stage_bytes_b);
+                tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
+              }
+              if (++stage == p.stages_b) {
+                stage = 0;
+                phase ^= 1u;
+              }
             }
           }
         }
       }
     }
+    __syncwarp();
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
-    if (lane == 0 && kiters > 0) {
+    // The k-steps of one operand stage are issued from a compile-time unrolled group: a run-time inner loop
+    // around the MMA instruction was measured to cost several hundred cycles per iteration.
+    auto mma_role = [&](auto kk_tag) {
+      constexpr int KK = decltype(kk_tag)::value;
       int stage = 0, bstage = 0;
       uint32_t phase = 0, bphase = 0;
       int local_tile = 0;
       bool ok = true;
       const bool sw64 = p.swizzle64 != 0;
-      const int kk = p.BK / 32;
+      const uint64_t bdesc0 = make_smem_desc(ring_b, sw64);
+      const int ntaps = p.ntaps, stages_b = p.stages_b;
+      const bool resident = p.b_resident != 0;
+      const uint32_t idesc = p.idesc;
+      const uint32_t bstep16 = p.stage_bytes_b >> 4;
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
         const int buf = local_tile & 1;
         const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait)) break;
+        ok = warp_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait, 200u);
+        if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * p.tmem_buf_stride;
+        uint32_t acc = 0;
         if (halo) {
           int n0, o0, w0, col0;
           decode(tile, n0, o0, w0, col0);
-          const int rel0 = o0 - (o0 / p.P) * p.P;
-          int ki = 0;
-          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
-            if (!mbar_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait)) {
-              ok = false;
-              break;
-            }
+          const uint32_t rel_bytes = (uint32_t)(o0 - fdiv(o0, p.fd_P) * p.P) * (uint32_t)p.BK;
+          if (p.b_resident && local_tile == 0) {   // the whole weight matrix arrives once
+            for (int ki = 0; ki < kiters && ok; ++ki) ok = warp_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+            if (!ok) break;
             tc_fence_after();
-            const uint32_t patch = ring_a + stage * a_stride;
-            for (int t = 0; t < p.ntaps; ++t, ++ki) {
-              const int shift = rel0 + (p.tap_dh[t] - p.dh_min) * p.P + (p.tap_dw[t] - p.dw_min);
-              uint32_t sb;
-              if (p.b_resident) {
-                sb = ring_b + ki * p.stage_bytes_b;
-                if (local_tile == 0) {
-                  if (!mbar_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait)) {
-                    ok = false;
-                    break;
-                  }
-                  tc_fence_after();
+          }
+          uint64_t bres = bdesc0;
+          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
+            ok = warp_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait, 200u);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t abase = make_smem_desc(ring_a + stage * a_stride + rel_bytes, sw64);
+            if (resident) {
+              if (elect_one()) {
+                for (int t = 0; t < ntaps; ++t) {
+                  const uint64_t adesc = abase + tapoff_s[t];
+#pragma unroll
+                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                  bres += bstep16;
                 }
-              } else {
-                sb = ring_b + bstage * p.stage_bytes_b;
-                if (!mbar_wait(b_full(bstage), bphase, abort_flag, p.status, kAsyncMmaBFullWait)) {
-                  ok = false;
-                  break;
-                }
-                tc_fence_after();
               }
-              const uint64_t adesc = make_smem_desc(patch + (uint32_t)shift * (uint32_t)p.BK, sw64);
-              const uint64_t bdesc = make_smem_desc(sb, sw64);
-              for (int k = 0; k < kk; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (ki | k) != 0 ? 1u : 0u);
-              if (!p.b_resident) {
-                umma_commit(b_empty(bstage));
-                if (++bstage == p.stages_b) {
+              __syncwarp();
+              acc = 1;
+            } else {
+              for (int t = 0; t < ntaps; ++t) {
+                ok = warp_wait(b_full(bstage), bphase, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t bdesc = bdesc0 + (uint64_t)bstage * bstep16;
+                const uint64_t adesc = abase + tapoff_s[t];
+                if (elect_one()) {
+#pragma unroll
+                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
+                  umma_commit(b_empty(bstage));
+                }
+                acc = 1;
+                if (++bstage == stages_b) {
                   bstage = 0;
                   bphase ^= 1u;
                 }
               }
             }
             if (!ok) break;
-            umma_commit(a_empty(stage));
+            if (elect_one()) umma_commit(a_empty(stage));
             if (++stage == p.stages_a) {
               stage = 0;
               phase ^= 1u;
@@ -386,16 +411,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           if (!ok) break;
         } else {
           for (int ki = 0; ki < kiters; ++ki) {
-            if (!mbar_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait)) {
-              ok = false;
-              break;
-            }
+            ok = warp_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait, 200u);
+            if (!ok) break;
             tc_fence_after();
             const uint32_t sa = ring_a + stage * a_stride;
             const uint64_t adesc = make_smem_desc(sa, sw64);
             const uint64_t bdesc = make_smem_desc(sa + p.stage_bytes_a, sw64);
-            for (int k = 0; k < kk; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, p.idesc, (ki | k) != 0 ? 1u : 0u);
-            umma_commit(a_empty(stage));
+            if (elect_one()) {
+#pragma unroll
+              for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
+              umma_commit(a_empty(stage));
+            }
+            acc = 1;
             if (++stage == p.stages_a) {
               stage = 0;
               phase ^= 1u;
@@ -403,9 +430,14 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           }
           if (!ok) break;
         }
-        umma_commit(tfull_bar(buf));
+        if (elect_one()) umma_commit(tfull_bar(buf));
       }
+    };
+    if (kiters > 0) {
+      if (p.BK == 64) mma_role(std::integral_constant<int, 2>{});
+      else mma_role(std::integral_constant<int, 4>{});
     }
+    __syncwarp();
   } else if (warp >= kFirstEpilogueWarp) {
     // ------------------------------ epilogue ------------------------------
     const int quarter = warp & 3;                         // TMEM lanes 32*quarter .. +31 belong to this warp
@@ -418,8 +450,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       const float s_w = *p.w_scale;
       q.s_acc = __fmul_rn(s_x, s_w);
       q.zx = p.xq->zero_point;
-      q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 0.0f;
+      q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
       q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+      qparams_finish(q);
     }
     if (blockIdx.x == 0 && ew == 0 && lane == 0) p.yq->acc_scale = q.s_acc;
     int mn = INT32_MAX, mx = INT32_MIN;
@@ -438,7 +471,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       if (halo) {
         const int o = h0 + row;
         n = n0;
-        i = o / p.P;
+        i = fdiv(o, p.fd_P);
         j = o - i * p.P;
         row_valid = (o < p.L) && (j < p.TW);
       } else {
@@ -450,15 +483,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       const int64_t pix = ((int64_t)n * p.out_H + (i * p.os_h + p.oa_h)) * p.out_W + (j * p.os_w + p.oa_w);
       const int32_t* corr_row = nullptr;
       if (p.corr != nullptr && q.zx != 0 && row_valid) {
-        const int rc = p.rowcls ? p.rowcls[i] : 0;
-        const int cc = p.colcls ? p.colcls[j] : 0;
-        corr_row = p.corr + (int64_t)(rc * p.ncolcls + cc) * p.corr_ld + col0;
+        const int rc = p.cls_in_smem ? cls_s[i] : (p.rowcls ? p.rowcls[i] : 0);
+        const int cc = p.cls_in_smem ? cls_s[512 + j] : (p.colcls ? p.colcls[j] : 0);
+        const int off = (rc * p.ncolcls + cc) * p.corr_ld + col0;
+        corr_row = (p.zc_in_smem ? zc_s : p.corr) + off;
       }
+      const int zmul = p.zc_in_smem ? 1 : q.zx;   // the shared table is already multiplied by zx
       const int buf = local_tile & 1;
       const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
       if (kiters > 0) {
-        bool w = mbar_wait(tfull_bar(buf), tph, abort_flag, p.status, kAsyncEpilogueTmemFullWait);
-        w = __all_sync(0xffffffffu, w);
+        int w = 1;
+        if (lane == 0) w = mbar_wait(tfull_bar(buf), tph, abort_flag, p.status, kAsyncEpilogueTmemFullWait, 2000u) ? 1 : 0;
+        w = __shfl_sync(0xffffffffu, w, 0);
         if (!w) break;
         tc_fence_after();
       }
@@ -483,10 +519,10 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           for (int e = 0; e < 32; e += 4) {
             if (e < lim) {
               const int4 cr = *reinterpret_cast<const int4*>(corr_row + c0 + e);
-              v[e + 0] -= q.zx * cr.x;
-              v[e + 1] -= q.zx * cr.y;
-              v[e + 2] -= q.zx * cr.z;
-              v[e + 3] -= q.zx * cr.w;
+              v[e + 0] -= zmul * cr.x;
+              v[e + 1] -= zmul * cr.y;
+              v[e + 2] -= zmul * cr.z;
+              v[e + 3] -= zmul * cr.w;
             }
           }
         }
@@ -513,10 +549,17 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         if (nvalid > 0) {
           if constexpr (kOut == kOutInt8) {
             uint32_t w[8];
+            if (q.fast) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-              w[e] = pack_sat4(requant_unclamped(v[4 * e + 0], q), requant_unclamped(v[4 * e + 1], q), requant_unclamped(v[4 * e + 2], q),
-                               requant_unclamped(v[4 * e + 3], q));
+              for (int e = 0; e < 8; ++e)
+                w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
+                                 requant_acc<true>(v[4 * e + 3], q));
+            } else {
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                w[e] = pack_sat4(requant_acc<false>(v[4 * e + 0], q), requant_acc<false>(v[4 * e + 1], q), requant_acc<false>(v[4 * e + 2], q),
+                                 requant_acc<false>(v[4 * e + 3], q));
+            }
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0 + c0;
             if (out_vec == 16) store_bytes32<16>(dst, w, nvalid);
             else if (out_vec == 8) store_bytes32<8>(dst, w, nvalid);

@@ -19,7 +19,8 @@ constexpr int kFirstEpilogueWarp = 4; // warps 0..3: A producer, MMA issuer, B p
 constexpr int kGemmThreads = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr int kMaxStagesA = 12;
 constexpr int kMaxStagesB = 32;
-constexpr uint32_t kSmemBudget = 212 * 1024;              // operand rings; barriers sit in static shared memory
+constexpr uint32_t kSmemBudget = 212 * 1024;              // operand rings + correction table; barriers sit in static shared memory
+constexpr uint32_t kMaxZcBytes = 20 * 1024;               // largest correction table kept in shared memory
 constexpr uint64_t kWaitLimitNs = 2000000000ull;          // bound of every device-side wait
 
 // status-word codes written by kernels when a bounded wait expires
@@ -31,6 +32,10 @@ enum AsyncCode : int32_t {
   kAsyncEpilogueTmemFullWait = 4,
   kAsyncProducerBEmptyWait = 5,
   kAsyncMmaBFullWait = 6,
+};
+
+struct FastDiv {                      // n / d == (umulhi(m, n) + n) >> l for 0 <= n < 2^31
+  uint32_t m, l;
 };
 
 enum OutMode : int { kOutInt8 = 0, kOutF32 = 1, kOutAcc = 2 };
@@ -69,6 +74,7 @@ struct GemmParams {
   int32_t corr_ld, ncolcls;
   const uint8_t* rowcls;              // [TH] or null (single class)
   const uint8_t* colcls;              // [TW] or null
+  int32_t cls_in_smem;                // both tables are non-null and fit the kernel's shared copy (TH, TW <= 512)
   const int32_t* bias;                // [Nout] or null
   const hq_range_state* xq;
   const float* w_scale;
@@ -81,6 +87,9 @@ struct GemmParams {
   uint32_t stage_bytes_a, stage_bytes_b;   // kModeTap: A and B part of one stage; kModeHalo: patch stage, B stage
   int32_t swizzle64;                  // 1: 64-byte swizzle (BK = 64), 0: 128-byte swizzle (BK = 128)
   int32_t producer_lanes;             // kModeTap: lanes of the producer warp that issue copies
+  FastDiv fd_tiles_col, fd_tiles_per_img, fd_tiles_w, fd_tiles_h, fd_P;
+  int32_t zc_in_smem, zc_elems;       // zero-point correction table copied (pre-multiplied) into shared memory
+  uint32_t zc_offset;                 // its byte offset from the ring base
 };
 
 struct DwParams {                     // depthwise (CUDA cores)
