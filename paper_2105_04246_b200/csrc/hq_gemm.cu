@@ -53,9 +53,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           uint32_t hint_ns = 200u) {
   if (mbar_try(bar, parity, hint_ns)) return true;
   const uint64_t t0 = global_timer_ns();
-  uint32_t spins = 0;
+  uint32_t spins = 0, nap = 32;
   for (;;) {
     if (mbar_try(bar, parity, hint_ns)) return true;
+    // back off: a waiting warp that keeps issuing takes issue slots from the epilogue warps of its sub-partition
+    __nanosleep(nap);
+    if (nap < hint_ns) nap += nap;
     if ((++spins & 15u) == 0u) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -123,37 +126,32 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int* v) {
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int* v) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
-        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
-        "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
-        "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr)
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 template <int V>
-__device__ __forceinline__ void store_bytes32(int8_t* p, const uint32_t* w, int nvalid) {
-  // w: 8 words = 32 output bytes; store the first nvalid bytes in pieces of V bytes
+__device__ __forceinline__ void store_bytes16(int8_t* p, const uint32_t* w, int nvalid) {
+  // w: 4 words = 16 output bytes; store the first nvalid bytes in pieces of V bytes
   if constexpr (V == 16) {
-#pragma unroll
-    for (int g = 0; g < 2; ++g)
-      if ((g + 1) * 16 <= nvalid) *reinterpret_cast<uint4*>(p + 16 * g) = make_uint4(w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+    if (nvalid >= 16) *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
   } else if constexpr (V == 8) {
 #pragma unroll
-    for (int g = 0; g < 4; ++g)
+    for (int g = 0; g < 2; ++g)
       if ((g + 1) * 8 <= nvalid) *reinterpret_cast<uint2*>(p + 8 * g) = make_uint2(w[2 * g], w[2 * g + 1]);
   } else if constexpr (V == 4) {
 #pragma unroll
-    for (int g = 0; g < 8; ++g)
+    for (int g = 0; g < 4; ++g)
       if ((g + 1) * 4 <= nvalid) *reinterpret_cast<uint32_t*>(p + 4 * g) = w[g];
   } else {
 #pragma unroll
-    for (int g = 0; g < 32; ++g)
+    for (int g = 0; g < 16; ++g)
       if (g < nvalid) p[g] = (int8_t)((w[g >> 2] >> (8 * (g & 3))) & 0xffu);
   }
 }
@@ -441,7 +439,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   } else if (warp >= kFirstEpilogueWarp) {
     // ------------------------------ epilogue ------------------------------
     const int quarter = warp & 3;                         // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int half = (warp - kFirstEpilogueWarp) >> 2;    // the two warps of a quarter split the column chunks
+    const int slice = (warp - kFirstEpilogueWarp) >> 2;   // the warps of a quarter split the column chunks
     const int ew = warp - kFirstEpilogueWarp;
     const int row = quarter * 32 + lane;
     QParams q;
@@ -459,9 +457,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int rn = row / (p.Ht * p.Wt);
     const int rh = (row / p.Wt) % p.Ht;
     const int rw = row % p.Wt;
-    const int nchunks = (p.BN + 31) / 32;
-    const int c_begin = half == 0 ? 0 : (nchunks + 1) / 2;
-    const int c_end = half == 0 ? (nchunks + 1) / 2 : nchunks;
+    const int nchunks = p.BN / 16;                      // BN is a multiple of 16
+    const int c_begin = (slice * nchunks) / kEpilogueSlices;
+    const int c_end = ((slice + 1) * nchunks) / kEpilogueSlices;
     int local_tile = 0;
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
       int n0, h0, w0, col0;
@@ -482,13 +480,14 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       }
       const int64_t pix = ((int64_t)n * p.out_H + (i * p.os_h + p.oa_h)) * p.out_W + (j * p.os_w + p.oa_w);
       const int32_t* corr_row = nullptr;
+      const int32_t* zrow_s = nullptr;
       if (p.corr != nullptr && q.zx != 0 && row_valid) {
         const int rc = p.cls_in_smem ? cls_s[i] : (p.rowcls ? p.rowcls[i] : 0);
         const int cc = p.cls_in_smem ? cls_s[512 + j] : (p.colcls ? p.colcls[j] : 0);
         const int off = (rc * p.ncolcls + cc) * p.corr_ld + col0;
-        corr_row = (p.zc_in_smem ? zc_s : p.corr) + off;
+        if (p.zc_in_smem) zrow_s = zc_s + off;   // shared copy, already multiplied by zx
+        else corr_row = p.corr + off;
       }
-      const int zmul = p.zc_in_smem ? 1 : q.zx;   // the shared table is already multiplied by zx
       const int buf = local_tile & 1;
       const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
       if (kiters > 0) {
@@ -499,47 +498,49 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         tc_fence_after();
       }
       const uint32_t taddr = tmem_base + buf * p.tmem_buf_stride + ((uint32_t)(quarter * 32) << 16);
-      for (int ch = c_begin; ch < c_end; ++ch) {
-        const int c0 = ch * 32;
-        int v[32];
-        if (kiters > 0) {
-          tmem_ld32(taddr + c0, v);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) v[e] = 0;
-        }
+      constexpr int CW = 16;   // columns per pass: 16 accumulators per thread keep the warp's register count low
+      // one pass over CW columns held in v: correction, statistics, requantization, store
+      auto process = [&](int c0, int (&v)[CW]) {
         int nvalid = p.Nout - (col0 + c0);
-        nvalid = nvalid < 0 ? 0 : (nvalid > 32 ? 32 : nvalid);
-        if (c0 + nvalid > p.BN) nvalid = p.BN - c0;
+        nvalid = nvalid < 0 ? 0 : (nvalid > CW ? CW : nvalid);
         if (!row_valid) nvalid = 0;
-        if (corr_row != nullptr) {
-          const int lim = (p.BN - c0 < 32) ? p.BN - c0 : 32;   // the table is padded to whole column tiles
+        if (zrow_s != nullptr) {   // the tables are padded to whole column tiles
 #pragma unroll
-          for (int e = 0; e < 32; e += 4) {
-            if (e < lim) {
-              const int4 cr = *reinterpret_cast<const int4*>(corr_row + c0 + e);
-              v[e + 0] -= zmul * cr.x;
-              v[e + 1] -= zmul * cr.y;
-              v[e + 2] -= zmul * cr.z;
-              v[e + 3] -= zmul * cr.w;
-            }
+          for (int e = 0; e < CW; e += 4) {
+            const int4 cr = *reinterpret_cast<const int4*>(zrow_s + c0 + e);
+            v[e + 0] -= cr.x;
+            v[e + 1] -= cr.y;
+            v[e + 2] -= cr.z;
+            v[e + 3] -= cr.w;
+          }
+        } else if (corr_row != nullptr) {
+#pragma unroll
+          for (int e = 0; e < CW; e += 4) {
+            const int4 cr = *reinterpret_cast<const int4*>(corr_row + c0 + e);
+            v[e + 0] -= q.zx * cr.x;
+            v[e + 1] -= q.zx * cr.y;
+            v[e + 2] -= q.zx * cr.z;
+            v[e + 3] -= q.zx * cr.w;
           }
         }
         if (p.bias != nullptr) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
+          for (int e = 0; e < CW; ++e)
             if (e < nvalid) v[e] += p.bias[col0 + c0 + e];
         }
-        if (nvalid == 32) {
+        if (nvalid == CW) {   // two independent chains, then merged: short dependency depth
+          int lo[2], hi[2];
 #pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            mn = __vimin3_s32(mn, v[e], v[e + 1]);
-            mx = __vimax3_s32(mx, v[e], v[e + 1]);
+          for (int g = 0; g < 2; ++g) {
+            const int* x = v + 8 * g;
+            lo[g] = min(__vimin3_s32(__vimin3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimin3_s32(x[5], x[6], x[7]));
+            hi[g] = max(__vimax3_s32(__vimax3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimax3_s32(x[5], x[6], x[7]));
           }
+          mn = __vimin3_s32(mn, lo[0], lo[1]);
+          mx = __vimax3_s32(mx, hi[0], hi[1]);
         } else {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
+          for (int e = 0; e < CW; ++e) {
             if (e < nvalid) {
               mn = min(mn, v[e]);
               mx = max(mx, v[e]);
@@ -548,28 +549,28 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         }
         if (nvalid > 0) {
           if constexpr (kOut == kOutInt8) {
-            uint32_t w[8];
+            uint32_t w[CW / 4];
             if (q.fast) {
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
+              for (int e = 0; e < CW / 4; ++e)
                 w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
                                  requant_acc<true>(v[4 * e + 3], q));
             } else {
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
+              for (int e = 0; e < CW / 4; ++e)
                 w[e] = pack_sat4(requant_acc<false>(v[4 * e + 0], q), requant_acc<false>(v[4 * e + 1], q), requant_acc<false>(v[4 * e + 2], q),
                                  requant_acc<false>(v[4 * e + 3], q));
             }
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16) store_bytes32<16>(dst, w, nvalid);
-            else if (out_vec == 8) store_bytes32<8>(dst, w, nvalid);
-            else if (out_vec == 4) store_bytes32<4>(dst, w, nvalid);
-            else store_bytes32<1>(dst, w, nvalid);
+            if (out_vec == 16) store_bytes16<16>(dst, w, nvalid);
+            else if (out_vec == 8) store_bytes16<8>(dst, w, nvalid);
+            else if (out_vec == 4) store_bytes16<4>(dst, w, nvalid);
+            else store_bytes16<1>(dst, w, nvalid);
           } else {
             uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16 && nvalid == 32) {
+            if (out_vec == 16 && nvalid == CW) {
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
+              for (int e = 0; e < CW / 4; ++e) {
                 uint32_t w[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k)
@@ -578,11 +579,22 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
               }
             } else {
 #pragma unroll
-              for (int e = 0; e < 32; ++e)
+              for (int e = 0; e < CW; ++e)
                 if (e < nvalid) dst[e] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[e]), q.s_acc)) : (uint32_t)v[e];
             }
           }
         }
+      };
+      for (int ch = c_begin; ch < c_end; ++ch) {
+        int v[CW];
+        if (kiters > 0) {
+          tmem_ld16(taddr + ch * CW, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int e = 0; e < CW; ++e) v[e] = 0;
+        }
+        process(ch * CW, v);
       }
       if (kiters > 0) {
         tc_fence_before();

@@ -14,7 +14,8 @@ namespace hq {
 
 constexpr int kMaxTaps = 49;          // 7x7
 constexpr int kTileM = 128;           // rows of one accumulator tile = TMEM lanes
-constexpr int kEpilogueWarps = 8;     // two per TMEM lane quarter; they split the columns
+constexpr int kEpilogueSlices = 4;    // epilogue warps per TMEM lane quarter; they split the columns
+constexpr int kEpilogueWarps = 4 * kEpilogueSlices;
 constexpr int kFirstEpilogueWarp = 4; // warps 0..3: A producer, MMA issuer, B producer, spare
 constexpr int kGemmThreads = 32 * (kFirstEpilogueWarp + kEpilogueWarps);
 constexpr int kMaxStagesA = 12;

@@ -20,10 +20,13 @@ __device__ __forceinline__ void qparams_finish(QParams& q) {
   q.fast = (isfinite(q.inv_scale) && q.inv_scale != 0.0f && isfinite(q.s_acc)) ? 1 : 0;
 }
 
-// rint(u) + zp without the (slow) float-to-int conversion pipe: clamp to +-2^22, add 1.5 * 2^23 (the sum is rounded
-// to an integer, ties to even) and read the integer out of the mantissa.  Values that were clamped saturate anyway.
+// rint(u) + zp without the (slow) float-to-int conversion pipe: add 1.5 * 2^23 (for |u| <= 2^22 the sum is rounded to
+// an integer, ties to even) and read the integer out of the mantissa.  Only a lower clamp is needed: it keeps the sum
+// positive, and bit patterns of positive floats are ordered like their values, so any u above the exact range yields
+// an integer above 127 (up to +inf, no wrap) and any u below it an integer below -128 -- the saturating pack that
+// follows gives the same code as the reference form.
 __device__ __forceinline__ int round_add_zp_fast(float u, const QParams& q) {
-  u = fminf(fmaxf(u, -4194304.0f), 4194304.0f);
+  u = fmaxf(u, -4194304.0f);
   const float rf = __fadd_rn(u, 12582912.0f);
   return __float_as_int(rf) - q.magic_sub;
 }
