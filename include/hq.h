@@ -144,7 +144,9 @@ hq_status hq_weights_release(hq_ctx* ctx, hq_prepared_weights* pw);
  *   y = float(acc) * s_acc;  q = clamp(rint(y * inv_scale) + zero_point, -128, 127)
  * (round half to even, one binary32 rounding per operation).  Merges min/max of acc into
  * yq->acc_min/acc_max (Sec. 4 step 2) and writes yq->acc_scale.  bias may be NULL.
- * Requires K % 16 == 0.  Backward data of a linear layer is this call with W transposed. */
+ * K that is not a multiple of 16 is served through zero-padded copies of X and W in context-owned scratch
+ * (grown with cudaMalloc when a larger layer is first seen).  Backward data of a linear layer is this call
+ * with W transposed. */
 hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K,
                         const int8_t* X, const hq_range_state* xq,
                         const int8_t* W, const float* w_scale, const int32_t* bias,
@@ -152,7 +154,9 @@ hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t
 
 /* Forward convolution as an implicit GEMM (Sec. 3.1), same epilogue as hq_linear_fwd.
  * Padding is zero in the real domain.  pw must come from hq_weights_prepare(.., HQ_DIR_FWD, ..)
- * with the same descriptor.  groups == C selects the depthwise kernel. */
+ * with the same descriptor.  groups == C selects the depthwise kernel.  Spatial filters over a channel
+ * count that is not a multiple of 16 (an RGB stem) run a gather pre-pass into a library-owned
+ * [pixels][R*S*C] matrix that the handle allocates at preparation time. */
 hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                       const int8_t* X, const hq_range_state* xq,
                       const hq_prepared_weights* pw, const float* w_scale,

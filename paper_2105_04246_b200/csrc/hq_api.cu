@@ -398,6 +398,12 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     CUtensorMap ta;
     if (sub.p.ntaps == 0) {
       ta = CUtensorMap{};
+    } else if (sub.patch_matrix != nullptr) {
+      // channel counts that no TMA box can address (C = 3): gather the filter windows into rows first
+      HQ_CUDA(ctx, launch_patch_matrix(in, sub.patch_matrix, inq, desc->N, desc->H, desc->W, desc->C, Ho, Wo, desc->R, desc->S, desc->stride_h,
+                                       desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, s));
+      ctx->launches += 1;
+      st = encode_a(ctx, sub, sub.patch_matrix, sub.patch_K, desc->N * Ho * Wo, 1, 1, &ta);
     } else if (sub.a_flat) {
       const int64_t rows = (int64_t)desc->N * aH * aW / sub.gfold;
       st = encode_a(ctx, sub, in, aC * sub.gfold, (int)rows, 1, 1, &ta);
@@ -415,9 +421,28 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
                      const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode) {
   if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
   if (!X || !xq || !W || !w_scale || !out || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
-  if (K % 16 != 0) return fail(ctx, HQ_ERR_ALIGNMENT, "K (%d) must be a multiple of 16", K);
   if (!aligned16(X) || !aligned16(W) || !aligned16(out) || !aligned16(xq) || !aligned16(yq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
+  if (K % 16 != 0) {
+    // rows whose length no TMA box can address: zero-padded copies of both operands in context-owned scratch
+    const int Kp = round_up(K, 16);
+    const size_t need = ((size_t)M + (size_t)N) * Kp;
+    if (need > ctx->pad_bytes) {
+      if (ctx->d_pad) HQ_CUDA(ctx, cudaFree(ctx->d_pad));
+      ctx->d_pad = nullptr;
+      ctx->pad_bytes = 0;
+      HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_pad, need));
+      ctx->pad_bytes = need;
+    }
+    int8_t* Xp = ctx->d_pad;
+    int8_t* Wp = ctx->d_pad + (size_t)M * Kp;
+    HQ_CUDA(ctx, launch_pad_rows(X, Xp, M, K, Kp, s));
+    HQ_CUDA(ctx, launch_pad_rows(W, Wp, N, K, Kp, s));
+    ctx->launches += 2;
+    X = Xp;
+    W = Wp;
+    K = Kp;
+  }
   SubSpec sp{};
   sp.n_img = 1; sp.TH = 1; sp.TW = M; sp.in_mul_h = 1; sp.in_mul_w = 1;
   sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = M; sp.Cin = K; sp.Nout = N;
@@ -524,6 +549,7 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_scratch);
+  if (ctx->d_pad) cudaFree(ctx->d_pad);
   delete ctx;
   return HQ_OK;
 }
@@ -614,7 +640,26 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
       sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = (int64_t)g * d.K; sp.flat = true;
       tr = {0}; ts = {0};
     } else {
-      if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "C = %d: spatial filters need C %% 16 == 0", d.C));
+      if (d.C % 16 != 0) {
+        // rows of [R*S*C] input bytes (padded to a multiple of 16, padding taps holding the input zero point) are
+        // gathered by a pre-pass into a library-owned matrix; the layer is then a flat GEMM over it
+        const int64_t rows = (int64_t)d.N * Ho * Wo;
+        const int rsc = d.R * d.S * d.C;
+        const int Kp = round_up(rsc, 16);
+        if (rows > INT32_MAX) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many pixels"));
+        sp.n_img = 1; sp.TH = 1; sp.TW = (int)rows; sp.in_mul_h = sp.in_mul_w = 1; sp.dh = {0}; sp.dw = {0};
+        sp.a_H = 1; sp.a_W = (int)rows; sp.Cin = Kp; sp.Nout = d.K;
+        sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.K; sp.flat = true;
+        hq_conv_desc flatd = d;
+        flatd.R = flatd.S = 1;
+        flatd.C = rsc;   // the filter [K][R][S][C] read as [K][R*S*C]
+        if ((st = build_sub(ctx, pw, s, sp, flatd, W, {0}, {0}, false, 1)) != HQ_OK) return bail(st);
+        hq_sub_problem& sub = pw->subs.back();
+        sub.patch_K = Kp;
+        if ((st = dev_alloc(ctx, pw, (void**)&sub.patch_matrix, (size_t)rows * Kp)) != HQ_OK) return bail(st);
+        *out = pw;
+        return HQ_OK;
+      }
       sp.n_img = d.N; sp.TH = Ho; sp.TW = Wo; sp.in_mul_h = d.stride_h; sp.in_mul_w = d.stride_w;
       for (int r = 0; r < d.R; ++r) { sp.dh.push_back(r - d.pad_h); tr.push_back(r); }
       for (int q = 0; q < d.S; ++q) { sp.dw.push_back(q - d.pad_w); ts.push_back(q); }
@@ -757,6 +802,9 @@ extern "C" __attribute__((visibility("default"))) hq_status hq_dynamic_quant_sta
     if (st != HQ_OK) return st;
   } else if (op->M <= 0 || op->N <= 0 || op->K <= 0) {
     return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
+  } else if (op->K % 16 != 0) {
+    return fail(ctx, HQ_ERR_UNSUPPORTED, "K = %d: rows that are not a multiple of 16 bytes need padded copies, which this call may not allocate",
+                op->K);
   }
   const int64_t elems = op_out_elems(op);
   if (elems > (int64_t)HQ_STATIC_WORKSPACE_ELEMS)

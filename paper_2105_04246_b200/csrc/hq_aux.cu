@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+
 #include "hq_internal.h"
 #include "hq_quant.cuh"
 
@@ -161,6 +163,47 @@ __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict_
   }
 }
 
+// ---- operand repacking for shapes no TMA box can address ------------------------------------------
+// A[m][j], j = (r*S + s)*C + c: the filter window of output pixel m; taps on padding hold the input zero point
+// (real zero), columns beyond R*S*C hold 0 (their weights are 0).  One thread builds 16 consecutive bytes.
+__global__ void patch_matrix_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ A, const hq_range_state* xq, int N, int H, int W, int C,
+                                    int Ho, int Wo, int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int Kp) {
+  const int groups = Kp / 16;
+  const int64_t total = (int64_t)N * Ho * Wo * groups;
+  const int zx = xq->zero_point;
+  const int rsc = R * S * C, sc = S * C;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int g = (int)(idx % groups);
+    int64_t m = idx / groups;
+    const int wo = (int)(m % Wo);
+    const int ho = (int)((m / Wo) % Ho);
+    const int n = (int)(m / ((int64_t)Wo * Ho));
+    uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int b = 0; b < 16; ++b) {
+      const int j = g * 16 + b;
+      int val = 0;
+      if (j < rsc) {
+        const int r = j / sc, rem = j - r * sc;
+        const int q = rem / C, c = rem - q * C;
+        const int hi = ho * stride_h - pad_h + r, wi = wo * stride_w - pad_w + q;
+        val = (hi >= 0 && hi < H && wi >= 0 && wi < W) ? (int)x[(((int64_t)n * H + hi) * W + wi) * C + c] : zx;
+      }
+      w[b >> 2] |= ((uint32_t)val & 0xffu) << (8 * (b & 3));
+    }
+    *reinterpret_cast<uint4*>(A + m * Kp + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+__global__ void pad_rows_kernel(const int8_t* __restrict__ src, int8_t* __restrict__ dst, int rows, int K, int Kp) {
+  const int64_t total = (int64_t)rows * Kp;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int j = (int)(idx % Kp);
+    const int64_t r = idx / Kp;
+    dst[idx] = j < K ? src[r * K + j] : (int8_t)0;
+  }
+}
+
 // ---- depthwise convolution on CUDA cores --------------------------------------------------------
 // One thread: one output pixel x 16 consecutive channels.  Same epilogue as the tensor-core kernel.
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xffu); }
@@ -310,6 +353,23 @@ cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, in
   int total = nrowcls * ncolcls * C;
   if (C * R * S > total) total = C * R * S;
   dw_prep_kernel<<<(total + 127) / 128, 128, 0, s>>>(W, Wt, corr, C, R, S, m, nrowcls, ncolcls);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
+                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, cudaStream_t s) {
+  const int64_t total = (int64_t)N * Ho * Wo * (Kp / 16);
+  int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+  if (blocks < 1) blocks = 1;
+  patch_matrix_kernel<<<blocks, 256, 0, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s) {
+  const int64_t total = (int64_t)rows * Kp;
+  int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
+  if (blocks < 1) blocks = 1;
+  pad_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, rows, K, Kp);
   return cudaGetLastError();
 }
 

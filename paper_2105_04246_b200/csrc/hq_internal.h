@@ -123,6 +123,9 @@ cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int nta
                                 const int8_t* tap_r, const int8_t* tap_s, int transposed, int blockdiag_g, cudaStream_t s);
 cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps, const uint32_t* rowmasks,
                         int nrowcls, const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s);
+cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
+                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, cudaStream_t s);
+cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
                            const uint32_t* colmasks, int ncolcls, cudaStream_t s);
 
@@ -134,6 +137,8 @@ struct hq_ctx {
   int32_t* d_status = nullptr;
   int32_t* d_scratch = nullptr;       // column sums of linear weights
   size_t scratch_elems = 0;
+  int8_t* d_pad = nullptr;            // zero-padded operand copies for linear layers whose K is not a multiple of 16
+  size_t pad_bytes = 0;
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
@@ -151,6 +156,8 @@ struct hq_sub_problem {               // one kernel launch of a prepared convolu
   int a_stride_h = 1, a_stride_w = 1; // traversal strides of the A tensor map
   int a_flat = 0;                     // 1: A is viewed as [pixels][C] (1x1 stride-1 layers and linear)
   int gfold = 1;                      // pixels folded into one GEMM row (channel counts that are not multiples of 16)
+  int8_t* patch_matrix = nullptr;     // [pixels][patch_K]: filter windows gathered by a pre-pass (C not a multiple of 16)
+  int patch_K = 0;
 };
 
 struct hq_prepared_weights {

@@ -77,6 +77,8 @@ def test_cfg1_linear_ten_iterations_with_scale_drift(ctx):
     (1, 16, 16, -128, False),       # smallest
     (515, 272, 80, 127, True),      # two column tiles of 144 (second ragged), K = 64 + 16
     (384, 8, 64, 3, False),         # N not a multiple of 16
+    (128, 512, 1000, -3, False),    # K not a multiple of 16 (backward of a 512 -> 1000 classifier): padded copies
+    (70, 40, 40, 9, True),
 ])
 def test_linear_ragged(ctx, M, N, K, zx, use_bias):
     r = synth.rng(102, M, N, K)
@@ -100,6 +102,8 @@ FWD_CASES = {
     "3x3_c512_k512_7x7": dict(N=4, H=7, W=7, Cin=512, K=512, R=3, S=3, stride=1, pad=1),
     "7x7_c16_s1": dict(N=1, H=20, W=23, Cin=16, K=32, R=7, S=7, stride=1, pad=3),
     "5x5_c16": dict(N=1, H=11, W=11, Cin=16, K=48, R=5, S=5, stride=1, pad=2),
+    "7x7_s2_c3_stem": dict(N=2, H=30, W=26, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
+    "3x3_c5": dict(N=2, H=9, W=9, Cin=5, K=24, R=3, S=3, stride=1, pad=1),
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
     "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
@@ -206,9 +210,6 @@ def test_rejected_calls_launch_nothing(ctx):
     ws = torch.ones(1, dtype=torch.float32, device=dev)
     n0 = ctx.launch_count()
     with pytest.raises(hq.HqError) as e:
-        ctx.linear_fwd(None, 64, 64, 40, x, st, x, ws, None, x, st[48:])          # K not a multiple of 16
-    assert e.value.status == 3
-    with pytest.raises(hq.HqError) as e:
         ctx.linear_fwd(None, 64, 64, 64, x[1:], st, x, ws, None, x, st[48:])      # misaligned X
     assert e.value.status == 3
     with pytest.raises(hq.HqError) as e:
@@ -218,7 +219,7 @@ def test_rejected_calls_launch_nothing(ctx):
         ctx.linear_fwd(None, 64, 64, 64, x, None, x, ws, None, x, st[48:])
     assert e.value.status == 1
     with pytest.raises(hq.HqError) as e:
-        ctx.weights_prepare(None, hq.conv_desc(1, 8, 8, 3, 16, 3, 3, 1, 1), hq.DIR_FWD, x)   # C = 3 with a spatial filter
+        ctx.weights_prepare(None, hq.conv_desc(1, 8, 8, 16, 3, 3, 3, 1, 1), hq.DIR_BWD_DATA, x)   # backward data with K = 3
     assert e.value.status == 2
     with pytest.raises(hq.HqError) as e:
         ctx.range_update(None, st, 2, 1.5)
