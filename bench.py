@@ -8,7 +8,7 @@ int8 tera-operations per second (2 x MACs of the dense definition) of the in-hin
 same run also times the dynamic-quantization comparison path and reports algorithmic HBM bytes
 per layer for both (Eq. 4 / Eq. 5 of arxiv 2105.04246).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4|cfg5]
     python bench.py --impl reference ...      # the CPU oracle on the host cores
 
 Prints ONE JSON line on rank 0.
@@ -60,6 +60,14 @@ def workload_layers(name: str, batch_div: int = 1):
         return [("conv_bwd", b(wl.CFG3_BWD), "grad")], False
     if name == "cfg4":
         return [("conv_fwd", b(wl.CFG4_EXPAND), "signed"), ("conv_fwd", b(wl.CFG4_DW), None), ("conv_fwd", b(wl.CFG4_PROJECT), None)], True
+    if name == "cfg5":
+        # every convolution of ResNet-18 at 224x224 and the classifier, forward and backward-data (none for the stem);
+        # each call has its own synthetic input: what sits between the layers (BN, ReLU, pooling, adds) is not on the path
+        convs, fc = wl.resnet18_layers(max(1, 128 // batch_div))
+        fwd = [("conv_fwd", c, "image" if c.C == 3 else "relu") for c in convs] + [("linear", fc, "relu")]
+        fc_bwd = wl.LinearShape("fc.bwd", fc.M, fc.K, fc.N)
+        bwd = [("conv_bwd", wl.replace(c, name=c.name + ".bwd"), "grad") for c in convs[1:]] + [("linear", fc_bwd, "grad")]
+        return fwd + bwd, False
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -72,6 +80,8 @@ def make_input(recipe: str, g, shape):
         return synth.tiled(synth.signed_activations, g, shape)
     if recipe == "grad":
         return synth.tiled(synth.gradients, g, shape)
+    if recipe == "image":
+        return synth.tiled(synth.image_like, g, shape)
     raise ValueError(recipe)
 
 
@@ -294,7 +304,7 @@ def run_gpu(args):
     ctx = hq.Context(local)
     peaks, peak_kind = load_peaks()
     name = args.workload
-    pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2}[name]
+    pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg5": 2}[name]
     wk = GpuWorkload(name, ctx, dev, pool, seed_key=rank)
     K, W = args.steps, max(3, args.warmup)
     stream = torch.cuda.current_stream(dev)
@@ -479,7 +489,7 @@ def main():
     ap.add_argument("--steps", type=int, default=600)
     ap.add_argument("--warmup", type=int, default=24)
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profile", action="store_true",
                     help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
