@@ -127,7 +127,9 @@ __global__ void prep_weights_kernel(const int8_t* __restrict__ W, int8_t* __rest
 // what the zero-filled padding taps did NOT contribute.
 __global__ void corr_kernel(const int8_t* __restrict__ Wmat, int32_t* __restrict__ corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps,
                             ClassMasks m, int nrowcls, int ncolcls, int corr_ld) {
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  // one warp per (class, output channel); Cpad is a multiple of 16, rows are 16-byte aligned
+  const int idx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
   if (idx >= nrowcls * ncolcls * Nout) return;
   const int n = idx % Nout;
   const int cls = idx / Nout;
@@ -137,11 +139,18 @@ __global__ void corr_kernel(const int8_t* __restrict__ Wmat, int32_t* __restrict
     if (!((m.row[rc] >> ri) & 1u)) continue;
     for (int si = 0; si < ncoltaps; ++si) {
       if (!((m.col[cc] >> si) & 1u)) continue;
-      const int8_t* w = Wmat + ((int64_t)n * ntaps + (ri * ncoltaps + si)) * Cpad;
-      for (int c = 0; c < Cpad; ++c) sum += w[c];
+      const uint4* w = reinterpret_cast<const uint4*>(Wmat + ((int64_t)n * ntaps + (ri * ncoltaps + si)) * Cpad);
+      for (int c = lane; c < Cpad / 16; c += 32) {
+        const uint4 q = w[c];
+        sum = __dp4a((int)q.x, 0x01010101, sum);
+        sum = __dp4a((int)q.y, 0x01010101, sum);
+        sum = __dp4a((int)q.z, 0x01010101, sum);
+        sum = __dp4a((int)q.w, 0x01010101, sum);
+      }
     }
   }
-  corr[(int64_t)cls * corr_ld + n] = sum;
+  sum = __reduce_add_sync(0xffffffffu, sum);
+  if (lane == 0) corr[(int64_t)cls * corr_ld + n] = sum;
 }
 
 // depthwise: weights to tap-major [R*S][C]; corr[cls][c] = sum of valid taps
@@ -165,33 +174,48 @@ __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict_
 
 // ---- operand repacking for shapes no TMA box can address ------------------------------------------
 // A[m][j], j = (r*S + s)*C + c: the filter window of output pixel m; taps on padding hold the input zero point
-// (real zero), columns beyond R*S*C hold 0 (their weights are 0).  One thread builds 16 consecutive bytes.
-__global__ void patch_matrix_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ A, const hq_range_state* xq, int N, int H, int W, int C,
-                                    int Ho, int Wo, int R, int S, int stride_h, int stride_w, int pad_h, int pad_w, int Kp) {
-  const int groups = Kp / 16;
-  const int64_t total = (int64_t)N * Ho * Wo * groups;
+// (real zero), columns beyond R*S*C hold 0 (their weights are 0).  For a fixed filter row r the S*C input bytes are
+// contiguous in NHWC, so thread (pixel, r) copies that run into the pixel's row in shared memory; the block then
+// writes its rows out with 16-byte stores.
+constexpr int kPatchPixels = 32;   // output pixels per block iteration
+__global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ A, const hq_range_state* xq, int N,
+                                                           int H, int W, int C, int Ho, int Wo, int R, int S, int stride_h, int stride_w,
+                                                           int pad_h, int pad_w, int Kp) {
+  extern __shared__ __align__(16) int8_t rows_s[];   // [kPatchPixels][Kp]
   const int zx = xq->zero_point;
-  const int rsc = R * S * C, sc = S * C;
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-    const int g = (int)(idx % groups);
-    int64_t m = idx / groups;
-    const int wo = (int)(m % Wo);
-    const int ho = (int)((m / Wo) % Ho);
-    const int n = (int)(m / ((int64_t)Wo * Ho));
-    uint32_t w[4] = {0, 0, 0, 0};
-#pragma unroll
-    for (int b = 0; b < 16; ++b) {
-      const int j = g * 16 + b;
-      int val = 0;
-      if (j < rsc) {
-        const int r = j / sc, rem = j - r * sc;
-        const int q = rem / C, c = rem - q * C;
-        const int hi = ho * stride_h - pad_h + r, wi = wo * stride_w - pad_w + q;
-        val = (hi >= 0 && hi < H && wi >= 0 && wi < W) ? (int)x[(((int64_t)n * H + hi) * W + wi) * C + c] : zx;
+  const int sc = S * C, rsc = R * sc;
+  const int64_t M = (int64_t)N * Ho * Wo;
+  for (int64_t m0 = (int64_t)blockIdx.x * kPatchPixels; m0 < M; m0 += (int64_t)gridDim.x * kPatchPixels) {
+    // zero the padding columns once per iteration (cheap: Kp - rsc < 16 bytes per pixel)
+    for (int t = threadIdx.x; t < kPatchPixels * (Kp - rsc); t += blockDim.x)
+      rows_s[(t / (Kp - rsc)) * Kp + rsc + t % (Kp - rsc)] = 0;
+    for (int t = threadIdx.x; t < kPatchPixels * R; t += blockDim.x) {
+      const int pl = t / R, r = t - pl * R;
+      const int64_t m = m0 + pl;
+      if (m >= M) continue;
+      const int wo = (int)(m % Wo);
+      const int ho = (int)((m / Wo) % Ho);
+      const int n = (int)(m / ((int64_t)Wo * Ho));
+      const int hi = ho * stride_h - pad_h + r;
+      const int wi0 = wo * stride_w - pad_w;
+      int8_t* dst = rows_s + pl * Kp + r * sc;
+      if (hi < 0 || hi >= H) {
+        for (int b = 0; b < sc; ++b) dst[b] = (int8_t)zx;
+      } else {
+        const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
+        for (int q = 0; q < S; ++q) {
+          const bool in = (wi0 + q >= 0) && (wi0 + q < W);
+          for (int c = 0; c < C; ++c) dst[q * C + c] = in ? src[q * C + c] : (int8_t)zx;
+        }
       }
-      w[b >> 2] |= ((uint32_t)val & 0xffu) << (8 * (b & 3));
     }
-    *reinterpret_cast<uint4*>(A + m * Kp + g * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+    __syncthreads();
+    const int chunks = kPatchPixels * Kp / 16;
+    for (int t = threadIdx.x; t < chunks; t += blockDim.x) {
+      const int64_t byte = (int64_t)t * 16;
+      if (m0 * Kp + byte < M * Kp) *reinterpret_cast<uint4*>(A + m0 * Kp + byte) = *reinterpret_cast<const uint4*>(rows_s + byte);
+    }
+    __syncthreads();
   }
 }
 
@@ -341,7 +365,7 @@ cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, 
   for (int i = 0; i < nrowcls; ++i) m.row[i] = rowmasks[i];
   for (int i = 0; i < ncolcls; ++i) m.col[i] = colmasks[i];
   const int total = nrowcls * ncolcls * Nout;
-  corr_kernel<<<(total + 127) / 128, 128, 0, s>>>(Wmat, corr, Nout, ntaps, Cpad, nrowtaps, ncoltaps, m, nrowcls, ncolcls, corr_ld);
+  corr_kernel<<<(total + 7) / 8, 256, 0, s>>>(Wmat, corr, Nout, ntaps, Cpad, nrowtaps, ncoltaps, m, nrowcls, ncolcls, corr_ld);
   return cudaGetLastError();
 }
 
@@ -358,10 +382,10 @@ cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, in
 
 cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
                                 int stride_h, int stride_w, int pad_h, int pad_w, int Kp, cudaStream_t s) {
-  const int64_t total = (int64_t)N * Ho * Wo * (Kp / 16);
-  int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+  const int64_t groups = ((int64_t)N * Ho * Wo + kPatchPixels - 1) / kPatchPixels;
+  int blocks = (int)std::min<int64_t>(groups, 148 * 8);
   if (blocks < 1) blocks = 1;
-  patch_matrix_kernel<<<blocks, 256, 0, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp);
+  patch_matrix_kernel<<<blocks, 256, (size_t)kPatchPixels * Kp, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp);
   return cudaGetLastError();
 }
 
