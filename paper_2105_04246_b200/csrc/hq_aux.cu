@@ -325,6 +325,126 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
   }
 }
 
+
+// 3x3, stride 1: thread = one 32-bit word of channels (4 channels) x 8 consecutive output pixels of a row.
+// The 36 weights of its channels stay in registers, each already shifted into its byte lane so that one dp4a
+// against the input word multiplies exactly one channel (the other three lanes meet zeros).  Input words are
+// read once per row of the window and reused by the three taps and the neighbouring pixels; a warp's lanes hold
+// consecutive channel words, so loads and stores are contiguous.  Out-of-image taps read as 0 and are settled by
+// the same border-class correction as in the tensor-core kernel.
+constexpr int kDwPix = 8;
+template <int kOut>
+__global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int slots, int groups_w) {
+  __shared__ int red_min[8], red_max[8];
+  QParams q;
+  q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
+  q.zx = p.xq->zero_point;
+  q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
+  q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  qparams_finish(q);
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
+  const int CW = p.C / 4;
+  const int cw = threadIdx.x % CW, slot = threadIdx.x / CW;
+  int mn = INT32_MAX, mx = INT32_MIN;
+  if (slot < slots) {
+    int wsel[9][4];   // weight of (tap, channel k) in byte lane k
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+      const uint32_t w4 = *reinterpret_cast<const uint32_t*>(p.w + (int64_t)t * p.C + cw * 4);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) wsel[t][k] = (int)(w4 & (0xffu << (8 * k)));
+    }
+    const int64_t items = (int64_t)p.N * p.Ho * groups_w;
+    const int cstride = p.C;
+    for (int64_t item = (int64_t)blockIdx.x * slots + slot; item < items; item += (int64_t)gridDim.x * slots) {
+      const int pg = (int)(item % groups_w);
+      const int ho = (int)((item / groups_w) % p.Ho);
+      const int n = (int)(item / ((int64_t)groups_w * p.Ho));
+      const int wo0 = pg * kDwPix;
+      int acc[kDwPix][4];
+#pragma unroll
+      for (int j = 0; j < kDwPix; ++j)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc[j][k] = 0;
+#pragma unroll
+      for (int r = 0; r < 3; ++r) {
+        const int hi = ho - p.pad_h + r;
+        if (hi < 0 || hi >= p.H) continue;
+        const int wi0 = wo0 - p.pad_w;
+        const int8_t* pj = p.x + (((int64_t)n * p.H + hi) * p.W + wi0) * p.C + cw * 4;   // not dereferenced where masked
+        int xw[kDwPix + 2];
+        if (wi0 >= 0 && wi0 + kDwPix + 2 <= p.W) {   // whole window inside the row: no per-pixel tests
+#pragma unroll
+          for (int j = 0; j < kDwPix + 2; ++j) {
+            xw[j] = *reinterpret_cast<const int*>(pj);
+            pj += cstride;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < kDwPix + 2; ++j) {
+            const int wi = wi0 + j;
+            xw[j] = (wi >= 0 && wi < p.W) ? *reinterpret_cast<const int*>(pj) : 0;
+            pj += cstride;
+          }
+        }
+#pragma unroll
+        for (int s = 0; s < 3; ++s)
+#pragma unroll
+          for (int j = 0; j < kDwPix; ++j)
+#pragma unroll
+            for (int k = 0; k < 4; ++k) acc[j][k] = __dp4a(xw[j + s], wsel[r * 3 + s][k], acc[j][k]);
+      }
+      const int rcls = q.zx != 0 ? p.rowcls[ho] * p.ncolcls : 0;
+#pragma unroll
+      for (int j = 0; j < kDwPix; ++j) {
+        const int wo = wo0 + j;
+        if (wo >= p.Wo) break;
+        if (q.zx != 0) {
+          const int4 cr = *reinterpret_cast<const int4*>(p.corr + (int64_t)(rcls + p.colcls[wo]) * p.C + cw * 4);
+          acc[j][0] -= q.zx * cr.x;
+          acc[j][1] -= q.zx * cr.y;
+          acc[j][2] -= q.zx * cr.z;
+          acc[j][3] -= q.zx * cr.w;
+        }
+        mn = min(__vimin3_s32(mn, acc[j][0], acc[j][1]), min(acc[j][2], acc[j][3]));
+        mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
+        const int64_t o = (((int64_t)n * p.Ho + ho) * p.Wo + wo) * p.C + cw * 4;
+        if constexpr (kOut == kOutInt8) {
+          const uint32_t w = q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q), requant_acc<true>(acc[j][2], q),
+                                                requant_acc<true>(acc[j][3], q))
+                                    : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
+                                                requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+          *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
+        } else {
+          uint32_t w[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(acc[j][k]), q.s_acc)) : (uint32_t)acc[j][k];
+          *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+    }
+  }
+  mn = __reduce_min_sync(0xffffffffu, mn);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    red_min[warp] = mn;
+    red_max[warp] = mx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int e = 1; e < (int)((blockDim.x + 31) >> 5); ++e) {
+      mn = min(mn, red_min[e]);
+      mx = max(mx, red_max[e]);
+    }
+    if (mn <= mx) {
+      atomicMin(&p.yq->acc_min, mn);
+      atomicMax(&p.yq->acc_max, mx);
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s) {
@@ -398,6 +518,21 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
 }
 
 cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s) {
+  const int CW = p.C / 4;
+  if (p.R == 3 && p.S == 3 && p.stride_h == 1 && p.stride_w == 1 && CW <= 256) {
+    const int slots = 256 / CW;                           // pixel groups per block
+    const int threads = ((slots * CW + 31) / 32) * 32;
+    const int groups_w = (p.Wo + kDwPix - 1) / kDwPix;
+    const int64_t items = (int64_t)p.N * p.Ho * groups_w;
+    int blocks = (int)std::min<int64_t>((items + slots - 1) / slots, (int64_t)num_sms * 8);
+    if (blocks < 1) blocks = 1;
+    switch (out_mode) {
+      case kOutInt8: depthwise3x3_kernel<kOutInt8><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
+      case kOutF32: depthwise3x3_kernel<kOutF32><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
+      default: depthwise3x3_kernel<kOutAcc><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
+    }
+    return cudaGetLastError();
+  }
   const int64_t total = (int64_t)p.N * p.Ho * p.Wo * (p.C / 16);
   int64_t want = (total + 255) / 256;
   int blocks = (int)(want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want);
