@@ -159,14 +159,13 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   p.corr_ld = p.tiles_col * p.BN;
   // instruction descriptor: D = s32, A = B = signed 8-bit, both K-major, N = BN, M = 128
   p.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-  if (p.BN > 128) {
-    p.tmem_buf_stride = 256;
-    p.tmem_cols = 512;
-  } else {
+  {
     uint32_t s = 32;
     while ((int)s < p.BN) s <<= 1;
     p.tmem_buf_stride = s;
-    p.tmem_cols = 2 * s;
+    p.tmem_bufs = (int)std::min<uint32_t>(8, 512 / s);
+    p.tmem_bufs_log2 = p.tmem_bufs == 8 ? 3 : (p.tmem_bufs == 4 ? 2 : 1);
+    p.tmem_cols = (uint32_t)p.tmem_bufs * s;
   }
   // border classes first: the size of the correction table decides how much shared memory the rings get
   if (sp.flat) {
@@ -251,6 +250,19 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   sub.a_stride_h = sp.in_mul_h;
   sub.a_stride_w = sp.in_mul_w;
   p.status = ctx->d_status;
+  {
+    // Two MMA issuer warps alternate tiles.  An issuer that waits for ring iteration `it` must find iteration
+    // `it - stages` already delivered, or the phase parity of an older delivery would satisfy its wait; that holds
+    // when the issuer's own previous tile covers it: two tiles' worth of stages must fit in the ring.
+    const int kiters = p.ntaps * p.chunks_per_tap;
+    const int a_per_tile = p.mode == kModeHalo ? p.chunks_per_tap : kiters;
+    const int b_per_tile = (p.mode == kModeHalo && !p.b_resident) ? kiters : 0;
+    const bool rings_ok = 2 * a_per_tile <= p.stages_a && (b_per_tile == 0 || 2 * b_per_tile <= p.stages_b);
+    p.mma_issuers = (rings_ok && kiters > 0 && p.num_tiles >= 2 * ctx->num_sms) ? 2 : 1;
+    // many small tiles per CTA: four epilogue groups; few large ones: all warps on every tile (shortest tail)
+    const int tiles_per_cta = ceil_div(p.num_tiles, ctx->num_sms);
+    p.epi_groups_log2 = tiles_per_cta >= 8 ? std::min(2, p.tmem_bufs_log2) : 0;
+  }
   p.fd_tiles_col = make_fastdiv(p.tiles_col);
   p.fd_tiles_per_img = make_fastdiv(p.mode == kModeHalo ? p.tiles_per_img : 1);
   p.fd_tiles_w = make_fastdiv(p.tiles_w);

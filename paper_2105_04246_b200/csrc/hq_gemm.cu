@@ -161,7 +161,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int out_vec) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * kMaxStagesA + 2 * kMaxStagesB + 4];
+  __shared__ __align__(8) uint64_t bars[2 * kMaxStagesA + 2 * kMaxStagesB + 16];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int red_min[kEpilogueWarps], red_max[kEpilogueWarps];
@@ -183,7 +183,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   auto b_full = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + s); };
   auto b_empty = [&](int s) { return bar0 + 8u * (2 * kMaxStagesA + kMaxStagesB + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + b); };
-  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + 2 + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + 8 + b); };
+  const int nbuf = p.tmem_bufs, nbuf_log2 = p.tmem_bufs_log2;   // accumulator buffers in TMEM (2 or 4)
 
   const int kiters = p.ntaps * p.chunks_per_tap;
 
@@ -197,9 +198,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       mbar_init(b_full(s), 1);
       mbar_init(b_empty(s), 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < nbuf; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), kEpilogueWarps);
+      mbar_init(tempty_bar(b), kEpilogueWarps >> p.epi_groups_log2);   // one arrival per warp of the group that drains it
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -330,25 +331,45 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+  } else if (warp == 1 || (warp == 3 && p.mma_issuers == 2)) {
+    // ------------------------------ MMA issuer(s) ------------------------------
+    // With two issuers, warp 1 takes the CTA's even tiles and warp 3 the odd ones (different accumulator buffers):
+    // the fixed per-tile latency of one issuer (decode, waits, commits) hides behind the other's MMA stream.
+    const int issuer = warp == 1 ? 0 : 1;
+    const int nissuers = p.mma_issuers;
     // The k-steps of one operand stage are issued from a compile-time unrolled group: a run-time inner loop
     // around the MMA instruction was measured to cost several hundred cycles per iteration.
     auto mma_role = [&](auto kk_tag) {
       constexpr int KK = decltype(kk_tag)::value;
       int stage = 0, bstage = 0;
       uint32_t phase = 0, bphase = 0;
-      int local_tile = 0;
       bool ok = true;
+      // ring positions are global over the CTA's tiles: skipping a tile advances them by that tile's stage count
+      auto advance = [](int& st, uint32_t& ph, int n, int stages) {
+        st += n;
+        while (st >= stages) {
+          st -= stages;
+          ph ^= 1u;
+        }
+      };
+      const int a_per_tile = halo ? p.chunks_per_tap : kiters;
+      const int b_per_tile = (halo && !p.b_resident) ? kiters : 0;
+      if (issuer > 0) {
+        advance(stage, phase, issuer * a_per_tile, p.stages_a);
+        if (b_per_tile) advance(bstage, bphase, issuer * b_per_tile, p.stages_b);
+      }
+      bool first = true;
       const bool sw64 = p.swizzle64 != 0;
       const uint64_t bdesc0 = make_smem_desc(ring_b, sw64);
       const int ntaps = p.ntaps, stages_b = p.stages_b;
       const bool resident = p.b_resident != 0;
       const uint32_t idesc = p.idesc;
       const uint32_t bstep16 = p.stage_bytes_b >> 4;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local_tile) {
-        const int buf = local_tile & 1;
-        const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
+      for (int local_tile = issuer; ok; local_tile += nissuers) {
+        const int tile = (int)blockIdx.x + local_tile * (int)gridDim.x;
+        if (tile >= p.num_tiles) break;
+        const int buf = local_tile & (nbuf - 1);
+        const uint32_t tph = (uint32_t)(local_tile >> nbuf_log2) & 1u;
         ok = warp_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait, 200u);
         if (!ok) break;
         tc_fence_after();
@@ -358,7 +379,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           int n0, o0, w0, col0;
           decode(tile, n0, o0, w0, col0);
           const uint32_t rel_bytes = (uint32_t)(o0 - fdiv(o0, p.fd_P) * p.P) * (uint32_t)p.BK;
-          if (p.b_resident && local_tile == 0) {   // the whole weight matrix arrives once
+          if (p.b_resident && first) {   // the whole weight matrix arrives once
             for (int ki = 0; ki < kiters && ok; ++ki) ok = warp_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
             if (!ok) break;
             tc_fence_after();
@@ -429,6 +450,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           if (!ok) break;
         }
         if (elect_one()) umma_commit(tfull_bar(buf));
+        first = false;
+        if (nissuers > 1) {   // step over the other issuer's tile
+          advance(stage, phase, (nissuers - 1) * a_per_tile, p.stages_a);
+          if (b_per_tile) advance(bstage, bphase, (nissuers - 1) * b_per_tile, p.stages_b);
+        }
       }
     };
     if (kiters > 0) {
@@ -438,9 +464,15 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp >= kFirstEpilogueWarp) {
     // ------------------------------ epilogue ------------------------------
+    // The 16 warps form G (1, 2 or 4, at most the number of accumulator buffers) groups; group g drains the CTA's tiles
+    // g, g + G, ...  Within a group the warps of a TMEM lane quarter split the column chunks.  More groups mean fewer
+    // hand-offs per warp (good for many small tiles); one group means the shortest tail (good for few large tiles).
     const int quarter = warp & 3;                         // TMEM lanes 32*quarter .. +31 belong to this warp
-    const int slice = (warp - kFirstEpilogueWarp) >> 2;   // the warps of a quarter split the column chunks
     const int ew = warp - kFirstEpilogueWarp;
+    const int ngroups = 1 << p.epi_groups_log2;
+    const int group = (ew >> 2) & (ngroups - 1);
+    const int slice = (ew >> 2) >> p.epi_groups_log2;
+    const int slices = kEpilogueSlices >> p.epi_groups_log2;
     const int row = quarter * 32 + lane;
     QParams q;
     {
@@ -458,10 +490,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int rh = (row / p.Wt) % p.Ht;
     const int rw = row % p.Wt;
     const int nchunks = p.BN / 16;                      // BN is a multiple of 16
-    const int c_begin = (slice * nchunks) / kEpilogueSlices;
-    const int c_end = ((slice + 1) * nchunks) / kEpilogueSlices;
-    int local_tile = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++local_tile) {
+    const int c_begin = (slice * nchunks) / slices;
+    const int c_end = ((slice + 1) * nchunks) / slices;
+    for (int local_tile = group; ; local_tile += ngroups) {
+      const int tile = (int)blockIdx.x + local_tile * (int)gridDim.x;
+      if (tile >= p.num_tiles) break;
       int n0, h0, w0, col0;
       decode(tile, n0, h0, w0, col0);
       int n, i, j;
@@ -488,8 +521,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         if (p.zc_in_smem) zrow_s = zc_s + off;   // shared copy, already multiplied by zx
         else corr_row = p.corr + off;
       }
-      const int buf = local_tile & 1;
-      const uint32_t tph = (uint32_t)(local_tile >> 1) & 1u;
+      const int buf = local_tile & (nbuf - 1);
+      const uint32_t tph = (uint32_t)(local_tile >> nbuf_log2) & 1u;
       if (kiters > 0) {
         int w = 1;
         if (lane == 0) w = mbar_wait(tfull_bar(buf), tph, abort_flag, p.status, kAsyncEpilogueTmemFullWait, 2000u) ? 1 : 0;

@@ -84,6 +84,9 @@ struct GemmParams {
   int32_t* status;
   uint32_t idesc;
   uint32_t tmem_cols, tmem_buf_stride;
+  int32_t mma_issuers;                // 1 or 2 warps issuing MMAs (alternate tiles)
+  int32_t tmem_bufs, tmem_bufs_log2;   // accumulator buffers in TMEM (2, 4 or 8)
+  int32_t epi_groups_log2;             // epilogue warp groups: 1, 2 or 4 (<= buffers)
   int32_t stages_a, stages_b;
   uint32_t stage_bytes_a, stage_bytes_b;   // kModeTap: A and B part of one stage; kModeHalo: patch stage, B stage
   int32_t swizzle64;                  // 1: 64-byte swizzle (BK = 64), 0: 128-byte swizzle (BK = 128)
