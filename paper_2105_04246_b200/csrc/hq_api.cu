@@ -413,7 +413,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     } else if (sub.patch_matrix != nullptr) {
       // channel counts that no TMA box can address (C = 3): gather the filter windows into rows first
       HQ_CUDA(ctx, launch_patch_matrix(in, sub.patch_matrix, inq, desc->N, desc->H, desc->W, desc->C, Ho, Wo, desc->R, desc->S, desc->stride_h,
-                                       desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, s));
+                                       desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, sub.patch_RP, s));
       ctx->launches += 1;
       st = encode_a(ctx, sub, sub.patch_matrix, sub.patch_K, desc->N * Ho * Wo, 1, 1, &ta);
     } else if (sub.a_flat) {
@@ -656,18 +656,26 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
         // rows of [R*S*C] input bytes (padded to a multiple of 16, padding taps holding the input zero point) are
         // gathered by a pre-pass into a library-owned matrix; the layer is then a flat GEMM over it
         const int64_t rows = (int64_t)d.N * Ho * Wo;
-        const int rsc = d.R * d.S * d.C;
-        const int Kp = round_up(rsc, 16);
+        const int RP = round_up(d.S * d.C, 8);   // one filter row per 8-byte aligned slot
+        const int Kp = round_up(d.R * RP, 16);
         if (rows > INT32_MAX) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many pixels"));
         sp.n_img = 1; sp.TH = 1; sp.TW = (int)rows; sp.in_mul_h = sp.in_mul_w = 1; sp.dh = {0}; sp.dw = {0};
         sp.a_H = 1; sp.a_W = (int)rows; sp.Cin = Kp; sp.Nout = d.K;
         sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.K; sp.flat = true;
         hq_conv_desc flatd = d;
         flatd.R = flatd.S = 1;
-        flatd.C = rsc;   // the filter [K][R][S][C] read as [K][R*S*C]
+        flatd.C = d.R * d.S * d.C;
         if ((st = build_sub(ctx, pw, s, sp, flatd, W, {0}, {0}, false, 1)) != HQ_OK) return bail(st);
         hq_sub_problem& sub = pw->subs.back();
         sub.patch_K = Kp;
+        sub.patch_RP = RP;
+        {  // the weight matrix in the slot layout of the patch rows, and its column sums
+          const uint32_t one = 1u;
+          cudaError_t e = launch_prep_patch_weights(W, sub.wmat, d.K, d.R, d.S * d.C, RP, sub.p.Cpad, s);
+          if (e == cudaSuccess) e = launch_corr(sub.wmat, sub.corr, d.K, 1, sub.p.Cpad, 1, 1, &one, 1, &one, 1, sub.p.corr_ld, s);
+          if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "patch weight preparation failed: %s", cudaGetErrorString(e)));
+          ctx->launches += 2;
+        }
         if ((st = dev_alloc(ctx, pw, (void**)&sub.patch_matrix, (size_t)rows * Kp)) != HQ_OK) return bail(st);
         *out = pw;
         return HQ_OK;

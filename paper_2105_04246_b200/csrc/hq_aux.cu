@@ -173,22 +173,24 @@ __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict_
 }
 
 // ---- operand repacking for shapes no TMA box can address ------------------------------------------
-// A[m][j], j = (r*S + s)*C + c: the filter window of output pixel m; taps on padding hold the input zero point
-// (real zero), columns beyond R*S*C hold 0 (their weights are 0).  For a fixed filter row r the S*C input bytes are
-// contiguous in NHWC, so thread (pixel, r) copies that run into the pixel's row in shared memory; the block then
-// writes its rows out with 16-byte stores.
+// A[m][r*RP + j], j = s*C + c < S*C: the filter window of output pixel m, one filter row per RP-byte slot
+// (RP = S*C rounded up to 8).  Taps on padding hold the input zero point (real zero); slot bytes beyond S*C hold
+// whatever follows in the input row -- their weights are zero.  For a fixed filter row the S*C input bytes are
+// contiguous in NHWC, so thread (pixel, r) moves that run with aligned 32-bit loads and a funnel shift into the
+// pixel's row in shared memory; the block then writes its rows out with 16-byte stores.
 constexpr int kPatchPixels = 32;   // output pixels per block iteration
 __global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ A, const hq_range_state* xq, int N,
                                                            int H, int W, int C, int Ho, int Wo, int R, int S, int stride_h, int stride_w,
-                                                           int pad_h, int pad_w, int Kp) {
+                                                           int pad_h, int pad_w, int Kp, int RP) {
   extern __shared__ __align__(16) int8_t rows_s[];   // [kPatchPixels][Kp]
   const int zx = xq->zero_point;
-  const int sc = S * C, rsc = R * sc;
+  const uint32_t zx4 = ((uint32_t)zx & 0xffu) * 0x01010101u;
+  const int sc = S * C, used = R * RP, nw = RP / 4;
   const int64_t M = (int64_t)N * Ho * Wo;
+  const int8_t* x_end = x + (int64_t)N * H * W * C;   // no load starts at or beyond this address
   for (int64_t m0 = (int64_t)blockIdx.x * kPatchPixels; m0 < M; m0 += (int64_t)gridDim.x * kPatchPixels) {
-    // zero the padding columns once per iteration (cheap: Kp - rsc < 16 bytes per pixel)
-    for (int t = threadIdx.x; t < kPatchPixels * (Kp - rsc); t += blockDim.x)
-      rows_s[(t / (Kp - rsc)) * Kp + rsc + t % (Kp - rsc)] = 0;
+    for (int t = threadIdx.x; t < kPatchPixels * (Kp - used); t += blockDim.x)   // columns after the last slot
+      rows_s[(t / (Kp - used)) * Kp + used + t % (Kp - used)] = 0;
     for (int t = threadIdx.x; t < kPatchPixels * R; t += blockDim.x) {
       const int pl = t / R, r = t - pl * R;
       const int64_t m = m0 + pl;
@@ -198,15 +200,29 @@ __global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restr
       const int n = (int)(m / ((int64_t)Wo * Ho));
       const int hi = ho * stride_h - pad_h + r;
       const int wi0 = wo * stride_w - pad_w;
-      int8_t* dst = rows_s + pl * Kp + r * sc;
+      int8_t* dst = rows_s + pl * Kp + r * RP;   // 8-byte aligned
+      uint32_t* dst4 = reinterpret_cast<uint32_t*>(dst);
       if (hi < 0 || hi >= H) {
-        for (int b = 0; b < sc; ++b) dst[b] = (int8_t)zx;
+        for (int i = 0; i < nw; ++i) dst4[i] = zx4;
+      } else if (wi0 >= 0 && wi0 + S <= W) {
+        const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
+        const uint32_t sh = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 3u) * 8u;
+        const uint32_t* a4 = reinterpret_cast<const uint32_t*>(reinterpret_cast<uintptr_t>(src) & ~(uintptr_t)3);
+        uint32_t prev = *a4;
+        for (int i = 0; i < nw; ++i) {
+          const uint32_t* nxt = a4 + i + 1;
+          // an aligned word that starts inside the tensor is readable to its end (the base is 16-byte aligned)
+          const uint32_t next = (reinterpret_cast<const int8_t*>(nxt) < x_end) ? *nxt : 0u;
+          dst4[i] = __funnelshift_r(prev, next, sh);
+          prev = next;
+        }
       } else {
         const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
         for (int q = 0; q < S; ++q) {
           const bool in = (wi0 + q >= 0) && (wi0 + q < W);
           for (int c = 0; c < C; ++c) dst[q * C + c] = in ? src[q * C + c] : (int8_t)zx;
         }
+        for (int b = sc; b < RP; ++b) dst[b] = 0;
       }
     }
     __syncthreads();
@@ -216,6 +232,17 @@ __global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restr
       if (m0 * Kp + byte < M * Kp) *reinterpret_cast<uint4*>(A + m0 * Kp + byte) = *reinterpret_cast<const uint4*>(rows_s + byte);
     }
     __syncthreads();
+  }
+}
+
+// weight matrix for the patch layout: Wmat[k][r*RP + j] = W[k][r][j], zero elsewhere (row pitch `ld` bytes)
+__global__ void prep_patch_weights_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wmat, int K, int R, int SC, int RP, int ld) {
+  const int64_t total = (int64_t)K * ld;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int j = (int)(idx % ld);
+    const int k = (int)(idx / ld);
+    const int r = j / RP, b = j - r * RP;
+    Wmat[idx] = (r < R && b < SC) ? W[((int64_t)k * R + r) * SC + b] : (int8_t)0;
   }
 }
 
@@ -500,12 +527,18 @@ cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, in
   return cudaGetLastError();
 }
 
+cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s) {
+  const int64_t total = (int64_t)K * ld;
+  prep_patch_weights_kernel<<<(int)std::min<int64_t>((total + 255) / 256, 1024), 256, 0, s>>>(W, Wmat, K, R, SC, RP, ld);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
-                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, cudaStream_t s) {
+                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, int RP, cudaStream_t s) {
   const int64_t groups = ((int64_t)N * Ho * Wo + kPatchPixels - 1) / kPatchPixels;
   int blocks = (int)std::min<int64_t>(groups, 148 * 8);
   if (blocks < 1) blocks = 1;
-  patch_matrix_kernel<<<blocks, 256, (size_t)kPatchPixels * Kp, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp);
+  patch_matrix_kernel<<<blocks, 256, (size_t)kPatchPixels * Kp, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp, RP);
   return cudaGetLastError();
 }
 

@@ -127,7 +127,8 @@ cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int nta
 cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps, const uint32_t* rowmasks,
                         int nrowcls, const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s);
 cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
-                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, cudaStream_t s);
+                                int stride_h, int stride_w, int pad_h, int pad_w, int Kp, int RP, cudaStream_t s);
+cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s);
 cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
                            const uint32_t* colmasks, int ncolcls, cudaStream_t s);
@@ -161,6 +162,7 @@ struct hq_sub_problem {               // one kernel launch of a prepared convolu
   int gfold = 1;                      // pixels folded into one GEMM row (channel counts that are not multiples of 16)
   int8_t* patch_matrix = nullptr;     // [pixels][patch_K]: filter windows gathered by a pre-pass (C not a multiple of 16)
   int patch_K = 0;
+  int patch_RP = 0;                   // bytes per filter-row slot in a patch-matrix row
 };
 
 struct hq_prepared_weights {
