@@ -36,6 +36,11 @@ from paper_2105_04246_b200 import workloads as wl
 METRIC = "int8 TOPS & HBM bytes/layer: hindsight-fused vs dynamic quant, % of roofline"
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 peak / dense bf16 peak on B200 (4.5 / 2.25 POPS)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the named layer's kernel, from the ncu captures
+# summarised under profiles/ (taken with the kernels as committed; set an entry to None when its kernel changes).
+# Output lines still dirty in L2 when the kernel ends are not in these counters.
+NCU_TRAFFIC = {"resnet_conv3x3_64": 12953344, "resnet_conv3x3_256_bwd": 13514496, "mbv2_dw3x3": 191312128,
+               "mbv2_expand": 78326528, "mbv2_project": 124691200}
 
 
 def load_peaks():
@@ -416,7 +421,7 @@ def run_gpu(args):
         ach = s.ops / layer_us[dom] / 1e6
         roof = {"bound": "tensor", "achieved": round(ach, 1), "peak": round(int8_peak, 1), "unit": "TOP/s", "frac": round(ach / int8_peak, 4)}
     roof.update({"kernel": "depthwise_kernel" if getattr(s, "depthwise", False) else "hq_gemm_kernel", "layer": s.name,
-                 "launch_us": round(layer_us[dom], 3), "traffic": None, "peak_source": f"{peak_kind} (int8 = bf16 burst x {NOMINAL_INT8_OVER_BF16})",
+                 "launch_us": round(layer_us[dom], 3), "traffic": NCU_TRAFFIC.get(s.name), "peak_source": f"{peak_kind} (int8 = bf16 burst x {NOMINAL_INT8_OVER_BF16})",
                  "frac_of": f"of {peak_kind}"})
 
     out = {
