@@ -307,6 +307,8 @@ def run_gpu(args):
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
     ctx = hq.Context(local)
+    if args.no_overlap:
+        ctx.set_option("overlap_launches", 0)
     peaks, peak_kind = load_peaks()
     name = args.workload
     pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg5": 2}[name]
@@ -430,6 +432,7 @@ def run_gpu(args):
         "data": "synthetic", "impl": "hq",
         "config": {"workload": f"{name}: " + ", ".join(s.name for _, s, _ in wk.layers), "path": "in-hindsight (static requant in the epilogue + min/max)",
                    "l2": f"inputs and outputs rotate over a pool of {pool} buffer sets (> L2) inside CUDA graphs", "eta": 0.9,
+                   "launch": "ordinary" if args.no_overlap else "programmatic stream serialization",
                    "parallelism": f"dp{world} (batch shards; one int32 min/max all-reduce per step before the range update)" if world > 1 else "dp1"},
         "gpu_launches": int(launches_per_step * K),
         "launches_per_step": int(launches_per_step),
@@ -456,6 +459,8 @@ def run_profile(args):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     ctx = hq.Context(0)
+    if args.no_overlap:
+        ctx.set_option("overlap_launches", 0)
     wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0)
     stream = torch.cuda.current_stream(dev)
     for j in range(2):
@@ -496,6 +501,8 @@ def main():
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="ordinary launches instead of programmatic stream serialization (set-up of a kernel overlapping its predecessor's tail)")
     ap.add_argument("--profile", action="store_true",
                     help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
                          "then --steps in-hindsight steps, then --steps dynamic steps")

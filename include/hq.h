@@ -120,7 +120,11 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
 /* Tuning knob (HOST key string), for tests and experiments; results are identical for every value.
  *   "staging": how convolutions prepared AFTER this call bring their input to the MAC array (the
  *              paper's "loaded into the MAC array", Sec. 3.1): -1 = chosen per layer (default),
- *              0 = one copy per filter tap, 1 = input rows kept resident wherever the layer allows. */
+ *              0 = one copy per filter tap, 1 = input rows kept resident wherever the layer allows.
+ *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their
+ *              set-up may run while the previous kernel in the stream drains; each waits for that
+ *              kernel to finish before it reads memory, so stream order is unchanged.  0 = ordinary
+ *              launches. */
 hq_status hq_set_option(hq_ctx* ctx, const char* key, int32_t value);
 
 /* ---- weights ------------------------------------------------------------------------------ */

@@ -208,7 +208,7 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
       if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * p.stage_bytes_b + 2ull * stride <= ring_budget) {
         resident = 1;
         stages_b = kiters;
-        stages_a = (int)std::min<uint64_t>(4, (ring_budget - (uint64_t)kiters * p.stage_bytes_b) / stride);
+        stages_a = (int)std::min<uint64_t>(kMaxStagesA, (ring_budget - (uint64_t)kiters * p.stage_bytes_b) / stride);
       } else {
         stages_a = 2;
         while (stages_a < 4 && (uint64_t)(stages_a + 1) * stride + 4ull * p.stage_bytes_b <= ring_budget) ++stages_a;
@@ -378,7 +378,7 @@ hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, con
   p.out = out;
   p.yq = yq;
   const int grid = std::min(p.num_tiles, ctx->num_sms);
-  HQ_CUDA(ctx, launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s));
+  HQ_CUDA(ctx, launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s, ctx->overlap));
   ctx->launches += 1;
   return HQ_OK;
 }
@@ -398,7 +398,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     p.stride_h = desc->stride_h; p.stride_w = desc->stride_w; p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
     p.x = in; p.w = pw->dw_w; p.corr = pw->dw_corr; p.rowcls = pw->dw_rowcls; p.colcls = pw->dw_colcls; p.ncolcls = pw->dw_ncolcls;
     p.xq = inq; p.w_scale = w_scale; p.yq = outq; p.out = out;
-    HQ_CUDA(ctx, launch_depthwise(p, out_mode, ctx->num_sms, s));
+    HQ_CUDA(ctx, launch_depthwise(p, out_mode, ctx->num_sms, s, false));
     ctx->launches += 1;
     return HQ_OK;
   }
@@ -575,6 +575,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "staging") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "staging must be -1, 0 or 1");
     ctx->force_mode = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "overlap_launches") {
+    if (value < 0 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "overlap_launches must be 0 or 1");
+    ctx->overlap = value != 0;
     return HQ_OK;
   }
   return fail(ctx, HQ_ERR_INVALID_ARG, "unknown option '%s'", key);
@@ -758,7 +763,7 @@ __attribute__((visibility("default"))) hq_status hq_range_update(hq_ctx* ctx, vo
   if (!states || count <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "states is null or count is not positive");
   if (!aligned16(states)) return fail(ctx, HQ_ERR_ALIGNMENT, "range states must be 16-byte aligned");
   if (!(eta >= 0.0f && eta <= 1.0f)) return fail(ctx, HQ_ERR_INVALID_ARG, "eta must lie in [0, 1]");
-  HQ_CUDA(ctx, launch_range_update(states, count, eta, (cudaStream_t)stream));
+  HQ_CUDA(ctx, launch_range_update(states, count, eta, (cudaStream_t)stream, ctx->overlap));
   ctx->launches += 1;
   return HQ_OK;
 }
@@ -770,8 +775,8 @@ __attribute__((visibility("default"))) hq_status hq_dynamic_quant(hq_ctx* ctx, v
   cudaStream_t s = (cudaStream_t)stream;
   hq_status st = run_op(ctx, s, op, workspace, yq, kOutF32);
   if (st != HQ_OK) return st;
-  HQ_CUDA(ctx, launch_dynamic_derive(yq, s));
-  HQ_CUDA(ctx, launch_quantize_pass(workspace, Y, op_out_elems(op), yq, ctx->num_sms, s));
+  HQ_CUDA(ctx, launch_dynamic_derive(yq, s, ctx->overlap));
+  HQ_CUDA(ctx, launch_quantize_pass(workspace, Y, op_out_elems(op), yq, ctx->num_sms, s, false));
   ctx->launches += 2;
   return HQ_OK;
 }
@@ -844,8 +849,8 @@ extern "C" __attribute__((visibility("default"))) hq_status hq_dynamic_quant_sta
   cudaStream_t s = (cudaStream_t)stream;
   st = run_op(ctx, s, op, ws, yq, kOutF32);
   if (st != HQ_OK) return st;
-  HQ_CUDA(ctx, launch_dynamic_derive(yq, s));
-  HQ_CUDA(ctx, launch_quantize_pass(ws, Y, elems, yq, ctx->num_sms, s));
+  HQ_CUDA(ctx, launch_dynamic_derive(yq, s, ctx->overlap));
+  HQ_CUDA(ctx, launch_quantize_pass(ws, Y, elems, yq, ctx->num_sms, s, false));
   ctx->launches += 2;
   return HQ_OK;
 }

@@ -27,6 +27,8 @@ __device__ __forceinline__ void derive_grid(hq_range_state* s) {
 }
 
 __global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
+  grid_launch_dependents();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
   hq_range_state* s = st + i;
@@ -50,6 +52,8 @@ __global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
 
 // Eq. 1: the range is the min/max of the tensor that was just written.
 __global__ void dynamic_derive_kernel(hq_range_state* s) {
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
+  grid_launch_dependents();
   const int mn = s->acc_min, mx = s->acc_max;
   if (mn > mx) return;
   s->q_min = __fmul_rn(__int2float_rn(mn), s->acc_scale);
@@ -62,6 +66,7 @@ __global__ void dynamic_derive_kernel(hq_range_state* s) {
 
 // second pass of the dynamic path: read the binary32 output back and quantize it
 __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __restrict__ out, int64_t count, const hq_range_state* st) {
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
   QParams q;
   q.s_acc = 1.0f;
   q.zx = 0;
@@ -81,6 +86,7 @@ __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __rest
     }
     reinterpret_cast<uint4*>(out)[g] = make_uint4(w[0], w[1], w[2], w[3]);
   }
+  grid_launch_dependents();   // the successor may take the SMs that free up from here on
   if (blockIdx.x == 0) {
     for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x)
       out[i] = (int8_t)min(max(requant_real<false>(y[i], q), -128), 127);
@@ -262,6 +268,7 @@ __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w 
 template <int kOut>
 __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
   __shared__ int red_min[8], red_max[8];
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
   QParams q;
   q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
   q.zx = p.xq->zero_point;
@@ -332,6 +339,7 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
       }
     }
   }
+  grid_launch_dependents();   // the successor may take the SMs that free up from here on
   mn = __reduce_min_sync(0xffffffffu, mn);
   mx = __reduce_max_sync(0xffffffffu, mx);
   const int warp = threadIdx.x >> 5;
@@ -363,6 +371,7 @@ constexpr int kDwPix = 8;
 template <int kOut>
 __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int slots, int groups_w) {
   __shared__ int red_min[8], red_max[8];
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
   QParams q;
   q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
   q.zx = p.xq->zero_point;
@@ -452,6 +461,7 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
       }
     }
   }
+  grid_launch_dependents();   // the successor may take the SMs that free up from here on
   mn = __reduce_min_sync(0xffffffffu, mn);
   mx = __reduce_max_sync(0xffffffffu, mx);
   const int warp = threadIdx.x >> 5;
@@ -474,22 +484,20 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
 
 }  // namespace
 
-cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s) {
-  range_update_kernel<<<(count + 127) / 128, 128, 0, s>>>(st, count, eta);
-  return cudaGetLastError();
+cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap) {
+  return launch_overlapped(range_update_kernel, (count + 127) / 128, 128, 0, s, overlap, st, count, eta);
 }
 
-cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s) {
-  dynamic_derive_kernel<<<1, 1, 0, s>>>(st);
-  return cudaGetLastError();
+cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overlap) {
+  return launch_overlapped(dynamic_derive_kernel, 1, 1, 0, s, overlap, st);
 }
 
-cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s) {
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
+                                 bool overlap) {
   const int threads = 256;
   int64_t want = (count / 16 + threads - 1) / threads;
   int blocks = (int)(want < 1 ? 1 : (want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want));
-  quantize_pass_kernel<<<blocks, threads, 0, s>>>(y, out, count, st);
-  return cudaGetLastError();
+  return launch_overlapped(quantize_pass_kernel, blocks, threads, 0, s, overlap, y, out, count, st);
 }
 
 cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
@@ -550,7 +558,7 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
   return cudaGetLastError();
 }
 
-cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s) {
+cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s, bool overlap) {
   const int CW = p.C / 4;
   if (p.R == 3 && p.S == 3 && p.stride_h == 1 && p.stride_w == 1 && CW <= 256) {
     const int slots = 256 / CW;                           // pixel groups per block
@@ -560,22 +568,20 @@ cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaS
     int blocks = (int)std::min<int64_t>((items + slots - 1) / slots, (int64_t)num_sms * 8);
     if (blocks < 1) blocks = 1;
     switch (out_mode) {
-      case kOutInt8: depthwise3x3_kernel<kOutInt8><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
-      case kOutF32: depthwise3x3_kernel<kOutF32><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
-      default: depthwise3x3_kernel<kOutAcc><<<blocks, threads, 0, s>>>(p, slots, groups_w); break;
+      case kOutInt8: return launch_overlapped(depthwise3x3_kernel<kOutInt8>, blocks, threads, 0, s, overlap, p, slots, groups_w);
+      case kOutF32: return launch_overlapped(depthwise3x3_kernel<kOutF32>, blocks, threads, 0, s, overlap, p, slots, groups_w);
+      default: return launch_overlapped(depthwise3x3_kernel<kOutAcc>, blocks, threads, 0, s, overlap, p, slots, groups_w);
     }
-    return cudaGetLastError();
   }
   const int64_t total = (int64_t)p.N * p.Ho * p.Wo * (p.C / 16);
   int64_t want = (total + 255) / 256;
   int blocks = (int)(want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want);
   if (blocks < 1) blocks = 1;
   switch (out_mode) {
-    case kOutInt8: depthwise_kernel<kOutInt8><<<blocks, 256, 0, s>>>(p); break;
-    case kOutF32: depthwise_kernel<kOutF32><<<blocks, 256, 0, s>>>(p); break;
-    default: depthwise_kernel<kOutAcc><<<blocks, 256, 0, s>>>(p); break;
+    case kOutInt8: return launch_overlapped(depthwise_kernel<kOutInt8>, blocks, 256, 0, s, overlap, p);
+    case kOutF32: return launch_overlapped(depthwise_kernel<kOutF32>, blocks, 256, 0, s, overlap, p);
+    default: return launch_overlapped(depthwise_kernel<kOutAcc>, blocks, 256, 0, s, overlap, p);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace hq

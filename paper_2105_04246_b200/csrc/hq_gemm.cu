@@ -209,13 +209,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     tapoff_s[threadIdx.x] =
         (uint32_t)(((p.tap_dh[threadIdx.x] - p.dh_min) * p.P + (p.tap_dw[threadIdx.x] - p.dw_min)) * p.BK) >> 4;
   int32_t* zc_s = reinterpret_cast<int32_t*>(smem_raw + ((ring_a - smem_u32(smem_raw)) + p.zc_offset));
-  if (p.zc_in_smem) {   // zx * (sum of in-image weights) per border class and output channel
-    const int zx = p.xq->zero_point;
-    for (int i = threadIdx.x; i < p.zc_elems; i += blockDim.x) zc_s[i] = zx * p.corr[i];
-  }
-  if (p.cls_in_smem) {
-    for (int i = threadIdx.x; i < p.TH; i += blockDim.x) cls_s[i] = p.rowcls[i];
-    for (int i = threadIdx.x; i < p.TW; i += blockDim.x) cls_s[512 + i] = p.colcls[i];
+  if (warp == 0 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap_b) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(p.tmem_cols)
@@ -226,6 +222,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  // Everything above touched only kernel parameters and this CTA's own resources.  From here on the kernel reads
+  // what earlier kernels in the stream wrote (operands, range states), so it waits for them.
+  grid_dependency_wait();
 
   // tile index -> origin.  kModeTap: (n0, h0, w0) of the pixel box; kModeHalo: image n0, first linear pixel h0
   auto decode = [&](int tile, int& n0, int& h0, int& w0, int& col0) {
@@ -462,6 +461,10 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       else mma_role(std::integral_constant<int, 4>{});
     }
     __syncwarp();
+    // All MMAs of this CTA are issued; what is left is the epilogue of the last tiles.  The next kernel in the stream
+    // may become resident as SMs free up (it waits for this grid to finish before it reads anything).  Releasing it
+    // earlier only parks its waiting CTAs beside this one, where they compete for issue slots.
+    grid_launch_dependents();
   } else if (warp >= kFirstEpilogueWarp) {
     // ------------------------------ epilogue ------------------------------
     // The 16 warps form G (1, 2 or 4, at most the number of accumulator buffers) groups; group g drains the CTA's tiles
@@ -485,6 +488,19 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       qparams_finish(q);
     }
     if (blockIdx.x == 0 && ew == 0 && lane == 0) p.yq->acc_scale = q.s_acc;
+    // The epilogue's tables are filled here, by the epilogue warps alone, while the first operand tiles are in flight:
+    // zx * (sum of in-image weights) per border class and output channel, and the border classes of rows and columns.
+    {
+      const int et = (int)threadIdx.x - kFirstEpilogueWarp * 32;
+      constexpr int kEpiThreads = kEpilogueWarps * 32;
+      if (p.zc_in_smem)
+        for (int i = et; i < p.zc_elems; i += kEpiThreads) zc_s[i] = q.zx * p.corr[i];
+      if (p.cls_in_smem) {
+        for (int i = et; i < p.TH; i += kEpiThreads) cls_s[i] = p.rowcls[i];
+        for (int i = et; i < p.TW; i += kEpiThreads) cls_s[512 + i] = p.colcls[i];
+      }
+      asm volatile("bar.sync 1, %0;" ::"r"(kEpiThreads) : "memory");
+    }
     int mn = INT32_MAX, mx = INT32_MIN;
     const int rn = row / (p.Ht * p.Wt);
     const int rh = (row / p.Wt) % p.Ht;
@@ -674,7 +690,7 @@ cudaError_t gemm_set_smem_attr(uint32_t smem_bytes) {
 }
 
 cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int out_mode, int grid, uint32_t smem_bytes,
-                        cudaStream_t s) {
+                        cudaStream_t s, bool overlap) {
   // widest aligned store the output rows allow
   int out_vec;
   const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out);
@@ -687,11 +703,10 @@ cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtens
     out_vec = (p.ldY % 4 == 0 && addr % 16 == 0) ? 16 : 4;
   }
   switch (out_mode) {
-    case kOutInt8: hq_gemm_kernel<kOutInt8><<<grid, kGemmThreads, smem_bytes, s>>>(p, ta, tb, out_vec); break;
-    case kOutF32: hq_gemm_kernel<kOutF32><<<grid, kGemmThreads, smem_bytes, s>>>(p, ta, tb, out_vec); break;
-    default: hq_gemm_kernel<kOutAcc><<<grid, kGemmThreads, smem_bytes, s>>>(p, ta, tb, out_vec); break;
+    case kOutInt8: return launch_overlapped(hq_gemm_kernel<kOutInt8>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
+    case kOutF32: return launch_overlapped(hq_gemm_kernel<kOutF32>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
+    default: return launch_overlapped(hq_gemm_kernel<kOutAcc>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
   }
-  return cudaGetLastError();
 }
 
 }  // namespace hq

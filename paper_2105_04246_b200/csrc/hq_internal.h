@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "hq.h"
@@ -114,14 +115,40 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// kernel launchers (defined in the .cu files)
+// Launch that lets the kernel become resident while its predecessor in the stream is still draining (programmatic
+// stream serialization).  Kernels launched this way run their set-up (barrier initialisation, TMEM allocation,
+// descriptor prefetch) early and execute grid_dependency_wait() before they touch any memory a predecessor may
+// have written; they also release their own successor at once, which then waits the same way, so the order of
+// memory effects in the stream is unchanged.  overlap = false is an ordinary launch (the two device calls are
+// no-ops then).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool overlap, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1u : 0u;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+
+// kernel launchers (defined in the .cu files); `overlap` as in launch_overlapped
 cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int out_mode, int grid, uint32_t smem_bytes,
-                        cudaStream_t s);
+                        cudaStream_t s, bool overlap);
 cudaError_t gemm_set_smem_attr(uint32_t smem_bytes);
-cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s);
-cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s);
-cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s);
-cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s);
+cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s, bool overlap);
+cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap);
+cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overlap);
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
+                                 bool overlap);
 cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
                                 const int8_t* tap_r, const int8_t* tap_s, int transposed, int blockdiag_g, cudaStream_t s);
 cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, int Cpad, int nrowtaps, int ncoltaps, const uint32_t* rowmasks,
@@ -146,6 +173,7 @@ struct hq_ctx {
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
+  bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
   std::string err;
 };
 

@@ -226,3 +226,63 @@ def test_rejected_calls_launch_nothing(ctx):
     assert e.value.status == 1
     assert ctx.launch_count() == n0
     torch.cuda.synchronize()
+
+
+# ---- two layers chained on one stream with no host synchronisation in between ----------------------
+@pytest.mark.parametrize("overlap", [1, 0])
+def test_chained_layers_without_host_sync(ctx, overlap):
+    """Layer B consumes layer A's int8 output and A's range state directly from device memory; the calls of
+    all iterations are enqueued back to back.  Checks the ordering of memory effects between consecutive
+    kernels (also when a kernel's set-up is allowed to overlap its predecessor's tail) against the oracle."""
+    r = synth.rng(77, overlap)
+    shpA = dict(N=3, H=20, W=20, Cin=32, K=64, R=3, S=3, stride=1, pad=1)
+    shpB = dict(N=3, H=20, W=20, Cin=64, K=48, R=1, S=1, stride=1, pad=0)
+    WA = synth.weights(r, (64, 3, 3, 32))
+    WB = synth.weights(r, (48, 1, 1, 64))
+    iters = 4
+    xs = [synth.signed_activations(r, (3, 20, 20, 32)) for _ in range(iters)]
+    dev = torch.device("cuda", ctx.device)
+    stream = torch.cuda.current_stream(dev)
+    ctx.set_option("overlap_launches", overlap)
+    try:
+        dA, dB = hq.conv_desc(**shpA), hq.conv_desc(**shpB)
+        wA = torch.from_numpy(WA.q).to(dev)
+        wB = torch.from_numpy(WB.q).to(dev)
+        sA = torch.tensor([WA.scale], dtype=torch.float32, device=dev)
+        sB = torch.tensor([WB.scale], dtype=torch.float32, device=dev)
+        pA = ctx.weights_prepare(stream, dA, hq.DIR_FWD, wA)
+        pB = ctx.weights_prepare(stream, dB, hq.DIR_FWD, wB)
+        states = hq.states_to_device(hq.new_states(2), dev)          # [A's output, B's output]
+        nbytes = hq.RANGE_STATE_DTYPE.itemsize
+        stA, stB = states[:nbytes], states[nbytes:]
+        xd = [torch.from_numpy(x.q).to(dev) for x in xs]
+        xq = [hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev) for x in xs]
+        y1 = [torch.full((3, 20, 20, 64), 99, dtype=torch.int8, device=dev) for _ in range(iters)]
+        y2 = [torch.full((3, 20, 20, 48), 99, dtype=torch.int8, device=dev) for _ in range(iters)]
+        ws1 = torch.empty((3, 20, 20, 64), dtype=torch.float32, device=dev)
+        ws2 = torch.empty((3, 20, 20, 48), dtype=torch.float32, device=dev)
+        torch.cuda.synchronize()
+        for t in range(iters):                                       # nothing below waits for the device
+            if t == 0:
+                ctx.dynamic_quant(stream, hq.conv_op(hq.OP_CONV_FWD, dA, xd[t], xq[t], pA, sA), ws1, y1[t], stA)
+                ctx.dynamic_quant(stream, hq.conv_op(hq.OP_CONV_FWD, dB, y1[t], stA, pB, sB), ws2, y2[t], stB)
+            else:
+                ctx.conv_fwd(stream, dA, xd[t], xq[t], pA, sA, y1[t], stA)
+                ctx.conv_fwd(stream, dB, y1[t], stA, pB, sB, y2[t], stB)
+                ctx.range_update(stream, states, 2, 0.9)
+        torch.cuda.synchronize()
+        assert ctx.get_async_error() == 0
+    finally:
+        ctx.set_option("overlap_launches", 1)
+    oA, oB = OracleLayer("conv_fwd", WA, shpA), OracleLayer("conv_fwd", WB, shpB)
+    for t in range(iters):
+        gridA = oA.layer.state.copy()                                # the range A's output is quantized with (t >= 1)
+        resA = oA.step(xs[t])
+        if t == 0:
+            gridA = oA.layer.state.copy()                            # dynamic: the range of the tensor itself
+        resB = oB.step(synth.QTensor(resA.q, gridA.scale, gridA.zero_point))
+        assert np.array_equal(y1[t].cpu().numpy(), resA.q), f"layer A, iteration {t}"
+        assert np.array_equal(y2[t].cpu().numpy(), resB.q), f"layer B, iteration {t}"
+    got = hq.states_from_device(states)
+    assert_state_close(got[0], oA.layer.state)
+    assert_state_close(got[1], oB.layer.state)
