@@ -121,6 +121,10 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
  *   "staging": how convolutions prepared AFTER this call bring their input to the MAC array (the
  *              paper's "loaded into the MAC array", Sec. 3.1): -1 = chosen per layer (default),
  *              0 = one copy per filter tap, 1 = input rows kept resident wherever the layer allows.
+ *   "repack":  how spatial filters over a channel count that is not a multiple of 16 (the RGB stem),
+ *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
+ *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows
+ *              per input row where the shape allows.
  *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their
  *              set-up may run while the previous kernel in the stream drains; each waits for that
  *              kernel to finish before it reads memory, so stream order is unchanged.  0 = ordinary

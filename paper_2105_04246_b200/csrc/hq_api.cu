@@ -7,6 +7,7 @@
 #include <stdio.h>
 
 #include <algorithm>
+#include <functional>
 #include <new>
 #include <string>
 #include <vector>
@@ -325,9 +326,12 @@ hq_status upload(hq_ctx* ctx, hq_prepared_weights* pw, const std::vector<uint8_t
   return HQ_OK;
 }
 
-// builds weight matrix, correction table and class maps of one sub-problem
+// builds weight matrix, correction table and class maps of one sub-problem; `custom` replaces the standard
+// [Nout][tap][Cpad] weight layout (repacked operands), the correction table is always summed from the matrix
+using WeightPrep = std::function<cudaError_t(hq_sub_problem&)>;
 hq_status build_sub(hq_ctx* ctx, hq_prepared_weights* pw, cudaStream_t s, const SubSpec& sp, const hq_conv_desc& d, const int8_t* W,
-                    const std::vector<int>& tap_r, const std::vector<int>& tap_s, bool transposed, int gfold) {
+                    const std::vector<int>& tap_r, const std::vector<int>& tap_s, bool transposed, int gfold,
+                    const WeightPrep* custom = nullptr) {
   pw->subs.emplace_back();
   hq_sub_problem& sub = pw->subs.back();
   sub.gfold = gfold;
@@ -343,12 +347,16 @@ hq_status build_sub(hq_ctx* ctx, hq_prepared_weights* pw, cudaStream_t s, const 
   st = dev_alloc(ctx, pw, (void**)&sub.corr, (size_t)rowmasks.size() * colmasks.size() * p.corr_ld * sizeof(int32_t));
   if (st != HQ_OK) return st;
   HQ_CUDA(ctx, cudaMemsetAsync(sub.corr, 0, (size_t)rowmasks.size() * colmasks.size() * p.corr_ld * sizeof(int32_t), s));
-  int8_t tr[kMaxTaps], ts[kMaxTaps];
-  for (int t = 0; t < p.ntaps; ++t) {
-    tr[t] = (int8_t)tap_r[t / (int)sp.dw.size()];
-    ts[t] = (int8_t)tap_s[t % (int)sp.dw.size()];
+  if (custom != nullptr) {
+    HQ_CUDA(ctx, (*custom)(sub));
+  } else {
+    int8_t tr[kMaxTaps], ts[kMaxTaps];
+    for (int t = 0; t < p.ntaps; ++t) {
+      tr[t] = (int8_t)tap_r[t / (int)sp.dw.size()];
+      ts[t] = (int8_t)tap_s[t % (int)sp.dw.size()];
+    }
+    HQ_CUDA(ctx, launch_prep_weights(W, sub.wmat, p.Nout, p.ntaps, p.Cpad, d.K, d.R, d.S, d.C, tr, ts, transposed ? 1 : 0, gfold, s));
   }
-  HQ_CUDA(ctx, launch_prep_weights(W, sub.wmat, p.Nout, p.ntaps, p.Cpad, d.K, d.R, d.S, d.C, tr, ts, transposed ? 1 : 0, gfold, s));
   HQ_CUDA(ctx, launch_corr(sub.wmat, sub.corr, p.Nout, p.ntaps, p.Cpad, (int)sp.dh.size(), (int)sp.dw.size(), rowmasks.data(),
                            (int)rowmasks.size(), colmasks.data(), (int)colmasks.size(), p.corr_ld, s));
   ctx->launches += 2;
@@ -416,6 +424,11 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
                                        desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, sub.patch_RP, s));
       ctx->launches += 1;
       st = encode_a(ctx, sub, sub.patch_matrix, sub.patch_K, desc->N * Ho * Wo, 1, 1, &ta);
+    } else if (sub.window != nullptr) {
+      HQ_CUDA(ctx, launch_row_window(in, sub.window, inq, desc->N, desc->H, desc->W, desc->C, sub.win_Hg, Wo, desc->S, sub.win_sh,
+                                     desc->stride_w, desc->pad_w, sub.win_SB, s));
+      ctx->launches += 1;
+      st = encode_a(ctx, sub, sub.window, sub.win_sh * sub.win_SB, Wo, sub.win_Hg, desc->N, &ta);
     } else if (sub.a_flat) {
       const int64_t rows = (int64_t)desc->N * aH * aW / sub.gfold;
       st = encode_a(ctx, sub, in, aC * sub.gfold, (int)rows, 1, 1, &ta);
@@ -577,6 +590,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     ctx->force_mode = value;
     return HQ_OK;
   }
+  if (std::string(key) == "repack") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "repack must be -1, 0 or 1");
+    ctx->force_repack = value;
+    return HQ_OK;
+  }
   if (std::string(key) == "overlap_launches") {
     if (value < 0 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "overlap_launches must be 0 or 1");
     ctx->overlap = value != 0;
@@ -658,29 +676,53 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
       tr = {0}; ts = {0};
     } else {
       if (d.C % 16 != 0) {
-        // rows of [R*S*C] input bytes (padded to a multiple of 16, padding taps holding the input zero point) are
-        // gathered by a pre-pass into a library-owned matrix; the layer is then a flat GEMM over it
+        // Channel counts no TMA box can address (the RGB stem).  Preferred: a pre-pass gathers, per output column, the
+        // horizontal filter windows of stride_h consecutive input rows into a library-owned tensor X2 of
+        // Cg = stride_h * SB bytes per pixel; over X2 the layer is a stride-1 convolution with vertical taps only.
+        const int sh = d.stride_h, sc = d.S * d.C;
+        int SB = round_up(sc, 16), Cg = 0;
+        if (64 % sh == 0 && sh * SB <= 64) { SB = 64 / sh; Cg = 64; }
+        else if (128 % sh == 0 && sh * SB <= 128) { SB = 128 / sh; Cg = 128; }
+        auto floordiv = [](int a, int b) { return a >= 0 ? a / b : -((-a + b - 1) / b); };
+        const int dh_min = floordiv(-d.pad_h, sh), dh_max = floordiv(d.R - 1 - d.pad_h, sh);
+        const int Hg = (d.H + sh - 1) / sh;
+        if (Cg != 0 && dh_max - dh_min + 1 <= kMaxTaps && ctx->force_repack != 0) {
+          sp.n_img = d.N; sp.TH = Ho; sp.TW = Wo; sp.in_mul_h = sp.in_mul_w = 1;
+          for (int t = dh_min; t <= dh_max; ++t) sp.dh.push_back(t);
+          sp.dw = {0};
+          sp.a_H = Hg; sp.a_W = Wo; sp.Cin = Cg; sp.Nout = d.K;
+          sp.out_H = Ho; sp.out_W = Wo; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.K; sp.flat = false;
+          const int ntaps = dh_max - dh_min + 1;
+          const WeightPrep prep = [&](hq_sub_problem& sub) {
+            ctx->launches += 1;
+            return launch_prep_window_weights(W, sub.wmat, d.K, d.R, sc, sh, SB, ntaps, dh_min, d.pad_h, s);
+          };
+          if ((st = build_sub(ctx, pw, s, sp, d, W, std::vector<int>(ntaps, 0), {0}, false, 1, &prep)) != HQ_OK) return bail(st);
+          hq_sub_problem& sub = pw->subs.back();
+          sub.win_sh = sh;
+          sub.win_SB = SB;
+          sub.win_Hg = Hg;
+          if ((st = dev_alloc(ctx, pw, (void**)&sub.window, (size_t)d.N * Hg * Wo * Cg)) != HQ_OK) return bail(st);
+          *out = pw;
+          return HQ_OK;
+        }
+        // Fallback: whole patch rows of [R*S*C] input bytes (one filter row per 8-byte aligned slot, padded to a multiple
+        // of 16, padding taps holding the input zero point) in a library-owned matrix; the layer is a flat GEMM over it
         const int64_t rows = (int64_t)d.N * Ho * Wo;
-        const int RP = round_up(d.S * d.C, 8);   // one filter row per 8-byte aligned slot
+        const int RP = round_up(d.S * d.C, 8);
         const int Kp = round_up(d.R * RP, 16);
         if (rows > INT32_MAX) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many pixels"));
         sp.n_img = 1; sp.TH = 1; sp.TW = (int)rows; sp.in_mul_h = sp.in_mul_w = 1; sp.dh = {0}; sp.dw = {0};
         sp.a_H = 1; sp.a_W = (int)rows; sp.Cin = Kp; sp.Nout = d.K;
         sp.out_H = 1; sp.out_W = (int)rows; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.K; sp.flat = true;
-        hq_conv_desc flatd = d;
-        flatd.R = flatd.S = 1;
-        flatd.C = d.R * d.S * d.C;
-        if ((st = build_sub(ctx, pw, s, sp, flatd, W, {0}, {0}, false, 1)) != HQ_OK) return bail(st);
+        const WeightPrep prep = [&](hq_sub_problem& sub) {
+          ctx->launches += 1;
+          return launch_prep_patch_weights(W, sub.wmat, d.K, d.R, d.S * d.C, RP, sub.p.Cpad, s);
+        };
+        if ((st = build_sub(ctx, pw, s, sp, d, W, {0}, {0}, false, 1, &prep)) != HQ_OK) return bail(st);
         hq_sub_problem& sub = pw->subs.back();
         sub.patch_K = Kp;
         sub.patch_RP = RP;
-        {  // the weight matrix in the slot layout of the patch rows, and its column sums
-          const uint32_t one = 1u;
-          cudaError_t e = launch_prep_patch_weights(W, sub.wmat, d.K, d.R, d.S * d.C, RP, sub.p.Cpad, s);
-          if (e == cudaSuccess) e = launch_corr(sub.wmat, sub.corr, d.K, 1, sub.p.Cpad, 1, 1, &one, 1, &one, 1, sub.p.corr_ld, s);
-          if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "patch weight preparation failed: %s", cudaGetErrorString(e)));
-          ctx->launches += 2;
-        }
         if ((st = dev_alloc(ctx, pw, (void**)&sub.patch_matrix, (size_t)rows * Kp)) != HQ_OK) return bail(st);
         *out = pw;
         return HQ_OK;

@@ -241,6 +241,88 @@ __global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restr
   }
 }
 
+// Second repacking for spatial filters over few channels (the RGB stem), cheaper than whole patch rows:
+// X2[n][m][j][u*SB + b], b = s*C + c < S*C, holds for output column j the horizontal filter window of input row
+// m*sh + u (sh = vertical stride; rows beyond the image and taps on horizontal padding hold the input zero point).
+// Over X2 the layer is a stride-1 convolution with ceil-range(R/sh) vertical taps, one output column wide, with
+// sh*SB "channels" -- a shape the tensor-core kernel stages by itself.  X2 is about the size of the layer's output.
+// Thread = one SB-byte slot: the S*C input bytes are contiguous, moved with aligned word loads and a funnel shift.
+__global__ void __launch_bounds__(256) row_window_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ X2, const hq_range_state* xq, int N,
+                                                         int H, int W, int C, int Hg, int Wo, int S, int sh, int stride_w, int pad_w, int SB) {
+  const int zx = xq->zero_point;
+  const uint32_t zx4 = ((uint32_t)zx & 0xffu) * 0x01010101u;
+  const int sc = S * C, nq = SB / 16;
+  const int64_t total = (int64_t)N * Hg * Wo * sh;
+  const int8_t* x_end = x + (int64_t)N * H * W * C;   // no load starts at or beyond this address
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int u = (int)(idx % sh);
+    int64_t t = idx / sh;
+    const int j = (int)(t % Wo);
+    t /= Wo;
+    const int m = (int)(t % Hg);
+    const int n = (int)(t / Hg);
+    const int hi = m * sh + u;
+    const int wi0 = j * stride_w - pad_w;
+    uint4* dst = reinterpret_cast<uint4*>(X2 + idx * SB);
+    if (hi >= H) {
+      for (int i = 0; i < nq; ++i) dst[i] = make_uint4(zx4, zx4, zx4, zx4);
+    } else if (wi0 >= 0 && wi0 + S <= W) {
+      const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
+      const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 3u) * 8u;
+      const uint32_t* a4 = reinterpret_cast<const uint32_t*>(reinterpret_cast<uintptr_t>(src) & ~(uintptr_t)3);
+      uint32_t prev = *a4;
+      for (int i = 0; i < nq; ++i) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const uint32_t* nxt = a4 + 4 * i + k + 1;
+          // bytes past the window only meet zero weights; an aligned word that starts inside the tensor is readable
+          const uint32_t next = (4 * (4 * i + k) < sc && reinterpret_cast<const int8_t*>(nxt) < x_end) ? *nxt : 0u;
+          w[k] = __funnelshift_r(prev, next, shb);
+          prev = next;
+        }
+        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    } else {
+      const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
+      for (int i = 0; i < nq; ++i) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          uint32_t word = 0;
+          for (int e = 0; e < 4; ++e) {
+            const int b = 16 * i + 4 * k + e;
+            int v = 0;
+            if (b < sc) {
+              const int q = b / C;
+              v = (wi0 + q >= 0 && wi0 + q < W) ? (int)src[b] : zx;
+            }
+            word |= ((uint32_t)v & 0xffu) << (8 * e);
+          }
+          w[k] = word;
+        }
+        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+}
+
+// weight matrix over the window tensor: Wmat[k][t][u*SB + b] = W[k][r][b] with r = (dh_min + t)*sh + u + pad_h, zero
+// where r is outside the filter or b >= S*C
+__global__ void prep_window_weights_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wmat, int K, int R, int SC, int sh, int SB, int ntaps,
+                                           int dh_min, int pad_h) {
+  const int Cg = sh * SB, ld = ntaps * Cg;
+  const int64_t total = (int64_t)K * ld;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int col = (int)(idx % ld);
+    const int k = (int)(idx / ld);
+    const int t = col / Cg, within = col - t * Cg;
+    const int u = within / SB, b = within - u * SB;
+    const int r = (dh_min + t) * sh + u + pad_h;
+    Wmat[idx] = (r >= 0 && r < R && b < SC) ? W[((int64_t)k * R + r) * SC + b] : (int8_t)0;
+  }
+}
+
 // weight matrix for the patch layout: Wmat[k][r*RP + j] = W[k][r][j], zero elsewhere (row pitch `ld` bytes)
 __global__ void prep_patch_weights_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wmat, int K, int R, int SC, int RP, int ld) {
   const int64_t total = (int64_t)K * ld;
@@ -547,6 +629,22 @@ cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state
   int blocks = (int)std::min<int64_t>(groups, 148 * 8);
   if (blocks < 1) blocks = 1;
   patch_matrix_kernel<<<blocks, 256, (size_t)kPatchPixels * Kp, s>>>(x, A, xq, N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w, Kp, RP);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_row_window(const int8_t* x, int8_t* X2, const hq_range_state* xq, int N, int H, int W, int C, int Hg, int Wo, int S, int sh,
+                              int stride_w, int pad_w, int SB, cudaStream_t s) {
+  const int64_t total = (int64_t)N * Hg * Wo * sh;
+  int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+  if (blocks < 1) blocks = 1;
+  row_window_kernel<<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w, SB);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_prep_window_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int sh, int SB, int ntaps, int dh_min, int pad_h,
+                                       cudaStream_t s) {
+  const int64_t total = (int64_t)K * ntaps * sh * SB;
+  prep_window_weights_kernel<<<(int)std::min<int64_t>((total + 255) / 256, 1024), 256, 0, s>>>(W, Wmat, K, R, SC, sh, SB, ntaps, dh_min, pad_h);
   return cudaGetLastError();
 }
 

@@ -155,6 +155,10 @@ cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, 
                         int nrowcls, const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s);
 cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state* xq, int N, int H, int W, int C, int Ho, int Wo, int R, int S,
                                 int stride_h, int stride_w, int pad_h, int pad_w, int Kp, int RP, cudaStream_t s);
+cudaError_t launch_row_window(const int8_t* x, int8_t* X2, const hq_range_state* xq, int N, int H, int W, int C, int Hg, int Wo, int S, int sh,
+                              int stride_w, int pad_w, int SB, cudaStream_t s);
+cudaError_t launch_prep_window_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int sh, int SB, int ntaps, int dh_min, int pad_h,
+                                       cudaStream_t s);
 cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s);
 cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
@@ -173,6 +177,7 @@ struct hq_ctx {
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
+  int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
   bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
   std::string err;
 };
@@ -191,6 +196,8 @@ struct hq_sub_problem {               // one kernel launch of a prepared convolu
   int8_t* patch_matrix = nullptr;     // [pixels][patch_K]: filter windows gathered by a pre-pass (C not a multiple of 16)
   int patch_K = 0;
   int patch_RP = 0;                   // bytes per filter-row slot in a patch-matrix row
+  int8_t* window = nullptr;           // [N][Hg][Wo][win_sh * win_SB]: horizontal filter windows of win_sh input rows per pixel
+  int win_sh = 0, win_SB = 0, win_Hg = 0;
 };
 
 struct hq_prepared_weights {

@@ -25,12 +25,14 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1):
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1):
     ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
+    ctx.set_option("repack", repack)        # how few-channel inputs are repacked; likewise
     try:
         g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
     finally:
         ctx.set_option("staging", -1)
+        ctx.set_option("repack", -1)
     o = OracleLayer(kind, W, shape, bias=bias, eta=eta)
     for t in range(iters):
         x = make_x(t)
@@ -104,6 +106,10 @@ FWD_CASES = {
     "5x5_c16": dict(N=1, H=11, W=11, Cin=16, K=48, R=5, S=5, stride=1, pad=2),
     "7x7_s2_c3_stem": dict(N=2, H=30, W=26, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
     "3x3_c5": dict(N=2, H=9, W=9, Cin=5, K=24, R=3, S=3, stride=1, pad=1),
+    "7x7_s2_c3_odd": dict(N=2, H=29, W=27, Cin=3, K=32, R=7, S=7, stride=2, pad=3),
+    "5x5_s2_c4_p1": dict(N=1, H=17, W=22, Cin=4, K=16, R=5, S=5, stride=2, pad=1),
+    "3x3_s4_c3": dict(N=2, H=21, W=19, Cin=3, K=16, R=3, S=3, stride=4, pad=1),
+    "5x5_s3_c3": dict(N=1, H=20, W=20, Cin=3, K=16, R=5, S=5, stride=3, pad=2),
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
     "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
@@ -126,6 +132,18 @@ def test_conv_fwd(ctx, name, staging):
     in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
     makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
     _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, staging=staging)
+
+
+@pytest.mark.parametrize("repack", [0, 1])
+@pytest.mark.parametrize("name", [n for n, c in FWD_CASES.items() if c["Cin"] % 16 != 0 and c.get("R", 1) > 1])
+def test_conv_fwd_few_channels_repacking(ctx, name, repack):
+    """Both repackings of few-channel inputs (whole filter patches; horizontal windows per input row) give the oracle's bytes."""
+    shape = dict(FWD_CASES[name])
+    r = synth.rng(104, len(name), shape["H"], repack)
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.image_like, synth.signed_activations, synth.relu_activations]
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, repack=repack)
 
 
 BWD_CASES = {
