@@ -686,7 +686,7 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
         auto floordiv = [](int a, int b) { return a >= 0 ? a / b : -((-a + b - 1) / b); };
         const int dh_min = floordiv(-d.pad_h, sh), dh_max = floordiv(d.R - 1 - d.pad_h, sh);
         const int Hg = (d.H + sh - 1) / sh;
-        if (Cg != 0 && dh_max - dh_min + 1 <= kMaxTaps && ctx->force_repack != 0) {
+        if (Cg != 0 && dh_max - dh_min + 1 <= kMaxTaps && ctx->force_repack != 0 && (int64_t)d.N * Hg * Wo * sh < ((int64_t)1 << 31)) {
           sp.n_img = d.N; sp.TH = Ho; sp.TW = Wo; sp.in_mul_h = sp.in_mul_w = 1;
           for (int t = dh_min; t <= dh_max; ++t) sp.dh.push_back(t);
           sp.dw = {0};

@@ -247,63 +247,71 @@ __global__ void __launch_bounds__(256) patch_matrix_kernel(const int8_t* __restr
 // Over X2 the layer is a stride-1 convolution with ceil-range(R/sh) vertical taps, one output column wide, with
 // sh*SB "channels" -- a shape the tensor-core kernel stages by itself.  X2 is about the size of the layer's output.
 // Thread = one SB-byte slot: the S*C input bytes are contiguous, moved with aligned word loads and a funnel shift.
+// Slot indices fit 32 bits (checked by the launcher); kWords = SB / 4 is a compile-time constant so that the slot
+// stays in registers.
+template <int kWords>
 __global__ void __launch_bounds__(256) row_window_kernel(const int8_t* __restrict__ x, int8_t* __restrict__ X2, const hq_range_state* xq, int N,
-                                                         int H, int W, int C, int Hg, int Wo, int S, int sh, int stride_w, int pad_w, int SB) {
+                                                         int H, int W, int C, int Hg, int Wo, int S, int sh, int stride_w, int pad_w) {
+  constexpr int SB = 4 * kWords;
   const int zx = xq->zero_point;
   const uint32_t zx4 = ((uint32_t)zx & 0xffu) * 0x01010101u;
-  const int sc = S * C, nq = SB / 16;
-  const int64_t total = (int64_t)N * Hg * Wo * sh;
-  const int8_t* x_end = x + (int64_t)N * H * W * C;   // no load starts at or beyond this address
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
-    const int u = (int)(idx % sh);
-    int64_t t = idx / sh;
-    const int j = (int)(t % Wo);
-    t /= Wo;
-    const int m = (int)(t % Hg);
-    const int n = (int)(t / Hg);
+  const int sc = S * C;
+  const int nload = (sc + 3) / 4 + 1;                       // aligned words that can hold window bytes
+  const int64_t total_words = ((int64_t)N * H * W * C + 3) >> 2;   // aligned words that start inside the tensor
+  const uint32_t per_row = (uint32_t)Wo * sh;             // slots of one (image, row group)
+  const int sh_log2 = 31 - __clz(sh);                     // sh is a power of two (checked when the layer is prepared)
+  // block = one (image, row group) at a time; thread = slot (output column j, sub-row u)
+  for (uint32_t rowi = blockIdx.x, rem = threadIdx.x; rowi < (uint32_t)N * Hg;) {
+    if (rem >= per_row) {   // next row group of this block
+      rowi += gridDim.x;
+      rem = threadIdx.x;
+      continue;
+    }
+    const uint32_t idx = rowi * per_row + rem;
+    const int j = (int)(rem >> sh_log2);
+    const int u = (int)(rem & (uint32_t)(sh - 1));
+    const int n = (int)(rowi / (uint32_t)Hg);
+    const int m = (int)(rowi - (uint32_t)n * Hg);
+    rem += blockDim.x;
     const int hi = m * sh + u;
     const int wi0 = j * stride_w - pad_w;
-    uint4* dst = reinterpret_cast<uint4*>(X2 + idx * SB);
+    uint32_t w[kWords];
     if (hi >= H) {
-      for (int i = 0; i < nq; ++i) dst[i] = make_uint4(zx4, zx4, zx4, zx4);
-    } else if (wi0 >= 0 && wi0 + S <= W) {
-      const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
-      const uint32_t shb = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 3u) * 8u;
-      const uint32_t* a4 = reinterpret_cast<const uint32_t*>(reinterpret_cast<uintptr_t>(src) & ~(uintptr_t)3);
-      uint32_t prev = *a4;
-      for (int i = 0; i < nq; ++i) {
-        uint32_t w[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const uint32_t* nxt = a4 + 4 * i + k + 1;
-          // bytes past the window only meet zero weights; an aligned word that starts inside the tensor is readable
-          const uint32_t next = (4 * (4 * i + k) < sc && reinterpret_cast<const int8_t*>(nxt) < x_end) ? *nxt : 0u;
-          w[k] = __funnelshift_r(prev, next, shb);
-          prev = next;
-        }
-        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
-      }
+      for (int i = 0; i < kWords; ++i) w[i] = zx4;
     } else {
-      const int8_t* src = x + (((int64_t)n * H + hi) * W + wi0) * C;
-      for (int i = 0; i < nq; ++i) {
-        uint32_t w[4];
+      // byte offset of the window's first tap from the tensor base (negative for windows that start on left padding of
+      // the first row), split into an aligned word index and a shift
+      const int64_t off = (((int64_t)n * H + hi) * W + wi0) * C;
+      const int64_t woff = off >> 2;                          // floor
+      const uint32_t shb = (uint32_t)(off & 3) * 8u;
+      const uint32_t* a4 = reinterpret_cast<const uint32_t*>(x) + woff;
+      // words [first, last) of this run exist in the tensor (an aligned word that starts inside it is readable)
+      const int first = woff < 0 ? (int)-woff : 0;
+      const int64_t left = total_words - woff;
+      const int last = left < (int64_t)nload ? (int)left : nload;
+      uint32_t ld[kWords + 1];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          uint32_t word = 0;
-          for (int e = 0; e < 4; ++e) {
-            const int b = 16 * i + 4 * k + e;
-            int v = 0;
-            if (b < sc) {
-              const int q = b / C;
-              v = (wi0 + q >= 0 && wi0 + q < W) ? (int)src[b] : zx;
-            }
-            word |= ((uint32_t)v & 0xffu) << (8 * e);
-          }
-          w[k] = word;
+      for (int i = 0; i <= kWords; ++i) ld[i] = (i >= first && i < last) ? __ldg(a4 + i) : 0u;
+#pragma unroll
+      for (int i = 0; i < kWords; ++i) w[i] = __funnelshift_r(ld[i], ld[i + 1], shb);
+      // taps on horizontal padding: bytes outside [lo_b, hi_b) of the slot hold the zero point
+      const int lo_b = (wi0 < 0 ? -wi0 : 0) * C;
+      const int hi_b = (wi0 + S > W ? W - wi0 : S) * C;
+      if (lo_b > 0 || hi_b < sc) {
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) {
+          const int klo = min(max(lo_b - 4 * i, 0), 4), khi = min(max(hi_b - 4 * i, 0), 4);   // valid bytes: [klo, khi)
+          const uint32_t below_hi = khi >= 4 ? 0xffffffffu : ((1u << (8 * khi)) - 1u);
+          const uint32_t below_lo = klo >= 4 ? 0xffffffffu : ((1u << (8 * klo)) - 1u);
+          const uint32_t keep = below_hi & ~below_lo;
+          w[i] = (w[i] & keep) | (zx4 & ~keep);
         }
-        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
+    uint4* dst = reinterpret_cast<uint4*>(X2 + (size_t)idx * SB);
+#pragma unroll
+    for (int i = 0; i < kWords / 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
   }
 }
 
@@ -635,9 +643,17 @@ cudaError_t launch_patch_matrix(const int8_t* x, int8_t* A, const hq_range_state
 cudaError_t launch_row_window(const int8_t* x, int8_t* X2, const hq_range_state* xq, int N, int H, int W, int C, int Hg, int Wo, int S, int sh,
                               int stride_w, int pad_w, int SB, cudaStream_t s) {
   const int64_t total = (int64_t)N * Hg * Wo * sh;
-  int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 32);
+  if (total >= (int64_t)1 << 31) return cudaErrorInvalidValue;   // checked when the layer is prepared
+  if ((sh & (sh - 1)) != 0) return cudaErrorInvalidValue;
+  int blocks = (int)std::min<int64_t>((int64_t)N * Hg, 148 * 64);
   if (blocks < 1) blocks = 1;
-  row_window_kernel<<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w, SB);
+  switch (SB) {
+    case 16: row_window_kernel<4><<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w); break;
+    case 32: row_window_kernel<8><<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w); break;
+    case 64: row_window_kernel<16><<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w); break;
+    case 128: row_window_kernel<32><<<blocks, 256, 0, s>>>(x, X2, xq, N, H, W, C, Hg, Wo, S, sh, stride_w, pad_w); break;
+    default: return cudaErrorInvalidValue;
+  }
   return cudaGetLastError();
 }
 

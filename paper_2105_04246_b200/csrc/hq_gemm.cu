@@ -53,12 +53,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
                                           uint32_t hint_ns = 200u) {
   if (mbar_try(bar, parity, hint_ns)) return true;
   const uint64_t t0 = global_timer_ns();
-  uint32_t spins = 0, nap = 32;
+  uint32_t spins = 0;
   for (;;) {
     if (mbar_try(bar, parity, hint_ns)) return true;
-    // back off: a waiting warp that keeps issuing takes issue slots from the epilogue warps of its sub-partition
-    __nanosleep(nap);
-    if (nap < hint_ns) nap += nap;
+    // A short fixed pause: the suspended try above already keeps a waiting warp off the issue slots; a growing
+    // back-off only adds wake-up latency to waits that sit on the critical path of every tile.
+    __nanosleep(32);
     if ((++spins & 15u) == 0u) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
@@ -634,16 +634,69 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           }
         }
       };
-      for (int ch = c_begin; ch < c_end; ++ch) {
-        int v[CW];
-        if (kiters > 0) {
+      // Warp-uniform conditions under which a pass is straight-line code: int8 output with 16-byte stores, finite
+      // parameters, no bias, every column of the pass inside the layer, correction table in shared memory (it holds
+      // zeros when the input zero point is 0).  Rows outside the image (tile padding) are computed like the others
+      // and only kept out of the statistics and the store.
+      const bool lean = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.zc_in_smem &&
+                        p.corr != nullptr && col0 + c_end * CW <= p.Nout;
+      if (lean) {
+        const int32_t* zrow = zc_s;
+        if (row_valid) {
+          const int rc = p.cls_in_smem ? cls_s[i] : (p.rowcls ? p.rowcls[i] : 0);
+          const int cc = p.cls_in_smem ? cls_s[512 + j] : (p.colcls ? p.colcls[j] : 0);
+          zrow = zc_s + (rc * p.ncolcls + cc) * p.corr_ld;
+        }
+        zrow += col0;
+        int8_t* dst_row = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0;
+        int tmn = INT32_MAX, tmx = INT32_MIN;
+        for (int ch = c_begin; ch < c_end; ++ch) {
+          int v[CW];
           tmem_ld16(taddr + ch * CW, v);
           tmem_ld_wait();
-        } else {
+          const int c0 = ch * CW;
+#pragma unroll
+          for (int e = 0; e < CW; e += 4) {
+            const int4 cr = *reinterpret_cast<const int4*>(zrow + c0 + e);
+            v[e + 0] -= cr.x;
+            v[e + 1] -= cr.y;
+            v[e + 2] -= cr.z;
+            v[e + 3] -= cr.w;
+          }
+          int lo[2], hi[2];
+#pragma unroll
+          for (int g = 0; g < 2; ++g) {
+            const int* x = v + 8 * g;
+            lo[g] = min(__vimin3_s32(__vimin3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimin3_s32(x[5], x[6], x[7]));
+            hi[g] = max(__vimax3_s32(__vimax3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimax3_s32(x[5], x[6], x[7]));
+          }
+          tmn = __vimin3_s32(tmn, lo[0], lo[1]);
+          tmx = __vimax3_s32(tmx, hi[0], hi[1]);
+          uint32_t w[CW / 4];
+#pragma unroll
+          for (int e = 0; e < CW / 4; ++e)
+            w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
+                             requant_acc<true>(v[4 * e + 3], q));
+          if (row_valid) *reinterpret_cast<uint4*>(dst_row + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (row_valid) {
+          mn = min(mn, tmn);
+          mx = max(mx, tmx);
+        }
+      } else if (kiters > 0) {
+        for (int ch = c_begin; ch < c_end; ++ch) {
+          int v[CW];
+          tmem_ld16(taddr + ch * CW, v);
+          tmem_ld_wait();
+          process(ch * CW, v);
+        }
+      } else {
+        for (int ch = c_begin; ch < c_end; ++ch) {
+          int v[CW];
 #pragma unroll
           for (int e = 0; e < CW; ++e) v[e] = 0;
+          process(ch * CW, v);
         }
-        process(ch * CW, v);
       }
       if (kiters > 0) {
         tc_fence_before();
