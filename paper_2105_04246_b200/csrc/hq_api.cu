@@ -140,11 +140,16 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     }
   if (sp.Cin % 16 != 0) return fail(ctx, HQ_ERR_UNSUPPORTED, "reduction length per tap (%d) must be a multiple of 16", sp.Cin);
   p.BK = (sp.Cin % 128 == 0) ? 128 : 64;
+  // a single-tap layer moves few bytes per copy-engine request: prefer 128-byte rows when that takes fewer copies
+  // (the padded reduction steps meet zero weights and zero-filled operand bytes)
+  if (p.ntaps == 1 && ceil_div(sp.Cin, 128) < ceil_div(sp.Cin, 64)) p.BK = 128;
   p.swizzle64 = p.BK == 64;
   p.Cpad = round_up(sp.Cin, p.BK);
   p.chunks_per_tap = p.Cpad / p.BK;
   p.Nout = sp.Nout;
-  const int ncol = ceil_div(sp.Nout, 256);
+  // column tiles: as wide as the MMA allows, except for very short reductions, where the epilogue is the bottleneck and
+  // narrower tiles give it four or more accumulator buffers to work on
+  const int ncol = ceil_div(sp.Nout, p.ntaps * p.Cpad <= 128 ? 128 : 256);
   p.BN = round_up(ceil_div(sp.Nout, ncol), 16);
   p.tiles_col = ceil_div(sp.Nout, p.BN);
   const int64_t nt = (int64_t)p.tiles_n * p.tiles_h * p.tiles_w * p.tiles_col;
@@ -241,8 +246,17 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   }
   if (p.mode == kModeTap) {
     p.stage_bytes_a = (uint32_t)kTileM * p.BK;
-    p.stages_a = (int)std::min<uint32_t>(kMaxStagesA, ring_budget / (p.stage_bytes_a + p.stage_bytes_b));
-    p.stages_b = 0;
+    // a small weight matrix stays in shared memory for the whole kernel; the ring then carries operand A only
+    const int kiters = p.ntaps * p.chunks_per_tap;
+    const uint64_t b_all = (uint64_t)p.tiles_col * kiters * p.stage_bytes_b;
+    if (kiters > 0 && p.tiles_col * kiters <= kMaxStagesB && b_all <= 64u * 1024u && b_all + 6ull * p.stage_bytes_a <= ring_budget) {
+      p.b_resident = 1;
+      p.stages_b = p.tiles_col * kiters;
+      p.stages_a = (int)std::min<uint64_t>(kMaxStagesA, (ring_budget - b_all) / p.stage_bytes_a);
+    } else {
+      p.stages_a = (int)std::min<uint32_t>(kMaxStagesA, ring_budget / (p.stage_bytes_a + p.stage_bytes_b));
+      p.stages_b = 0;
+    }
     if (p.stages_a < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
     p.producer_lanes = std::min(4, p.stages_a);
   }

@@ -174,8 +174,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 
   const uint32_t ring_a = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const bool halo = p.mode == kModeHalo;
-  // kModeTap: one ring, stage = [A tile | B tile]; kModeHalo: patch ring, then weight ring
-  const uint32_t a_stride = halo ? p.stage_bytes_a : p.stage_bytes_a + p.stage_bytes_b;
+  // kModeTap: one ring, stage = [A tile | B tile] (A tile alone when the weights are resident, which then follow
+  // the ring); kModeHalo: patch ring, then weight ring
+  const uint32_t a_stride = (halo || p.b_resident) ? p.stage_bytes_a : p.stage_bytes_a + p.stage_bytes_b;
   const uint32_t ring_b = ring_a + (uint32_t)p.stages_a * a_stride;
   const uint32_t bar0 = smem_u32(bars);
   auto a_full = [&](int s) { return bar0 + 8u * s; };
@@ -281,7 +282,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
               if (elect_one()) {
                 mbar_expect_tx(a_full(stage), a_stride);
                 tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
-                tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+                if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
               }
               if (++stage == p.stages_a) {
                 stage = 0;
@@ -295,7 +296,20 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     __syncwarp();
   } else if (warp == 2) {
     // ------------------------------ weight producer (kModeHalo) ------------------------------
-    if (halo && kiters > 0) {
+    if (!halo && p.b_resident && kiters > 0) {
+      // kModeTap with a small weight matrix: every (column tile, tap, chunk) box once, in the order the issuer uses them
+      if (my_tiles > 0) {
+        for (int ct = 0; ct < p.tiles_col; ++ct)
+          for (int ki = 0; ki < kiters; ++ki) {
+            const int t = ki / p.chunks_per_tap, cc = ki - t * p.chunks_per_tap;
+            const int slot = ct * kiters + ki;
+            if (elect_one()) {
+              mbar_expect_tx(b_full(slot), p.stage_bytes_b);
+              tma_load_2d(ring_b + slot * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, ct * p.BN, b_full(slot));
+            }
+          }
+      }
+    } else if (halo && kiters > 0) {
       if (p.b_resident) {
         if (my_tiles > 0) {
           for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
@@ -428,13 +442,23 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           }
           if (!ok) break;
         } else {
+          uint64_t bres = bdesc0;
+          if (resident) {
+            if (first) {   // the whole weight matrix arrives once
+              for (int ki = 0; ki < p.stages_b && ok; ++ki) ok = warp_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            const int t0 = fdiv(tile, p.fd_tiles_col);
+            bres += (uint64_t)((tile - t0 * p.tiles_col) * kiters) * bstep16;
+          }
           for (int ki = 0; ki < kiters; ++ki) {
             ok = warp_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait, 200u);
             if (!ok) break;
             tc_fence_after();
             const uint32_t sa = ring_a + stage * a_stride;
             const uint64_t adesc = make_smem_desc(sa, sw64);
-            const uint64_t bdesc = make_smem_desc(sa + p.stage_bytes_a, sw64);
+            const uint64_t bdesc = resident ? bres + (uint64_t)ki * bstep16 : make_smem_desc(sa + p.stage_bytes_a, sw64);
             if (elect_one()) {
 #pragma unroll
               for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
