@@ -309,6 +309,7 @@ def run_gpu(args):
     ctx = hq.Context(local)
     if args.no_overlap:
         ctx.set_option("overlap_launches", 0)
+    ctx.set_option("depthwise", args.depthwise)
     peaks, peak_kind = load_peaks()
     name = args.workload
     pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg5": 2}[name]
@@ -461,6 +462,7 @@ def run_profile(args):
     ctx = hq.Context(0)
     if args.no_overlap:
         ctx.set_option("overlap_launches", 0)
+    ctx.set_option("depthwise", args.depthwise)
     wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0)
     stream = torch.cuda.current_stream(dev)
     for j in range(2):
@@ -501,6 +503,8 @@ def main():
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--depthwise", type=int, default=-1, choices=[-1, 0, 1],
+                    help="depthwise layers: -1 library's choice, 0 CUDA-core kernel, 1 dense slices on the tensor cores")
     ap.add_argument("--no-overlap", action="store_true",
                     help="ordinary launches instead of programmatic stream serialization (set-up of a kernel overlapping its predecessor's tail)")
     ap.add_argument("--profile", action="store_true",

@@ -121,6 +121,9 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
  *   "staging": how convolutions prepared AFTER this call bring their input to the MAC array (the
  *              paper's "loaded into the MAC array", Sec. 3.1): -1 = chosen per layer (default),
  *              0 = one copy per filter tap, 1 = input rows kept resident wherever the layer allows.
+ *   "depthwise": how depthwise layers prepared AFTER this call run: -1 = library's choice (default; the
+ *              CUDA-core kernel), 0 = CUDA-core kernel, 1 = on the tensor cores as dense layers with
+ *              diagonal filters, one per 64-channel slice.
  *   "repack":  how spatial filters over a channel count that is not a multiple of 16 (the RGB stem),
  *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows

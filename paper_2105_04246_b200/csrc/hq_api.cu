@@ -306,10 +306,11 @@ hq_status encode_b(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* wmat, i
 }
 
 // operand A: flat [rows][C] view, or NHWC image with one box per tile (traversal strides for strided layers)
-hq_status encode_a(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* base, int C, int W, int H, int N, CUtensorMap* m) {
+hq_status encode_a(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* base, int C, int W, int H, int N, CUtensorMap* m, int pitch = 0) {
   const GemmParams& p = sub.p;
+  if (pitch == 0) pitch = C;   // bytes from one pixel to the next (a channel slice of a wider tensor has pitch > C)
   uint64_t dims[4] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)N};
-  uint64_t strides[3] = {(uint64_t)C, (uint64_t)C * W, (uint64_t)C * W * H};
+  uint64_t strides[3] = {(uint64_t)pitch, (uint64_t)pitch * W, (uint64_t)pitch * W * H};
   uint32_t box[4] = {(uint32_t)p.BK, (uint32_t)(p.Wt * sub.a_stride_w), (uint32_t)(p.Ht * sub.a_stride_h), (uint32_t)p.Nt};
   uint32_t es[4] = {1, (uint32_t)sub.a_stride_w, (uint32_t)sub.a_stride_h, 1};
   if (p.mode == kModeHalo) {  // NR padded rows of P pixels of one image
@@ -443,6 +444,14 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
                                      desc->stride_w, desc->pad_w, sub.win_SB, s));
       ctx->launches += 1;
       st = encode_a(ctx, sub, sub.window, sub.win_sh * sub.win_SB, Wo, sub.win_Hg, desc->N, &ta);
+    } else if (sub.chans > 0) {
+      // depthwise: this launch is the dense layer over the channel slice [chan0, chan0 + chans) of input and output
+      st = encode_a(ctx, sub, in + sub.chan0, sub.chans, aW, aH, desc->N, &ta, desc->C);
+      if (st != HQ_OK) return st;
+      void* o = out_mode == kOutInt8 ? (void*)((int8_t*)out + sub.chan0) : (void*)((uint32_t*)out + sub.chan0);
+      st = launch_sub(ctx, s, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode);
+      if (st != HQ_OK) return st;
+      continue;
     } else if (sub.a_flat) {
       const int64_t rows = (int64_t)desc->N * aH * aW / sub.gfold;
       st = encode_a(ctx, sub, in, aC * sub.gfold, (int)rows, 1, 1, &ta);
@@ -604,6 +613,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     ctx->force_mode = value;
     return HQ_OK;
   }
+  if (std::string(key) == "depthwise") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "depthwise must be -1, 0 or 1");
+    ctx->force_depthwise = value;
+    return HQ_OK;
+  }
   if (std::string(key) == "repack") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "repack must be -1, 0 or 1");
     ctx->force_repack = value;
@@ -653,6 +667,38 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   if (d.groups != 1) {
     if (dir != HQ_DIR_FWD) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data is not implemented"));
     if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise needs C %% 16 == 0"));
+  }
+  // Optional form of a depthwise layer on the tensor cores: ceil(C / 64) dense layers, one per 64-channel slice of
+  // input and output, each with a weight matrix that is zero off the channel diagonal (the int32 sums are the same).
+  // Measured on the 56x56x144 layer it is only on a par with the CUDA-core kernel (N = 64 MMAs are bound by
+  // shared-memory reads of the pixel operand), so it is not chosen by default.
+  const bool dw_dense = d.groups != 1 && ctx->force_depthwise == 1;
+  if (dw_dense) {
+    for (int c0 = 0; c0 < d.C; c0 += 64) {
+      const int cw = std::min(64, d.C - c0);
+      int8_t* Wd = nullptr;
+      if ((st = dev_alloc(ctx, pw, (void**)&Wd, (size_t)cw * d.R * d.S * cw)) != HQ_OK) return bail(st);
+      cudaError_t e = launch_dw_dense(W, Wd, d.R * d.S, c0, cw, s);
+      if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "depthwise weight expansion failed: %s", cudaGetErrorString(e)));
+      ctx->launches += 1;
+      hq_conv_desc dd = d;
+      dd.C = dd.K = cw;
+      dd.groups = 1;
+      SubSpec sp{};
+      std::vector<int> tr, ts;
+      sp.n_img = d.N; sp.TH = Ho; sp.TW = Wo; sp.in_mul_h = d.stride_h; sp.in_mul_w = d.stride_w;
+      for (int r = 0; r < d.R; ++r) { sp.dh.push_back(r - d.pad_h); tr.push_back(r); }
+      for (int q = 0; q < d.S; ++q) { sp.dw.push_back(q - d.pad_w); ts.push_back(q); }
+      sp.a_H = d.H; sp.a_W = d.W; sp.Cin = cw; sp.Nout = cw;
+      sp.out_H = Ho; sp.out_W = Wo; sp.os_h = sp.os_w = 1; sp.oa_h = sp.oa_w = 0; sp.ldY = d.C; sp.flat = false;
+      if ((st = build_sub(ctx, pw, s, sp, dd, Wd, tr, ts, false, 1)) != HQ_OK) return bail(st);
+      pw->subs.back().chan0 = c0;
+      pw->subs.back().chans = cw;
+    }
+    *out = pw;
+    return HQ_OK;
+  }
+  if (d.groups != 1 && !dw_dense) {
     pw->depthwise = true;
     std::vector<int> dh, dw;
     for (int r = 0; r < d.R; ++r) dh.push_back(r - d.pad_h);

@@ -178,6 +178,17 @@ __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict_
   }
 }
 
+// dense form of the depthwise filter of channels [c0, c0 + cw): Wd[k][tap][c] = (c == k) ? W[c0 + k][tap] : 0
+__global__ void dw_dense_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wd, int taps, int c0, int cw) {
+  const int total = cw * taps * cw;
+  for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+    const int c = idx % cw;
+    const int kt = idx / cw;
+    const int k = kt / taps, t = kt - k * taps;
+    Wd[idx] = c == k ? W[(int64_t)(c0 + k) * taps + t] : (int8_t)0;
+  }
+}
+
 // ---- operand repacking for shapes no TMA box can address ------------------------------------------
 // A[m][r*RP + j], j = s*C + c < S*C: the filter window of output pixel m, one filter row per RP-byte slot
 // (RP = S*C rounded up to 8).  Taps on padding hold the input zero point (real zero); slot bytes beyond S*C hold
@@ -611,6 +622,12 @@ cudaError_t launch_corr(const int8_t* Wmat, int32_t* corr, int Nout, int ntaps, 
   for (int i = 0; i < ncolcls; ++i) m.col[i] = colmasks[i];
   const int total = nrowcls * ncolcls * Nout;
   corr_kernel<<<(total + 7) / 8, 256, 0, s>>>(Wmat, corr, Nout, ntaps, Cpad, nrowtaps, ncoltaps, m, nrowcls, ncolcls, corr_ld);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s) {
+  const int total = cw * taps * cw;
+  dw_dense_kernel<<<std::min((total + 255) / 256, 1024), 256, 0, s>>>(W, Wd, taps, c0, cw);
   return cudaGetLastError();
 }
 

@@ -161,6 +161,7 @@ cudaError_t launch_prep_window_weights(const int8_t* W, int8_t* Wmat, int K, int
                                        cudaStream_t s);
 cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s);
 cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
+cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
                            const uint32_t* colmasks, int ncolcls, cudaStream_t s);
 
@@ -177,6 +178,7 @@ struct hq_ctx {
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
+  int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
   bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
   std::string err;
@@ -198,6 +200,7 @@ struct hq_sub_problem {               // one kernel launch of a prepared convolu
   int patch_RP = 0;                   // bytes per filter-row slot in a patch-matrix row
   int8_t* window = nullptr;           // [N][Hg][Wo][win_sh * win_SB]: horizontal filter windows of win_sh input rows per pixel
   int win_sh = 0, win_SB = 0, win_Hg = 0;
+  int chan0 = 0, chans = 0;           // depthwise on the tensor cores: this launch covers channels [chan0, chan0 + chans)
 };
 
 struct hq_prepared_weights {

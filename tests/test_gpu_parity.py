@@ -25,14 +25,16 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1):
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1):
     ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
     ctx.set_option("repack", repack)        # how few-channel inputs are repacked; likewise
+    ctx.set_option("depthwise", depthwise)  # CUDA-core kernel or dense expansion on the tensor cores; likewise
     try:
         g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
     finally:
         ctx.set_option("staging", -1)
         ctx.set_option("repack", -1)
+        ctx.set_option("depthwise", -1)
     o = OracleLayer(kind, W, shape, bias=bias, eta=eta)
     for t in range(iters):
         x = make_x(t)
@@ -113,6 +115,8 @@ FWD_CASES = {
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
     "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
+    "dw5x5_c48": dict(N=1, H=13, W=9, Cin=48, K=48, R=5, S=5, stride=1, pad=2, groups=48),
+    "dw3x3_c320": dict(N=1, H=7, W=7, Cin=320, K=320, R=3, S=3, stride=1, pad=1, groups=320),
 }
 
 
@@ -132,6 +136,18 @@ def test_conv_fwd(ctx, name, staging):
     in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
     makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
     _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, staging=staging)
+
+
+@pytest.mark.parametrize("depthwise", [0, 1])
+@pytest.mark.parametrize("name", [n for n, c in FWD_CASES.items() if c.get("groups", 1) != 1])
+def test_depthwise_both_paths(ctx, name, depthwise):
+    """The CUDA-core depthwise kernel and the dense (diagonal filter) form on the tensor cores give the oracle's bytes."""
+    shape = dict(FWD_CASES[name])
+    r = synth.rng(105, len(name), shape["H"], depthwise)
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, depthwise=depthwise)
 
 
 @pytest.mark.parametrize("repack", [0, 1])
