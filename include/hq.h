@@ -124,6 +124,9 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
  *   "depthwise": how depthwise layers prepared AFTER this call run: -1 = library's choice (default; the
  *              CUDA-core kernel), 0 = CUDA-core kernel, 1 = on the tensor cores as dense layers with
  *              diagonal filters, one per 64-channel slice.
+ *   "depthwise_staging": CUDA-core depthwise 3x3 stride-1 layers (read at every call): -1 = library's
+ *              choice (default), 0 = direct global loads, 1 = input patches staged in shared memory by TMA
+ *              where the shape allows.
  *   "repack":  how spatial filters over a channel count that is not a multiple of 16 (the RGB stem),
  *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows

@@ -421,6 +421,46 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     p.stride_h = desc->stride_h; p.stride_w = desc->stride_w; p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
     p.x = in; p.w = pw->dw_w; p.corr = pw->dw_corr; p.rowcls = pw->dw_rowcls; p.colcls = pw->dw_colcls; p.ncolcls = pw->dw_ncolcls;
     p.xq = inq; p.w_scale = w_scale; p.yq = outq; p.out = out;
+    p.status = ctx->d_status;
+    // 3x3 stride 1 with at most 256 channels: output tiles of 4 rows whose input patch one TMA box stages in shared memory
+    if (desc->R == 3 && desc->S == 3 && desc->stride_h == 1 && desc->stride_w == 1 && desc->C <= 256 && ctx->force_dw_tiled != 0) {
+      p.TR = 4;
+      const int budget = 50 * 1024;   // two patches + tables per CTA, two CTAs per SM
+      int twt = (budget / (desc->C * (p.TR + 2)) - 2) / 8 * 8;
+      twt = std::min(twt, std::min(round_up(Wo, 8), 248));
+      if (twt >= 8) {
+        p.TWt = twt;
+        p.tiles_h = ceil_div(Ho, p.TR);
+        p.tiles_w = ceil_div(Wo, p.TWt);
+        p.ncls = pw->dw_ncls;
+        p.patch_bytes = (uint32_t)desc->C * (uint32_t)(p.TWt + 2) * (uint32_t)(p.TR + 2);
+        p.patch_stride = (p.patch_bytes + 127u) & ~127u;
+        // strips of 8 pixels per tile are dealt to `slots` thread groups: the divisor of the strip count that gives
+        // the most threads within 512
+        const int strips = p.TR * (p.TWt / 8), cwords = desc->C / 4;
+        p.slots = 1;
+        for (int k = 1; k <= strips; ++k)
+          if (strips % k == 0 && k * cwords <= 512 && k * cwords <= 320) p.slots = k;
+        if (p.slots * cwords < 128)
+          for (int k = 1; k <= strips; ++k)
+            if (k * cwords <= 512) p.slots = k;
+        const int64_t n_tiles = (int64_t)desc->N * p.tiles_h * p.tiles_w;
+        if (n_tiles <= INT32_MAX && depthwise_tiled_smem_bytes(p) <= 200u * 1024u) {
+          CUtensorMap tm;
+          uint64_t dims[4] = {(uint64_t)desc->C, (uint64_t)desc->W, (uint64_t)desc->H, (uint64_t)desc->N};
+          uint64_t strides[3] = {(uint64_t)desc->C, (uint64_t)desc->C * desc->W, (uint64_t)desc->C * desc->W * desc->H};
+          uint32_t box[4] = {(uint32_t)desc->C, (uint32_t)(p.TWt + 2), (uint32_t)(p.TR + 2), 1u};
+          uint32_t es[4] = {1, 1, 1, 1};
+          CUresult r = ctx->encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(in), dims, strides, box, es,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+          if (r != CUDA_SUCCESS) return fail(ctx, HQ_ERR_CUDA, "tensor map encoding failed (CUresult %d)", (int)r);
+          HQ_CUDA(ctx, launch_depthwise_tiled(p, tm, out_mode, ctx->num_sms, s));
+          ctx->launches += 1;
+          return HQ_OK;
+        }
+      }
+    }
     HQ_CUDA(ctx, launch_depthwise(p, out_mode, ctx->num_sms, s, false));
     ctx->launches += 1;
     return HQ_OK;
@@ -583,7 +623,7 @@ __attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int dev
   ctx->scratch_elems = 4096;
   if (cudaMalloc((void**)&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc((void**)&ctx->d_scratch, ctx->scratch_elems * sizeof(int32_t)) != cudaSuccess ||
-      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess) {
+      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_scratch) cudaFree(ctx->d_scratch);
     delete ctx;
@@ -611,6 +651,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "staging") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "staging must be -1, 0 or 1");
     ctx->force_mode = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "depthwise_staging") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "depthwise_staging must be -1, 0 or 1");
+    ctx->force_dw_tiled = value;
     return HQ_OK;
   }
   if (std::string(key) == "depthwise") {
@@ -709,6 +754,7 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
     border_classes(Wo, d.stride_w, dw, d.W, colcls, cm);
     if (rm.size() > 16 || cm.size() > 16) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes"));
     pw->dw_ncolcls = (int)cm.size();
+    pw->dw_ncls = (int)(rm.size() * cm.size());
     if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_w, (size_t)d.C * d.R * d.S)) != HQ_OK) return bail(st);
     if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_corr, rm.size() * cm.size() * d.C * sizeof(int32_t))) != HQ_OK) return bail(st);
     cudaError_t e = launch_dw_prep(W, pw->dw_w, pw->dw_corr, d.C, d.R, d.S, rm.data(), (int)rm.size(), cm.data(), (int)cm.size(), s);

@@ -6,6 +6,7 @@
 
 #include <algorithm>
 
+#include "hq_device.cuh"
 #include "hq_internal.h"
 #include "hq_quant.cuh"
 
@@ -583,6 +584,166 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
   }
 }
 
+// 3x3 stride-1 depthwise with the input staged in shared memory.  A CTA walks over output tiles of TR rows x TWt
+// columns; one TMA box brings the (TR + 2) x (TWt + 2) pixel patch of all C channels (padding pixels arrive as
+// zeros), double buffered, so the loads of the next tile run under the arithmetic of this one.  Thread = one
+// 32-bit channel word (4 channels) x strips of 8 consecutive output pixels of one row; its 36 weights stay in
+// registers, each pre-shifted into its byte lane so that one dp4a against an input word multiplies exactly one
+// channel.  The accumulators start at minus the zero-point correction of the pixel's border class (table in
+// shared memory, already multiplied by the input zero point), so the epilogue is statistics, requantization, store.
+template <int kOut>
+__global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams p, const __grid_constant__ CUtensorMap tmap) {
+  extern __shared__ uint8_t dsm_raw[];
+  __shared__ __align__(8) uint64_t full_bar[2];
+  __shared__ int abort_s;
+  __shared__ int red_min[16], red_max[16];
+  const uint32_t patch0 = (smem_u32(dsm_raw) + 127u) & ~127u;
+  uint8_t* gen = dsm_raw + (patch0 - smem_u32(dsm_raw));
+  int32_t* zc_s = reinterpret_cast<int32_t*>(gen + 2u * p.patch_stride);
+  uint8_t* rcls_s = reinterpret_cast<uint8_t*>(zc_s + p.ncls * p.C);
+  uint8_t* ccls_s = rcls_s + p.Ho;
+  volatile int* abort_flag = &abort_s;
+  const int CW = p.C / 4;
+  const int cw = threadIdx.x % CW, slot = threadIdx.x / CW;
+  const uint32_t bar0 = smem_u32(full_bar);
+  if (threadIdx.x == 0) {
+    abort_s = 0;
+    mbar_init(bar0, 1);
+    mbar_init(bar0 + 8u, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap) : "memory");
+  }
+  __syncthreads();
+  grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
+
+  const int total = p.N * p.tiles_h * p.tiles_w;
+  auto issue = [&](int tile, int buf) {   // one thread: the patch of `tile` into buffer `buf`
+    const int tw = tile % p.tiles_w;
+    const int th = (tile / p.tiles_w) % p.tiles_h;
+    const int n = tile / (p.tiles_w * p.tiles_h);
+    mbar_expect_tx(bar0 + 8u * buf, p.patch_bytes);
+    tma_load_4d(patch0 + buf * p.patch_stride, &tmap, 0, tw * p.TWt - p.pad_w, th * p.TR - p.pad_h, n, bar0 + 8u * buf);
+  };
+  if (threadIdx.x == 0) {
+    if ((int)blockIdx.x < total) issue(blockIdx.x, 0);
+    if ((int)(blockIdx.x + gridDim.x) < total) issue(blockIdx.x + gridDim.x, 1);
+  }
+  QParams q;
+  q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
+  q.zx = p.xq->zero_point;
+  q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
+  q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  qparams_finish(q);
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
+  for (int i = threadIdx.x; i < p.ncls * p.C; i += blockDim.x) zc_s[i] = q.zx * p.corr[i];
+  for (int i = threadIdx.x; i < p.Ho; i += blockDim.x) rcls_s[i] = p.rowcls[i];
+  for (int i = threadIdx.x; i < p.Wo; i += blockDim.x) ccls_s[i] = p.colcls[i];
+  int wsel[9][4];   // weight of (tap, channel k) in byte lane k
+  const bool worker = slot < p.slots;
+  if (worker) {
+#pragma unroll
+    for (int t = 0; t < 9; ++t) {
+      const uint32_t w4 = *reinterpret_cast<const uint32_t*>(p.w + (int64_t)t * p.C + cw * 4);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) wsel[t][k] = (int)(w4 & (0xffu << (8 * k)));
+    }
+  }
+  __syncthreads();   // tables complete
+
+  int mn = INT32_MAX, mx = INT32_MIN;
+  const int box_w = p.TWt + 2;
+  const int ngw = p.TWt / kDwPix;
+  const int strips = p.TR * ngw;
+  const int pix_stride = p.C;   // bytes from one patch pixel to the next
+  int it = 0;
+  for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++it) {
+    const int buf = it & 1;
+    bool ok = mbar_wait(bar0 + 8u * buf, (uint32_t)(it >> 1) & 1u, abort_flag, p.status, kAsyncDepthwiseFullWait, 1000u);
+    ok = __syncthreads_and(ok) != 0;   // one decision for the whole CTA
+    if (!ok) break;
+    const int tw = tile % p.tiles_w;
+    const int th = (tile / p.tiles_w) % p.tiles_h;
+    const int n = tile / (p.tiles_w * p.tiles_h);
+    const uint8_t* patch = gen + buf * p.patch_stride + cw * 4;
+    if (worker) {
+      for (int s = slot; s < strips; s += p.slots) {
+        const int row = s / ngw, g = s - row * ngw;
+        const int ho = th * p.TR + row;
+        const int wo0 = tw * p.TWt + g * kDwPix;
+        if (ho >= p.Ho || wo0 >= p.Wo) continue;
+        const int rc = rcls_s[ho] * p.ncolcls;
+        int acc[kDwPix][4];
+#pragma unroll
+        for (int j = 0; j < kDwPix; ++j) {
+          const int wo = min(wo0 + j, p.Wo - 1);
+          const int4 zc = *reinterpret_cast<const int4*>(zc_s + (rc + ccls_s[wo]) * p.C + cw * 4);
+          acc[j][0] = -zc.x;
+          acc[j][1] = -zc.y;
+          acc[j][2] = -zc.z;
+          acc[j][3] = -zc.w;
+        }
+#pragma unroll
+        for (int r = 0; r < 3; ++r) {
+          const uint8_t* pr = patch + ((row + r) * box_w + g * kDwPix) * pix_stride;
+          int xw[kDwPix + 2];
+#pragma unroll
+          for (int j = 0; j < kDwPix + 2; ++j) xw[j] = *reinterpret_cast<const int*>(pr + j * pix_stride);
+#pragma unroll
+          for (int sx = 0; sx < 3; ++sx)
+#pragma unroll
+            for (int j = 0; j < kDwPix; ++j)
+#pragma unroll
+              for (int k = 0; k < 4; ++k) acc[j][k] = __dp4a(xw[j + sx], wsel[r * 3 + sx][k], acc[j][k]);
+        }
+        const int64_t o0 = (((int64_t)n * p.Ho + ho) * p.Wo + wo0) * p.C + cw * 4;
+#pragma unroll
+        for (int j = 0; j < kDwPix; ++j) {
+          if (wo0 + j < p.Wo) {
+            mn = min(__vimin3_s32(mn, acc[j][0], acc[j][1]), min(acc[j][2], acc[j][3]));
+            mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
+            const int64_t o = o0 + (int64_t)j * p.C;
+            if constexpr (kOut == kOutInt8) {
+              const uint32_t w = q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q),
+                                                    requant_acc<true>(acc[j][2], q), requant_acc<true>(acc[j][3], q))
+                                        : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
+                                                    requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+              *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
+            } else {
+              uint32_t w[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(acc[j][k]), q.s_acc)) : (uint32_t)acc[j][k];
+              *reinterpret_cast<uint4*>(reinterpret_cast<uint32_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+    }
+    __syncthreads();   // every thread is done with this buffer
+    if (threadIdx.x == 0 && tile + 2 * (int)gridDim.x < total) issue(tile + 2 * gridDim.x, buf);
+  }
+  grid_launch_dependents();   // the successor may take the SMs that free up from here on
+  mn = __reduce_min_sync(0xffffffffu, mn);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    red_min[warp] = mn;
+    red_max[warp] = mx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int e = 1; e < (int)((blockDim.x + 31) >> 5); ++e) {
+      mn = min(mn, red_min[e]);
+      mx = max(mx, red_max[e]);
+    }
+    if (mn <= mx) {
+      atomicMin(&p.yq->acc_min, mn);
+      atomicMax(&p.yq->acc_max, mx);
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap) {
@@ -686,6 +847,32 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
   int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
   if (blocks < 1) blocks = 1;
   pad_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, rows, K, Kp);
+  return cudaGetLastError();
+}
+
+uint32_t depthwise_tiled_smem_bytes(const DwParams& p) {
+  return 2u * p.patch_stride + (uint32_t)p.ncls * p.C * 4u + (uint32_t)p.Ho + (uint32_t)p.Wo + 256u;
+}
+
+cudaError_t depthwise_tiled_set_smem_attr(uint32_t smem_bytes) {
+  cudaError_t e = cudaFuncSetAttribute(depthwise3x3_tiled_kernel<kOutInt8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(depthwise3x3_tiled_kernel<kOutF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(depthwise3x3_tiled_kernel<kOutAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+}
+
+cudaError_t launch_depthwise_tiled(const DwParams& p, const CUtensorMap& tmap, int out_mode, int num_sms, cudaStream_t s) {
+  const int total = p.N * p.tiles_h * p.tiles_w;
+  const uint32_t smem = depthwise_tiled_smem_bytes(p);
+  const int per_sm = smem <= 110u * 1024u ? 2 : 1;
+  const int grid = std::max(1, std::min(total, num_sms * per_sm));
+  const int threads = ((p.C / 4) * p.slots + 31) / 32 * 32;
+  switch (out_mode) {
+    case kOutInt8: depthwise3x3_tiled_kernel<kOutInt8><<<grid, threads, smem, s>>>(p, tmap); break;
+    case kOutF32: depthwise3x3_tiled_kernel<kOutF32><<<grid, threads, smem, s>>>(p, tmap); break;
+    default: depthwise3x3_tiled_kernel<kOutAcc><<<grid, threads, smem, s>>>(p, tmap); break;
+  }
   return cudaGetLastError();
 }
 

@@ -34,6 +34,7 @@ enum AsyncCode : int32_t {
   kAsyncEpilogueTmemFullWait = 4,
   kAsyncProducerBEmptyWait = 5,
   kAsyncMmaBFullWait = 6,
+  kAsyncDepthwiseFullWait = 7,
 };
 
 struct FastDiv {                      // n / d == (umulhi(m, n) + n) >> l for 0 <= n < 2^31
@@ -109,6 +110,11 @@ struct DwParams {                     // depthwise (CUDA cores)
   const float* w_scale;
   hq_range_state* yq;
   void* out;
+  // tiled 3x3 kernel: output tile of TR rows x TWt columns, input patch of (TR + 2) x (TWt + 2) pixels in shared memory
+  int32_t TR, TWt, tiles_h, tiles_w, slots, ncls;
+  uint32_t patch_bytes;               // bytes one TMA box delivers
+  uint32_t patch_stride;              // patch_bytes rounded up to 128: distance of the two buffers (TMA destinations are 128-byte aligned)
+  int32_t* status;                    // device status word (expired waits)
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -145,6 +151,10 @@ cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtens
                         cudaStream_t s, bool overlap);
 cudaError_t gemm_set_smem_attr(uint32_t smem_bytes);
 cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s, bool overlap);
+// 3x3 stride-1 depthwise with the input patch staged by TMA (p.TR ... p.status filled in); tmap covers the NHWC input
+cudaError_t launch_depthwise_tiled(const DwParams& p, const CUtensorMap& tmap, int out_mode, int num_sms, cudaStream_t s);
+cudaError_t depthwise_tiled_set_smem_attr(uint32_t smem_bytes);
+uint32_t depthwise_tiled_smem_bytes(const DwParams& p);
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap);
 cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overlap);
 cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
@@ -178,6 +188,7 @@ struct hq_ctx {
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
+  int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
   bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
@@ -214,5 +225,6 @@ struct hq_prepared_weights {
   uint8_t* dw_rowcls = nullptr;
   uint8_t* dw_colcls = nullptr;
   int dw_ncolcls = 1;
+  int dw_ncls = 1;                    // border classes (rows x columns) of the depthwise correction table
   std::vector<void*> allocs;          // everything to cudaFree on release
 };

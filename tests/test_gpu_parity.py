@@ -115,6 +115,9 @@ FWD_CASES = {
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
     "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
+    "dw3x3_c64_wide": dict(N=2, H=9, W=150, Cin=64, K=64, R=3, S=3, stride=1, pad=1, groups=64),
+    "dw3x3_c32_ragged": dict(N=3, H=13, W=21, Cin=32, K=32, R=3, S=3, stride=1, pad=1, groups=32),
+    "dw3x3_c256_nopad": dict(N=1, H=11, W=12, Cin=256, K=256, R=3, S=3, stride=1, pad=0, groups=256),
     "dw5x5_c48": dict(N=1, H=13, W=9, Cin=48, K=48, R=5, S=5, stride=1, pad=2, groups=48),
     "dw3x3_c320": dict(N=1, H=7, W=7, Cin=320, K=320, R=3, S=3, stride=1, pad=1, groups=320),
 }
@@ -148,6 +151,22 @@ def test_depthwise_both_paths(ctx, name, depthwise):
     in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
     makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
     _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, depthwise=depthwise)
+
+
+@pytest.mark.parametrize("dw_staging", [0, 1])
+@pytest.mark.parametrize("name", ["dw3x3_c144", "dw3x3_c64_wide", "dw3x3_c32_ragged", "dw3x3_c256_nopad"])
+def test_depthwise_cuda_core_staging(ctx, name, dw_staging):
+    """CUDA-core depthwise 3x3: direct global loads and TMA-staged patches (several tiles, ragged edges) give the oracle's bytes."""
+    shape = dict(FWD_CASES[name])
+    r = synth.rng(106, len(name), shape["H"], dw_staging)
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
+    ctx.set_option("depthwise_staging", dw_staging)
+    try:
+        _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, depthwise=0)
+    finally:
+        ctx.set_option("depthwise_staging", -1)
 
 
 @pytest.mark.parametrize("repack", [0, 1])
