@@ -124,6 +124,9 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
  *   "depthwise": how depthwise layers prepared AFTER this call run: -1 = library's choice (default; the
  *              CUDA-core kernel), 0 = CUDA-core kernel, 1 = on the tensor cores as dense layers with
  *              diagonal filters, one per 64-channel slice.
+ *   "side_by_side": 1 (default) = the independent launches of one call (parity classes of a strided
+ *              backward pass) run concurrently on shares of the SMs, forked from and joined into the
+ *              caller's stream; 0 = one after the other.
  *   "depthwise_staging": CUDA-core depthwise 3x3 stride-1 layers (read at every call): -1 = library's
  *              choice (default), 0 = direct global loads, 1 = input patches staged in shared memory by TMA
  *              where the shape allows.

@@ -393,14 +393,14 @@ int fold_factor(int channels, int64_t pixels) {
 }
 
 hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, const CUtensorMap& ta, const CUtensorMap& tb, const hq_range_state* xq,
-                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode) {
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, int max_ctas = 0) {
   GemmParams p = sub.p;
   p.xq = xq;
   p.w_scale = w_scale;
   p.bias = bias;
   p.out = out;
   p.yq = yq;
-  const int grid = std::min(p.num_tiles, ctx->num_sms);
+  const int grid = std::max(1, std::min(p.num_tiles, max_ctas > 0 ? max_ctas : ctx->num_sms));
   HQ_CUDA(ctx, launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s, ctx->overlap));
   ctx->launches += 1;
   return HQ_OK;
@@ -469,7 +469,46 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
   const int aC = dir == HQ_DIR_FWD ? desc->C : desc->K;
   const int aH = dir == HQ_DIR_FWD ? desc->H : Ho;
   const int aW = dir == HQ_DIR_FWD ? desc->W : Wo;
+  // Several launches of one call (parity classes of a strided backward pass, channel slices) write disjoint outputs:
+  // they run side by side, each on its share of the SMs (every CTA needs a whole SM's shared memory), forked from and
+  // joined back into the caller's stream with events.
+  const int nsub = (int)pw->subs.size();
+  constexpr int kMaxSideBySide = 64;
+  bool side_by_side = nsub > 1 && nsub <= kMaxSideBySide && ctx->parallel_subs;
+  int share[kMaxSideBySide] = {0};
+  if (side_by_side) {
+    double total = 0.0;
+    double cost[kMaxSideBySide];
+    for (int i = 0; i < nsub; ++i) {
+      const GemmParams& gp = pw->subs[i].p;
+      cost[i] = (double)gp.num_tiles * (6.0 + (double)gp.ntaps * gp.chunks_per_tap * (gp.BK / 64.0) * (gp.BN / 128.0));
+      total += cost[i];
+    }
+    int used = 0;
+    for (int i = 0; i < nsub; ++i) {
+      share[i] = std::max(1, (int)(ctx->num_sms * cost[i] / total));
+      used += share[i];
+    }
+    for (int i = 0; used < ctx->num_sms; i = (i + 1) % nsub, ++used) ++share[i];
+    HQ_CUDA(ctx, cudaEventRecord(ctx->ev_fork, s));
+  }
+  int sub_index = -1;
+  auto join = [&]() -> hq_status {
+    if (!side_by_side) return HQ_OK;
+    for (int k = 0; k < std::min(nsub - 1, 3); ++k) {
+      HQ_CUDA(ctx, cudaEventRecord(ctx->ev_join[k], ctx->side[k]));
+      HQ_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
+    }
+    return HQ_OK;
+  };
   for (const hq_sub_problem& sub : pw->subs) {
+    ++sub_index;
+    cudaStream_t ss = s;
+    if (side_by_side && sub_index > 0) {
+      ss = ctx->side[(sub_index - 1) % 3];
+      if (sub_index <= 3) HQ_CUDA(ctx, cudaStreamWaitEvent(ss, ctx->ev_fork, 0));
+    }
+    const int max_ctas = side_by_side ? share[sub_index] : 0;
     CUtensorMap ta;
     if (sub.p.ntaps == 0) {
       ta = CUtensorMap{};
@@ -489,7 +528,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       st = encode_a(ctx, sub, in + sub.chan0, sub.chans, aW, aH, desc->N, &ta, desc->C);
       if (st != HQ_OK) return st;
       void* o = out_mode == kOutInt8 ? (void*)((int8_t*)out + sub.chan0) : (void*)((uint32_t*)out + sub.chan0);
-      st = launch_sub(ctx, s, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode);
+      st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas);
       if (st != HQ_OK) return st;
       continue;
     } else if (sub.a_flat) {
@@ -499,10 +538,10 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       st = encode_a(ctx, sub, in, aC, aW, aH, desc->N, &ta);
     }
     if (st != HQ_OK) return st;
-    st = launch_sub(ctx, s, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode);
+    st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas);
     if (st != HQ_OK) return st;
   }
-  return HQ_OK;
+  return join();
 }
 
 hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
@@ -596,6 +635,22 @@ __attribute__((visibility("default"))) const char* hq_status_string(hq_status s)
   return "unknown status";
 }
 
+static bool make_side_streams(hq_ctx* ctx) {
+  if (cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess) return false;
+  for (int k = 0; k < 3; ++k) {
+    if (cudaStreamCreateWithFlags(&ctx->side[k], cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaEventCreateWithFlags(&ctx->ev_join[k], cudaEventDisableTiming) != cudaSuccess) return false;
+  }
+  return true;
+}
+static void free_side_streams(hq_ctx* ctx) {
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  for (int k = 0; k < 3; ++k) {
+    if (ctx->ev_join[k]) cudaEventDestroy(ctx->ev_join[k]);
+    if (ctx->side[k]) cudaStreamDestroy(ctx->side[k]);
+  }
+}
+
 __attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int device) {
   if (!out) return HQ_ERR_INVALID_ARG;
   *out = nullptr;
@@ -623,9 +678,11 @@ __attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int dev
   ctx->scratch_elems = 4096;
   if (cudaMalloc((void**)&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc((void**)&ctx->d_scratch, ctx->scratch_elems * sizeof(int32_t)) != cudaSuccess ||
-      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess) {
+      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess ||
+      !make_side_streams(ctx)) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_scratch) cudaFree(ctx->d_scratch);
+    free_side_streams(ctx);
     delete ctx;
     return HQ_ERR_CUDA;
   }
@@ -638,6 +695,7 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_scratch);
   if (ctx->d_pad) cudaFree(ctx->d_pad);
+  free_side_streams(ctx);
   delete ctx;
   return HQ_OK;
 }
@@ -651,6 +709,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "staging") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "staging must be -1, 0 or 1");
     ctx->force_mode = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "side_by_side") {
+    if (value < 0 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "side_by_side must be 0 or 1");
+    ctx->parallel_subs = value != 0;
     return HQ_OK;
   }
   if (std::string(key) == "depthwise_staging") {

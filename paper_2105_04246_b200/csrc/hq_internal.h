@@ -191,6 +191,9 @@ struct hq_ctx {
   int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
+  cudaStream_t side[3] = {nullptr, nullptr, nullptr};   // independent launches of one call run side by side (see run_conv)
+  cudaEvent_t ev_fork = nullptr, ev_join[3] = {nullptr, nullptr, nullptr};
+  bool parallel_subs = true;
   bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
   std::string err;
 };
