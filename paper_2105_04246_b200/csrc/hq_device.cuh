@@ -45,9 +45,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try(bar, parity, hint_ns)) return true;
-    // A short fixed pause: the suspended try above already keeps a waiting warp off the issue slots; a growing
-    // back-off only adds wake-up latency to waits that sit on the critical path of every tile.
-    __nanosleep(32);
+    // A pause between polls: the try above returns after some tens of nanoseconds even with a long hint, and a warp
+    // that polls back to back takes issue slots from the epilogue warps of its scheduler.  A quarter of the hint keeps
+    // the wake-up latency of waits on the critical path (short hints) small.
+    __nanosleep(hint_ns >> 2);
     if ((++spins & 15u) == 0u) {
       if (*abort_flag) return false;
       if (global_timer_ns() - t0 > kWaitLimitNs) {
