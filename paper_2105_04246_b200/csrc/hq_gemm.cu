@@ -454,6 +454,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int nchunks = p.BN / 16;                      // BN is a multiple of 16
     const int c_begin = (slice * nchunks) / slices;
     const int c_end = ((slice + 1) * nchunks) / slices;
+    const bool has_corr = p.corr != nullptr;
+    // per-layer part of the condition for the straight-line pass (see below)
+    const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.zc_in_smem && has_corr;
     for (int local_tile = group; ; local_tile += ngroups) {
       const int tile = (int)blockIdx.x + local_tile * (int)gridDim.x;
       if (tile >= p.num_tiles) break;
@@ -474,14 +477,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         row_valid = (n < p.n_img) && (i < p.TH) && (j < p.TW);
       }
       const int64_t pix = ((int64_t)n * p.out_H + (i * p.os_h + p.oa_h)) * p.out_W + (j * p.os_w + p.oa_w);
-      const int32_t* corr_row = nullptr;
-      const int32_t* zrow_s = nullptr;
-      if (p.corr != nullptr && q.zx != 0 && row_valid) {
+      // correction row of this pixel's border class (row 0 for pixels of tile padding, whose results are dropped)
+      int zoff = col0;
+      if (has_corr && row_valid) {
         const int rc = p.cls_in_smem ? cls_s[i] : (p.rowcls ? p.rowcls[i] : 0);
         const int cc = p.cls_in_smem ? cls_s[512 + j] : (p.colcls ? p.colcls[j] : 0);
-        const int off = (rc * p.ncolcls + cc) * p.corr_ld + col0;
-        if (p.zc_in_smem) zrow_s = zc_s + off;   // shared copy, already multiplied by zx
-        else corr_row = p.corr + off;
+        zoff += (rc * p.ncolcls + cc) * p.corr_ld;
+      }
+      const int32_t* corr_row = nullptr;
+      const int32_t* zrow_s = nullptr;
+      if (has_corr && q.zx != 0 && row_valid) {
+        if (p.zc_in_smem) zrow_s = zc_s + zoff;   // shared copy, already multiplied by zx
+        else corr_row = p.corr + zoff;
       }
       const int buf = local_tile & (nbuf - 1);
       const uint32_t tph = (uint32_t)(local_tile >> nbuf_log2) & 1u;
@@ -584,16 +591,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       // parameters, no bias, every column of the pass inside the layer, correction table in shared memory (it holds
       // zeros when the input zero point is 0).  Rows outside the image (tile padding) are computed like the others
       // and only kept out of the statistics and the store.
-      const bool lean = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.zc_in_smem &&
-                        p.corr != nullptr && col0 + c_end * CW <= p.Nout;
+      const bool lean = lean_layer && col0 + c_end * CW <= p.Nout;
       if (lean) {
-        const int32_t* zrow = zc_s;
-        if (row_valid) {
-          const int rc = p.cls_in_smem ? cls_s[i] : (p.rowcls ? p.rowcls[i] : 0);
-          const int cc = p.cls_in_smem ? cls_s[512 + j] : (p.colcls ? p.colcls[j] : 0);
-          zrow = zc_s + (rc * p.ncolcls + cc) * p.corr_ld;
-        }
-        zrow += col0;
+        const int32_t* zrow = zc_s + zoff;
         int8_t* dst_row = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0;
         int tmn = INT32_MAX, tmx = INT32_MIN;
         for (int ch = c_begin; ch < c_end; ++ch) {
