@@ -314,18 +314,28 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           int n0, o0, w0, col0;
           decode(tile, n0, o0, w0, col0);
           const uint32_t rel_bytes = (uint32_t)(o0 - fdiv(o0, p.fd_P) * p.P) * (uint32_t)p.BK;
-          if (p.b_resident && first) {   // the whole weight matrix arrives once
-            for (int ki = 0; ki < kiters && ok; ++ki) ok = warp_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
-            if (!ok) break;
-            tc_fence_after();
-          }
           uint64_t bres = bdesc0;
           for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
             ok = warp_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait, 200u);
             if (!ok) break;
             tc_fence_after();
             const uint64_t abase = make_smem_desc(ring_a + stage * a_stride + rel_bytes, sw64);
-            if (resident) {
+            if (resident && first) {
+              // the weight matrix arrives once, tap by tap: the first tile starts on each tap as soon as it is there
+              for (int t = 0; t < ntaps; ++t) {
+                ok = warp_wait(b_full(cc * ntaps + t), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t adesc = abase + tapoff_s[t];
+                if (elect_one()) {
+#pragma unroll
+                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                }
+                bres += bstep16;
+              }
+              __syncwarp();
+              acc = 1;
+            } else if (resident) {
               if (elect_one()) {
                 for (int t = 0; t < ntaps; ++t) {
                   const uint64_t adesc = abase + tapoff_s[t];
