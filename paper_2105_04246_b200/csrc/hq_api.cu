@@ -393,8 +393,10 @@ int fold_factor(int channels, int64_t pixels) {
 }
 
 hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, const CUtensorMap& ta, const CUtensorMap& tb, const hq_range_state* xq,
-                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, int max_ctas = 0) {
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, int max_ctas = 0,
+                     bool weights_early = false) {
   GemmParams p = sub.p;
+  p.weights_early = weights_early ? 1 : 0;
   p.xq = xq;
   p.w_scale = w_scale;
   p.bias = bias;
@@ -472,6 +474,8 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
   // Several launches of one call (parity classes of a strided backward pass, channel slices) write disjoint outputs:
   // they run side by side, each on its share of the SMs (every CTA needs a whole SM's shared memory), forked from and
   // joined back into the caller's stream with events.
+  const bool weights_early = ctx->overlap && pw->used;
+  pw->used = true;
   const int nsub = (int)pw->subs.size();
   constexpr int kMaxSideBySide = 64;
   bool side_by_side = nsub > 1 && nsub <= kMaxSideBySide && ctx->parallel_subs;
@@ -528,7 +532,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       st = encode_a(ctx, sub, in + sub.chan0, sub.chans, aW, aH, desc->N, &ta, desc->C);
       if (st != HQ_OK) return st;
       void* o = out_mode == kOutInt8 ? (void*)((int8_t*)out + sub.chan0) : (void*)((uint32_t*)out + sub.chan0);
-      st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas);
+      st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas, weights_early);
       if (st != HQ_OK) return st;
       continue;
     } else if (sub.a_flat) {
@@ -538,7 +542,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       st = encode_a(ctx, sub, in, aC, aW, aH, desc->N, &ta);
     }
     if (st != HQ_OK) return st;
-    st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas);
+    st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas, weights_early);
     if (st != HQ_OK) return st;
   }
   return join();

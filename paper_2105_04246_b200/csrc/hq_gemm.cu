@@ -146,8 +146,10 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   // Everything above touched only kernel parameters and this CTA's own resources.  From here on the kernel reads
-  // what earlier kernels in the stream wrote (operands, range states), so it waits for them.
-  grid_dependency_wait();
+  // what earlier kernels in the stream wrote (operands, range states), so it waits for them.  The weight producer
+  // reads nothing but the prepared weight matrix; where the host knows that matrix to be older than the previous
+  // kernel (any call after the first with these prepared weights) it starts copying at once.
+  if (!(warp == 2 && p.weights_early)) grid_dependency_wait();
 
   // tile index -> origin.  kModeTap: (n0, h0, w0) of the pixel box; kModeHalo: image n0, first linear pixel h0
   auto decode = [&](int tile, int& n0, int& h0, int& w0, int& col0) {

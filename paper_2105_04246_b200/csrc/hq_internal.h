@@ -69,6 +69,7 @@ struct GemmParams {
   uint32_t patch_chunk_stride;        // bytes between channel chunks of one patch (1024-aligned)
   uint32_t patch_box_bytes;           // bytes one patch TMA delivers
   int32_t b_resident;
+  int32_t weights_early;              // the weight producer may start before the previous kernel in the stream has finished
   // common
   int32_t Nout, BN;
   int32_t out_H, out_W, os_h, os_w, oa_h, oa_w;
@@ -221,6 +222,7 @@ struct hq_prepared_weights {
   hq_conv_desc desc{};
   hq_direction dir = HQ_DIR_FWD;
   bool depthwise = false;
+  mutable bool used = false;          // set by the first layer call: later calls know that the tables were complete long before
   std::vector<hq_sub_problem> subs;
   // depthwise tables
   int8_t* dw_w = nullptr;
