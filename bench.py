@@ -371,22 +371,39 @@ def run_gpu(args):
     sampler.stop_flag = True
     sampler.join(timeout=2)
 
-    # end to end through the binding with host buffers: H2D of the step's inputs, the step, D2H of its result
+    # end to end through the binding with host buffers: every step copies its inputs from pinned host memory, runs, and
+    # copies its result back to pinned host memory.  Copies run on their own streams, ordered against the compute stream
+    # with events per pool slot, so the H2D of step k+1 and the D2H of step k-1 overlap step k (as a serving loop would).
     e2e_steps = min(K, 50)
     host_in = [[x.cpu().pin_memory() for x in xs] if xs is not None else None for xs in wk.x_pool]
-    host_out = torch.empty(wk.y_pool[-1][0].shape, dtype=torch.int8).pin_memory()
+    host_out = [torch.empty(wk.y_pool[-1][0].shape, dtype=torch.int8).pin_memory() for _ in range(pool)]
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    ev_in = [torch.cuda.Event() for _ in range(pool)]
+    ev_done = [torch.cuda.Event() for _ in range(pool)]
+    ev_out = [torch.cuda.Event() for _ in range(pool)]
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     t0 = time.perf_counter()
     for k in range(e2e_steps):
         j = k % pool
-        for i in range(n_layers):
-            if host_in[i] is not None:
-                wk.x_pool[i][j].copy_(host_in[i][j], non_blocking=True)
+        with torch.cuda.stream(s_in):
+            if k >= pool:
+                s_in.wait_event(ev_done[j])          # the step that last read this slot's inputs has finished
+            for i in range(n_layers):
+                if host_in[i] is not None:
+                    wk.x_pool[i][j].copy_(host_in[i][j], non_blocking=True)
+            ev_in[j].record(s_in)
+        stream.wait_event(ev_in[j])
+        if k >= pool:
+            stream.wait_event(ev_out[j])             # the slot's previous result has left the device
         wk.step(stream, j)
-        host_out.copy_(wk.y_pool[-1][j], non_blocking=True)
-        torch.cuda.synchronize()
+        ev_done[j].record(stream)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(ev_done[j])
+            host_out[j].copy_(wk.y_pool[-1][j], non_blocking=True)
+            ev_out[j].record(s_out)
+    torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     assert ctx.get_async_error() == 0, "a device-side wait expired during the benchmark"
 
