@@ -1,6 +1,7 @@
 """Parity at the full sizes of the workloads, in the launch configuration the benchmark times
 (default staging, whole batch, persistent grid).  The oracle evaluates these tensors in full in a
-few seconds each, so every output element is compared, not a sample."""
+few seconds each (under a minute for the whole ResNet-18-shaped stack), so every output element is
+compared, not a sample."""
 import numpy as np
 import pytest
 
@@ -73,3 +74,28 @@ def test_cfg4_inverted_residual_chain_full_batch(ctx):
             st = g.state()
             xg = synth.QTensor(y, float(st["scale"]), int(st["zero_point"]))          # each output feeds the next layer
             xo = synth.QTensor(res.q, o.layer.state.scale, o.layer.state.zero_point)
+
+
+def test_cfg5_resnet18_stack_full_batch(ctx):
+    """Every layer call of the ResNet-18-shaped workload at its full batch (the configuration the benchmark times:
+    window repacking of the stem, side-by-side parity classes, padded classifier rows), dynamic initialisation and one
+    in-hindsight iteration, every output element against the oracle."""
+    import bench
+    layers, _ = bench.workload_layers("cfg5", 1)
+    r = synth.rng(204)
+    for kind, s, recipe in layers:
+        xsh, ysh, wsh = bench.layer_shapes(kind, s)
+        if kind == "linear":
+            W, shape = synth.uniform_int8(r, wsh, scale=0.01), None
+        else:
+            W, shape = synth.weights(r, wsh), _shape(s)
+        g, o = GpuLayer(ctx, kind, W, shape), OracleLayer(kind, W, shape)
+        for t in range(2):
+            x = bench.make_input(recipe, r, xsh)
+            x.scale *= float(np.exp(r.normal(0.0, 0.3)))
+            y, res = g.step(x), o.step(x)
+            assert y.shape == tuple(ysh)
+            bad = int((y != res.q).sum())
+            assert bad == 0, f"{s.name} iteration {t}: {bad} of {y.size} int8 codes differ"
+            assert_state_close(g.state(), o.layer.state)
+        del g, o
