@@ -180,6 +180,39 @@ def dynamic(acc: np.ndarray, s_acc: float, q: Range):
     return yf, out
 
 
+def philox4x32_10(counter, key):
+    """Four 32-bit words of Philox4x32-10 for a 4-word counter and a 2-word key."""
+    c = (C.c_uint32 * 4)(*[int(x) & 0xFFFFFFFF for x in counter])
+    k = (C.c_uint32 * 2)(*[int(x) & 0xFFFFFFFF for x in key])
+    out = (C.c_uint32 * 4)()
+    lib().hqo_philox4x32_10(c, k, out)
+    return [int(x) for x in out]
+
+
+def draw16(seed: int, iteration: int, e: int) -> int:
+    """The 16-bit draw of the output element with linear index e."""
+    lib().hqo_draw16.restype = C.c_uint32
+    return int(lib().hqo_draw16(C.c_uint32(seed), C.c_uint32(iteration), C.c_int64(e)))
+
+
+def quantize_sr(acc: np.ndarray, s_acc: float, q: Range, seed: int, iteration: int, first: int = 0) -> np.ndarray:
+    """Static quantization with stochastic rounding; element i (C order) has linear index first + i."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    out = np.empty(acc.shape, np.int8)
+    lib().hqo_quantize_sr(_p(acc, C.c_int32), C.c_int64(acc.size), C.c_float(s_acc), C.byref(q), C.c_uint32(seed), C.c_uint32(iteration),
+                          C.c_int64(first), _p(out, C.c_int8))
+    return out
+
+
+def dynamic_sr(acc: np.ndarray, s_acc: float, q: Range, seed: int):
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    yf = np.empty(acc.shape, np.float32)
+    out = np.empty(acc.shape, np.int8)
+    lib().hqo_dynamic_sr(_p(acc, C.c_int32), C.c_int64(acc.size), C.c_float(s_acc), C.byref(q), C.c_uint32(seed), _p(yf, C.c_float),
+                         _p(out, C.c_int8))
+    return yf, out
+
+
 def acc_scale(s_x: float, s_w: float) -> float:
     return float(lib().hqo_acc_scale(C.c_float(s_x), C.c_float(s_w)))
 
@@ -206,17 +239,26 @@ class Layer:
     previous iterations, then apply Eq. 2-3 with this tensor's min/max.
     """
 
-    def __init__(self, eta: float = 0.9):
+    def __init__(self, eta: float = 0.9, sr_seed: int | None = None):
+        """sr_seed: None = round to nearest even; an integer = stochastic rounding with that seed
+        (the iteration number of the draws is the state's update count)."""
         self.eta = float(eta)
         self.state = Range()
+        self.sr_seed = sr_seed
 
     def step(self, acc: np.ndarray, s_acc: float, force_state: Range | None = None) -> StepResult:
         if force_state is not None:
             self.state = force_state.copy()
         mn, mx = minmax(acc)
         if self.state.step == 0:
-            _, q = dynamic(acc, s_acc, self.state)
+            if self.sr_seed is None:
+                _, q = dynamic(acc, s_acc, self.state)
+            else:
+                _, q = dynamic_sr(acc, s_acc, self.state, self.sr_seed)
             return StepResult(acc, mn, mx, s_acc, q, "dynamic")
-        q = quantize(acc, s_acc, self.state)
+        if self.sr_seed is None:
+            q = quantize(acc, s_acc, self.state)
+        else:
+            q = quantize_sr(acc, s_acc, self.state, self.sr_seed, self.state.step)
         range_update(self.state, mn, mx, s_acc, self.eta)
         return StepResult(acc, mn, mx, s_acc, q, "hindsight")

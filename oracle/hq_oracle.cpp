@@ -37,6 +37,7 @@
 //   R-9  t = 0 runs the dynamic path; from t = 1 the range of t-1 is used.
 //   R-13 a degenerate range (hi - lo not > 0) gives s = 1.
 //   R-15 the dynamic path materialises binary32 y = fl(float(acc) * s_acc).
+//   R-18..R-20 stochastic rounding for gradients: see the section further down.
 //
 // Pins (tests/ -m "not gpu"): brute-force and readable-by-eye cases for the index
 // arithmetic, the forward/backward adjoint identity, library convolutions in float64,
@@ -311,6 +312,91 @@ void hqo_dynamic(const int32_t* acc, int64_t count, float s_acc, hqo_range* q, f
   q->step += 1;
   hqo_derive(q);
   for (int64_t i = 0; i < count; ++i) out[i] = quantize_real(yf[i], q);
+}
+
+// ------------------------------------------------------------------------------------
+// Stochastic rounding for gradients (the paper quantizes gradients with stochastic rounding;
+// it gives no formula, so the conventions below are readings):
+//   R-18  q = sat8(floor(fl(u + r)) + z) with u as in O4 (R-4) and r uniform in [0,1);
+//         the sum is one binary32 round-to-nearest-even addition.
+//   R-19  r = h / 65536 with h a 16-bit draw, so r is exact in binary32.
+//   R-20  draws come from the counter-based generator Philox4x32-10 (Salmon, Moraes, Dror,
+//         Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11): key = (seed, 0),
+//         counter = (low and high word of e >> 3, iteration, 0) for the element with linear
+//         index e in the output tensor; of the call's four 32-bit words, element e takes half
+//         number (e & 7): word (e & 7) >> 1, low half when e is even, high half when odd.
+//         `iteration` is the number of range updates the output's state has seen.
+// Pins: the generator against the known-answer vectors published with it; floor(u+r) is one
+// of the two neighbours of u; exact for integer u; unbiased over draws; reproducible.
+// ------------------------------------------------------------------------------------
+static inline void mulhilo32(uint32_t a, uint32_t b, uint32_t* hi, uint32_t* lo) {
+  uint64_t p = (uint64_t)a * (uint64_t)b;
+  *hi = (uint32_t)(p >> 32);
+  *lo = (uint32_t)p;
+}
+
+void hqo_philox4x32_10(const uint32_t counter[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = counter[0], c1 = counter[1], c2 = counter[2], c3 = counter[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    uint32_t hi0, lo0, hi1, lo1;
+    mulhilo32(0xD2511F53u, c0, &hi0, &lo0);
+    mulhilo32(0xCD9E8D57u, c2, &hi1, &lo1);
+    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += 0x9E3779B9u;   // key schedule: golden-ratio and sqrt(3)-1 Weyl constants
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// the 16-bit draw of element e (R-20)
+uint32_t hqo_draw16(uint32_t seed, uint32_t iteration, int64_t e) {
+  uint64_t block = (uint64_t)e >> 3;
+  uint32_t counter[4] = {(uint32_t)block, (uint32_t)(block >> 32), iteration, 0u};
+  uint32_t key[2] = {seed, 0u};
+  uint32_t w[4];
+  hqo_philox4x32_10(counter, key, w);
+  uint32_t word = w[((uint32_t)e & 7u) >> 1];
+  return (e & 1) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+static inline int32_t floor_to_i32(float t) {   // floor, then to int32 with saturation; NaN -> 0
+  if (t != t) return 0;
+  float f = std::floor(t);
+  if (f >= 2147483648.0f) return std::numeric_limits<int32_t>::max();
+  if (f <= -2147483648.0f) return std::numeric_limits<int32_t>::min();
+  return (int32_t)f;
+}
+
+static inline int8_t quantize_real_sr(float y, const hqo_range* q, uint32_t seed, uint32_t iteration, int64_t e) {
+  float u = y * q->inv_scale;
+  float r = (float)hqo_draw16(seed, iteration, e) * (1.0f / 65536.0f);
+  float t = u + r;
+  return (int8_t)clamp_i64((int64_t)floor_to_i32(t) + q->zero_point, -128, 127);
+}
+
+// static quantization with stochastic rounding; element i of `acc` has linear index first + i
+void hqo_quantize_sr(const int32_t* acc, int64_t count, float s_acc, const hqo_range* q, uint32_t seed, uint32_t iteration, int64_t first,
+                     int8_t* out) {
+  for (int64_t i = 0; i < count; ++i) out[i] = quantize_real_sr((float)acc[i] * s_acc, q, seed, iteration, first + i);
+}
+
+// dynamic path with stochastic rounding: as hqo_dynamic; the draws use the iteration count before this call
+void hqo_dynamic_sr(const int32_t* acc, int64_t count, float s_acc, hqo_range* q, uint32_t seed, float* yf, int8_t* out) {
+  for (int64_t i = 0; i < count; ++i) yf[i] = (float)acc[i] * s_acc;
+  float lo = std::numeric_limits<float>::infinity(), hi = -lo;
+  for (int64_t i = 0; i < count; ++i) {
+    if (yf[i] < lo) lo = yf[i];
+    if (yf[i] > hi) hi = yf[i];
+  }
+  if (count == 0) return;
+  const uint32_t iteration = q->step;
+  q->q_min = lo;
+  q->q_max = hi;
+  q->step += 1;
+  hqo_derive(q);
+  for (int64_t i = 0; i < count; ++i) out[i] = quantize_real_sr(yf[i], q, seed, iteration, i);
 }
 
 // s_acc = fl(s_x * s_w): scale of one accumulator unit in real terms
