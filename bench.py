@@ -181,14 +181,19 @@ class ClockSampler(threading.Thread):
 class GpuWorkload:
     """All device buffers of one workload plus the calls of one step (hindsight or dynamic)."""
 
-    def __init__(self, name: str, ctx, dev, pool: int, seed_key: int):
+    def __init__(self, name: str, ctx, dev, pool: int, seed_key: int, stochastic: bool = False):
         import torch
         from paper_2105_04246_b200 import hq
         self.hq, self.torch, self.ctx, self.dev, self.name = hq, torch, ctx, dev, name
         self.layers, self.chained = workload_layers(name)
         n = len(self.layers)
         g = synth.rng(1000 + seed_key)
-        self.states = hq.states_to_device(hq.new_states(n), dev)
+        st = hq.new_states(n)
+        if stochastic:                      # the paper's rounding for gradients: backward-data layers only
+            for i, (kind, _s, _r) in enumerate(self.layers):
+                if kind == "conv_bwd" or _s.name.endswith(".bwd"):
+                    st[i]["rounding"], st[i]["seed"] = hq.ROUND_STOCHASTIC, 0x2105 + i
+        self.states = hq.states_to_device(st, dev)
         self.state_ptr = [self.states.data_ptr() + 48 * i for i in range(n)]
         self.W, self.w_scale, self.pw, self.desc, self.x_pool, self.xq_pool, self.y_pool, self.ws = [], [], [], [], [], [], [], []
         stream = torch.cuda.current_stream(dev)
@@ -313,7 +318,7 @@ def run_gpu(args):
     peaks, peak_kind = load_peaks()
     name = args.workload
     pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg5": 2}[name]
-    wk = GpuWorkload(name, ctx, dev, pool, seed_key=rank)
+    wk = GpuWorkload(name, ctx, dev, pool, seed_key=rank, stochastic=args.rounding == "stochastic")
     K, W = args.steps, max(3, args.warmup)
     stream = torch.cuda.current_stream(dev)
     n_layers = len(wk.layers)
@@ -451,6 +456,7 @@ def run_gpu(args):
         "config": {"workload": f"{name}: " + ", ".join(s.name for _, s, _ in wk.layers), "path": "in-hindsight (static requant in the epilogue + min/max)",
                    "l2": f"inputs and outputs rotate over a pool of {pool} buffer sets (> L2) inside CUDA graphs", "eta": 0.9,
                    "launch": "ordinary" if args.no_overlap else "programmatic stream serialization",
+                   "rounding": "nearest even" if args.rounding == "nearest" else "stochastic for gradient layers, nearest even otherwise",
                    "parallelism": f"dp{world} (batch shards; one int32 min/max all-reduce per step before the range update)" if world > 1 else "dp1"},
         "gpu_launches": int(launches_per_step * K),
         "launches_per_step": int(launches_per_step),
@@ -480,7 +486,7 @@ def run_profile(args):
     if args.no_overlap:
         ctx.set_option("overlap_launches", 0)
     ctx.set_option("depthwise", args.depthwise)
-    wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0)
+    wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0, stochastic=args.rounding == "stochastic")
     stream = torch.cuda.current_stream(dev)
     for j in range(2):
         wk.step(stream, j, dynamic=True)
@@ -520,6 +526,8 @@ def main():
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rounding", default="nearest", choices=["nearest", "stochastic"],
+                    help="stochastic: backward-data (gradient) layers use stochastic rounding, the paper's choice for gradients")
     ap.add_argument("--depthwise", type=int, default=-1, choices=[-1, 0, 1],
                     help="depthwise layers: -1 library's choice, 0 CUDA-core kernel, 1 dense slices on the tensor cores")
     ap.add_argument("--no-overlap", action="store_true",

@@ -61,7 +61,16 @@ typedef enum {
  *   scale, inv_scale, zero_point   the 2^8-level grid derived from the running range:
  *                    lo = min(q_min,0), hi = max(q_max,0), scale = (hi-lo)/255 (1 if not > 0),
  *                    inv_scale = 1/scale, zero_point = clamp(-128 - rint(lo/scale), -128, 127).
+ *   rounding, seed   how a layer call that WRITES this tensor rounds: HQ_ROUND_NEAREST_EVEN (0), or
+ *                    HQ_ROUND_STOCHASTIC (1) -- the paper's choice for gradients: code =
+ *                    sat8(floor(fl(u + r)) + zero_point) with u as for nearest-even and r = h / 65536,
+ *                    h the 16-bit draw of Philox4x32-10 (Salmon et al., SC'11) with key (seed, 0) and
+ *                    counter (e >> 3 as two words, step, 0) for the element with linear index e in the
+ *                    output tensor: half number (e & 7) of the call's four words, low half first.
+ *                    `step` is the value at the time of the call, so every iteration draws anew.
  * For a layer INPUT only scale and zero_point are read.                                      */
+#define HQ_ROUND_NEAREST_EVEN 0u
+#define HQ_ROUND_STOCHASTIC 1u
 typedef struct {
   int32_t acc_min, acc_max;
   float acc_scale;
@@ -69,7 +78,9 @@ typedef struct {
   float q_min, q_max;
   float scale, inv_scale;
   int32_t zero_point;
-  uint32_t reserved[3];
+  uint32_t rounding;
+  uint32_t seed;
+  uint32_t reserved;
 } hq_range_state;
 
 /* Forward-convolution geometry.  Input N x H x W x C, output N x Ho x Wo x K with

@@ -396,6 +396,7 @@ hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, con
                      const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, int max_ctas = 0,
                      bool weights_early = false) {
   GemmParams p = sub.p;
+  p.out_col0 = sub.chan0;
   p.weights_early = weights_early ? 1 : 0;
   p.xq = xq;
   p.w_scale = w_scale;

@@ -74,23 +74,45 @@ __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __rest
   q.inv_scale = st->inv_scale;
   q.zp = st->zero_point;
   qparams_finish(q);
+  if (st->rounding == HQ_ROUND_STOCHASTIC) {   // the derive kernel has already counted this iteration
+    q.sr = 1;
+    q.sr_seed = st->seed;
+    q.sr_iter = st->step - 1u;
+  }
   const int64_t groups = count / 16;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) {
     const float4* src = reinterpret_cast<const float4*>(y) + 4 * g;
     uint32_t w[4];
+    if (q.sr) {   // elements 16g .. 16g + 15: two blocks of eight draws
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float4 f = __ldcs(src + e);
-      w[e] = q.fast ? pack_sat4(requant_real<true>(f.x, q), requant_real<true>(f.y, q), requant_real<true>(f.z, q), requant_real<true>(f.w, q))
-                    : pack_sat4(requant_real<false>(f.x, q), requant_real<false>(f.y, q), requant_real<false>(f.z, q), requant_real<false>(f.w, q));
+      for (int b = 0; b < 2; ++b) {
+        uint32_t h[8];
+        sr_draws8(q, (uint64_t)(2 * g + b), h);
+        const float4 f0 = __ldcs(src + 2 * b), f1 = __ldcs(src + 2 * b + 1);
+        w[2 * b] = q.fast ? pack_sat4(requant_real_sr<true>(f0.x, h[0], q), requant_real_sr<true>(f0.y, h[1], q),
+                                      requant_real_sr<true>(f0.z, h[2], q), requant_real_sr<true>(f0.w, h[3], q))
+                          : pack_sat4(requant_real_sr<false>(f0.x, h[0], q), requant_real_sr<false>(f0.y, h[1], q),
+                                      requant_real_sr<false>(f0.z, h[2], q), requant_real_sr<false>(f0.w, h[3], q));
+        w[2 * b + 1] = q.fast ? pack_sat4(requant_real_sr<true>(f1.x, h[4], q), requant_real_sr<true>(f1.y, h[5], q),
+                                          requant_real_sr<true>(f1.z, h[6], q), requant_real_sr<true>(f1.w, h[7], q))
+                              : pack_sat4(requant_real_sr<false>(f1.x, h[4], q), requant_real_sr<false>(f1.y, h[5], q),
+                                          requant_real_sr<false>(f1.z, h[6], q), requant_real_sr<false>(f1.w, h[7], q));
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 f = __ldcs(src + e);
+        w[e] = q.fast ? pack_sat4(requant_real<true>(f.x, q), requant_real<true>(f.y, q), requant_real<true>(f.z, q), requant_real<true>(f.w, q))
+                      : pack_sat4(requant_real<false>(f.x, q), requant_real<false>(f.y, q), requant_real<false>(f.z, q), requant_real<false>(f.w, q));
+      }
     }
     reinterpret_cast<uint4*>(out)[g] = make_uint4(w[0], w[1], w[2], w[3]);
   }
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
   if (blockIdx.x == 0) {
     for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x)
-      out[i] = (int8_t)min(max(requant_real<false>(y[i], q), -128), 127);
+      out[i] = (int8_t)min(max(q.sr ? requant_real_sr<false>(y[i], sr_draw1(q, i), q) : requant_real<false>(y[i], q), -128), 127);
   }
 }
 
@@ -377,6 +399,11 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
+  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
+    q.sr = 1;
+    q.sr_seed = p.yq->seed;
+    q.sr_iter = p.yq->step;
+  }
   const float s_acc = q.s_acc;
   const int zx = q.zx;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = s_acc;
@@ -426,7 +453,7 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
         int c[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) c[k] = q.fast ? requant_acc<true>(acc[4 * e + k], q) : requant_acc<false>(acc[4 * e + k], q);
-        w[e] = pack_sat4(c[0], c[1], c[2], c[3]);
+        w[e] = q.sr ? pack4_sr(acc[4 * e], acc[4 * e + 1], acc[4 * e + 2], acc[4 * e + 3], o + 4 * e, q) : pack_sat4(c[0], c[1], c[2], c[3]);
       }
       *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
     } else {
@@ -480,6 +507,11 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
+  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
+    q.sr = 1;
+    q.sr_seed = p.yq->seed;
+    q.sr_iter = p.yq->step;
+  }
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
   const int CW = p.C / 4;
   const int cw = threadIdx.x % CW, slot = threadIdx.x / CW;
@@ -548,10 +580,11 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
         mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
         const int64_t o = (((int64_t)n * p.Ho + ho) * p.Wo + wo) * p.C + cw * 4;
         if constexpr (kOut == kOutInt8) {
-          const uint32_t w = q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q), requant_acc<true>(acc[j][2], q),
-                                                requant_acc<true>(acc[j][3], q))
-                                    : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
-                                                requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+          const uint32_t w = q.sr     ? pack4_sr(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q)
+                             : q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q), requant_acc<true>(acc[j][2], q),
+                                                  requant_acc<true>(acc[j][3], q))
+                                      : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
+                                                  requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
           *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
         } else {
           uint32_t w[4];
@@ -635,6 +668,11 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
+  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
+    q.sr = 1;
+    q.sr_seed = p.yq->seed;
+    q.sr_iter = p.yq->step;
+  }
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
   for (int i = threadIdx.x; i < p.ncls * p.C; i += blockDim.x) zc_s[i] = q.zx * p.corr[i];
   for (int i = threadIdx.x; i < p.Ho; i += blockDim.x) rcls_s[i] = p.rowcls[i];
@@ -704,10 +742,11 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
             mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
             const int64_t o = o0 + (int64_t)j * p.C;
             if constexpr (kOut == kOutInt8) {
-              const uint32_t w = q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q),
-                                                    requant_acc<true>(acc[j][2], q), requant_acc<true>(acc[j][3], q))
-                                        : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
-                                                    requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+              const uint32_t w = q.sr     ? pack4_sr(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q)
+                                 : q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q),
+                                                      requant_acc<true>(acc[j][2], q), requant_acc<true>(acc[j][3], q))
+                                          : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
+                                                      requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
               *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
             } else {
               uint32_t w[4];

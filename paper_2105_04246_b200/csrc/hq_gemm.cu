@@ -444,6 +444,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
       q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
       qparams_finish(q);
+      if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
+        q.sr = 1;
+        q.sr_seed = p.yq->seed;
+        q.sr_iter = p.yq->step;
+      }
     }
     if (blockIdx.x == 0 && ew == 0 && lane == 0) p.yq->acc_scale = q.s_acc;
     // The epilogue's tables are filled here, by the epilogue warps alone, while the first operand tiles are in flight:
@@ -564,7 +569,28 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         if (nvalid > 0) {
           if constexpr (kOut == kOutInt8) {
             uint32_t w[CW / 4];
-            if (q.fast) {
+            if (q.sr) {   // stochastic rounding, one draw per element (shapes that miss the straight-line pass)
+              const int64_t e0 = pix * p.ldY + p.out_col0 + col0 + c0;
+              int r[CW];
+              if (nvalid == CW && (e0 & 7) == 0) {   // two aligned blocks of eight elements: one generator call each
+#pragma unroll
+                for (int b = 0; b < 2; ++b) {
+                  uint32_t h[8];
+                  sr_draws8(q, ((uint64_t)e0 >> 3) + b, h);
+#pragma unroll
+                  for (int e = 0; e < 8; ++e)
+                    r[8 * b + e] = q.fast ? requant_acc_sr<true>(v[8 * b + e], h[e], q) : requant_acc_sr<false>(v[8 * b + e], h[e], q);
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < CW; ++e)
+                  r[e] = e < nvalid
+                             ? (q.fast ? requant_acc_sr<true>(v[e], sr_draw1(q, e0 + e), q) : requant_acc_sr<false>(v[e], sr_draw1(q, e0 + e), q))
+                             : 0;
+              }
+#pragma unroll
+              for (int e = 0; e < CW / 4; ++e) w[e] = pack_sat4(r[4 * e + 0], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
+            } else if (q.fast) {
 #pragma unroll
               for (int e = 0; e < CW / 4; ++e)
                 w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
@@ -607,6 +633,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       if (lean) {
         const int32_t* zrow = zc_s + zoff;
         int8_t* dst_row = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0;
+        const int64_t elem_row = pix * p.ldY + p.out_col0 + col0;   // linear index in the output tensor of this row's first column
         int tmn = INT32_MAX, tmx = INT32_MIN;
         for (int ch = c_begin; ch < c_end; ++ch) {
           int v[CW];
@@ -631,10 +658,23 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           tmn = __vimin3_s32(tmn, lo[0], lo[1]);
           tmx = __vimax3_s32(tmx, hi[0], hi[1]);
           uint32_t w[CW / 4];
+          if (q.sr) {   // stochastic rounding: the pass covers two aligned blocks of eight elements, one generator call each
+            const uint64_t block = (uint64_t)(elem_row + c0) >> 3;
 #pragma unroll
-          for (int e = 0; e < CW / 4; ++e)
-            w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
-                             requant_acc<true>(v[4 * e + 3], q));
+            for (int b = 0; b < 2; ++b) {
+              uint32_t h[8];
+              sr_draws8(q, block + b, h);
+              w[2 * b] = pack_sat4(requant_acc_sr<true>(v[8 * b + 0], h[0], q), requant_acc_sr<true>(v[8 * b + 1], h[1], q),
+                                   requant_acc_sr<true>(v[8 * b + 2], h[2], q), requant_acc_sr<true>(v[8 * b + 3], h[3], q));
+              w[2 * b + 1] = pack_sat4(requant_acc_sr<true>(v[8 * b + 4], h[4], q), requant_acc_sr<true>(v[8 * b + 5], h[5], q),
+                                       requant_acc_sr<true>(v[8 * b + 6], h[6], q), requant_acc_sr<true>(v[8 * b + 7], h[7], q));
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < CW / 4; ++e)
+              w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
+                               requant_acc<true>(v[4 * e + 3], q));
+          }
           if (row_valid) *reinterpret_cast<uint4*>(dst_row + c0) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         if (row_valid) {

@@ -69,6 +69,7 @@ struct GemmParams {
   uint32_t patch_chunk_stride;        // bytes between channel chunks of one patch (1024-aligned)
   uint32_t patch_box_bytes;           // bytes one patch TMA delivers
   int32_t b_resident;
+  int32_t out_col0;                   // column of the output tensor that column 0 of this launch writes (channel slices)
   int32_t weights_early;              // the weight producer may start before the previous kernel in the stream has finished
   // common
   int32_t Nout, BN;

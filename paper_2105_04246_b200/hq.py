@@ -28,7 +28,7 @@ EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_g
 
 # numpy view of hq_range_state (48 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
-                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("reserved", "<u4", (3,))])
+                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("rounding", "<u4"), ("seed", "<u4"), ("reserved", "<u4")])
 assert RANGE_STATE_DTYPE.itemsize == 48
 INT32_MAX, INT32_MIN = 2**31 - 1, -2**31
 
@@ -204,11 +204,18 @@ def conv_op(kind: int, desc: ConvDesc, X, xq, pw: PreparedWeights, w_scale) -> O
 
 
 # ---- range-state helpers (host-side packing of the plain-data struct) -------------------------------
-def new_states(count: int) -> np.ndarray:
-    """`count` empty states: no range yet (step 0), empty statistics slot."""
+ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
+
+
+def new_states(count: int, sr_seed: int | None = None) -> np.ndarray:
+    """`count` empty states: no range yet (step 0), empty statistics slot.  sr_seed: None = round to nearest even,
+    an integer = stochastic rounding with that seed for the tensors these states describe."""
     s = np.zeros(count, RANGE_STATE_DTYPE)
     s["acc_min"] = INT32_MAX
     s["acc_max"] = INT32_MIN
+    if sr_seed is not None:
+        s["rounding"] = ROUND_STOCHASTIC
+        s["seed"] = int(sr_seed) & 0xFFFFFFFF
     return s
 
 

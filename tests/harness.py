@@ -13,13 +13,14 @@ from paper_2105_04246_b200.synth import QTensor
 class GpuLayer:
     """kind: 'linear' | 'conv_fwd' | 'conv_bwd'.  For conv kinds `shape` is a dict of conv_desc arguments."""
 
-    def __init__(self, ctx: hq.Context, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9):
+    def __init__(self, ctx: hq.Context, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9,
+                 sr_seed: int | None = None):
         self.ctx, self.kind, self.eta = ctx, kind, eta
         self.dev = torch.device("cuda", ctx.device)
         self.W = torch.from_numpy(np.ascontiguousarray(W.q)).to(self.dev)
         self.w_scale = torch.tensor([W.scale], dtype=torch.float32, device=self.dev)
         self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias, dtype=np.int32)).to(self.dev)
-        self.yq = hq.states_to_device(hq.new_states(1), self.dev)
+        self.yq = hq.states_to_device(hq.new_states(1, sr_seed), self.dev)   # sr_seed: stochastic rounding of this layer's output
         self.stream = torch.cuda.current_stream(self.dev)
         if kind == "linear":
             self.N, self.K = W.q.shape
@@ -98,9 +99,10 @@ class GpuLayer:
 
 
 class OracleLayer:
-    def __init__(self, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9):
+    def __init__(self, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9,
+                 sr_seed: int | None = None):
         self.kind, self.W, self.bias = kind, W, bias
-        self.layer = O.Layer(eta)
+        self.layer = O.Layer(eta, sr_seed)
         self.desc = None if kind == "linear" else O.conv_desc(shape["N"], shape["H"], shape["W"], shape["Cin"], shape["K"], shape.get("R", 1),
                                                               shape.get("S", 1), shape.get("stride", 1), shape.get("pad", 0),
                                                               shape.get("groups", 1))

@@ -59,6 +59,18 @@ def test_cfg3_bwd_data_256_full_batch(ctx):
         _compare(t, g.step(x), o.step(x), g, o)
 
 
+def test_cfg3_bwd_data_256_full_batch_stochastic_rounding(ctx):
+    """The gradient layer with the paper's rounding for gradients: same draws on both sides, every code equal."""
+    s = wl.CFG3_BWD
+    r = synth.rng(205)
+    W = synth.weights(r, (s.K, s.R, s.S, s.C))
+    g = GpuLayer(ctx, "conv_bwd", W, _shape(s), sr_seed=424242)
+    o = OracleLayer("conv_bwd", W, _shape(s), sr_seed=424242)
+    for t in range(3):
+        x = synth.tiled(synth.gradients, r, (s.N, s.Ho, s.Wo, s.K))
+        _compare(t, g.step(x), o.step(x), g, o)
+
+
 def test_cfg4_inverted_residual_chain_full_batch(ctx):
     r = synth.rng(203)
     specs = [wl.CFG4_EXPAND, wl.CFG4_DW, wl.CFG4_PROJECT]

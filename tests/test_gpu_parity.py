@@ -25,17 +25,17 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1):
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1, sr_seed=None):
     ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
     ctx.set_option("repack", repack)        # how few-channel inputs are repacked; likewise
     ctx.set_option("depthwise", depthwise)  # CUDA-core kernel or dense expansion on the tensor cores; likewise
     try:
-        g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta)
+        g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
     finally:
         ctx.set_option("staging", -1)
         ctx.set_option("repack", -1)
         ctx.set_option("depthwise", -1)
-    o = OracleLayer(kind, W, shape, bias=bias, eta=eta)
+    o = OracleLayer(kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
     for t in range(iters):
         x = make_x(t)
         if t == 0:
@@ -339,3 +339,42 @@ def test_chained_layers_without_host_sync(ctx, overlap):
     got = hq.states_from_device(states)
     assert_state_close(got[0], oA.layer.state)
     assert_state_close(got[1], oB.layer.state)
+
+
+# ---- stochastic rounding (the paper's rounding for gradients): same draws on both sides, bit-exact codes -----------
+SR_BWD = ["3x3_c64_k64", "3x3_c256_k256_14x14", "3x3_s2_c64_k128", "3x3_s2_odd"]
+
+
+@pytest.mark.parametrize("name", [n for n in SR_BWD if n in BWD_CASES])
+def test_stochastic_rounding_conv_bwd_data(ctx, name):
+    shape = dict(BWD_CASES[name])
+    r = synth.rng(401, len(name), shape["H"])
+    W = _weights(r, shape)
+    Ho = (shape["H"] + 2 * shape["pad"] - shape["R"]) // shape["stride"] + 1
+    Wo = (shape["W"] + 2 * shape["pad"] - shape["S"]) // shape["stride"] + 1
+    in_shape = (shape["N"], Ho, Wo, shape["K"])
+    g, o = _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 4, sr_seed=20210504 + len(name))
+    # the draws differ between iterations and from nearest-even: the codes of the last tensor under nearest-even
+    x = synth.gradients(r, in_shape)
+    acc = o.accumulate(x)
+    rne = O.quantize(acc, o.s_acc(x), o.layer.state)
+    sr = O.quantize_sr(acc, o.s_acc(x), o.layer.state, o.layer.sr_seed, o.layer.state.step)
+    assert 0.05 < (rne != sr).mean() < 0.95
+    assert np.abs(rne.astype(np.int32) - sr.astype(np.int32)).max() <= 1
+
+
+@pytest.mark.parametrize("name", ["1x1_c144_k24", "3x3_c5", "3x3_c64_56x56", "dw3x3_c144", "dw3x3_s2_c32", "dw3x3_c64_wide"])
+def test_stochastic_rounding_conv_fwd_shapes(ctx, name):
+    """Shapes that leave the straight-line pass (ragged columns, 8-byte stores), a depthwise kernel of each kind."""
+    shape = dict(FWD_CASES[name])
+    shape.setdefault("R", 1); shape.setdefault("S", 1)
+    r = synth.rng(402, len(name), shape["H"])
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: synth.signed_activations(r, in_shape), 3, sr_seed=7 + len(name))
+
+
+def test_stochastic_rounding_linear_ragged(ctx):
+    r = synth.rng(403)
+    W = synth.uniform_int8(r, (72, 160), scale=0.02)
+    _run_iterations(ctx, "linear", W, None, lambda t: synth.uniform_int8(r, (300, 160), scale=0.05, zero_point=3), 3, sr_seed=99)
