@@ -68,6 +68,9 @@ typedef enum {
  *                    counter (e >> 3 as two words, step, 0) for the element with linear index e in the
  *                    output tensor: half number (e & 7) of the call's four words, low half first.
  *                    `step` is the value at the time of the call, so every iteration draws anew.
+ *   dynamic_eta      read by hq_dynamic_quant only: 0 (default) = current min-max (Eq. 1); eta in (0,1) =
+ *                    running min-max (Sec. 4.1): the range that quantizes the tensor is
+ *                    (1-eta) * its own min/max + eta * the previous range (first tensor: its min/max).
  * For a layer INPUT only scale and zero_point are read.                                      */
 #define HQ_ROUND_NEAREST_EVEN 0u
 #define HQ_ROUND_STOCHASTIC 1u
@@ -80,7 +83,7 @@ typedef struct {
   int32_t zero_point;
   uint32_t rounding;
   uint32_t seed;
-  uint32_t reserved;
+  float dynamic_eta;
 } hq_range_state;
 
 /* Forward-convolution geometry.  Input N x H x W x C, output N x Ho x Wo x K with

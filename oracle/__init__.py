@@ -213,6 +213,16 @@ def dynamic_sr(acc: np.ndarray, s_acc: float, q: Range, seed: int):
     return yf, out
 
 
+def dynamic_running(acc: np.ndarray, s_acc: float, q: Range, eta: float):
+    """Running min-max: the dynamic path with the moving average of Eq. 2-3 taken over the current tensor's min/max."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    yf = np.empty(acc.shape, np.float32)
+    out = np.empty(acc.shape, np.int8)
+    lib().hqo_dynamic_running(_p(acc, C.c_int32), C.c_int64(acc.size), C.c_float(s_acc), C.byref(q), C.c_float(eta), _p(yf, C.c_float),
+                              _p(out, C.c_int8))
+    return yf, out
+
+
 def acc_scale(s_x: float, s_w: float) -> float:
     return float(lib().hqo_acc_scale(C.c_float(s_x), C.c_float(s_w)))
 

@@ -399,6 +399,36 @@ void hqo_dynamic_sr(const int32_t* acc, int64_t count, float s_acc, hqo_range* q
   for (int64_t i = 0; i < count; ++i) out[i] = quantize_real_sr(yf[i], q, seed, iteration, i);
 }
 
+// ------------------------------------------------------------------------------------
+// Running min-max (Sec. 4.1, last sentences): Eq. 2-3 with the statistics of the CURRENT tensor
+// G^t in place of G^{t-1}: the range that quantizes tensor t is (1-eta) * minmax(G^t) +
+// eta * q^{t-1}.  It is a dynamic method (the tensor's min/max must be known before it can be
+// quantized), so it runs on the dynamic path; eta = 0 is current min-max (Eq. 1); t = 0 takes
+// the min/max of the first tensor.  Same binary32 op order as hqo_range_update.
+// ------------------------------------------------------------------------------------
+void hqo_dynamic_running(const int32_t* acc, int64_t count, float s_acc, hqo_range* q, float eta, float* yf, int8_t* out) {
+  for (int64_t i = 0; i < count; ++i) yf[i] = (float)acc[i] * s_acc;
+  float lo = std::numeric_limits<float>::infinity(), hi = -lo;
+  for (int64_t i = 0; i < count; ++i) {
+    if (yf[i] < lo) lo = yf[i];
+    if (yf[i] > hi) hi = yf[i];
+  }
+  if (count == 0) return;
+  if (q->step == 0 || eta == 0.0f) {
+    q->q_min = lo;
+    q->q_max = hi;
+  } else {
+    float one_minus_eta = 1.0f - eta;
+    float a_lo = one_minus_eta * lo, b_lo = eta * q->q_min;
+    float a_hi = one_minus_eta * hi, b_hi = eta * q->q_max;
+    q->q_min = a_lo + b_lo;
+    q->q_max = a_hi + b_hi;
+  }
+  q->step += 1;
+  hqo_derive(q);
+  for (int64_t i = 0; i < count; ++i) out[i] = quantize_real(yf[i], q);
+}
+
 // s_acc = fl(s_x * s_w): scale of one accumulator unit in real terms
 float hqo_acc_scale(float s_x, float s_w) { return s_x * s_w; }
 

@@ -51,14 +51,23 @@ __global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
   s->acc_max = INT32_MIN;
 }
 
-// Eq. 1: the range is the min/max of the tensor that was just written.
+// Eq. 1: the range is the min/max of the tensor that was just written; with dynamic_eta > 0, its moving average.
 __global__ void dynamic_derive_kernel(hq_range_state* s) {
   grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
   grid_launch_dependents();
   const int mn = s->acc_min, mx = s->acc_max;
   if (mn > mx) return;
-  s->q_min = __fmul_rn(__int2float_rn(mn), s->acc_scale);
-  s->q_max = __fmul_rn(__int2float_rn(mx), s->acc_scale);
+  const float m_lo = __fmul_rn(__int2float_rn(mn), s->acc_scale);
+  const float m_hi = __fmul_rn(__int2float_rn(mx), s->acc_scale);
+  const float eta = s->dynamic_eta;
+  if (s->step == 0 || eta == 0.0f) {   // current min-max
+    s->q_min = m_lo;
+    s->q_max = m_hi;
+  } else {   // running min-max (Sec. 4.1): Eq. 2-3 over the current tensor's statistics
+    const float ome = __fsub_rn(1.0f, eta);
+    s->q_min = __fadd_rn(__fmul_rn(ome, m_lo), __fmul_rn(eta, s->q_min));
+    s->q_max = __fadd_rn(__fmul_rn(ome, m_hi), __fmul_rn(eta, s->q_max));
+  }
   s->step += 1;
   derive_grid(s);
   s->acc_min = INT32_MAX;

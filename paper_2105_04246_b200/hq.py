@@ -28,7 +28,7 @@ EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_g
 
 # numpy view of hq_range_state (48 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
-                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("rounding", "<u4"), ("seed", "<u4"), ("reserved", "<u4")])
+                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("rounding", "<u4"), ("seed", "<u4"), ("dynamic_eta", "<f4")])
 assert RANGE_STATE_DTYPE.itemsize == 48
 INT32_MAX, INT32_MIN = 2**31 - 1, -2**31
 

@@ -378,3 +378,26 @@ def test_stochastic_rounding_linear_ragged(ctx):
     r = synth.rng(403)
     W = synth.uniform_int8(r, (72, 160), scale=0.02)
     _run_iterations(ctx, "linear", W, None, lambda t: synth.uniform_int8(r, (300, 160), scale=0.05, zero_point=3), 3, sr_seed=99)
+
+
+# ---- running min-max on the dynamic path (Sec. 4.1) ----------------------------------------------------------------
+@pytest.mark.parametrize("eta", [0.9, 0.0])
+def test_dynamic_path_running_minmax(ctx, eta):
+    r = synth.rng(404, int(eta * 10))
+    shape = dict(N=2, H=12, W=12, Cin=32, K=48, R=3, S=3, stride=1, pad=1)
+    W = synth.weights(r, (48, 3, 3, 32))
+    g = GpuLayer(ctx, "conv_fwd", W, shape)
+    st = g.state().copy()
+    st["dynamic_eta"] = np.float32(eta)
+    g.set_state(st)
+    o = OracleLayer("conv_fwd", W, shape)
+    q = O.Range()
+    for t in range(5):
+        x = synth.signed_activations(r, (2, 12, 12, 32))
+        x.scale *= float(np.exp(r.normal(0.0, 0.4)))
+        y, ws = g.dynamic(x)
+        acc = o.accumulate(x)
+        yf, codes = O.dynamic_running(acc, o.s_acc(x), q, eta)
+        assert np.array_equal(ws, yf)
+        assert np.array_equal(y, codes), f"iteration {t}"
+        assert_state_close(g.state(), q)

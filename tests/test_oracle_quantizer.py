@@ -175,3 +175,45 @@ def test_hindsight_uses_previous_range_not_current():
     assert np.array_equal(res.q, O.quantize(big, 1.0, before))                # quantized with the OLD range ...
     assert ((res.q == -128) | (res.q == 127)).sum() > 150                    # ... so most of it saturates
     assert layer.state.q_max == pytest.approx(0.1 * 1000 + 0.9 * 100, rel=1e-6)   # and the range then follows
+
+
+# ---- running min-max (Sec. 4.1: Eq. 2-3 over the current tensor's statistics, a dynamic method) ---------------
+def test_running_minmax_eta_zero_is_current_minmax():
+    g = synth.rng(23)
+    acc = g.integers(-7000, 3000, size=777).astype(np.int32)
+    a, b = O.Range(), O.Range(q_min=-50.0, q_max=70.0, step=4)
+    b = O.derive(b)
+    _, cur = O.dynamic(acc, 2e-3, a)
+    _, run0 = O.dynamic_running(acc, 2e-3, b, 0.0)
+    assert np.array_equal(cur, run0)
+    assert (a.q_min, a.q_max) == (b.q_min, b.q_max) and b.step == 5
+
+
+@pytest.mark.parametrize("eta", [0.9, 0.5])
+def test_running_minmax_recurrence_and_use_of_the_current_tensor(eta):
+    g = synth.rng(24, int(eta * 10))
+    s_acc = 1e-3
+    q = O.Range()
+    e = float(np.float32(eta)); s = float(np.float32(s_acc))
+    lo = hi = None
+    for t in range(12):
+        acc = (g.integers(-9000, 9000, size=400) * (1 + t % 3)).astype(np.int32)
+        mn, mx = O.minmax(acc)
+        _, codes = O.dynamic_running(acc, s_acc, q, eta)
+        if t == 0:
+            lo, hi = mn * s, mx * s                                  # first tensor: its own min/max
+        else:
+            lo, hi = (1 - e) * mn * s + e * lo, (1 - e) * mx * s + e * hi   # the CURRENT tensor's statistics enter at once
+        assert q.q_min == pytest.approx(lo, rel=2e-6) and q.q_max == pytest.approx(hi, rel=2e-6)
+        assert q.step == t + 1
+        assert np.array_equal(codes, O.quantize(acc, s_acc, q))      # quantized with the range that already contains it
+    # in contrast to in-hindsight min-max, which quantizes with the range BEFORE the update
+    layer = O.Layer(eta)
+    layer.step(np.arange(-100, 101, dtype=np.int32), 1.0)
+    before = layer.state.copy()
+    big = np.arange(-1000, 1001, 10, dtype=np.int32)
+    res = layer.step(big, 1.0)
+    run = before.copy()
+    _, run_codes = O.dynamic_running(big, 1.0, run, eta)
+    assert not np.array_equal(res.q, run_codes)
+    assert (run.q_min, run.q_max) == (layer.state.q_min, layer.state.q_max)    # same Eq. 2-3 numbers, used one step earlier
