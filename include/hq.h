@@ -131,6 +131,8 @@ const char* hq_last_error(const hq_ctx* ctx);    /* HOST string of the last reje
 hq_status hq_get_async_error(hq_ctx* ctx, void* stream, int32_t* code);
 /* Number of kernel launches this context has enqueued so far (HOST counter). */
 uint64_t hq_launch_count(const hq_ctx* ctx);
+/* Of those, the layer-kernel launches that ran as pairs of CTAs on 256-row tiles (option "pair"). */
+uint64_t hq_pair_launch_count(const hq_ctx* ctx);
 /* Tuning knob (HOST key string), for tests and experiments; results are identical for every value.
  *   "staging": how convolutions prepared AFTER this call bring their input to the MAC array (the
  *              paper's "loaded into the MAC array", Sec. 3.1): -1 = chosen per layer (default),
@@ -148,6 +150,10 @@ uint64_t hq_launch_count(const hq_ctx* ctx);
  *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows
  *              per input row where the shape allows.
+ *   "pair":    layers prepared AFTER this call whose weights stream through shared memory: -1 = chosen per layer
+ *              (default), 0 = every CTA works on its own 128-row tile, 1 = pairs of CTAs on neighbouring SMs share
+ *              256-row tiles (one tensor-core instruction for both, each CTA holding half of the weight rows)
+ *              wherever the layer allows.
  *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their
  *              set-up may run while the previous kernel in the stream drains; each waits for that
  *              kernel to finish before it reads memory, so stream order is unchanged.  0 = ordinary

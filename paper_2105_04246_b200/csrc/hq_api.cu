@@ -191,8 +191,12 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   const uint32_t ring_budget = kSmemBudget - zc_bytes;
   p.zc_offset = ring_budget;
   // ---- operand staging: resident input rows (kModeHalo) where the tile space is stride-1, else one box per tap ----
+  // With CTA pairs (b_rows = BN / 2) each CTA stages half of the rows of B; resident weights are never paired.
+  auto plan_staging = [&](bool pair) -> hq_status {
   p.mode = kModeTap;
-  p.stage_bytes_b = (uint32_t)p.BN * p.BK;
+  p.b_resident = 0;
+  const uint32_t full_stage_b = (uint32_t)p.BN * p.BK;
+  p.stage_bytes_b = pair ? full_stage_b / 2 : full_stage_b;
   bool halo = !sp.flat && sp.in_mul_h == 1 && sp.in_mul_w == 1 && p.ntaps >= 2 && ctx->force_mode != kModeTap;
   if (halo) {
     const int dh_min = *std::min_element(sp.dh.begin(), sp.dh.end()), dh_max = *std::max_element(sp.dh.begin(), sp.dh.end());
@@ -211,15 +215,15 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
            (util >= 0.6 || ctx->force_mode == kModeHalo);
     int stages_a = 0, stages_b = 0, resident = 0;
     if (halo) {
-      if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * p.stage_bytes_b + 2ull * stride <= ring_budget) {
+      if (kiters <= kMaxStagesB && p.tiles_col == 1 && (uint64_t)kiters * full_stage_b + 2ull * stride <= ring_budget) {
         resident = 1;
         stages_b = kiters;
-        stages_a = (int)std::min<uint64_t>(kMaxStagesA, (ring_budget - (uint64_t)kiters * p.stage_bytes_b) / stride);
+        stages_a = (int)std::min<uint64_t>(kMaxStagesA, (ring_budget - (uint64_t)kiters * full_stage_b) / stride);
       } else {
         stages_a = 2;
         while (stages_a < 4 && (uint64_t)(stages_a + 1) * stride + 4ull * p.stage_bytes_b <= ring_budget) ++stages_a;
         if ((uint64_t)stages_a * stride < ring_budget)
-          stages_b = (int)std::min<uint64_t>(8, (ring_budget - (uint64_t)stages_a * stride) / p.stage_bytes_b);
+          stages_b = (int)std::min<uint64_t>(pair ? 12 : 8, (ring_budget - (uint64_t)stages_a * stride) / p.stage_bytes_b);
         if (stages_b < 2) halo = false;
       }
     }
@@ -241,14 +245,18 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
       p.Ht = 1;
       p.Wt = kTileM;
       p.num_tiles = sp.n_img * tiles_per_img * p.tiles_col;
+      p.num_pair_tiles = ceil_div(sp.n_img, 2) * tiles_per_img * p.tiles_col;
       p.producer_lanes = 1;
     }
   }
   if (p.mode == kModeTap) {
+    pick_tile(sp.n_img, sp.TH, sp.TW, sp.in_mul_h, sp.in_mul_w, p.Nt, p.Ht, p.Wt);
+    p.num_tiles = (int)nt;
+    p.num_pair_tiles = ceil_div(p.tiles_n * p.tiles_h * p.tiles_w, 2) * p.tiles_col;
     p.stage_bytes_a = (uint32_t)kTileM * p.BK;
     // a small weight matrix stays in shared memory for the whole kernel; the ring then carries operand A only
     const int kiters = p.ntaps * p.chunks_per_tap;
-    const uint64_t b_all = (uint64_t)p.tiles_col * kiters * p.stage_bytes_b;
+    const uint64_t b_all = (uint64_t)p.tiles_col * kiters * full_stage_b;
     if (kiters > 0 && p.tiles_col * kiters <= kMaxStagesB && b_all <= 64u * 1024u && b_all + 6ull * p.stage_bytes_a <= ring_budget) {
       p.b_resident = 1;
       p.stages_b = p.tiles_col * kiters;
@@ -260,6 +268,23 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     if (p.stages_a < 2) return fail(ctx, HQ_ERR_UNSUPPORTED, "operand tiles do not fit in shared memory");
     p.producer_lanes = std::min(4, p.stages_a);
   }
+  return HQ_OK;
+  };
+  // CTA pairs pay where the weights stream through shared memory and the tile is wide: each CTA then copies and reads
+  // half of the rows of B per 128 rows of output.  Never for flat (1x1 / linear) layers, which the epilogue bounds.
+  bool want_pair = ctx->force_pair != 0 && !sp.flat && p.ntaps >= 1 && p.tiles_n * p.tiles_h * p.tiles_w >= 2 &&
+                   (p.BN >= 128 || ctx->force_pair == 1);
+  {
+    hq_status pst = plan_staging(want_pair);
+    if (pst != HQ_OK) return pst;
+    if (want_pair && (p.b_resident || (p.mode == kModeHalo && sp.n_img < 2))) {
+      want_pair = false;
+      pst = plan_staging(false);
+      if (pst != HQ_OK) return pst;
+    }
+  }
+  p.pair = want_pair ? 1 : 0;
+  if (p.pair) p.idesc = (p.idesc & ~(0x1Fu << 24)) | ((uint32_t)(2 * kTileM >> 4) << 24);   // M = 256 across the pair
   sub.smem_bytes = kSmemBudget + 1024;
   sub.a_flat = sp.flat;
   sub.a_stride_h = sp.in_mul_h;
@@ -273,7 +298,7 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     const int a_per_tile = p.mode == kModeHalo ? p.chunks_per_tap : kiters;
     const int b_per_tile = (p.mode == kModeHalo && !p.b_resident) ? kiters : 0;
     const bool rings_ok = 2 * a_per_tile <= p.stages_a && (b_per_tile == 0 || 2 * b_per_tile <= p.stages_b);
-    p.mma_issuers = (rings_ok && kiters > 0 && p.num_tiles >= 2 * ctx->num_sms) ? 2 : 1;
+    p.mma_issuers = (rings_ok && kiters > 0 && p.num_tiles >= 2 * ctx->num_sms && !p.pair) ? 2 : 1;
     // many small tiles per CTA: four epilogue groups; few large ones: all warps on every tile (shortest tail)
     const int tiles_per_cta = ceil_div(p.num_tiles, ctx->num_sms);
     p.epi_groups_log2 = tiles_per_cta >= 8 ? std::min(2, p.tmem_bufs_log2) : 0;
@@ -300,7 +325,7 @@ hq_status encode_b(hq_ctx* ctx, const hq_sub_problem& sub, const int8_t* wmat, i
   const GemmParams& p = sub.p;
   uint64_t dims[2] = {(uint64_t)row_bytes, (uint64_t)p.Nout};
   uint64_t strides[1] = {(uint64_t)row_bytes};
-  uint32_t box[2] = {(uint32_t)p.BK, (uint32_t)p.BN};
+  uint32_t box[2] = {(uint32_t)p.BK, (uint32_t)(p.pair ? p.BN / 2 : p.BN)};   // a pair's CTAs fetch half of the rows each
   uint32_t es[2] = {1, 1};
   return encode_map(ctx, m, wmat, 2, dims, strides, box, es, p.swizzle64, true);
 }
@@ -403,9 +428,21 @@ hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, con
   p.bias = bias;
   p.out = out;
   p.yq = yq;
-  const int grid = std::max(1, std::min(p.num_tiles, max_ctas > 0 ? max_ctas : ctx->num_sms));
-  HQ_CUDA(ctx, launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s, ctx->overlap));
+  int grid = std::max(1, std::min(p.num_tiles, max_ctas > 0 ? max_ctas : ctx->num_sms));
+  if (p.pair) {   // clusters of two: one pair per two SMs
+    const int pairs = std::max(1, (max_ctas > 0 ? max_ctas : ctx->num_sms) / 2);
+    grid = 2 * std::max(1, std::min(p.num_pair_tiles, pairs));
+  }
+  {
+    const cudaError_t le = launch_gemm(p, ta, tb, out_mode, grid, sub.smem_bytes, s, ctx->overlap);
+    if (le != cudaSuccess) {
+      (void)cudaGetLastError();   // a rejected launch leaves no work behind; clear it so that later calls start clean
+      return fail(ctx, HQ_ERR_CUDA, "layer kernel launch failed: %s (grid %d, pair %d, tiles %d, pair tiles %d, mode %d, BN %d)",
+                  cudaGetErrorString(le), grid, p.pair, p.num_tiles, p.num_pair_tiles, p.mode, p.BN);
+    }
+  }
   ctx->launches += 1;
+  ctx->pair_launches += p.pair ? 1 : 0;
   return HQ_OK;
 }
 
@@ -708,6 +745,7 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
 __attribute__((visibility("default"))) const char* hq_last_error(const hq_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 
 __attribute__((visibility("default"))) uint64_t hq_launch_count(const hq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+__attribute__((visibility("default"))) uint64_t hq_pair_launch_count(const hq_ctx* ctx) { return ctx ? ctx->pair_launches : 0; }
 
 __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, const char* key, int32_t value) {
   if (!ctx || !key) return HQ_ERR_INVALID_ARG;
@@ -734,6 +772,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "repack") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "repack must be -1, 0 or 1");
     ctx->force_repack = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "pair") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "pair must be -1, 0 or 1");
+    ctx->force_pair = value;
     return HQ_OK;
   }
   if (std::string(key) == "overlap_launches") {

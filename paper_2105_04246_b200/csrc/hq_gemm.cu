@@ -47,6 +47,30 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// CTA pair: one instruction drives the tensor cores of both SMs (rows 0..127 of the 256-row tile come from this CTA's
+// operand A, rows 128..255 from the peer's at the same shared-memory offset; each CTA holds half of the rows of B);
+// the commit arrives on the barrier at the same offset in both CTAs.
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"((uint16_t)3)
+               : "memory");
+}
+template <bool kPair>
+__device__ __forceinline__ void mma_any(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (kPair) umma_i8_pair(d_tmem, adesc, bdesc, idesc, accumulate);
+  else umma_i8(d_tmem, adesc, bdesc, idesc, accumulate);
+}
+template <bool kPair>
+__device__ __forceinline__ void commit_any(uint32_t bar) {
+  if constexpr (kPair) umma_commit_pair(bar);
+  else umma_commit(bar);
+}
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int* v) {
   asm volatile(
@@ -78,7 +102,9 @@ __device__ __forceinline__ void store_bytes16(int8_t* p, const uint32_t* w, int 
   }
 }
 
-template <int kOut>
+// kPairK: the instantiation that runs as clusters of two CTAs (its cta_group::2 instructions make the launch
+// require an even cluster size, so single-CTA launches use the other instantiation).
+template <int kOut, bool kPairK>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                int out_vec) {
@@ -108,22 +134,36 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + 8 + b); };
   const int nbuf = p.tmem_bufs, nbuf_log2 = p.tmem_bufs_log2;   // accumulator buffers in TMEM (2 or 4)
+  // CTA pair (cluster of two): both CTAs walk over the same sequence of 256-row pair tiles, each with its own 128 rows
+  // of A and half of the rows of B; the MMA issuer of rank 0 drives both tensor cores.  "Full" barriers and the
+  // accumulator's "empty" barriers are those of rank 0 (the peer reports to them remotely); operand "empty" and
+  // accumulator "full" barriers are local in both CTAs and receive the issuer's multicast commits.
+  constexpr bool pair = kPairK;
+  uint32_t crank = 0u, bar0_lead = bar0;
+  if constexpr (kPairK) {
+    crank = cluster_cta_rank();
+    bar0_lead = map_to_cta(bar0, 0u);
+  }
+  auto a_full_lead = [&](int s) { return bar0_lead + 8u * s; };
+  auto b_full_lead = [&](int s) { return bar0_lead + 8u * (2 * kMaxStagesA + s); };
+  auto tempty_lead = [&](int b) { return bar0_lead + 8u * (2 * kMaxStagesA + 2 * kMaxStagesB + 8 + b); };
+  const int ncta = pair ? 2 : 1;
 
   const int kiters = p.ntaps * p.chunks_per_tap;
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < p.stages_a; ++s) {
-      mbar_init(a_full(s), 1);
+      mbar_init(a_full(s), ncta);   // one arrival (with its byte count) per producing CTA
       mbar_init(a_empty(s), 1);
     }
     for (int s = 0; s < p.stages_b; ++s) {
-      mbar_init(b_full(s), 1);
+      mbar_init(b_full(s), ncta);
       mbar_init(b_empty(s), 1);
     }
     for (int b = 0; b < nbuf; ++b) {
       mbar_init(tfull_bar(b), 1);
-      mbar_init(tempty_bar(b), kEpilogueWarps >> p.epi_groups_log2);   // one arrival per warp of the group that drains it
+      mbar_init(tempty_bar(b), ncta * (kEpilogueWarps >> p.epi_groups_log2));   // one arrival per warp of the group(s) that drain it
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -137,12 +177,19 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmap_b) : "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(p.tmem_cols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if constexpr (kPairK) {   // the pair's accumulators: the same columns in both CTAs' tensor memory
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(p.tmem_cols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(p.tmem_cols)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if constexpr (kPairK) cluster_sync_all();   // the peer's barriers exist before anything arrives on them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
   // Everything above touched only kernel parameters and this CTA's own resources.  From here on the kernel reads
@@ -167,7 +214,29 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       n0 = t3 * p.Nt;
     }
   };
-  const int my_tiles = (p.num_tiles > (int)blockIdx.x) ? (p.num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  // The CTA's it-th tile, or -1 when it has none left.  A pair takes pair tile (pair index + it * pairs): rank r gets
+  // row tile 2q + r (kModeTap) or the same tile of image 2a + r (kModeHalo: both halves of the pair then start at the
+  // same pixel of their patch, as the shared matrix descriptor requires).  Row tiles past the end are computed on
+  // zero-filled operands and dropped by the epilogue.
+  auto own_tile = [&](int it) -> int {
+    if (!pair) {
+      const int tile = (int)blockIdx.x + it * (int)gridDim.x;
+      return tile < p.num_tiles ? tile : -1;
+    }
+    const int pt = (int)(blockIdx.x >> 1) + it * (int)(gridDim.x >> 1);
+    if (pt >= p.num_pair_tiles) return -1;
+    const int q = fdiv(pt, p.fd_tiles_col);
+    const int ct = pt - q * p.tiles_col;
+    int mt;
+    if (halo) {
+      const int a = fdiv(q, p.fd_tiles_per_img);
+      mt = (2 * a + (int)crank) * p.tiles_per_img + (q - a * p.tiles_per_img);
+    } else {
+      mt = 2 * q + (int)crank;
+    }
+    return mt * p.tiles_col + ct;
+  };
+  const int my_tiles = own_tile(0) >= 0 ? 1 : 0;   // only "has any" is used
 
   // The three single-issuer roles below are executed by their WHOLE warp with warp-uniform control flow and
   // values; only the copy / MMA / commit instructions themselves sit under a one-lane predicate (elect.sync).
@@ -178,7 +247,10 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+      const int b_row_off = (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
+      for (int it = 0; ok; ++it) {
+        const int tile = own_tile(it);
+        if (tile < 0) break;
         int n0, h0, w0, col0;
         decode(tile, n0, h0, w0, col0);
         if (halo) {
@@ -187,8 +259,13 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
             ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
             if (!ok) break;
             if (elect_one()) {
-              mbar_expect_tx(a_full(stage), p.patch_box_bytes);
-              tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
+              if constexpr (kPairK) {
+                mbar_expect_tx_remote(a_full_lead(stage), p.patch_box_bytes);
+                tma_load_4d_pair(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full_lead(stage));
+              } else {
+                mbar_expect_tx(a_full(stage), p.patch_box_bytes);
+                tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
+              }
             }
             if (++stage == p.stages_a) {
               stage = 0;
@@ -204,9 +281,15 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
               if (!ok) break;
               const uint32_t sa = ring_a + stage * a_stride;
               if (elect_one()) {
-                mbar_expect_tx(a_full(stage), a_stride);
-                tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
-                if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+                if constexpr (kPairK) {   // never with resident weights
+                  mbar_expect_tx_remote(a_full_lead(stage), a_stride);
+                  tma_load_4d_pair(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full_lead(stage));
+                  tma_load_2d_pair(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0 + b_row_off, a_full_lead(stage));
+                } else {
+                  mbar_expect_tx(a_full(stage), a_stride);
+                  tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
+                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+                }
               }
               if (++stage == p.stages_a) {
                 stage = 0;
@@ -248,15 +331,22 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
-          const int col0 = (tile % p.tiles_col) * p.BN;
+        for (int it = 0; ok; ++it) {
+          const int tile = own_tile(it);
+          if (tile < 0) break;
+          const int col0 = (tile % p.tiles_col) * p.BN + (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
           for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
             for (int t = 0; t < p.ntaps; ++t) {
               ok = warp_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait, 1000u);
               if (!ok) break;
               if (elect_one()) {
-                mbar_expect_tx(b_full(stage), p.stage_bytes_b);
-                tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
+                if constexpr (kPairK) {
+                  mbar_expect_tx_remote(b_full_lead(stage), p.stage_bytes_b);
+                  tma_load_2d_pair(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full_lead(stage));
+                } else {
+                  mbar_expect_tx(b_full(stage), p.stage_bytes_b);
+                  tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
+                }
               }
               if (++stage == p.stages_b) {
                 stage = 0;
@@ -276,8 +366,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int nissuers = p.mma_issuers;
     // The k-steps of one operand stage are issued from a compile-time unrolled group: a run-time inner loop
     // around the MMA instruction was measured to cost several hundred cycles per iteration.
-    auto mma_role = [&](auto kk_tag) {
+    auto mma_role = [&](auto kk_tag, auto pair_tag) {
       constexpr int KK = decltype(kk_tag)::value;
+      constexpr bool kPair = decltype(pair_tag)::value;
       int stage = 0, bstage = 0;
       uint32_t phase = 0, bphase = 0;
       bool ok = true;
@@ -303,8 +394,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       const uint32_t idesc = p.idesc;
       const uint32_t bstep16 = p.stage_bytes_b >> 4;
       for (int local_tile = issuer; ok; local_tile += nissuers) {
-        const int tile = (int)blockIdx.x + local_tile * (int)gridDim.x;
-        if (tile >= p.num_tiles) break;
+        const int tile = own_tile(local_tile);
+        if (tile < 0) break;
         const int buf = local_tile & (nbuf - 1);
         const uint32_t tph = (uint32_t)(local_tile >> nbuf_log2) & 1u;
         ok = warp_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait, 200u);
@@ -331,7 +422,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                 const uint64_t adesc = abase + tapoff_s[t];
                 if (elect_one()) {
 #pragma unroll
-                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                  for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
                 }
                 bres += bstep16;
               }
@@ -342,7 +433,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                 for (int t = 0; t < ntaps; ++t) {
                   const uint64_t adesc = abase + tapoff_s[t];
 #pragma unroll
-                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                  for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
                   bres += bstep16;
                 }
               }
@@ -357,8 +448,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                 const uint64_t adesc = abase + tapoff_s[t];
                 if (elect_one()) {
 #pragma unroll
-                  for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
-                  umma_commit(b_empty(bstage));
+                  for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
+                  commit_any<kPair>(b_empty(bstage));
                 }
                 acc = 1;
                 if (++bstage == stages_b) {
@@ -368,7 +459,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
               }
             }
             if (!ok) break;
-            if (elect_one()) umma_commit(a_empty(stage));
+            if (elect_one()) commit_any<kPair>(a_empty(stage));
             if (++stage == p.stages_a) {
               stage = 0;
               phase ^= 1u;
@@ -395,8 +486,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
             const uint64_t bdesc = resident ? bres + (uint64_t)ki * bstep16 : make_smem_desc(sa + p.stage_bytes_a, sw64);
             if (elect_one()) {
 #pragma unroll
-              for (int k = 0; k < KK; ++k) umma_i8(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
-              umma_commit(a_empty(stage));
+              for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
+              commit_any<kPair>(a_empty(stage));
             }
             acc = 1;
             if (++stage == p.stages_a) {
@@ -406,7 +497,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           }
           if (!ok) break;
         }
-        if (elect_one()) umma_commit(tfull_bar(buf));
+        if (elect_one()) commit_any<kPair>(tfull_bar(buf));
         first = false;
         if (nissuers > 1) {   // step over the other issuer's tile
           advance(stage, phase, (nissuers - 1) * a_per_tile, p.stages_a);
@@ -414,9 +505,14 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         }
       }
     };
-    if (kiters > 0) {
-      if (p.BK == 64) mma_role(std::integral_constant<int, 2>{});
-      else mma_role(std::integral_constant<int, 4>{});
+    if (kiters > 0 && crank == 0) {   // in a pair, rank 0 issues for both CTAs
+      if constexpr (kPairK) {
+        if (p.BK == 64) mma_role(std::integral_constant<int, 2>{}, std::true_type{});
+        else mma_role(std::integral_constant<int, 4>{}, std::true_type{});
+      } else {
+        if (p.BK == 64) mma_role(std::integral_constant<int, 2>{}, std::false_type{});
+        else mma_role(std::integral_constant<int, 4>{}, std::false_type{});
+      }
     }
     __syncwarp();
     // All MMAs of this CTA are issued; what is left is the epilogue of the last tiles.  The next kernel in the stream
@@ -475,8 +571,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     // per-layer part of the condition for the straight-line pass (see below)
     const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.zc_in_smem && has_corr;
     for (int local_tile = group; ; local_tile += ngroups) {
-      const int tile = (int)blockIdx.x + local_tile * (int)gridDim.x;
-      if (tile >= p.num_tiles) break;
+      const int tile = own_tile(local_tile);
+      if (tile < 0) break;
       int n0, h0, w0, col0;
       decode(tile, n0, h0, w0, col0);
       int n, i, j;
@@ -486,7 +582,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         n = n0;
         i = fdiv(o, p.fd_P);
         j = o - i * p.P;
-        row_valid = (o < p.L) && (j < p.TW);
+        row_valid = (o < p.L) && (j < p.TW) && (n < p.n_img);
       } else {
         n = n0 + rn;
         i = h0 + rh;
@@ -699,7 +795,10 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       if (kiters > 0) {
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(buf));
+        if (lane == 0) {
+          if constexpr (kPairK) mbar_arrive_remote(tempty_lead(buf));
+          else mbar_arrive(tempty_bar(buf));
+        }
       }
     }
     // statistics: registers -> warp -> CTA -> one atomic pair per CTA
@@ -723,21 +822,29 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   }
 
   tc_fence_before();
-  __syncthreads();
+  if constexpr (kPairK) cluster_sync_all();   // neither CTA leaves while the other may still read its operands or arrive on its barriers
+  else __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    if constexpr (kPairK) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
   }
 }
 
 }  // namespace
 
+template <int kOut, bool kPairK>
+cudaError_t set_smem_attr_one(uint32_t smem_bytes) {
+  return cudaFuncSetAttribute(hq_gemm_kernel<kOut, kPairK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+}
 cudaError_t gemm_set_smem_attr(uint32_t smem_bytes) {
-  cudaError_t e = cudaFuncSetAttribute(hq_gemm_kernel<kOutInt8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(hq_gemm_kernel<kOutF32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(hq_gemm_kernel<kOutAcc>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  cudaError_t e;
+  if ((e = set_smem_attr_one<kOutInt8, false>(smem_bytes)) != cudaSuccess) return e;
+  if ((e = set_smem_attr_one<kOutF32, false>(smem_bytes)) != cudaSuccess) return e;
+  if ((e = set_smem_attr_one<kOutAcc, false>(smem_bytes)) != cudaSuccess) return e;
+  if ((e = set_smem_attr_one<kOutInt8, true>(smem_bytes)) != cudaSuccess) return e;
+  if ((e = set_smem_attr_one<kOutF32, true>(smem_bytes)) != cudaSuccess) return e;
+  return set_smem_attr_one<kOutAcc, true>(smem_bytes);
 }
 
 cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int out_mode, int grid, uint32_t smem_bytes,
@@ -753,10 +860,17 @@ cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtens
   } else {
     out_vec = (p.ldY % 4 == 0 && addr % 16 == 0) ? 16 : 4;
   }
+  if (p.pair) {   // grid is an even number of CTAs: clusters of two
+    switch (out_mode) {
+      case kOutInt8: return launch_overlapped_cluster(hq_gemm_kernel<kOutInt8, true>, grid, kGemmThreads, smem_bytes, s, overlap, 2u, p, ta, tb, out_vec);
+      case kOutF32: return launch_overlapped_cluster(hq_gemm_kernel<kOutF32, true>, grid, kGemmThreads, smem_bytes, s, overlap, 2u, p, ta, tb, out_vec);
+      default: return launch_overlapped_cluster(hq_gemm_kernel<kOutAcc, true>, grid, kGemmThreads, smem_bytes, s, overlap, 2u, p, ta, tb, out_vec);
+    }
+  }
   switch (out_mode) {
-    case kOutInt8: return launch_overlapped(hq_gemm_kernel<kOutInt8>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
-    case kOutF32: return launch_overlapped(hq_gemm_kernel<kOutF32>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
-    default: return launch_overlapped(hq_gemm_kernel<kOutAcc>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
+    case kOutInt8: return launch_overlapped(hq_gemm_kernel<kOutInt8, false>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
+    case kOutF32: return launch_overlapped(hq_gemm_kernel<kOutF32, false>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
+    default: return launch_overlapped(hq_gemm_kernel<kOutAcc, false>, grid, kGemmThreads, smem_bytes, s, overlap, p, ta, tb, out_vec);
   }
 }
 

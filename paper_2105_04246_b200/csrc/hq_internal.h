@@ -89,6 +89,9 @@ struct GemmParams {
   uint32_t idesc;
   uint32_t tmem_cols, tmem_buf_stride;
   int32_t mma_issuers;                // 1 or 2 warps issuing MMAs (alternate tiles)
+  int32_t pair;                       // 1: launched as clusters of two CTAs that share 256-row tiles (tcgen05 cta_group::2);
+                                      //    stage_bytes_b and the B tensor map's box then cover BN/2 rows
+  int32_t num_pair_tiles;             // pair tiles (two row tiles x one column tile)
   int32_t tmem_bufs, tmem_bufs_log2;   // accumulator buffers in TMEM (2, 4 or 8)
   int32_t epi_groups_log2;             // epilogue warp groups: 1, 2 or 4 (<= buffers)
   int32_t stages_a, stages_b;
@@ -143,6 +146,26 @@ cudaError_t launch_overlapped(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
   cfg.numAttrs = overlap ? 1u : 0u;
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
+// the same, as thread-block clusters of `cluster` consecutive CTAs (grid.x a multiple of it)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_overlapped_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool overlap, unsigned cluster,
+                                      Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 2u : 1u;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 #ifdef __CUDACC__
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -189,10 +212,12 @@ struct hq_ctx {
   size_t pad_bytes = 0;
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
+  uint64_t pair_launches = 0;         // of those, layer kernels launched as CTA pairs
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
   int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
+  int force_pair = -1;                // CTA pairs on 256-row tiles: -1 choose per layer, 0 never, 1 wherever the layer allows
   cudaStream_t side[3] = {nullptr, nullptr, nullptr};   // independent launches of one call run side by side (see run_conv)
   cudaEvent_t ev_fork = nullptr, ev_join[3] = {nullptr, nullptr, nullptr};
   bool parallel_subs = true;

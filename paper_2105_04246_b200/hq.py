@@ -22,7 +22,8 @@ DIR_FWD, DIR_BWD_DATA = 0, 1
 OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 
 # every extern "C" symbol include/hq.h declares
-EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_set_option",
+EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_pair_launch_count",
+           "hq_set_option",
            "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
            "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate"]
 
@@ -66,6 +67,7 @@ def lib():
         L.hq_last_error.argtypes = [vp]; L.hq_last_error.restype = C.c_char_p
         L.hq_get_async_error.argtypes = [vp, vp, C.POINTER(i32)]
         L.hq_launch_count.argtypes = [vp]; L.hq_launch_count.restype = C.c_uint64
+        L.hq_pair_launch_count.argtypes = [vp]; L.hq_pair_launch_count.restype = C.c_uint64
         L.hq_set_option.argtypes = [vp, C.c_char_p, i32]
         L.hq_weights_prepare.argtypes = [vp, vp, C.POINTER(ConvDesc), C.c_int, vp, C.POINTER(vp)]
         L.hq_weights_release.argtypes = [vp, vp]
@@ -77,7 +79,7 @@ def lib():
         L.hq_debug_accumulate.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
         L.hq_dynamic_quant_static.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
         for name in EXPORTS:
-            if name not in ("hq_status_string", "hq_last_error", "hq_launch_count"):
+            if name not in ("hq_status_string", "hq_last_error", "hq_launch_count", "hq_pair_launch_count"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -191,6 +193,9 @@ class Context:
 
     def launch_count(self) -> int:
         return int(lib().hq_launch_count(self.handle))
+
+    def pair_launch_count(self) -> int:
+        return int(lib().hq_pair_launch_count(self.handle))
 
 
 def linear_op(M, N, K, X, xq, W, w_scale, bias=None) -> OpDesc:

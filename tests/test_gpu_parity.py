@@ -25,14 +25,16 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1, sr_seed=None):
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1, sr_seed=None, pair=-1):
     ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
+    ctx.set_option("pair", pair)            # one CTA per 128-row tile or CTA pairs on 256-row tiles; likewise
     ctx.set_option("repack", repack)        # how few-channel inputs are repacked; likewise
     ctx.set_option("depthwise", depthwise)  # CUDA-core kernel or dense expansion on the tensor cores; likewise
     try:
         g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
     finally:
         ctx.set_option("staging", -1)
+        ctx.set_option("pair", -1)
         ctx.set_option("repack", -1)
         ctx.set_option("depthwise", -1)
     o = OracleLayer(kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
@@ -202,6 +204,45 @@ def test_conv_bwd_data(ctx, name, staging):
     Wo = (shape["W"] + 2 * shape.get("pad", 0) - shape["S"]) // shape.get("stride", 1) + 1
     in_shape = (shape["N"], Ho, Wo, shape["K"])
     _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3, staging=staging)
+
+
+# CTA pairs (tcgen05 cta_group::2): layers whose weights stream through shared memory, in both staging modes; odd image
+# and tile counts leave the second CTA of the last pair with a tile of padding only
+PAIR_FWD = ["3x3_c128_k256", "3x3_c256_k512_7x7", "3x3_c512_k512_7x7", "3x3_s2_c64_k128_30x30", "3x3_c256_k256_14x14_n5", "3x3_c128_k128_20x20_n3"]
+PAIR_EXTRA = {
+    "3x3_s2_c64_k128_30x30": dict(N=3, H=30, W=30, Cin=64, K=128, R=3, S=3, stride=2, pad=1),
+    "3x3_s2_c128_k256_18x18": dict(N=3, H=18, W=18, Cin=128, K=256, R=3, S=3, stride=2, pad=1),
+    "3x3_c256_k256_14x14_n5": dict(N=5, H=14, W=14, Cin=256, K=256, R=3, S=3, stride=1, pad=1),
+    "3x3_c128_k128_20x20_n3": dict(N=3, H=20, W=20, Cin=128, K=320, R=3, S=3, stride=1, pad=1),
+}
+
+
+@pytest.mark.parametrize("staging", [0, 1])
+@pytest.mark.parametrize("name", PAIR_FWD)
+def test_conv_fwd_cta_pairs(ctx, name, staging):
+    shape = dict(FWD_CASES.get(name) or PAIR_EXTRA[name])
+    r = synth.rng(107, len(name), shape["H"], shape["Cin"])
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
+    n0 = ctx.pair_launch_count()
+    _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, staging=staging, pair=1)
+    assert ctx.pair_launch_count() > n0, "the layer did not run as CTA pairs"
+
+
+@pytest.mark.parametrize("staging", [0, 1])
+@pytest.mark.parametrize("name", ["3x3_c256_k256_14x14", "3x3_s2_c128_k256_18x18"])
+def test_conv_bwd_data_cta_pairs(ctx, name, staging):
+    shape = dict(BWD_CASES.get(name) or PAIR_EXTRA[name])
+    r = synth.rng(108, len(name), shape["H"], shape["Cin"])
+    W = _weights(r, shape)
+    Ho = (shape["H"] + 2 * shape.get("pad", 0) - shape["R"]) // shape.get("stride", 1) + 1
+    Wo = (shape["W"] + 2 * shape.get("pad", 0) - shape["S"]) // shape.get("stride", 1) + 1
+    in_shape = (shape["N"], Ho, Wo, shape["K"])
+    n0 = ctx.pair_launch_count()
+    _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3, staging=staging, pair=1)
+    if staging == 0 or "s2" not in name:   # with resident input rows the small parity classes keep their weights resident: no pairs
+        assert ctx.pair_launch_count() > n0, "the layer did not run as CTA pairs"
 
 
 # ---- protocol and edge cases ---------------------------------------------------------------------
