@@ -150,6 +150,9 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows
  *              per input row where the shape allows.
+ *   "col_tiles": into how many column tiles (each a multiple of 16 columns, at most 256) the output channels of
+ *              layers prepared AFTER this call are split: -1 = chosen per layer by estimated duration (default),
+ *              0 = as few as possible, n > 0 = at least n.
  *   "pair":    layers prepared AFTER this call whose weights stream through shared memory: -1 = chosen per layer
  *              (default), 0 = every CTA works on its own 128-row tile, 1 = pairs of CTAs on neighbouring SMs share
  *              256-row tiles (one tensor-core instruction for both, each CTA holding half of the weight rows)

@@ -116,11 +116,13 @@ struct SubSpec {            // geometry of one launch, before tiling
   int out_H, out_W, os_h, os_w, oa_h, oa_w;
   int64_t ldY;
   bool flat;
+  bool whole_gpu = true;    // false: the launch shares the SMs with other launches of the same call
 };
 
-// fills everything in sub.p that does not depend on per-call pointers
-hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
-                   std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks) {
+// fills everything in sub.p that does not depend on per-call pointers, for a given number of column tiles
+// (ncol_req = 0: as few as the MMA allows) and a given answer to "CTA pairs?" (pair_req: 0 no, 1 where the layer allows)
+hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
+                         std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks, int ncol_req, int pair_req) {
   GemmParams& p = sub.p;
   p.n_img = sp.n_img;
   p.TH = sp.TH;
@@ -149,7 +151,7 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   p.Nout = sp.Nout;
   // column tiles: as wide as the MMA allows, except for very short reductions, where the epilogue is the bottleneck and
   // narrower tiles give it four or more accumulator buffers to work on
-  const int ncol = ceil_div(sp.Nout, p.ntaps * p.Cpad <= 128 ? 128 : 256);
+  const int ncol = std::max(ncol_req, ceil_div(sp.Nout, p.ntaps * p.Cpad <= 128 ? 128 : 256));
   p.BN = round_up(ceil_div(sp.Nout, ncol), 16);
   p.tiles_col = ceil_div(sp.Nout, p.BN);
   const int64_t nt = (int64_t)p.tiles_n * p.tiles_h * p.tiles_w * p.tiles_col;
@@ -272,8 +274,7 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   };
   // CTA pairs pay where the weights stream through shared memory and the tile is wide: each CTA then copies and reads
   // half of the rows of B per 128 rows of output.  Never for flat (1x1 / linear) layers, which the epilogue bounds.
-  bool want_pair = ctx->force_pair != 0 && !sp.flat && p.ntaps >= 1 && p.tiles_n * p.tiles_h * p.tiles_w >= 2 &&
-                   (p.BN >= 128 || ctx->force_pair == 1);
+  bool want_pair = pair_req != 0 && !sp.flat && p.ntaps >= 1 && p.tiles_n * p.tiles_h * p.tiles_w >= 2;
   {
     hq_status pst = plan_staging(want_pair);
     if (pst != HQ_OK) return pst;
@@ -309,6 +310,34 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
   p.fd_tiles_h = make_fastdiv(p.tiles_h);
   p.fd_P = make_fastdiv(p.mode == kModeHalo ? p.P : 1);
   return HQ_OK;
+}
+
+// Chooses the number of column tiles and single CTAs or CTA pairs, by rules taken from measurements on B200:
+//  * CTA pairs pay where the input rows are resident and the weights stream through shared memory (each SM then copies
+//    half of the weight rows per 128 rows of output); with one copy per filter tap they do not, and on strided or
+//    single-tap layers they cost time;
+//  * narrower column tiles only pay where the widest ones leave SMs without any tile (few row tiles: 7x7 images): then
+//    as many column tiles as still fit in one round, none narrower than 64 columns.  Everywhere else splitting the
+//    columns multiplies the traffic of operand A and is much slower.
+hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
+                   std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks) {
+  if (sp.flat) return plan_sub_fixed(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks, std::max(0, ctx->force_cols), 0);
+  int ncol = std::max(0, ctx->force_cols);
+  int pair = ctx->force_pair;
+  if (ctx->force_cols < 0 || ctx->force_pair < 0) {
+    hq_sub_problem trial = sub;
+    std::vector<uint8_t> rc, cc;
+    std::vector<uint32_t> rm, cm;
+    hq_status st = plan_sub_fixed(ctx, sp, trial, rc, cc, rm, cm, ncol, 0);
+    if (st != HQ_OK) return st;
+    const GemmParams& t = trial.p;
+    if (ctx->force_pair < 0) pair = (t.mode == kModeHalo && !t.b_resident && sp.Nout >= 128) ? 1 : 0;
+    if (ctx->force_cols < 0 && sp.whole_gpu && pair == 0 && t.ntaps > 0 && t.num_tiles < ctx->num_sms) {
+      const int row_tiles = t.num_tiles / t.tiles_col;
+      for (int k = t.tiles_col + 1; k <= 16 && row_tiles * k <= ctx->num_sms && ceil_div(sp.Nout, k) >= 64; ++k) ncol = k;
+    }
+  }
+  return plan_sub_fixed(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks, ncol, pair);
 }
 
 hq_status encode_map(hq_ctx* ctx, CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
@@ -426,6 +455,7 @@ hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, con
   p.xq = xq;
   p.w_scale = w_scale;
   p.bias = bias;
+  p.acc_bound = (float)p.ntaps * (float)p.Cpad * 255.0f * 128.0f;
   p.out = out;
   p.yq = yq;
   int grid = std::max(1, std::min(p.num_tiles, max_ctas > 0 ? max_ctas : ctx->num_sms));
@@ -774,6 +804,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     ctx->force_repack = value;
     return HQ_OK;
   }
+  if (std::string(key) == "col_tiles") {
+    if (value < -1 || value > 16) return fail(ctx, HQ_ERR_INVALID_ARG, "col_tiles must be -1 .. 16");
+    ctx->force_cols = value;
+    return HQ_OK;
+  }
   if (std::string(key) == "pair") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "pair must be -1, 0 or 1");
     ctx->force_pair = value;
@@ -984,6 +1019,7 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
           }
           sp.a_H = Ho; sp.a_W = Wo; sp.Cin = d.K; sp.Nout = d.C;
           sp.out_H = d.H; sp.out_W = d.W; sp.os_h = d.stride_h; sp.os_w = d.stride_w; sp.oa_h = a; sp.oa_w = b; sp.ldY = d.C; sp.flat = false;
+          sp.whole_gpu = d.stride_h * d.stride_w == 1;   // the parity classes of a strided layer run side by side
           if ((st = build_sub(ctx, pw, s, sp, d, W, tr, ts, true, 1)) != HQ_OK) return bail(st);
         }
     }

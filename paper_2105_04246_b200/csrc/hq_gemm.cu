@@ -81,6 +81,20 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int* v) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// eight columns; the matching wait names the registers, so that no use of them can be scheduled ahead of it while
+// another load is in flight
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait8(int (&v)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7])
+               :
+               : "memory");
+}
 
 template <int V>
 __device__ __forceinline__ void store_bytes16(int8_t* p, const uint32_t* w, int nvalid) {
@@ -540,6 +554,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
       q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
       qparams_finish(q);
+      qparams_bound(q, p.acc_bound);
       if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
         q.sr = 1;
         q.sr_seed = p.yq->seed;
@@ -731,46 +746,42 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         int8_t* dst_row = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0;
         const int64_t elem_row = pix * p.ldY + p.out_col0 + col0;   // linear index in the output tensor of this row's first column
         int tmn = INT32_MAX, tmx = INT32_MIN;
-        for (int ch = c_begin; ch < c_end; ++ch) {
-          int v[CW];
-          tmem_ld16(taddr + ch * CW, v);
-          tmem_ld_wait();
-          const int c0 = ch * CW;
-#pragma unroll
-          for (int e = 0; e < CW; e += 4) {
-            const int4 cr = *reinterpret_cast<const int4*>(zrow + c0 + e);
-            v[e + 0] -= cr.x;
-            v[e + 1] -= cr.y;
-            v[e + 2] -= cr.z;
-            v[e + 3] -= cr.w;
-          }
-          int lo[2], hi[2];
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            const int* x = v + 8 * g;
-            lo[g] = min(__vimin3_s32(__vimin3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimin3_s32(x[5], x[6], x[7]));
-            hi[g] = max(__vimax3_s32(__vimax3_s32(x[0], x[1], x[2]), x[3], x[4]), __vimax3_s32(x[5], x[6], x[7]));
-          }
-          tmn = __vimin3_s32(tmn, lo[0], lo[1]);
-          tmx = __vimax3_s32(tmx, hi[0], hi[1]);
-          uint32_t w[CW / 4];
-          if (q.sr) {   // stochastic rounding: the pass covers two aligned blocks of eight elements, one generator call each
-            const uint64_t block = (uint64_t)(elem_row + c0) >> 3;
-#pragma unroll
-            for (int b = 0; b < 2; ++b) {
-              uint32_t h[8];
-              sr_draws8(q, block + b, h);
-              w[2 * b] = pack_sat4(requant_acc_sr<true>(v[8 * b + 0], h[0], q), requant_acc_sr<true>(v[8 * b + 1], h[1], q),
-                                   requant_acc_sr<true>(v[8 * b + 2], h[2], q), requant_acc_sr<true>(v[8 * b + 3], h[3], q));
-              w[2 * b + 1] = pack_sat4(requant_acc_sr<true>(v[8 * b + 4], h[4], q), requant_acc_sr<true>(v[8 * b + 5], h[5], q),
-                                       requant_acc_sr<true>(v[8 * b + 6], h[6], q), requant_acc_sr<true>(v[8 * b + 7], h[7], q));
-            }
+        // eight columns at a time, two register sets: the load of the next eight is in flight while these are processed
+        const QPacked qk = qpacked(q);
+        auto half = [&](int (&x)[8], int c, uint32_t& w0, uint32_t& w1) {
+          const int4 ca = *reinterpret_cast<const int4*>(zrow + c), cb = *reinterpret_cast<const int4*>(zrow + c + 4);
+          x[0] -= ca.x; x[1] -= ca.y; x[2] -= ca.z; x[3] -= ca.w;
+          x[4] -= cb.x; x[5] -= cb.y; x[6] -= cb.z; x[7] -= cb.w;
+          tmn = __vimin3_s32(tmn, x[0], x[1]); tmx = __vimax3_s32(tmx, x[0], x[1]);
+          tmn = __vimin3_s32(tmn, x[2], x[3]); tmx = __vimax3_s32(tmx, x[2], x[3]);
+          tmn = __vimin3_s32(tmn, x[4], x[5]); tmx = __vimax3_s32(tmx, x[4], x[5]);
+          tmn = __vimin3_s32(tmn, x[6], x[7]); tmx = __vimax3_s32(tmx, x[6], x[7]);
+          if (q.sr) {   // stochastic rounding: one aligned block of eight elements, one generator call
+            uint32_t h[8];
+            sr_draws8(q, (uint64_t)(elem_row + c) >> 3, h);
+            w0 = pack_sat4(requant_acc_sr<true>(x[0], h[0], q), requant_acc_sr<true>(x[1], h[1], q), requant_acc_sr<true>(x[2], h[2], q),
+                           requant_acc_sr<true>(x[3], h[3], q));
+            w1 = pack_sat4(requant_acc_sr<true>(x[4], h[4], q), requant_acc_sr<true>(x[5], h[5], q), requant_acc_sr<true>(x[6], h[6], q),
+                           requant_acc_sr<true>(x[7], h[7], q));
+          } else if (q.noclamp) {
+            w0 = requant_pack4<false>(x[0], x[1], x[2], x[3], q, qk);
+            w1 = requant_pack4<false>(x[4], x[5], x[6], x[7], q, qk);
           } else {
-#pragma unroll
-            for (int e = 0; e < CW / 4; ++e)
-              w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
-                               requant_acc<true>(v[4 * e + 3], q));
+            w0 = requant_pack4<true>(x[0], x[1], x[2], x[3], q, qk);
+            w1 = requant_pack4<true>(x[4], x[5], x[6], x[7], q, qk);
           }
+        };
+        int va[8], vb[8];
+        tmem_ld8(taddr + c_begin * CW, va);
+        for (int ch = c_begin; ch < c_end; ++ch) {
+          const int c0 = ch * CW;
+          uint32_t w[4];
+          tmem_ld_wait8(va);
+          tmem_ld8(taddr + c0 + 8, vb);
+          half(va, c0, w[0], w[1]);
+          tmem_ld_wait8(vb);
+          if (ch + 1 < c_end) tmem_ld8(taddr + c0 + CW, va);
+          half(vb, c0 + 8, w[2], w[3]);
           if (row_valid) *reinterpret_cast<uint4*>(dst_row + c0) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         if (row_valid) {

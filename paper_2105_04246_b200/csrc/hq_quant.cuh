@@ -13,6 +13,7 @@ struct QParams {
   int zx, zp;
   int magic_sub;   // 0x4B400000 - zp
   int fast;        // parameters finite and inv_scale != 0: u can never be NaN, so the magic-number rounding is exact
+  int noclamp;     // fast, and |u| < 2^22 for every accumulator the layer can produce: the lower clamp is not needed
   int sr;          // stochastic rounding (the output state's `rounding`); draws keyed on (sr_seed, sr_iter, element index)
   uint32_t sr_seed, sr_iter;
 };
@@ -22,6 +23,12 @@ __device__ __forceinline__ void qparams_finish(QParams& q) {
   q.sr_seed = q.sr_iter = 0u;
   q.magic_sub = 0x4B400000 - q.zp;
   q.fast = (isfinite(q.inv_scale) && q.inv_scale != 0.0f && isfinite(q.s_acc)) ? 1 : 0;
+  q.noclamp = 0;
+}
+// acc_bound: an upper bound of |accumulator| over every input the layer can see (reduction length x 255 x 128).
+// |y| <= fl(acc_bound * |s_acc|) (1 + 2^-23) and |u| <= that * |inv_scale| (1 + 2^-23); a margin of 2 covers the roundings.
+__device__ __forceinline__ void qparams_bound(QParams& q, float acc_bound) {
+  q.noclamp = (q.fast && fabsf(q.s_acc) * acc_bound * fabsf(q.inv_scale) * 2.0f < 4194304.0f) ? 1 : 0;
 }
 
 // rint(u) + zp without the (slow) float-to-int conversion pipe: add 1.5 * 2^23 (for |u| <= 2^22 the sum is rounded to
@@ -51,6 +58,47 @@ template <bool kFast>
 __device__ __forceinline__ int requant_acc(int a, const QParams& q) {
   return requant_real<kFast>(__fmul_rn(__int2float_rn(a), q.s_acc), q);
 }
+
+// Two accumulators at once with the packed binary32 instructions of sm_100 (mul.rn.f32x2 / fma.rn.f32x2: per lane
+// the same single round-to-nearest-even operation as the scalar forms, half the instruction slots).  kClamp as in
+// round_add_zp_fast; without it the caller guarantees |u| < 2^22 (QParams::noclamp).
+// The rounding add is written as fma(u, 1, magic): one rounding of u + magic, like the add, but a form the assembler
+// cannot merge with the multiplication before it (it was seen to turn mul.rn.f32x2 followed by add.rn.f32x2 into one
+// fused operation, which rounds once instead of twice and moves ties).
+struct QPacked {
+  unsigned long long s_acc2, inv2, magic2, one2;
+};
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ QPacked qpacked(const QParams& q) {
+  QPacked k;
+  k.s_acc2 = pack_f32x2(q.s_acc, q.s_acc);
+  k.inv2 = pack_f32x2(q.inv_scale, q.inv_scale);
+  k.magic2 = pack_f32x2(12582912.0f, 12582912.0f);
+  k.one2 = pack_f32x2(1.0f, 1.0f);
+  return k;
+}
+template <bool kClamp>
+__device__ __forceinline__ void requant_acc2(int a0, int a1, const QParams& q, const QPacked& k, int& r0, int& r1) {
+  unsigned long long x = pack_f32x2(__int2float_rn(a0), __int2float_rn(a1)), y, u, t;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(y) : "l"(x), "l"(k.s_acc2));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(u) : "l"(y), "l"(k.inv2));
+  if constexpr (kClamp) {
+    float u0, u1;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(u0), "=f"(u1) : "l"(u));
+    u = pack_f32x2(fmaxf(u0, -4194304.0f), fmaxf(u1, -4194304.0f));
+  }
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(t) : "l"(u), "l"(k.one2), "l"(k.magic2));
+  int b0, b1;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(b0), "=r"(b1) : "l"(t));
+  r0 = b0 - q.magic_sub;
+  r1 = b1 - q.magic_sub;
+}
+template <bool kClamp>
+__device__ __forceinline__ uint32_t requant_pack4(int a0, int a1, int a2, int a3, const QParams& q, const QPacked& k);
 
 // ---- stochastic rounding (the paper's rounding for gradients) ----------------------------------------------------
 // code = sat8(floor(fl(u + r)) + zp), r = h / 65536 with h a 16-bit draw of the counter-based generator
@@ -120,6 +168,14 @@ __device__ __forceinline__ uint32_t pack_sat4(int q0, int q1, int q2, int q3) {
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(q1), "r"(q0), "r"(hi));
   return d;
+}
+
+template <bool kClamp>
+__device__ __forceinline__ uint32_t requant_pack4(int a0, int a1, int a2, int a3, const QParams& q, const QPacked& k) {
+  int r0, r1, r2, r3;
+  requant_acc2<kClamp>(a0, a1, q, k, r0, r1);
+  requant_acc2<kClamp>(a2, a3, q, k, r2, r3);
+  return pack_sat4(r0, r1, r2, r3);
 }
 
 // four accumulators whose first element has linear index e (a multiple of 4) -> four codes with stochastic rounding

@@ -217,6 +217,23 @@ PAIR_EXTRA = {
 }
 
 
+@pytest.mark.parametrize("cols", [0, 2, 3])
+@pytest.mark.parametrize("name", ["3x3_c256_k512_7x7", "3x3_c128_k256", "3x3_c64_k64", "1x1_c144_k24"])
+def test_conv_fwd_column_tiles(ctx, name, cols):
+    """The split of the output channels into column tiles (option col_tiles) does not change a byte, ragged last tile included."""
+    shape = dict(FWD_CASES[name])
+    shape.setdefault("R", 1); shape.setdefault("S", 1)
+    r = synth.rng(109, len(name), shape["H"], cols)
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.relu_activations, synth.signed_activations, synth.relu_activations]
+    ctx.set_option("col_tiles", cols)
+    try:
+        _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3)
+    finally:
+        ctx.set_option("col_tiles", -1)
+
+
 @pytest.mark.parametrize("staging", [0, 1])
 @pytest.mark.parametrize("name", PAIR_FWD)
 def test_conv_fwd_cta_pairs(ctx, name, staging):
