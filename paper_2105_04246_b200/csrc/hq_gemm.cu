@@ -319,26 +319,24 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     // ------------------------------ weight producer (kModeHalo) ------------------------------
     if (!halo && p.b_resident && kiters > 0) {
       // kModeTap with a small weight matrix: every (column tile, tap, chunk) box once, in the order the issuer uses them
-      if (my_tiles > 0) {
+      if (my_tiles > 0) {   // all of them report to barrier 0: the issuer waits once
+        if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)(p.tiles_col * kiters) * p.stage_bytes_b);
+        __syncwarp();
         for (int ct = 0; ct < p.tiles_col; ++ct)
           for (int ki = 0; ki < kiters; ++ki) {
             const int t = ki / p.chunks_per_tap, cc = ki - t * p.chunks_per_tap;
             const int slot = ct * kiters + ki;
-            if (elect_one()) {
-              mbar_expect_tx(b_full(slot), p.stage_bytes_b);
-              tma_load_2d(ring_b + slot * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, ct * p.BN, b_full(slot));
-            }
+            if (elect_one()) tma_load_2d(ring_b + slot * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, ct * p.BN, b_full(0));
           }
       }
     } else if (halo && kiters > 0) {
       if (p.b_resident) {
         if (my_tiles > 0) {
+          if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)kiters * p.stage_bytes_b);
+          __syncwarp();
           for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
             const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
-            if (elect_one()) {
-              mbar_expect_tx(b_full(ki), p.stage_bytes_b);
-              tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(ki));
-            }
+            if (elect_one()) tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(0));
           }
         }
       } else {
@@ -380,9 +378,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int nissuers = p.mma_issuers;
     // The k-steps of one operand stage are issued from a compile-time unrolled group: a run-time inner loop
     // around the MMA instruction was measured to cost several hundred cycles per iteration.
-    auto mma_role = [&](auto kk_tag, auto pair_tag) {
+    auto mma_role = [&](auto kk_tag, auto pair_tag, auto nt_tag) {
       constexpr int KK = decltype(kk_tag)::value;
       constexpr bool kPair = decltype(pair_tag)::value;
+      // NT > 0: resident-row layers with exactly NT filter taps (3x3: 9).  Their tap loop is unrolled at compile time with
+      // the tap offsets in registers: as a run-time loop (shared-memory load of the offset, branch, descriptor arithmetic
+      // in per-thread registers) it cost about 200 clocks per tap, more than the MMAs of a tap on a 64-column tile take.
+      constexpr int NT = decltype(nt_tag)::value;
+      uint32_t toff[NT > 0 ? NT : 1];
+      if constexpr (NT > 0) {
+#pragma unroll
+        for (int t = 0; t < NT; ++t) toff[t] = tapoff_s[t];
+      }
       int stage = 0, bstage = 0;
       uint32_t phase = 0, bphase = 0;
       bool ok = true;
@@ -417,6 +424,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * p.tmem_buf_stride;
         uint32_t acc = 0;
+        if (resident && first) {   // the whole weight matrix arrives once
+          ok = warp_wait(b_full(0), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+          if (!ok) break;
+          tc_fence_after();
+        }
         if (halo) {
           int n0, o0, w0, col0;
           decode(tile, n0, o0, w0, col0);
@@ -427,32 +439,52 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
             if (!ok) break;
             tc_fence_after();
             const uint64_t abase = make_smem_desc(ring_a + stage * a_stride + rel_bytes, sw64);
-            if (resident && first) {
-              // the weight matrix arrives once, tap by tap: the first tile starts on each tap as soon as it is there
-              for (int t = 0; t < ntaps; ++t) {
-                ok = warp_wait(b_full(cc * ntaps + t), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
-                if (!ok) break;
-                tc_fence_after();
-                const uint64_t adesc = abase + tapoff_s[t];
+            if (resident) {
+              if constexpr (NT > 0) {
+#pragma unroll
+                for (int t = 0; t < NT; ++t) {
+                  const uint64_t adesc = abase + toff[t];
+                  const uint64_t bdesc = bres + (uint64_t)(t * bstep16);
+                  if (elect_one()) {
+#pragma unroll
+                    for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                  }
+                }
+                bres += (uint64_t)(NT * bstep16);
+              } else {
                 if (elect_one()) {
+                  for (int t = 0; t < ntaps; ++t) {
+                    const uint64_t adesc = abase + tapoff_s[t];
 #pragma unroll
-                  for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
-                }
-                bres += bstep16;
-              }
-              __syncwarp();
-              acc = 1;
-            } else if (resident) {
-              if (elect_one()) {
-                for (int t = 0; t < ntaps; ++t) {
-                  const uint64_t adesc = abase + tapoff_s[t];
-#pragma unroll
-                  for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
-                  bres += bstep16;
+                    for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bres + 2u * k, idesc, (k == 0 && t == 0) ? acc : 1u);
+                    bres += bstep16;
+                  }
                 }
               }
               __syncwarp();
               acc = 1;
+            } else if constexpr (NT > 0) {
+#pragma unroll
+              for (int t = 0; t < NT; ++t) {
+                if (ok) {
+                  ok = warp_wait(b_full(bstage), bphase, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
+                  if (ok) {
+                    tc_fence_after();
+                    const uint64_t bdesc = bdesc0 + (uint64_t)bstage * bstep16;
+                    const uint64_t adesc = abase + toff[t];
+                    if (elect_one()) {
+#pragma unroll
+                      for (int k = 0; k < KK; ++k) mma_any<kPair>(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, k == 0 ? acc : 1u);
+                      commit_any<kPair>(b_empty(bstage));
+                    }
+                    acc = 1;
+                    if (++bstage == stages_b) {
+                      bstage = 0;
+                      bphase ^= 1u;
+                    }
+                  }
+                }
+              }
             } else {
               for (int t = 0; t < ntaps; ++t) {
                 ok = warp_wait(b_full(bstage), bphase, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
@@ -483,11 +515,6 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         } else {
           uint64_t bres = bdesc0;
           if (resident) {
-            if (first) {   // the whole weight matrix arrives once
-              for (int ki = 0; ki < p.stages_b && ok; ++ki) ok = warp_wait(b_full(ki), 0u, abort_flag, p.status, kAsyncMmaBFullWait, 200u);
-              if (!ok) break;
-              tc_fence_after();
-            }
             const int t0 = fdiv(tile, p.fd_tiles_col);
             bres += (uint64_t)((tile - t0 * p.tiles_col) * kiters) * bstep16;
           }
@@ -520,12 +547,16 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       }
     };
     if (kiters > 0 && crank == 0) {   // in a pair, rank 0 issues for both CTAs
-      if constexpr (kPairK) {
-        if (p.BK == 64) mma_role(std::integral_constant<int, 2>{}, std::true_type{});
-        else mma_role(std::integral_constant<int, 4>{}, std::true_type{});
+      using PairTag = std::integral_constant<bool, kPairK>;
+      using T9 = std::integral_constant<int, 9>;
+      using T0 = std::integral_constant<int, 0>;
+      const bool nine = halo && p.ntaps == 9;
+      if (p.BK == 64) {
+        if (nine) mma_role(std::integral_constant<int, 2>{}, PairTag{}, T9{});
+        else mma_role(std::integral_constant<int, 2>{}, PairTag{}, T0{});
       } else {
-        if (p.BK == 64) mma_role(std::integral_constant<int, 2>{}, std::false_type{});
-        else mma_role(std::integral_constant<int, 4>{}, std::false_type{});
+        if (nine) mma_role(std::integral_constant<int, 4>{}, PairTag{}, T9{});
+        else mma_role(std::integral_constant<int, 4>{}, PairTag{}, T0{});
       }
     }
     __syncwarp();
@@ -545,6 +576,18 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int slice = (ew >> 2) >> p.epi_groups_log2;
     const int slices = kEpilogueSlices >> p.epi_groups_log2;
     const int row = quarter * 32 + lane;
+    // Everything the tables need is requested before the first use of any of it (a warp stalls at the first use of a
+    // pending load, and the loads behind it would only start then): one trip to memory instead of three.
+    const int et0 = (int)threadIdx.x - kFirstEpilogueWarp * 32;
+    constexpr int kCorrAhead = 4;
+    int32_t corr_ahead[kCorrAhead];
+#pragma unroll
+    for (int k = 0; k < kCorrAhead; ++k) {
+      const int i = et0 + k * kEpilogueWarps * 32;
+      corr_ahead[k] = (p.zc_in_smem && i < p.zc_elems) ? p.corr[i] : 0;
+    }
+    const uint8_t rowcls_ahead = (p.cls_in_smem && et0 < p.TH) ? p.rowcls[et0] : (uint8_t)0;
+    const uint8_t colcls_ahead = (p.cls_in_smem && et0 < p.TW) ? p.colcls[et0] : (uint8_t)0;
     QParams q;
     {
       const float s_x = p.xq->scale;
@@ -567,11 +610,15 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     {
       const int et = (int)threadIdx.x - kFirstEpilogueWarp * 32;
       constexpr int kEpiThreads = kEpilogueWarps * 32;
-      if (p.zc_in_smem)
-        for (int i = et; i < p.zc_elems; i += kEpiThreads) zc_s[i] = q.zx * p.corr[i];
-      if (p.cls_in_smem) {
-        for (int i = et; i < p.TH; i += kEpiThreads) cls_s[i] = p.rowcls[i];
-        for (int i = et; i < p.TW; i += kEpiThreads) cls_s[512 + i] = p.colcls[i];
+      if (p.zc_in_smem) {
+#pragma unroll
+        for (int k = 0; k < kCorrAhead; ++k)
+          if (et + k * kEpiThreads < p.zc_elems) zc_s[et + k * kEpiThreads] = q.zx * corr_ahead[k];
+        for (int i = et + kCorrAhead * kEpiThreads; i < p.zc_elems; i += kEpiThreads) zc_s[i] = q.zx * p.corr[i];
+      }
+      if (p.cls_in_smem) {   // TH, TW <= 512 = the number of epilogue threads
+        if (et < p.TH) cls_s[et] = rowcls_ahead;
+        if (et < p.TW) cls_s[512 + et] = colcls_ahead;
       }
       asm volatile("bar.sync 1, %0;" ::"r"(kEpiThreads) : "memory");
     }
