@@ -300,6 +300,11 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
     const int b_per_tile = (p.mode == kModeHalo && !p.b_resident) ? kiters : 0;
     const bool rings_ok = 2 * a_per_tile <= p.stages_a && (b_per_tile == 0 || 2 * b_per_tile <= p.stages_b);
     p.mma_issuers = (rings_ok && kiters > 0 && p.num_tiles >= 2 * ctx->num_sms && !p.pair) ? 2 : 1;
+    // narrow tiles (64 columns or fewer) keep the tensor core busy for so short a time per tile that a third issuer pays;
+    // the weight producer's warp takes that part once resident weights are on their way
+    if (p.mma_issuers == 2 && p.b_resident && p.BN <= 64 && 3 * a_per_tile <= p.stages_a && p.num_tiles >= 3 * ctx->num_sms &&
+        p.tmem_bufs >= 4)
+      p.mma_issuers = 3;
     // many small tiles per CTA: four epilogue groups; few large ones: all warps on every tile (shortest tail)
     const int tiles_per_cta = ceil_div(p.num_tiles, ctx->num_sms);
     p.epi_groups_log2 = tiles_per_cta >= 8 ? std::min(2, p.tmem_bufs_log2) : 0;

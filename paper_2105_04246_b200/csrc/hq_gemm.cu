@@ -206,11 +206,12 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
-  // Everything above touched only kernel parameters and this CTA's own resources.  From here on the kernel reads
-  // what earlier kernels in the stream wrote (operands, range states), so it waits for them.  The weight producer
-  // reads nothing but the prepared weight matrix; where the host knows that matrix to be older than the previous
-  // kernel (any call after the first with these prepared weights) it starts copying at once.
-  if (!(warp == 2 && p.weights_early)) grid_dependency_wait();
+  // Everything above touched only kernel parameters and this CTA's own resources.  What earlier kernels in the stream
+  // wrote (operands, range states) is read by the operand producers and the epilogue warps; each of them waits for
+  // those kernels (grid_dependency_wait) right before its first access to global memory, after its own set-up, so that
+  // the set-up runs while the previous kernel drains (the MMA issuers, which touch shared and tensor memory only, wait
+  // before their first barrier).  The weight producer reads nothing but the prepared weight matrix; where the host knows that matrix to be
+  // older than the previous kernel (any call after the first with these prepared weights) it starts copying at once.
 
   // tile index -> origin.  kModeTap: (n0, h0, w0) of the pixel box; kModeHalo: image n0, first linear pixel h0
   auto decode = [&](int tile, int& n0, int& h0, int& w0, int& col0) {
@@ -255,126 +256,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   // The three single-issuer roles below are executed by their WHOLE warp with warp-uniform control flow and
   // values; only the copy / MMA / commit instructions themselves sit under a one-lane predicate (elect.sync).
   // Uniform values stay in uniform registers, which is what the TMA and MMA instructions take their operands from.
-  if (warp == 0) {
-    // ------------------------------ operand A producer ------------------------------
-    if (kiters > 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      const int b_row_off = (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
-      for (int it = 0; ok; ++it) {
-        const int tile = own_tile(it);
-        if (tile < 0) break;
-        int n0, h0, w0, col0;
-        decode(tile, n0, h0, w0, col0);
-        if (halo) {
-          const int hp0 = fdiv(h0, p.fd_P);   // h0 is the tile's first linear pixel
-          for (int cb = 0; cb < p.chunks_per_tap; ++cb) {   // one ring stage per channel chunk of the patch
-            ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
-            if (!ok) break;
-            if (elect_one()) {
-              if constexpr (kPairK) {
-                mbar_expect_tx_remote(a_full_lead(stage), p.patch_box_bytes);
-                tma_load_4d_pair(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full_lead(stage));
-              } else {
-                mbar_expect_tx(a_full(stage), p.patch_box_bytes);
-                tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
-              }
-            }
-            if (++stage == p.stages_a) {
-              stage = 0;
-              phase ^= 1u;
-            }
-          }
-        } else {
-          for (int t = 0; t < p.ntaps && ok; ++t) {
-            const int ch = h0 * p.in_mul_h + p.tap_dh[t];
-            const int cw = w0 * p.in_mul_w + p.tap_dw[t];
-            for (int cc = 0; cc < p.chunks_per_tap; ++cc) {
-              ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
-              if (!ok) break;
-              const uint32_t sa = ring_a + stage * a_stride;
-              if (elect_one()) {
-                if constexpr (kPairK) {   // never with resident weights
-                  mbar_expect_tx_remote(a_full_lead(stage), a_stride);
-                  tma_load_4d_pair(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full_lead(stage));
-                  tma_load_2d_pair(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0 + b_row_off, a_full_lead(stage));
-                } else {
-                  mbar_expect_tx(a_full(stage), a_stride);
-                  tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
-                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
-                }
-              }
-              if (++stage == p.stages_a) {
-                stage = 0;
-                phase ^= 1u;
-              }
-            }
-          }
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 2) {
-    // ------------------------------ weight producer (kModeHalo) ------------------------------
-    if (!halo && p.b_resident && kiters > 0) {
-      // kModeTap with a small weight matrix: every (column tile, tap, chunk) box once, in the order the issuer uses them
-      if (my_tiles > 0) {   // all of them report to barrier 0: the issuer waits once
-        if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)(p.tiles_col * kiters) * p.stage_bytes_b);
-        __syncwarp();
-        for (int ct = 0; ct < p.tiles_col; ++ct)
-          for (int ki = 0; ki < kiters; ++ki) {
-            const int t = ki / p.chunks_per_tap, cc = ki - t * p.chunks_per_tap;
-            const int slot = ct * kiters + ki;
-            if (elect_one()) tma_load_2d(ring_b + slot * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, ct * p.BN, b_full(0));
-          }
-      }
-    } else if (halo && kiters > 0) {
-      if (p.b_resident) {
-        if (my_tiles > 0) {
-          if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)kiters * p.stage_bytes_b);
-          __syncwarp();
-          for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
-            const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
-            if (elect_one()) tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(0));
-          }
-        }
-      } else {
-        int stage = 0;
-        uint32_t phase = 0;
-        bool ok = true;
-        for (int it = 0; ok; ++it) {
-          const int tile = own_tile(it);
-          if (tile < 0) break;
-          const int col0 = (tile % p.tiles_col) * p.BN + (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
-          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
-            for (int t = 0; t < p.ntaps; ++t) {
-              ok = warp_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait, 1000u);
-              if (!ok) break;
-              if (elect_one()) {
-                if constexpr (kPairK) {
-                  mbar_expect_tx_remote(b_full_lead(stage), p.stage_bytes_b);
-                  tma_load_2d_pair(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full_lead(stage));
-                } else {
-                  mbar_expect_tx(b_full(stage), p.stage_bytes_b);
-                  tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
-                }
-              }
-              if (++stage == p.stages_b) {
-                stage = 0;
-                phase ^= 1u;
-              }
-            }
-          }
-        }
-      }
-    }
-    __syncwarp();
-  } else if (warp == 1 || (warp == 3 && p.mma_issuers == 2)) {
+  auto run_issuer = [&](const int issuer) __attribute__((always_inline)) {
     // ------------------------------ MMA issuer(s) ------------------------------
-    // With two issuers, warp 1 takes the CTA's even tiles and warp 3 the odd ones (different accumulator buffers):
-    // the fixed per-tile latency of one issuer (decode, waits, commits) hides behind the other's MMA stream.
-    const int issuer = warp == 1 ? 0 : 1;
+    // With several issuers (warps 1, 3 and, once resident weights are on their way, 2) issuer i takes the CTA's tiles
+    // i, i + n, ...: the fixed per-tile latency of one issuer (decode, waits, commits) hides behind the others' MMA
+    // streams.
     const int nissuers = p.mma_issuers;
     // The k-steps of one operand stage are issued from a compile-time unrolled group: a run-time inner loop
     // around the MMA instruction was measured to cost several hundred cycles per iteration.
@@ -414,6 +300,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       const bool resident = p.b_resident != 0;
       const uint32_t idesc = p.idesc;
       const uint32_t bstep16 = p.stage_bytes_b >> 4;
+      // nothing can arrive before the operand producers have passed the same point; waiting here keeps the bounded waits
+      // below from counting time that belongs to an earlier kernel
+      grid_dependency_wait();
       for (int local_tile = issuer; ok; local_tile += nissuers) {
         const int tile = own_tile(local_tile);
         if (tile < 0) break;
@@ -559,6 +448,131 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         else mma_role(std::integral_constant<int, 4>{}, PairTag{}, T0{});
       }
     }
+  };
+  if (warp == 0) {
+    // ------------------------------ operand A producer ------------------------------
+    if (kiters > 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      const int b_row_off = (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
+      for (int it = 0; ok; ++it) {
+        const int tile = own_tile(it);
+        if (tile < 0) break;
+        int n0, h0, w0, col0;
+        decode(tile, n0, h0, w0, col0);
+        if (it == 0) grid_dependency_wait();   // the first copy reads what the previous kernel may have written
+        if (halo) {
+          const int hp0 = fdiv(h0, p.fd_P);   // h0 is the tile's first linear pixel
+          for (int cb = 0; cb < p.chunks_per_tap; ++cb) {   // one ring stage per channel chunk of the patch
+            ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
+            if (!ok) break;
+            if (elect_one()) {
+              if constexpr (kPairK) {
+                mbar_expect_tx_remote(a_full_lead(stage), p.patch_box_bytes);
+                tma_load_4d_pair(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full_lead(stage));
+              } else {
+                mbar_expect_tx(a_full(stage), p.patch_box_bytes);
+                tma_load_4d(ring_a + stage * a_stride, &tmap_a, cb * p.BK, p.dw_min, hp0 + p.dh_min, n0, a_full(stage));
+              }
+            }
+            if (++stage == p.stages_a) {
+              stage = 0;
+              phase ^= 1u;
+            }
+          }
+        } else {
+          for (int t = 0; t < p.ntaps && ok; ++t) {
+            const int ch = h0 * p.in_mul_h + p.tap_dh[t];
+            const int cw = w0 * p.in_mul_w + p.tap_dw[t];
+            for (int cc = 0; cc < p.chunks_per_tap; ++cc) {
+              ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
+              if (!ok) break;
+              const uint32_t sa = ring_a + stage * a_stride;
+              if (elect_one()) {
+                if constexpr (kPairK) {   // never with resident weights
+                  mbar_expect_tx_remote(a_full_lead(stage), a_stride);
+                  tma_load_4d_pair(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full_lead(stage));
+                  tma_load_2d_pair(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0 + b_row_off, a_full_lead(stage));
+                } else {
+                  mbar_expect_tx(a_full(stage), a_stride);
+                  tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
+                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+                }
+              }
+              if (++stage == p.stages_a) {
+                stage = 0;
+                phase ^= 1u;
+              }
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 2) {
+    // ------------------------------ weight producer (kModeHalo) ------------------------------
+    if (!p.weights_early) grid_dependency_wait();
+    if (!halo && p.b_resident && kiters > 0) {
+      // kModeTap with a small weight matrix: every (column tile, tap, chunk) box once, in the order the issuer uses them
+      if (my_tiles > 0) {   // all of them report to barrier 0: the issuer waits once
+        if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)(p.tiles_col * kiters) * p.stage_bytes_b);
+        __syncwarp();
+        for (int ct = 0; ct < p.tiles_col; ++ct)
+          for (int ki = 0; ki < kiters; ++ki) {
+            const int t = ki / p.chunks_per_tap, cc = ki - t * p.chunks_per_tap;
+            const int slot = ct * kiters + ki;
+            if (elect_one()) tma_load_2d(ring_b + slot * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, ct * p.BN, b_full(0));
+          }
+      }
+    } else if (halo && kiters > 0) {
+      if (p.b_resident) {
+        if (my_tiles > 0) {
+          if (elect_one()) mbar_expect_tx(b_full(0), (uint32_t)kiters * p.stage_bytes_b);
+          __syncwarp();
+          for (int ki = 0; ki < kiters; ++ki) {   // chunk-major order, as the MMA issuer consumes them
+            const int cc = ki / p.ntaps, t = ki - cc * p.ntaps;
+            if (elect_one()) tma_load_2d(ring_b + ki * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, 0, b_full(0));
+          }
+        }
+      } else {
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int it = 0; ok; ++it) {
+          const int tile = own_tile(it);
+          if (tile < 0) break;
+          const int col0 = (tile % p.tiles_col) * p.BN + (int)crank * (p.BN >> 1);   // pair: this CTA's half of the rows of B
+          for (int cc = 0; cc < p.chunks_per_tap && ok; ++cc) {
+            for (int t = 0; t < p.ntaps; ++t) {
+              ok = warp_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerBEmptyWait, 1000u);
+              if (!ok) break;
+              if (elect_one()) {
+                if constexpr (kPairK) {
+                  mbar_expect_tx_remote(b_full_lead(stage), p.stage_bytes_b);
+                  tma_load_2d_pair(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full_lead(stage));
+                } else {
+                  mbar_expect_tx(b_full(stage), p.stage_bytes_b);
+                  tma_load_2d(ring_b + stage * p.stage_bytes_b, &tmap_b, t * p.Cpad + cc * p.BK, col0, b_full(stage));
+                }
+              }
+              if (++stage == p.stages_b) {
+                stage = 0;
+                phase ^= 1u;
+              }
+            }
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (p.mma_issuers == 3) {   // the weights are on their way and stay: nothing more to copy
+      run_issuer(2);
+      __syncwarp();
+      grid_launch_dependents();
+    }
+  } else if (warp == 1 || (warp == 3 && p.mma_issuers >= 2)) {
+    run_issuer(warp == 1 ? 0 : 1);
     __syncwarp();
     // All MMAs of this CTA are issued; what is left is the epilogue of the last tiles.  The next kernel in the stream
     // may become resident as SMs free up (it waits for this grid to finish before it reads anything).  Releasing it
@@ -576,6 +590,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int slice = (ew >> 2) >> p.epi_groups_log2;
     const int slices = kEpilogueSlices >> p.epi_groups_log2;
     const int row = quarter * 32 + lane;
+    grid_dependency_wait();   // range states, scales and tables may come from earlier kernels in the stream
     // Everything the tables need is requested before the first use of any of it (a warp stalls at the first use of a
     // pending load, and the loads behind it would only start then): one trip to memory instead of three.
     const int et0 = (int)threadIdx.x - kFirstEpilogueWarp * 32;

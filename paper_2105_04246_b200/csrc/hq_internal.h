@@ -89,7 +89,7 @@ struct GemmParams {
   int32_t* status;
   uint32_t idesc;
   uint32_t tmem_cols, tmem_buf_stride;
-  int32_t mma_issuers;                // 1 or 2 warps issuing MMAs (alternate tiles)
+  int32_t mma_issuers;                // 1, 2 or 3 warps issuing MMAs (tiles in turn)
   int32_t pair;                       // 1: launched as clusters of two CTAs that share 256-row tiles (tcgen05 cta_group::2);
                                       //    stage_bytes_b and the B tensor map's box then cover BN/2 rows
   int32_t num_pair_tiles;             // pair tiles (two row tiles x one column tile)
