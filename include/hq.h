@@ -150,6 +150,8 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows
  *              per input row where the shape allows.
+ *   "epilogue_groups": layers prepared AFTER this call: -1 = chosen per layer (default); g = 0, 1, 2: the sixteen
+ *              epilogue warps form 2^g groups that drain alternate tiles (at most one group per accumulator buffer).
  *   "col_tiles": into how many column tiles (each a multiple of 16 columns, at most 256) the output channels of
  *              layers prepared AFTER this call are split: -1 = chosen per layer by estimated duration (default),
  *              0 = as few as possible, n > 0 = at least n.

@@ -218,6 +218,7 @@ struct hq_ctx {
   int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
+  int force_epi_groups = -1;          // log2 of the epilogue warp groups: -1 chosen per layer, else min(value, log2 of the accumulator buffers)
   int force_cols = -1;                // column tiles: -1 chosen by estimated duration, 0 as wide as the MMA allows, n > 0 at least n
   int force_pair = -1;                // CTA pairs on 256-row tiles: -1 choose per layer, 0 never, 1 wherever the layer allows
   cudaStream_t side[3] = {nullptr, nullptr, nullptr};   // independent launches of one call run side by side (see run_conv)
