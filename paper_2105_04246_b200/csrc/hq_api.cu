@@ -340,6 +340,25 @@ hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vec
     if (st != HQ_OK) return st;
     const GemmParams& t = trial.p;
     if (ctx->force_pair < 0) pair = (t.mode == kModeHalo && !t.b_resident && sp.Nout >= 128) ? 1 : 0;
+    // Small images fill the 128-row tiles of the resident-row numbering badly (14x14: 77 %).  With one copy per filter
+    // tap the tiles are full; where that saves a fifth of the rounds or more, pairs with one copy per tap are faster
+    // (each SM then still copies only half of the weight rows).
+    if (ctx->force_pair < 0 && ctx->force_mode < 0 && pair == 1) {
+      hq_sub_problem halo_trial = sub, tap_trial = sub;
+      const int pairs = std::max(1, ctx->num_sms / 2);
+      if (plan_sub_fixed(ctx, sp, halo_trial, rc, cc, rm, cm, ncol, 1) == HQ_OK && halo_trial.p.pair) {
+        ctx->force_mode = kModeTap;
+        const hq_status ts = plan_sub_fixed(ctx, sp, tap_trial, rc, cc, rm, cm, ncol, 1);
+        ctx->force_mode = -1;
+        if (ts == HQ_OK && tap_trial.p.pair &&
+            5 * ceil_div(tap_trial.p.num_pair_tiles, pairs) <= 4 * ceil_div(halo_trial.p.num_pair_tiles, pairs)) {
+          ctx->force_mode = kModeTap;
+          const hq_status fs = plan_sub_fixed(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks, ncol, 1);
+          ctx->force_mode = -1;
+          return fs;
+        }
+      }
+    }
     if (ctx->force_cols < 0 && sp.whole_gpu && pair == 0 && t.ntaps > 0 && t.num_tiles < ctx->num_sms) {
       const int row_tiles = t.num_tiles / t.tiles_col;
       for (int k = t.tiles_col + 1; k <= 16 && row_tiles * k <= ctx->num_sms && ceil_div(sp.Nout, k) >= 64; ++k) ncol = k;
