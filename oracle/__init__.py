@@ -59,6 +59,8 @@ def lib():
         L.hqo_out_w.argtypes = [cp]; L.hqo_out_w.restype = C.c_int32
         L.hqo_derive.argtypes = [rp]; L.hqo_derive.restype = None
         L.hqo_linear_acc.argtypes = [C.c_int, C.c_int, C.c_int, i8p, C.c_int, i8p, C.c_int, i32p, i32p]; L.hqo_linear_acc.restype = C.c_int
+        L.hqo_linear_wgrad_acc.argtypes = [C.c_int, C.c_int, C.c_int, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_linear_wgrad_acc.restype = C.c_int
+        L.hqo_scale_to_real.argtypes = [i32p, C.c_int64, C.c_float, f32p]; L.hqo_scale_to_real.restype = None
         L.hqo_conv_fwd_acc.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_conv_fwd_acc.restype = C.c_int
         L.hqo_conv_bwd_data_acc.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_conv_bwd_data_acc.restype = C.c_int
         L.hqo_linear_acc_at.argtypes = [C.c_int, C.c_int, C.c_int, i8p, C.c_int, i8p, C.c_int, i32p, i64p, C.c_int64, i64p]; L.hqo_linear_acc_at.restype = None
@@ -109,6 +111,26 @@ def linear_acc(X, zx, W, zw=0, bias=None) -> np.ndarray:
     ovf = lib().hqo_linear_acc(M, N, K, _p(X, C.c_int8), int(zx), _p(W, C.c_int8), int(zw), b, _p(acc, C.c_int32))
     assert ovf == 0, "int32 accumulator overflow"
     return acc
+
+
+def linear_wgrad_acc(dY, zdy, X, zx) -> np.ndarray:
+    """int32 g[n,k] = sum_m (dy[m,n] - z_dy) * (x[m,k] - z_x): the weight gradient of a linear layer in accumulator units."""
+    dY, X = _i8(dY), _i8(X)
+    M, N = dY.shape
+    K = X.shape[1]
+    assert X.shape[0] == M
+    g = np.empty((N, K), np.int32)
+    ovf = lib().hqo_linear_wgrad_acc(M, N, K, _p(dY, C.c_int8), int(zdy), _p(X, C.c_int8), int(zx), _p(g, C.c_int32))
+    assert ovf == 0, "int32 accumulator overflow"
+    return g
+
+
+def scale_to_real(acc: np.ndarray, s_acc: float) -> np.ndarray:
+    """fl(float(acc) * s_acc) per element, in binary32 (the weight gradient is kept in FP32)."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    out = np.empty(acc.shape, np.float32)
+    lib().hqo_scale_to_real(_p(acc, C.c_int32), acc.size, C.c_float(s_acc), _p(out, C.c_float))
+    return out
 
 
 def conv_fwd_acc(d: Conv, X, zx, W, zw=0) -> np.ndarray:

@@ -10,6 +10,8 @@
 //                   is held in 32-bit accumulators and then quantized by Q_Y; backward,
 //                   the 8-bit output gradient and the weights give the input gradient
 //                   G_X, which is quantized by Q_G.
+//   Sec. 3.1        weight gradient of a linear layer from the quantized output gradient and
+//                   the quantized input, kept in binary32 (hqo_linear_wgrad_acc).
 //   Sec. 3.2, Eq. 1 dynamic quantization: range = (min G, max G) of the current tensor;
 //                   the 32-bit output is written out, reduced, read back and quantized.
 //   Sec. 3.2        static quantization: the range is known in advance, each
@@ -40,7 +42,8 @@
 //   R-18..R-20 stochastic rounding for gradients: see the section further down.
 //
 // Pins (tests/ -m "not gpu"): brute-force and readable-by-eye cases for the index
-// arithmetic, the forward/backward adjoint identity, library convolutions in float64,
+// arithmetic, the forward/backward adjoint identity, the trace identity <dY, X W^T> = <dY^T X, W>
+// that ties the weight gradient to the forward layer, library convolutions in float64,
 // the closed form of the Eq. 2-3 recurrence, grid invariants of the quantizer, and
 // static == dynamic when the ranges coincide.
 // PARITY UNPINNED: the tie rule of the rounding (R-4), the zero-point formula of
@@ -125,6 +128,25 @@ int hqo_linear_acc(int M, int N, int K, const int8_t* X, int zx, const int8_t* W
       acc[(int64_t)m * N + n] = (int32_t)a;
     }
   return ovf;
+}
+
+// weight gradient of a linear layer (Sec. 3.1, backward pass: the quantized output gradient G~_Y and the quantized layer
+// input X~ give G_W, which stays in binary32):  g[n,k] = sum_m (dy[m,n] - z_dy) * (x[m,k] - z_x)  in int32, and
+// G_W[n,k] = fl(float(g[n,k]) * fl(s_dy * s_x)).  dY is [M][N], X is [M][K], G_W is [N][K] like the weights.
+int hqo_linear_wgrad_acc(int M, int N, int K, const int8_t* dY, int zdy, const int8_t* X, int zx, int32_t* g) {
+  int ovf = 0;
+#pragma omp parallel for reduction(| : ovf)
+  for (int n = 0; n < N; ++n)
+    for (int k = 0; k < K; ++k) {
+      int64_t a = 0;
+      for (int m = 0; m < M; ++m) a += (int64_t)((int)dY[(int64_t)m * N + n] - zdy) * ((int)X[(int64_t)m * K + k] - zx);
+      if (a > INT32_MAX || a < INT32_MIN) ovf |= 1;
+      g[(int64_t)n * K + k] = (int32_t)a;
+    }
+  return ovf;
+}
+void hqo_scale_to_real(const int32_t* acc, int64_t count, float s_acc, float* out) {
+  for (int64_t i = 0; i < count; ++i) out[i] = (float)acc[i] * s_acc;
 }
 
 // forward convolution, X NHWC, W [K][R][S][C/groups], Y [N][Ho][Wo][K]:
