@@ -214,6 +214,18 @@ hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                            const hq_prepared_weights* pw, const float* w_scale,
                            int8_t* dX, hq_range_state* dxq);
 
+/* Weight gradient of a linear layer (Sec. 3.1, backward pass: the quantized output gradient and the quantized layer
+ * input give G_W, which the paper keeps in FP32):
+ *   GW[n][k] = fl( float( sum_m (dY[m][n] - z_dy) * (X[m][k] - z_x) ) * fl(s_dy * s_x) ),  one binary32 rounding per step,
+ * with (s_dy, z_dy) = scale / zero_point of *dyq and (s_x, z_x) of *xq.  dY is [M][N], X is [M][K], GW is [N][K] binary32,
+ * laid out like the weights.  The sum is exact in int32; M may not exceed 65536.  The reduction runs over the rows, so the
+ * call first transposes both operands into context-owned scratch (grown with cudaMalloc when a larger layer is first
+ * seen; calls on one context must not overlap) and runs the tensor-core layer kernel on them with a binary32
+ * epilogue.  Nothing is quantized and no range state is written. */
+hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K,
+                          const int8_t* dY, const hq_range_state* dyq,
+                          const int8_t* X, const hq_range_state* xq, float* GW);
+
 /* Eq. 2-3 for `count` consecutive states, to be enqueued after the layer calls of the iteration:
  *   m_lo = float(acc_min) * acc_scale, m_hi alike;
  *   step == 0:  q_min = m_lo, q_max = m_hi                      (initialisation, Sec. 4.1)

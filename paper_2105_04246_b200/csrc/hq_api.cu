@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdarg.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <stdio.h>
 
@@ -475,8 +476,9 @@ int fold_factor(int channels, int64_t pixels) {
 
 hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, const CUtensorMap& ta, const CUtensorMap& tb, const hq_range_state* xq,
                      const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, int max_ctas = 0,
-                     bool weights_early = false) {
+                     bool weights_early = false, const int32_t* row_term = nullptr) {
   GemmParams p = sub.p;
+  p.row_term = row_term;
   p.out_col0 = sub.chan0;
   p.weights_early = weights_early ? 1 : 0;
   p.xq = xq;
@@ -644,7 +646,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
 }
 
 hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
-                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode) {
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, const int32_t* row_term = nullptr) {
   if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
   if (!X || !xq || !W || !w_scale || !out || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(X) || !aligned16(W) || !aligned16(out) || !aligned16(xq) || !aligned16(yq))
@@ -696,7 +698,7 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
   if (st != HQ_OK) return st;
   st = encode_b(ctx, sub, W, K, &tb);
   if (st != HQ_OK) return st;
-  return launch_sub(ctx, s, sub, ta, tb, xq, w_scale, bias, out, yq, out_mode);
+  return launch_sub(ctx, s, sub, ta, tb, xq, w_scale, bias, out, yq, out_mode, 0, false, row_term);
 }
 
 hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, hq_range_state* yq, int out_mode) {
@@ -794,6 +796,7 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
   cudaFree(ctx->d_status);
   cudaFree(ctx->d_scratch);
   if (ctx->d_pad) cudaFree(ctx->d_pad);
+  if (ctx->d_wgrad) cudaFree(ctx->d_wgrad);
   free_side_streams(ctx);
   delete ctx;
   return HQ_OK;
@@ -1106,6 +1109,44 @@ __attribute__((visibility("default"))) hq_status hq_dynamic_quant(hq_ctx* ctx, v
   HQ_CUDA(ctx, launch_quantize_pass(workspace, Y, op_out_elems(op), yq, ctx->num_sms, s, false));
   ctx->launches += 2;
   return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K, const int8_t* dY,
+                                                                 const hq_range_state* dyq, const int8_t* X, const hq_range_state* xq, float* GW) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
+  if (!dY || !dyq || !X || !xq || !GW) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(GW) || !aligned16(dyq) || !aligned16(xq))
+    return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
+  // |sum_m (dy - z_dy) * x| <= M * 255 * 128 has to stay inside int32 before the input zero point is taken out
+  if (M > 65536) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient over more than 65536 rows (M = %d) could leave the int32 range", M);
+  cudaStream_t s = (cudaStream_t)stream;
+  // The reduction runs over the rows (the batch), so both operands are transposed first: A = dY^T [N][Mp] and
+  // B = X^T [K][Mp] (Mp = M rounded up to 16, zero filled).  The layer kernel removes the zero point of its first
+  // operand (dY) through the column sums of the second; the zero point of X costs one number per output row,
+  // z_x * sum_m (dy - z_dy), which a small kernel prepares and the epilogue subtracts before the conversion to binary32.
+  const int Mp = round_up(M, 16);
+  const size_t a_bytes = ((size_t)N * Mp + 255) & ~(size_t)255, b_bytes = ((size_t)K * Mp + 255) & ~(size_t)255;
+  const size_t t_bytes = ((size_t)N * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t need = a_bytes + b_bytes + t_bytes + 256;
+  if (need > ctx->wgrad_bytes) {
+    if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));
+    ctx->d_wgrad = nullptr;
+    ctx->wgrad_bytes = 0;
+    HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_wgrad, need));
+    ctx->wgrad_bytes = need;
+  }
+  int8_t* At = reinterpret_cast<int8_t*>(ctx->d_wgrad);
+  int8_t* Bt = At + a_bytes;
+  int32_t* terms = reinterpret_cast<int32_t*>(ctx->d_wgrad + a_bytes + b_bytes);
+  hq_range_state* tmp = reinterpret_cast<hq_range_state*>(ctx->d_wgrad + a_bytes + b_bytes + t_bytes);
+  HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, N, Mp, 0, s));
+  HQ_CUDA(ctx, launch_transpose_rows(X, Bt, M, K, Mp, 0, s));
+  HQ_CUDA(ctx, launch_wgrad_row_terms(dY, M, N, dyq, xq, terms, s));
+  ctx->launches += 3;
+  // GW[n][k] = fl(float(acc) * fl(s_dy * s_x)): the layer kernel's binary32 output mode; its "weight scale" is the scale of X
+  const float* x_scale = reinterpret_cast<const float*>(reinterpret_cast<const char*>(xq) + offsetof(hq_range_state, scale));
+  return run_linear(ctx, s, N, K, Mp, At, dyq, Bt, x_scale, nullptr, GW, tmp, kOutF32, terms);
 }
 
 __attribute__((visibility("default"))) hq_status hq_debug_accumulate(hq_ctx* ctx, void* stream, const hq_op_desc* op, int32_t* acc, hq_range_state* yq) {

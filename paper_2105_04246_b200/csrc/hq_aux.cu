@@ -394,6 +394,43 @@ __global__ void pad_rows_kernel(const int8_t* __restrict__ src, int8_t* __restri
   }
 }
 
+// ---- weight gradient of a linear layer: operand transposition and the final correction ---------------------------
+// out[c][r] = in[r][c] for r < R, c < C; every output row is Rp long (zeros from R on).  With `ones_row`, output row C
+// holds 1 for r < R and rows C+1 .. C+15 hold zeros (not used at present).
+__global__ void __launch_bounds__(256) transpose_rows_kernel(const int8_t* __restrict__ in, int8_t* __restrict__ out, int R, int C, int Rp,
+                                                              int ones_row) {
+  __shared__ int8_t tile[32][33];
+  const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8 threads
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int r = r0 + ty + 8 * j, c = c0 + tx;
+    int8_t v = 0;
+    if (r < R) {
+      if (c < C) v = in[(int64_t)r * C + c];
+      else if (ones_row && c == C) v = 1;
+    }
+    tile[ty + 8 * j][tx] = v;
+  }
+  __syncthreads();
+  const int Ctot = C + (ones_row ? 16 : 0);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = c0 + ty + 8 * j, r = r0 + tx;
+    if (c < Ctot && r < Rp) out[(int64_t)c * Rp + r] = tile[tx][ty + 8 * j];
+  }
+}
+// sum_m (dy - z_dy)(x - z_x) = sum_m (dy - z_dy) x  -  z_x * sum_m (dy - z_dy): the second term, one number per output
+// row n, which the layer kernel's epilogue subtracts from every accumulator of that row.
+__global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int N, const hq_range_state* __restrict__ dyq,
+                                       const hq_range_state* __restrict__ xq, int32_t* __restrict__ terms) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= N) return;
+  int sum = 0;
+  for (int m = 0; m < M; ++m) sum += dY[(int64_t)m * N + n];
+  terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
+}
+
 // ---- depthwise convolution on CUDA cores --------------------------------------------------------
 // One thread: one output pixel x 16 consecutive channels.  Same epilogue as the tensor-core kernel.
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xffu); }
@@ -895,6 +932,17 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
   int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 16);
   if (blocks < 1) blocks = 1;
   pad_rows_kernel<<<blocks, 256, 0, s>>>(src, dst, rows, K, Kp);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, int Rp, int ones_row, cudaStream_t s) {
+  dim3 grid((unsigned)((Rp + 31) / 32), (unsigned)((C + (ones_row ? 16 : 0) + 31) / 32));
+  transpose_rows_kernel<<<grid, 256, 0, s>>>(in, out, R, C, Rp, ones_row);
+  return cudaGetLastError();
+}
+cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
+                                   cudaStream_t s) {
+  wgrad_row_terms_kernel<<<(N + 127) / 128, 128, 0, s>>>(dY, M, N, dyq, xq, terms);
   return cudaGetLastError();
 }
 

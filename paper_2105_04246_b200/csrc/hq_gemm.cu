@@ -646,7 +646,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int c_end = ((slice + 1) * nchunks) / slices;
     const bool has_corr = p.corr != nullptr;
     // per-layer part of the condition for the straight-line pass (see below)
-    const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.zc_in_smem && has_corr;
+    const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.row_term == nullptr &&
+                            p.zc_in_smem && has_corr;
     for (int local_tile = group; ; local_tile += ngroups) {
       const int tile = own_tile(local_tile);
       if (tile < 0) break;
@@ -719,6 +720,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 #pragma unroll
           for (int e = 0; e < CW; ++e)
             if (e < nvalid) v[e] += p.bias[col0 + c0 + e];
+        }
+        if (p.row_term != nullptr && row_valid) {   // flat layers: the output row is the pixel index
+          const int rt = p.row_term[pix];
+#pragma unroll
+          for (int e = 0; e < CW; ++e) v[e] -= rt;
         }
         if (nvalid == CW) {   // two independent chains, then merged: short dependency depth
           int lo[2], hi[2];

@@ -81,6 +81,7 @@ struct GemmParams {
   const uint8_t* colcls;              // [TW] or null
   int32_t cls_in_smem;                // both tables are non-null and fit the kernel's shared copy (TH, TW <= 512)
   const int32_t* bias;                // [Nout] or null
+  const int32_t* row_term;            // [output rows] or null: subtracted from every accumulator of the row (flat layers only)
   float acc_bound;                    // upper bound of |accumulator| before the bias: reduction length x 255 x 128
   const hq_range_state* xq;
   const float* w_scale;
@@ -197,6 +198,9 @@ cudaError_t launch_prep_window_weights(const int8_t* W, int8_t* Wmat, int K, int
                                        cudaStream_t s);
 cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s);
 cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
+cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, int Rp, int ones_row, cudaStream_t s);
+cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
+                                   cudaStream_t s);
 cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
                            const uint32_t* colmasks, int ncolcls, cudaStream_t s);
@@ -211,6 +215,8 @@ struct hq_ctx {
   size_t scratch_elems = 0;
   int8_t* d_pad = nullptr;            // zero-padded operand copies for linear layers whose K is not a multiple of 16
   size_t pad_bytes = 0;
+  uint8_t* d_wgrad = nullptr;         // weight gradient: transposed operands, int32 accumulators, one range state
+  size_t wgrad_bytes = 0;
   hq::EncodeTiledFn encode = nullptr;
   uint64_t launches = 0;
   uint64_t pair_launches = 0;         // of those, layer kernels launched as CTA pairs

@@ -1,0 +1,50 @@
+"""Weight gradient of a linear layer on the GPU (hq_linear_wgrad) against the oracle: every binary32 value equal.
+Sizes span several 128-row tiles of the transposed problem, ragged tails in all three dimensions and both zero points."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2105_04246_b200 import hq, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = hq.Context(0)
+    yield c
+    assert c.get_async_error() == 0
+    c.close()
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 16, 16), (7, 5, 3), (50, 130, 70), (128, 1000, 512), (300, 144, 24), (513, 40, 272), (64, 300, 1000)])
+def test_linear_wgrad_matches_oracle(ctx, M, N, K):
+    dev = torch.device("cuda", ctx.device)
+    r = synth.rng(301, M, N, K)
+    dy = synth.gradients(r, (M, N))
+    x = synth.relu_activations(r, (M, K)) if (M + N) % 2 else synth.signed_activations(r, (M, K))
+    dy_d, x_d = torch.from_numpy(dy.q).to(dev), torch.from_numpy(x.q).to(dev)
+    dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
+    xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
+    want = O.scale_to_real(O.linear_wgrad_acc(dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
+    for _ in range(2):    # the second call reuses the context's scratch with stale contents
+        gw = torch.full((N, K), float("nan"), dtype=torch.float32, device=dev)
+        ctx.linear_wgrad(None, M, N, K, dy_d, dyq, x_d, xq, gw)
+        torch.cuda.synchronize(dev)
+        got = gw.cpu().numpy()
+        bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
+        assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
+    assert ctx.get_async_error() == 0
+
+
+def test_linear_wgrad_rejections_launch_nothing(ctx):
+    dev = torch.device("cuda", ctx.device)
+    t = torch.zeros(1024, dtype=torch.int8, device=dev)
+    st = hq.states_to_device(hq.input_state(0.1, 0), dev)
+    g = torch.zeros(256, dtype=torch.float32, device=dev)
+    n0 = ctx.launch_count()
+    for args in [(0, 4, 4, t, st, t, st, g), (4, 4, 4, None, st, t, st, g), (70000, 4, 4, t, st, t, st, g)]:
+        with pytest.raises(hq.HqError):
+            ctx.linear_wgrad(None, *args)
+    assert ctx.launch_count() == n0
