@@ -208,7 +208,9 @@ hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
  * quantized output gradient and the weights, always quantized by Q_G):
  *   dX[n][hi][wi][c] = Q_G( sum over (r,s,k) with ho*stride_h - pad_h + r == hi (wo alike)
  *                           of (dY[n][ho][wo][k] - z_dy) * W[k][r][s][c] ).
- * dY is N x Ho x Wo x K, dX is N x H x W x C.  pw from hq_weights_prepare(.., HQ_DIR_BWD_DATA, ..). */
+ * dY is N x Ho x Wo x K, dX is N x H x W x C.  pw from hq_weights_prepare(.., HQ_DIR_BWD_DATA, ..).
+ * Depthwise layers (groups == C): stride 1 and pad <= filter size - 1 only (HQ_ERR_UNSUPPORTED otherwise, from
+ * hq_weights_prepare); the sum then runs over (r,s) alone with k == c. */
 hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                            const int8_t* dY, const hq_range_state* dyq,
                            const hq_prepared_weights* pw, const float* w_scale,

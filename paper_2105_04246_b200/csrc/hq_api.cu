@@ -513,8 +513,12 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
   if (!aligned16(in) || !aligned16(out) || !aligned16(inq) || !aligned16(outq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
   if (pw->dir != dir || !same_desc(pw->desc, *desc)) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights were built for another layer");
-  const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
   if (pw->depthwise) {
+    // the geometry the kernel runs (see hq_weights_prepare): for backward data the forward layer over the output gradient
+    const hq_conv_desc* const caller_desc = desc;
+    desc = &pw->dw_run;
+    (void)caller_desc;
+    const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
     DwParams p{};
     p.N = desc->N; p.H = desc->H; p.W = desc->W; p.C = desc->C; p.Ho = Ho; p.Wo = Wo; p.R = desc->R; p.S = desc->S;
     p.stride_h = desc->stride_h; p.stride_w = desc->stride_w; p.pad_h = desc->pad_h; p.pad_w = desc->pad_w;
@@ -564,6 +568,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     ctx->launches += 1;
     return HQ_OK;
   }
+  const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
   // operand A is the forward input (fwd) or the output gradient (bwd data)
   const int aC = dir == HQ_DIR_FWD ? desc->C : desc->K;
   const int aH = dir == HQ_DIR_FWD ? desc->H : Ho;
@@ -890,15 +895,27 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
     return e;
   };
 
+  // Backward data of a stride-1 depthwise layer is a forward depthwise layer over the output gradient (Ho x Wo) with the
+  // filter turned by 180 degrees and padding R-1-pad: dx(hi) = sum_r dy(hi + pad - r) w(r) = sum_r' dy(hi - (R-1-pad) + r') w(R-1-r').
+  const bool dw_bwd = d.groups != 1 && dir == HQ_DIR_BWD_DATA;
+  hq_conv_desc dwd = d;
   if (d.groups != 1) {
-    if (dir != HQ_DIR_FWD) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data is not implemented"));
     if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise needs C %% 16 == 0"));
+    if (dw_bwd) {
+      if (d.stride_h != 1 || d.stride_w != 1) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data needs stride 1"));
+      if (d.pad_h > d.R - 1 || d.pad_w > d.S - 1) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data needs pad <= filter size - 1"));
+      dwd.H = Ho;
+      dwd.W = Wo;
+      dwd.pad_h = d.R - 1 - d.pad_h;
+      dwd.pad_w = d.S - 1 - d.pad_w;
+    }
   }
+  pw->dw_run = dwd;
   // Optional form of a depthwise layer on the tensor cores: ceil(C / 64) dense layers, one per 64-channel slice of
   // input and output, each with a weight matrix that is zero off the channel diagonal (the int32 sums are the same).
   // Measured on the 56x56x144 layer it is only on a par with the CUDA-core kernel (N = 64 MMAs are bound by
   // shared-memory reads of the pixel operand), so it is not chosen by default.
-  const bool dw_dense = d.groups != 1 && ctx->force_depthwise == 1;
+  const bool dw_dense = d.groups != 1 && ctx->force_depthwise == 1 && !dw_bwd;
   if (dw_dense) {
     for (int c0 = 0; c0 < d.C; c0 += 64) {
       const int cw = std::min(64, d.C - c0);
@@ -927,18 +944,20 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   if (d.groups != 1 && !dw_dense) {
     pw->depthwise = true;
     std::vector<int> dh, dw;
-    for (int r = 0; r < d.R; ++r) dh.push_back(r - d.pad_h);
-    for (int q = 0; q < d.S; ++q) dw.push_back(q - d.pad_w);
+    for (int r = 0; r < d.R; ++r) dh.push_back(r - dwd.pad_h);
+    for (int q = 0; q < d.S; ++q) dw.push_back(q - dwd.pad_w);
     std::vector<uint8_t> rowcls, colcls;
     std::vector<uint32_t> rm, cm;
-    border_classes(Ho, d.stride_h, dh, d.H, rowcls, rm);
-    border_classes(Wo, d.stride_w, dw, d.W, colcls, cm);
+    // output rows / columns of the layer the kernel runs (backward data: the input image of the original layer)
+    const int run_Ho = out_dim(dwd.H, dwd.pad_h, dwd.R, dwd.stride_h), run_Wo = out_dim(dwd.W, dwd.pad_w, dwd.S, dwd.stride_w);
+    border_classes(run_Ho, dwd.stride_h, dh, dwd.H, rowcls, rm);
+    border_classes(run_Wo, dwd.stride_w, dw, dwd.W, colcls, cm);
     if (rm.size() > 16 || cm.size() > 16) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "too many border classes"));
     pw->dw_ncolcls = (int)cm.size();
     pw->dw_ncls = (int)(rm.size() * cm.size());
     if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_w, (size_t)d.C * d.R * d.S)) != HQ_OK) return bail(st);
     if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_corr, rm.size() * cm.size() * d.C * sizeof(int32_t))) != HQ_OK) return bail(st);
-    cudaError_t e = launch_dw_prep(W, pw->dw_w, pw->dw_corr, d.C, d.R, d.S, rm.data(), (int)rm.size(), cm.data(), (int)cm.size(), s);
+    cudaError_t e = launch_dw_prep(W, pw->dw_w, pw->dw_corr, d.C, d.R, d.S, rm.data(), (int)rm.size(), cm.data(), (int)cm.size(), dw_bwd ? 1 : 0, s);
     if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "depthwise weight preparation failed: %s", cudaGetErrorString(e)));
     ctx->launches += 1;
     if ((st = upload(ctx, pw, rowcls, &pw->dw_rowcls, s)) != HQ_OK) return bail(st);

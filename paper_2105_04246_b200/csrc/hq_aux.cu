@@ -192,12 +192,14 @@ __global__ void corr_kernel(const int8_t* __restrict__ Wmat, int32_t* __restrict
 }
 
 // depthwise: weights to tap-major [R*S][C]; corr[cls][c] = sum of valid taps
+// flip: tap t of the prepared filter is tap R*S-1-t of W (the filter turned by 180 degrees, which makes backward data
+// of a stride-1 depthwise layer a forward depthwise layer over the output gradient)
 __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict__ Wt, int32_t* __restrict__ corr, int C, int R, int S, ClassMasks m,
-                               int nrowcls, int ncolcls) {
+                               int nrowcls, int ncolcls, int flip) {
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx < C * R * S) {
     const int c = idx % C, t = idx / C;
-    Wt[idx] = W[c * R * S + t];
+    Wt[idx] = W[c * R * S + (flip ? R * S - 1 - t : t)];
   }
   if (idx < nrowcls * ncolcls * C) {
     const int c = idx % C, cls = idx / C;
@@ -205,7 +207,7 @@ __global__ void dw_prep_kernel(const int8_t* __restrict__ W, int8_t* __restrict_
     int32_t sum = 0;
     for (int r = 0; r < R; ++r)
       for (int s = 0; s < S; ++s)
-        if (((m.row[rc] >> r) & 1u) && ((m.col[cc] >> s) & 1u)) sum += W[c * R * S + r * S + s];
+        if (((m.row[rc] >> r) & 1u) && ((m.col[cc] >> s) & 1u)) sum += W[c * R * S + (flip ? R * S - 1 - (r * S + s) : r * S + s)];
     corr[idx] = sum;
   }
 }
@@ -878,13 +880,13 @@ cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int c
 }
 
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
-                           const uint32_t* colmasks, int ncolcls, cudaStream_t s) {
+                           const uint32_t* colmasks, int ncolcls, int flip, cudaStream_t s) {
   ClassMasks m{};
   for (int i = 0; i < nrowcls; ++i) m.row[i] = rowmasks[i];
   for (int i = 0; i < ncolcls; ++i) m.col[i] = colmasks[i];
   int total = nrowcls * ncolcls * C;
   if (C * R * S > total) total = C * R * S;
-  dw_prep_kernel<<<(total + 127) / 128, 128, 0, s>>>(W, Wt, corr, C, R, S, m, nrowcls, ncolcls);
+  dw_prep_kernel<<<(total + 127) / 128, 128, 0, s>>>(W, Wt, corr, C, R, S, m, nrowcls, ncolcls, flip);
   return cudaGetLastError();
 }
 

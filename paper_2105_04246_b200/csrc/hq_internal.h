@@ -203,7 +203,7 @@ cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_rang
                                    cudaStream_t s);
 cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
-                           const uint32_t* colmasks, int ncolcls, cudaStream_t s);
+                           const uint32_t* colmasks, int ncolcls, int flip, cudaStream_t s);
 
 }  // namespace hq
 
@@ -257,6 +257,8 @@ struct hq_prepared_weights {
   hq_conv_desc desc{};
   hq_direction dir = HQ_DIR_FWD;
   bool depthwise = false;
+  hq_conv_desc dw_run{};              // geometry the depthwise kernel runs: desc itself (forward) or, for backward data of a stride-1
+                                      // layer, the forward layer over the output gradient with the turned filter
   mutable bool used = false;          // set by the first layer call: later calls know that the tables were complete long before
   std::vector<hq_sub_problem> subs;
   // depthwise tables

@@ -262,6 +262,42 @@ def test_conv_bwd_data_cta_pairs(ctx, name, staging):
         assert ctx.pair_launch_count() > n0, "the layer did not run as CTA pairs"
 
 
+DW_BWD_CASES = {
+    "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
+    "dw3x3_c32_ragged": dict(N=3, H=13, W=21, Cin=32, K=32, R=3, S=3, stride=1, pad=1, groups=32),
+    "dw3x3_c256_nopad": dict(N=1, H=11, W=12, Cin=256, K=256, R=3, S=3, stride=1, pad=0, groups=256),
+    "dw5x5_c48": dict(N=1, H=13, W=9, Cin=48, K=48, R=5, S=5, stride=1, pad=2, groups=48),
+    "dw3x3_c64_wide": dict(N=2, H=9, W=150, Cin=64, K=64, R=3, S=3, stride=1, pad=1, groups=64),
+    "dw5x5_c16_pad1": dict(N=2, H=9, W=8, Cin=16, K=16, R=5, S=5, stride=1, pad=1, groups=16),
+}
+
+
+@pytest.mark.parametrize("dw_staging", [0, 1])
+@pytest.mark.parametrize("name", list(DW_BWD_CASES))
+def test_depthwise_bwd_data(ctx, name, dw_staging):
+    """Input gradient of a stride-1 depthwise layer (run as a forward depthwise layer over the output gradient with the
+    filter turned by 180 degrees) against the oracle's backward-data definition, in both staging forms of the kernel."""
+    shape = dict(DW_BWD_CASES[name])
+    r = synth.rng(111, len(name), shape["H"], dw_staging)
+    W = _weights(r, shape)
+    Ho = shape["H"] + 2 * shape["pad"] - shape["R"] + 1
+    Wo = shape["W"] + 2 * shape["pad"] - shape["S"] + 1
+    in_shape = (shape["N"], Ho, Wo, shape["K"])
+    ctx.set_option("depthwise_staging", dw_staging)
+    try:
+        _run_iterations(ctx, "conv_bwd", W, shape, lambda t: synth.gradients(r, in_shape), 3)
+    finally:
+        ctx.set_option("depthwise_staging", -1)
+
+
+def test_depthwise_bwd_data_strided_is_refused(ctx):
+    dev = torch.device("cuda", ctx.device)
+    W = torch.zeros((32, 3, 3), dtype=torch.int8, device=dev)
+    with pytest.raises(hq.HqError) as e:
+        ctx.weights_prepare(None, hq.conv_desc(2, 11, 11, 32, 32, 3, 3, stride=2, pad=1, groups=32), hq.DIR_BWD_DATA, W)
+    assert e.value.status == 2
+
+
 # ---- protocol and edge cases ---------------------------------------------------------------------
 def test_teacher_forced_state_and_saturation(ctx):
     """The oracle is fed the GPU's own state before each step: isolates the layer kernel from the
