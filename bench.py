@@ -65,6 +65,9 @@ def workload_layers(name: str, batch_div: int = 1):
         return [("conv_bwd", b(wl.CFG3_BWD), "grad")], False
     if name == "cfg4":
         return [("conv_fwd", b(wl.CFG4_EXPAND), "signed"), ("conv_fwd", b(wl.CFG4_DW), None), ("conv_fwd", b(wl.CFG4_PROJECT), None)], True
+    if name == "cfg4b":
+        # backward data through the same inverted residual, last layer first; each input gradient feeds the layer before
+        return [("conv_bwd", b(wl.CFG4_PROJECT), "grad"), ("conv_bwd", b(wl.CFG4_DW), None), ("conv_bwd", b(wl.CFG4_EXPAND), None)], True
     if name == "cfg5":
         # every convolution of ResNet-18 at 224x224 and the classifier, forward and backward-data (none for the stem);
         # each call has its own synthetic input: what sits between the layers (BN, ReLU, pooling, adds) is not on the path
@@ -317,7 +320,7 @@ def run_gpu(args):
     ctx.set_option("depthwise", args.depthwise)
     peaks, peak_kind = load_peaks()
     name = args.workload
-    pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg5": 2}[name]
+    pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg4b": 2, "cfg5": 2}[name]
     wk = GpuWorkload(name, ctx, dev, pool, seed_key=rank, stochastic=args.rounding == "stochastic")
     K, W = args.steps, max(3, args.warmup)
     stream = torch.cuda.current_stream(dev)
@@ -611,8 +614,9 @@ def main():
     ap.add_argument("--steps", type=int, default=600)
     ap.add_argument("--warmup", type=int, default=24)
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5", "wgrad"],
-                    help="cfg1..cfg5: the five layer workloads; wgrad: the weight gradient of a linear layer (a later row of the scope)")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad"],
+                    help="cfg1..cfg5: the five layer workloads; cfg4b: backward data through cfg4's block; wgrad: the weight gradient "
+                         "of a linear layer (a later row of the scope)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--rounding", default="nearest", choices=["nearest", "stochastic"],
                     help="stochastic: backward-data (gradient) layers use stochastic rounding, the paper's choice for gradients")
