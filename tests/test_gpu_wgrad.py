@@ -48,3 +48,24 @@ def test_linear_wgrad_rejections_launch_nothing(ctx):
         with pytest.raises(hq.HqError):
             ctx.linear_wgrad(None, *args)
     assert ctx.launch_count() == n0
+
+
+def test_linear_wgrad_bench_size_sampled_rows(ctx):
+    """The benchmark's shape (4096 -> 4096 classifier layer at batch 256): output rows sampled over the whole matrix,
+    each compared in full with the oracle (the oracle computes a row block from the matching columns of dY)."""
+    dev = torch.device("cuda", ctx.device)
+    M, N, K = 256, 4096, 4096
+    r = synth.rng(302)
+    dy, x = synth.gradients(r, (M, N)), synth.relu_activations(r, (M, K))
+    dy_d, x_d = torch.from_numpy(dy.q).to(dev), torch.from_numpy(x.q).to(dev)
+    dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
+    xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
+    gw = torch.empty((N, K), dtype=torch.float32, device=dev)
+    ctx.linear_wgrad(None, M, N, K, dy_d, dyq, x_d, xq, gw)
+    torch.cuda.synchronize(dev)
+    got = gw.cpu().numpy()
+    rows = np.unique(np.concatenate([np.arange(0, 130), np.arange(2040, 2060), np.arange(N - 70, N), r.integers(0, N, 64)]))
+    want = O.scale_to_real(O.linear_wgrad_acc(np.ascontiguousarray(dy.q[:, rows]), dy.zero_point, x.q, x.zero_point),
+                           O.acc_scale(dy.scale, x.scale))
+    assert np.array_equal(got[rows].view(np.uint32), want.view(np.uint32))
+    assert np.isfinite(got).all()
