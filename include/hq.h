@@ -220,7 +220,8 @@ hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
  * input give G_W, which the paper keeps in FP32):
  *   GW[n][k] = fl( float( sum_m (dY[m][n] - z_dy) * (X[m][k] - z_x) ) * fl(s_dy * s_x) ),  one binary32 rounding per step,
  * with (s_dy, z_dy) = scale / zero_point of *dyq and (s_x, z_x) of *xq.  dY is [M][N], X is [M][K], GW is [N][K] binary32,
- * laid out like the weights.  The sum is exact in int32; M may not exceed 65536.  The reduction runs over the rows, so the
+ * laid out like the weights.  The sum is formed modulo 2^32, so it is exact whenever the true sum fits in int32 (partial
+ * sums may leave that range); M may not exceed 2^24.  The reduction runs over the rows, so the
  * call first transposes both operands into context-owned scratch (grown with cudaMalloc when a larger layer is first
  * seen; calls on one context must not overlap) and runs the tensor-core layer kernel on them with a binary32
  * epilogue.  Nothing is quantized and no range state is written. */

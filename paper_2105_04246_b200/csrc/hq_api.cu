@@ -1137,8 +1137,9 @@ __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, vo
   if (!dY || !dyq || !X || !xq || !GW) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(dY) || !aligned16(X) || !aligned16(GW) || !aligned16(dyq) || !aligned16(xq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
-  // |sum_m (dy - z_dy) * x| <= M * 255 * 128 has to stay inside int32 before the input zero point is taken out
-  if (M > 65536) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient over more than 65536 rows (M = %d) could leave the int32 range", M);
+  // The accumulator, the column-sum correction and the per-row term are all added modulo 2^32 (the MMA is issued without
+  // saturation), so a partial sum that leaves the int32 range does no harm as long as the gradient itself fits.
+  if (M > (1 << 24)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient over more than 2^24 rows (M = %d)", M);
   cudaStream_t s = (cudaStream_t)stream;
   // The reduction runs over the rows (the batch), so both operands are transposed first: A = dY^T [N][Mp] and
   // B = X^T [K][Mp] (Mp = M rounded up to 16, zero filled).  The layer kernel removes the zero point of its first

@@ -38,13 +38,32 @@ def test_linear_wgrad_matches_oracle(ctx, M, N, K):
     assert ctx.get_async_error() == 0
 
 
+def test_linear_wgrad_partial_sums_may_leave_int32(ctx):
+    """70000 rows of dy - z_dy = 255 against x = 127: the sum before the zero point of x is taken out is 2.27e9 > 2^31,
+    the gradient itself is 255 * 70000 * (127 - z_x).  All additions are modulo 2^32, so the result is exact."""
+    dev = torch.device("cuda", ctx.device)
+    M, N, K = 70000, 16, 32
+    dy = np.full((M, N), 127, np.int8)
+    x = np.full((M, K), 127, np.int8)
+    x[:, 1] = 126
+    dy_d, x_d = torch.from_numpy(dy).to(dev), torch.from_numpy(x).to(dev)
+    dyq = hq.states_to_device(hq.input_state(0.5, -128), dev)
+    xq = hq.states_to_device(hq.input_state(0.25, 127), dev)
+    gw = torch.full((N, K), float("nan"), dtype=torch.float32, device=dev)
+    ctx.linear_wgrad(None, M, N, K, dy_d, dyq, x_d, xq, gw)
+    torch.cuda.synchronize(dev)
+    want = O.scale_to_real(O.linear_wgrad_acc(dy, -128, x, 127), O.acc_scale(0.5, 0.25))
+    assert want[0, 0] == 0.0 and want[0, 1] == np.float32(-255 * M) * np.float32(0.125)
+    assert np.array_equal(gw.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
 def test_linear_wgrad_rejections_launch_nothing(ctx):
     dev = torch.device("cuda", ctx.device)
     t = torch.zeros(1024, dtype=torch.int8, device=dev)
     st = hq.states_to_device(hq.input_state(0.1, 0), dev)
     g = torch.zeros(256, dtype=torch.float32, device=dev)
     n0 = ctx.launch_count()
-    for args in [(0, 4, 4, t, st, t, st, g), (4, 4, 4, None, st, t, st, g), (70000, 4, 4, t, st, t, st, g)]:
+    for args in [(0, 4, 4, t, st, t, st, g), (4, 4, 4, None, st, t, st, g), ((1 << 24) + 1, 4, 4, t, st, t, st, g)]:
         with pytest.raises(hq.HqError):
             ctx.linear_wgrad(None, *args)
     assert ctx.launch_count() == n0
