@@ -60,6 +60,7 @@ def lib():
         L.hqo_derive.argtypes = [rp]; L.hqo_derive.restype = None
         L.hqo_linear_acc.argtypes = [C.c_int, C.c_int, C.c_int, i8p, C.c_int, i8p, C.c_int, i32p, i32p]; L.hqo_linear_acc.restype = C.c_int
         L.hqo_linear_wgrad_acc.argtypes = [C.c_int, C.c_int, C.c_int, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_linear_wgrad_acc.restype = C.c_int
+        L.hqo_conv_wgrad_acc.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_conv_wgrad_acc.restype = C.c_int
         L.hqo_scale_to_real.argtypes = [i32p, C.c_int64, C.c_float, f32p]; L.hqo_scale_to_real.restype = None
         L.hqo_conv_fwd_acc.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_conv_fwd_acc.restype = C.c_int
         L.hqo_conv_bwd_data_acc.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i32p]; L.hqo_conv_bwd_data_acc.restype = C.c_int
@@ -121,6 +122,18 @@ def linear_wgrad_acc(dY, zdy, X, zx) -> np.ndarray:
     assert X.shape[0] == M
     g = np.empty((N, K), np.int32)
     ovf = lib().hqo_linear_wgrad_acc(M, N, K, _p(dY, C.c_int8), int(zdy), _p(X, C.c_int8), int(zx), _p(g, C.c_int32))
+    assert ovf == 0, "int32 accumulator overflow"
+    return g
+
+
+def conv_wgrad_acc(d: Conv, dY, zdy, X, zx) -> np.ndarray:
+    """int32 g[k,r,s,c] = sum over output pixels of (dy - z_dy) * (x - z_x), padded taps skipped (dense layers)."""
+    assert d.groups == 1
+    dY, X = _i8(dY), _i8(X)
+    Ho, Wo = out_hw(d)
+    assert dY.shape == (d.N, Ho, Wo, d.K) and X.shape == (d.N, d.H, d.W, d.C)
+    g = np.empty((d.K, d.R, d.S, d.C), np.int32)
+    ovf = lib().hqo_conv_wgrad_acc(C.byref(d), _p(dY, C.c_int8), int(zdy), _p(X, C.c_int8), int(zx), _p(g, C.c_int32))
     assert ovf == 0, "int32 accumulator overflow"
     return g
 

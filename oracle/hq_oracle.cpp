@@ -145,6 +145,36 @@ int hqo_linear_wgrad_acc(int M, int N, int K, const int8_t* dY, int zdy, const i
     }
   return ovf;
 }
+// weight gradient of a convolution (Sec. 3.1, backward pass), W layout [K][R][S][C]:
+//   g(k,r,s,c) = sum over n,ho,wo of (dy(n,ho,wo,k) - z_dy) * (x(n,hi,wi,c) - z_x),  hi = ho*stride_h - pad_h + r (wi alike),
+//   over those output pixels whose (hi,wi) lies inside the image: padding is zero in the real domain (R-8), so a padded
+//   tap contributes nothing.  G_W = fl(float(g) * fl(s_dy * s_x)).  Dense layers only (groups == 1).
+int hqo_conv_wgrad_acc(const hqo_conv* d, const int8_t* dY, int zdy, const int8_t* X, int zx, int32_t* g) {
+  const int Ho = hqo_out_h(d), Wo = hqo_out_w(d);
+  int ovf = 0;
+#pragma omp parallel for collapse(2) reduction(| : ovf)
+  for (int k = 0; k < d->K; ++k)
+    for (int r = 0; r < d->R; ++r)
+      for (int s = 0; s < d->S; ++s)
+        for (int c = 0; c < d->C; ++c) {
+          int64_t a = 0;
+          for (int n = 0; n < d->N; ++n)
+            for (int ho = 0; ho < Ho; ++ho) {
+              const int hi = ho * d->stride_h - d->pad_h + r;
+              if (hi < 0 || hi >= d->H) continue;
+              for (int wo = 0; wo < Wo; ++wo) {
+                const int wi = wo * d->stride_w - d->pad_w + s;
+                if (wi < 0 || wi >= d->W) continue;
+                a += (int64_t)((int)dY[(((int64_t)n * Ho + ho) * Wo + wo) * d->K + k] - zdy) *
+                     ((int)X[(((int64_t)n * d->H + hi) * d->W + wi) * d->C + c] - zx);
+              }
+            }
+          if (a > INT32_MAX || a < INT32_MIN) ovf |= 1;
+          g[(((int64_t)k * d->R + r) * d->S + s) * d->C + c] = (int32_t)a;
+        }
+  return ovf;
+}
+
 void hqo_scale_to_real(const int32_t* acc, int64_t count, float s_acc, float* out) {
   for (int64_t i = 0; i < count; ++i) out[i] = (float)acc[i] * s_acc;
 }

@@ -50,3 +50,56 @@ def test_real_value_is_one_binary32_multiplication():
     want = acc.astype(np.float32) * s                               # int -> binary32 (round to nearest even), one multiplication
     assert got.dtype == np.float32 and np.array_equal(got, want)
     assert got[0, 0] == 0.0 and got[0, 1] == s and got[0, 2] == -s
+
+
+# ---- convolution weight gradient ------------------------------------------------------------------
+def _conv_cases():
+    return [dict(N=2, H=5, W=6, C=3, K=4, R=3, S=3, stride=1, pad=1), dict(N=1, H=7, W=7, C=2, K=3, R=3, S=3, stride=2, pad=1),
+            dict(N=2, H=6, W=5, C=4, K=2, R=1, S=1, stride=1, pad=0), dict(N=1, H=9, W=8, C=2, K=2, R=5, S=5, stride=2, pad=2),
+            dict(N=3, H=4, W=4, C=2, K=5, R=3, S=3, stride=1, pad=0)]
+
+
+def _desc(c):
+    return O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["K"], c["R"], c["S"], stride=c["stride"], pad=c["pad"])
+
+
+def test_conv_wgrad_pointwise_is_the_linear_gradient():
+    r = np.random.default_rng(21)
+    c = dict(N=2, H=6, W=5, C=4, K=3, R=1, S=1, stride=1, pad=0)
+    d = _desc(c)
+    dy, x = _rand(r, (2, 6, 5, 3)), _rand(r, (2, 6, 5, 4))
+    g = O.conv_wgrad_acc(d, dy, -3, x, 7)
+    assert np.array_equal(g.reshape(3, 4), O.linear_wgrad_acc(dy.reshape(-1, 3), -3, x.reshape(-1, 4), 7))
+
+
+def test_conv_wgrad_trace_identity_with_the_forward_convolution():
+    """<dY - z, conv_fwd(X, W)> == <conv_wgrad(dY, X), W> in exact integers, for every geometry: ties the gradient's
+    index arithmetic (strides, padding skipped, tap order) to the forward convolution, which has its own pins."""
+    r = np.random.default_rng(22)
+    for c in _conv_cases():
+        d = _desc(c)
+        Ho, Wo = O.out_hw(d)
+        dy, x = _rand(r, (c["N"], Ho, Wo, c["K"])), _rand(r, (c["N"], c["H"], c["W"], c["C"]))
+        w = _rand(r, (c["K"], c["R"], c["S"], c["C"]))
+        zdy, zx = int(r.integers(-128, 128)), int(r.integers(-128, 128))
+        y = O.conv_fwd_acc(d, x, zx, w).astype(np.int64)
+        lhs = int(((dy.astype(np.int64) - zdy) * y).sum())
+        rhs = int((O.conv_wgrad_acc(d, dy, zdy, x, zx).astype(np.int64) * w.astype(np.int64)).sum())
+        assert lhs == rhs, c
+
+
+def test_conv_wgrad_against_library_convolution():
+    """torch's weight gradient of conv2d in float64 on the zero-point-corrected integers (exact below 2^53); padding
+    there is zero AFTER the correction, which is the reading the oracle takes."""
+    import torch
+    r = np.random.default_rng(23)
+    for c in _conv_cases():
+        d = _desc(c)
+        Ho, Wo = O.out_hw(d)
+        dy, x = _rand(r, (c["N"], Ho, Wo, c["K"])), _rand(r, (c["N"], c["H"], c["W"], c["C"]))
+        zdy, zx = -5, 11
+        xt = torch.from_numpy((x.astype(np.float64) - zx).transpose(0, 3, 1, 2).copy())
+        gt = torch.from_numpy((dy.astype(np.float64) - zdy).transpose(0, 3, 1, 2).copy())
+        gw = torch.nn.grad.conv2d_weight(xt, (c["K"], c["C"], c["R"], c["S"]), gt, stride=c["stride"], padding=c["pad"])
+        want = gw.numpy().transpose(0, 2, 3, 1).round().astype(np.int64)
+        assert np.array_equal(O.conv_wgrad_acc(d, dy, zdy, x, zx).astype(np.int64), want), c
