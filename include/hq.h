@@ -229,6 +229,19 @@ hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32
                           const int8_t* dY, const hq_range_state* dyq,
                           const int8_t* X, const hq_range_state* xq, float* GW);
 
+/* Weight gradient of a dense convolution (Sec. 3.1, backward pass; kept in FP32 like the paper's):
+ *   GW[k][r][s][c] = fl( float( sum over n,ho,wo of (dY[n][ho][wo][k] - z_dy) * (X[n][hi][wi][c] - z_x) ) * fl(s_dy * s_x) ),
+ * hi = ho*stride_h - pad_h + r (wi alike), output pixels whose (hi,wi) lies outside the image contributing nothing (padding
+ * is zero in the real domain).  dY is N x Ho x Wo x K, X is N x H x W x C, GW has the layout of the weights, binary32.
+ * The sum is formed modulo 2^32: exact whenever the true sum fits in int32.  groups must be 1; at most 2^24 output pixels.
+ * How it runs: the filter windows of X and dY are written transposed (pixels innermost) into context-owned scratch (grown
+ * with cudaMalloc when a larger layer is first seen: R*S times the size of X; calls on one context must not overlap);
+ * the reduction over the pixels is cut into slices that the tensor-core layer kernel multiplies side by side, and a last
+ * pass sums the slices, removes both zero points and converts.  No range state is written. */
+hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
+                        const int8_t* dY, const hq_range_state* dyq,
+                        const int8_t* X, const hq_range_state* xq, float* GW);
+
 /* Eq. 2-3 for `count` consecutive states, to be enqueued after the layer calls of the iteration:
  *   m_lo = float(acc_min) * acc_scale, m_hi alike;
  *   step == 0:  q_min = m_lo, q_max = m_hi                      (initialisation, Sec. 4.1)

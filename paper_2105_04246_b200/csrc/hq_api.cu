@@ -118,6 +118,8 @@ struct SubSpec {            // geometry of one launch, before tiling
   int64_t ldY;
   bool flat;
   bool whole_gpu = true;    // false: the launch shares the SMs with other launches of the same call
+  int slices = 0;           // flat GEMM whose reduction is cut into `slices` pieces of `slice_len` bytes: n_img == slices, image n
+  int slice_len = 0;        // of the tile space multiplies reduction range [n * slice_len, (n + 1) * slice_len) into its own output slab
 };
 
 // fills everything in sub.p that does not depend on per-call pointers, for a given number of column tiles
@@ -130,7 +132,16 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
   p.TW = sp.TW;
   p.in_mul_h = sp.in_mul_h;
   p.in_mul_w = sp.in_mul_w;
-  pick_tile(sp.n_img, sp.TH, sp.TW, sp.in_mul_h, sp.in_mul_w, p.Nt, p.Ht, p.Wt);
+  auto tile_shape = [&]() {
+    pick_tile(sp.n_img, sp.TH, sp.TW, sp.in_mul_h, sp.in_mul_w, p.Nt, p.Ht, p.Wt);
+    if (sp.slices > 0) {   // one slice per tile: rows only
+      p.Nt = 1;
+      p.Ht = 1;
+      p.Wt = kTileM;
+    }
+  };
+  tile_shape();
+  p.b_slice = sp.slices > 0 ? sp.slice_len : 0;
   p.tiles_n = ceil_div(sp.n_img, p.Nt);
   p.tiles_h = ceil_div(sp.TH, p.Ht);
   p.tiles_w = ceil_div(sp.TW, p.Wt);
@@ -253,14 +264,15 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
     }
   }
   if (p.mode == kModeTap) {
-    pick_tile(sp.n_img, sp.TH, sp.TW, sp.in_mul_h, sp.in_mul_w, p.Nt, p.Ht, p.Wt);
+    tile_shape();
     p.num_tiles = (int)nt;
     p.num_pair_tiles = ceil_div(p.tiles_n * p.tiles_h * p.tiles_w, 2) * p.tiles_col;
     p.stage_bytes_a = (uint32_t)kTileM * p.BK;
     // a small weight matrix stays in shared memory for the whole kernel; the ring then carries operand A only
     const int kiters = p.ntaps * p.chunks_per_tap;
     const uint64_t b_all = (uint64_t)p.tiles_col * kiters * full_stage_b;
-    if (kiters > 0 && p.tiles_col * kiters <= kMaxStagesB && b_all <= 64u * 1024u && b_all + 6ull * p.stage_bytes_a <= ring_budget) {
+    if (kiters > 0 && sp.slices == 0 && p.tiles_col * kiters <= kMaxStagesB && b_all <= 64u * 1024u &&
+        b_all + 6ull * p.stage_bytes_a <= ring_budget) {
       p.b_resident = 1;
       p.stages_b = p.tiles_col * kiters;
       p.stages_a = (int)std::min<uint64_t>(kMaxStagesA, (ring_budget - b_all) / p.stage_bytes_a);
@@ -1167,6 +1179,89 @@ __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, vo
   // GW[n][k] = fl(float(acc) * fl(s_dy * s_x)): the layer kernel's binary32 output mode; its "weight scale" is the scale of X
   const float* x_scale = reinterpret_cast<const float*>(reinterpret_cast<const char*>(xq) + offsetof(hq_range_state, scale));
   return run_linear(ctx, s, N, K, Mp, At, dyq, Bt, x_scale, nullptr, GW, tmp, kOutF32, terms);
+}
+
+__attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* dY,
+                                                               const hq_range_state* dyq, const int8_t* X, const hq_range_state* xq, float* GW) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  hq_status st = check_desc(ctx, desc);
+  if (st != HQ_OK) return st;
+  if (!dY || !dyq || !X || !xq || !GW) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
+  if (!aligned16(dY) || !aligned16(X) || !aligned16(GW) || !aligned16(dyq) || !aligned16(xq))
+    return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
+  const hq_conv_desc& d = *desc;
+  if (d.groups != 1) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient of grouped convolutions is not implemented");
+  cudaStream_t s = (cudaStream_t)stream;
+  const int Ho = out_dim(d.H, d.pad_h, d.R, d.stride_h), Wo = out_dim(d.W, d.pad_w, d.S, d.stride_w);
+  const int64_t M64 = (int64_t)d.N * Ho * Wo;
+  const int64_t cols64 = (int64_t)d.R * d.S * d.C;
+  if (M64 > (1 << 24) || cols64 > (1 << 20)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels or filter elements");
+  const int M = (int)M64, rows = d.K, cols = (int)cols64;
+  // G_W as one GEMM over the output pixels m: rows k (dY^T [K][M]) x columns (r,s,c) (the filter windows of X,
+  // transposed: Bt [(r,s,c)][M]).  The output is as small as the weights while the reduction is long, so the reduction is
+  // cut into slices that run as the "images" of the layer kernel's tile space, each into an int32 slab of its own; a last
+  // pass sums the slabs, takes out both zero points and converts.  Slice length: a multiple of 128 bytes that gives the
+  // SMs about two tiles each.
+  const int tiles_one = ceil_div(rows, kTileM) * ceil_div(cols, 256);
+  int want_slices = std::max(1, (2 * ctx->num_sms + tiles_one - 1) / tiles_one);
+  int slice_len = std::max(128, round_up(ceil_div(M, want_slices), 128));
+  const int slices = ceil_div(M, slice_len);
+  const int64_t Mp = (int64_t)slices * slice_len;
+  const size_t a_bytes = ((size_t)rows * Mp + 255) & ~(size_t)255, b_bytes = ((size_t)cols * Mp + 255) & ~(size_t)255;
+  const size_t slab_bytes = ((size_t)slices * rows * cols * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t sum_bytes = (((size_t)rows + cols) * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t need = a_bytes + b_bytes + slab_bytes + sum_bytes + 256;
+  if (need > ctx->wgrad_bytes) {
+    if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));
+    ctx->d_wgrad = nullptr;
+    ctx->wgrad_bytes = 0;
+    HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_wgrad, need));
+    ctx->wgrad_bytes = need;
+  }
+  int8_t* At = reinterpret_cast<int8_t*>(ctx->d_wgrad);
+  int8_t* Bt = At + a_bytes;
+  int32_t* slabs = reinterpret_cast<int32_t*>(ctx->d_wgrad + a_bytes + b_bytes);
+  int32_t* rowsum = reinterpret_cast<int32_t*>(ctx->d_wgrad + a_bytes + b_bytes + slab_bytes);
+  int32_t* colsum = rowsum + rows;
+  hq_range_state* tmp = reinterpret_cast<hq_range_state*>(ctx->d_wgrad + a_bytes + b_bytes + slab_bytes + sum_bytes);
+  if (Mp > INT32_MAX) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels");
+  HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, rows, (int)Mp, 0, s));
+  HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, s));
+  const uint32_t one = 1u;
+  HQ_CUDA(ctx, launch_corr(At, rowsum, rows, 1, (int)Mp, 1, 1, &one, 1, &one, 1, rows, s));
+  HQ_CUDA(ctx, launch_corr(Bt, colsum, cols, 1, (int)Mp, 1, 1, &one, 1, &one, 1, cols, s));
+  ctx->launches += 4;
+  SubSpec sp{};
+  sp.n_img = slices; sp.TH = 1; sp.TW = rows; sp.in_mul_h = 1; sp.in_mul_w = 1;
+  sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = rows; sp.Cin = slice_len; sp.Nout = cols;
+  sp.out_H = 1; sp.out_W = rows; sp.os_h = 1; sp.os_w = 1; sp.oa_h = 0; sp.oa_w = 0; sp.ldY = cols; sp.flat = true;
+  sp.slices = slices; sp.slice_len = slice_len;
+  hq_sub_problem sub;
+  std::vector<uint8_t> rc, cc;
+  std::vector<uint32_t> rm, cm;
+  st = plan_sub(ctx, sp, sub, rc, cc, rm, cm);
+  if (st != HQ_OK) return st;
+  sub.p.corr = nullptr;       // both zero points are taken out after the slabs are summed
+  sub.p.zc_in_smem = 0;       // no correction table: nothing to copy into shared memory
+  sub.p.zc_elems = 0;
+  sub.p.Cpad = slice_len;
+  CUtensorMap ta, tb;
+  {   // operand A: [rows][Mp] seen as (reduction byte within the slice, row, 1, slice)
+    uint64_t dims[4] = {(uint64_t)slice_len, (uint64_t)rows, 1, (uint64_t)slices};
+    uint64_t strides[3] = {(uint64_t)Mp, (uint64_t)Mp * rows, (uint64_t)slice_len};
+    uint32_t box[4] = {(uint32_t)sub.p.BK, (uint32_t)sub.p.Wt, 1, 1};
+    uint32_t es[4] = {1, 1, 1, 1};
+    st = encode_map(ctx, &ta, At, 4, dims, strides, box, es, sub.p.swizzle64, false);
+    if (st != HQ_OK) return st;
+  }
+  st = encode_b(ctx, sub, Bt, Mp, &tb);
+  if (st != HQ_OK) return st;
+  const float* x_scale = reinterpret_cast<const float*>(reinterpret_cast<const char*>(xq) + offsetof(hq_range_state, scale));
+  st = launch_sub(ctx, s, sub, ta, tb, dyq, x_scale, nullptr, slabs, tmp, kOutAcc);
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, launch_wgrad_reduce(slabs, slices, rows, cols, colsum, rowsum, M, dyq, xq, GW, s));
+  ctx->launches += 1;
+  return HQ_OK;
 }
 
 __attribute__((visibility("default"))) hq_status hq_debug_accumulate(hq_ctx* ctx, void* stream, const hq_op_desc* op, int32_t* acc, hq_range_state* yq) {

@@ -422,6 +422,61 @@ __global__ void __launch_bounds__(256) transpose_rows_kernel(const int8_t* __res
     if (c < Ctot && r < Rp) out[(int64_t)c * Rp + r] = tile[tx][ty + 8 * j];
   }
 }
+// Weight gradient of a convolution: the second GEMM operand, transposed.  Bt[(r*S + s)*C + c][m] = x(n, hi, wi, c) for
+// output pixel m = (n, ho, wo) and hi = ho*stride_h - pad_h + r (wi alike); the input zero point where (hi, wi) lies
+// outside the image (real zero, which the zero-point correction then turns into no contribution); 0 for m >= M.
+// One block: 32 output pixels x 32 channels of one filter tap, transposed through shared memory.
+__global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict__ X, int8_t* __restrict__ Bt, const hq_range_state* __restrict__ xq,
+                                                        hq_conv_desc d, int Ho, int Wo, int64_t M, int64_t Mp) {
+  __shared__ int8_t tile[32][33];
+  const int64_t m0 = (int64_t)blockIdx.x * 32;
+  const int c0 = blockIdx.y * 32;
+  const int tap = blockIdx.z, r = tap / d.S, s = tap - r * d.S;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int8_t zx = (int8_t)xq->zero_point;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int64_t m = m0 + ty + 8 * j;
+    const int c = c0 + tx;
+    int8_t v = 0;
+    if (m < M && c < d.C) {
+      const int wo = (int)(m % Wo);
+      const int64_t t = m / Wo;
+      const int ho = (int)(t % Ho);
+      const int64_t n = t / Ho;
+      const int hi = ho * d.stride_h - d.pad_h + r, wi = wo * d.stride_w - d.pad_w + s;
+      v = (hi >= 0 && hi < d.H && wi >= 0 && wi < d.W) ? X[((n * d.H + hi) * d.W + wi) * d.C + c] : zx;
+    }
+    tile[ty + 8 * j][tx] = v;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = c0 + ty + 8 * j;
+    const int64_t m = m0 + tx;
+    if (c < d.C && m < Mp) Bt[((int64_t)tap * d.C + c) * Mp + m] = tile[tx][ty + 8 * j];
+  }
+}
+// The reduction was cut into slices that accumulated into slabs of their own: sum them (modulo 2^32, like everything
+// before), take out both zero points -- sum (a - za)(b - zb) = sum a b - za * sum b - zb * (sum a - za * M), with sum b
+// the row sums of the second operand (colsum) and sum a those of the first (rowsum) -- and convert:
+// G = fl(float(g) * fl(s_dy * s_x)).
+__global__ void wgrad_reduce_kernel(const int32_t* __restrict__ slabs, int nslabs, int rows, int cols, const int32_t* __restrict__ colsum,
+                                    const int32_t* __restrict__ rowsum, int M, const hq_range_state* __restrict__ dyq,
+                                    const hq_range_state* __restrict__ xq, float* __restrict__ G) {
+  const float sc = __fmul_rn(dyq->scale, xq->scale);
+  const int zdy = dyq->zero_point, zx = xq->zero_point;
+  const int64_t total = (int64_t)rows * cols;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int row = (int)(idx / cols), col = (int)(idx - (int64_t)row * cols);
+    uint32_t g = 0;
+    for (int sl = 0; sl < nslabs; ++sl) g += (uint32_t)slabs[(int64_t)sl * total + idx];
+    g -= (uint32_t)zdy * (uint32_t)colsum[col];
+    g -= (uint32_t)zx * ((uint32_t)rowsum[row] - (uint32_t)zdy * (uint32_t)M);
+    G[idx] = __fmul_rn(__int2float_rn((int)g), sc);
+  }
+}
+
 // sum_m (dy - z_dy)(x - z_x) = sum_m (dy - z_dy) x  -  z_x * sum_m (dy - z_dy): the second term, one number per output
 // row n, which the layer kernel's epilogue subtracts from every accumulator of that row.
 __global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int N, const hq_range_state* __restrict__ dyq,
@@ -940,6 +995,19 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
 cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, int Rp, int ones_row, cudaStream_t s) {
   dim3 grid((unsigned)((Rp + 31) / 32), (unsigned)((C + (ones_row ? 16 : 0) + 31) / 32));
   transpose_rows_kernel<<<grid, 256, 0, s>>>(in, out, R, C, Rp, ones_row);
+  return cudaGetLastError();
+}
+cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, cudaStream_t s) {
+  const int64_t M = (int64_t)d.N * Ho * Wo;
+  dim3 grid((unsigned)((Mp + 31) / 32), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
+  im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, M, Mp);
+  return cudaGetLastError();
+}
+cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
+                                const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s) {
+  const int64_t total = (int64_t)rows * cols;
+  const int blocks = (int)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 16));
+  wgrad_reduce_kernel<<<blocks, 256, 0, s>>>(slabs, nslabs, rows, cols, colsum, rowsum, M, dyq, xq, G);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,

@@ -493,11 +493,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                 if constexpr (kPairK) {   // never with resident weights
                   mbar_expect_tx_remote(a_full_lead(stage), a_stride);
                   tma_load_4d_pair(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full_lead(stage));
-                  tma_load_2d_pair(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0 + b_row_off, a_full_lead(stage));
+                  tma_load_2d_pair(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK + n0 * p.b_slice, col0 + b_row_off, a_full_lead(stage));
                 } else {
                   mbar_expect_tx(a_full(stage), a_stride);
                   tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
-                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK, col0, a_full(stage));
+                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK + n0 * p.b_slice, col0, a_full(stage));
                 }
               }
               if (++stage == p.stages_a) {
@@ -599,7 +599,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 #pragma unroll
     for (int k = 0; k < kCorrAhead; ++k) {
       const int i = et0 + k * kEpilogueWarps * 32;
-      corr_ahead[k] = (p.zc_in_smem && i < p.zc_elems) ? p.corr[i] : 0;
+      corr_ahead[k] = (p.zc_in_smem && p.corr != nullptr && i < p.zc_elems) ? p.corr[i] : 0;
     }
     const uint8_t rowcls_ahead = (p.cls_in_smem && et0 < p.TH) ? p.rowcls[et0] : (uint8_t)0;
     const uint8_t colcls_ahead = (p.cls_in_smem && et0 < p.TW) ? p.colcls[et0] : (uint8_t)0;
@@ -629,7 +629,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 #pragma unroll
         for (int k = 0; k < kCorrAhead; ++k)
           if (et + k * kEpiThreads < p.zc_elems) zc_s[et + k * kEpiThreads] = q.zx * corr_ahead[k];
-        for (int i = et + kCorrAhead * kEpiThreads; i < p.zc_elems; i += kEpiThreads) zc_s[i] = q.zx * p.corr[i];
+        if (p.corr != nullptr)
+          for (int i = et + kCorrAhead * kEpiThreads; i < p.zc_elems; i += kEpiThreads) zc_s[i] = q.zx * p.corr[i];
       }
       if (p.cls_in_smem) {   // TH, TW <= 512 = the number of epilogue threads
         if (et < p.TH) cls_s[et] = rowcls_ahead;

@@ -81,6 +81,8 @@ struct GemmParams {
   const uint8_t* colcls;              // [TW] or null
   int32_t cls_in_smem;                // both tables are non-null and fit the kernel's shared copy (TH, TW <= 512)
   const int32_t* bias;                // [Nout] or null
+  int32_t b_slice;                    // kModeTap, streamed weights: image n of the tile space reads operand B at reduction offset n * b_slice
+                                      // (the reduction of one GEMM cut into slices that run as "images"; 0 otherwise)
   const int32_t* row_term;            // [output rows] or null: subtracted from every accumulator of the row (flat layers only)
   float acc_bound;                    // upper bound of |accumulator| before the bias: reduction length x 255 x 128
   const hq_range_state* xq;
@@ -199,6 +201,9 @@ cudaError_t launch_prep_window_weights(const int8_t* W, int8_t* Wmat, int K, int
 cudaError_t launch_prep_patch_weights(const int8_t* W, int8_t* Wmat, int K, int R, int SC, int RP, int ld, cudaStream_t s);
 cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int Kp, cudaStream_t s);
 cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, int Rp, int ones_row, cudaStream_t s);
+cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, cudaStream_t s);
+cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
+                                const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
                                    cudaStream_t s);
 cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s);

@@ -25,7 +25,7 @@ OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_pair_launch_count",
            "hq_set_option",
            "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
-           "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate", "hq_linear_wgrad"]
+           "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate", "hq_linear_wgrad", "hq_conv_wgrad"]
 
 # numpy view of hq_range_state (48 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
@@ -75,6 +75,7 @@ def lib():
         L.hq_conv_fwd.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp, vp]
         L.hq_conv_bwd_data.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp, vp]
         L.hq_linear_wgrad.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.hq_conv_wgrad.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp]
         L.hq_range_update.argtypes = [vp, vp, vp, i32, C.c_float]
         L.hq_dynamic_quant.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp, vp]
         L.hq_debug_accumulate.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
@@ -162,6 +163,9 @@ class Context:
 
     def linear_wgrad(self, stream, M, N, K, dY, dyq, X, xq, GW):
         self._check(lib().hq_linear_wgrad(self.handle, _stream(stream), M, N, K, _ptr(dY), _ptr(dyq), _ptr(X), _ptr(xq), _ptr(GW)))
+
+    def conv_wgrad(self, stream, desc, dY, dyq, X, xq, GW):
+        self._check(lib().hq_conv_wgrad(self.handle, _stream(stream), C.byref(desc), _ptr(dY), _ptr(dyq), _ptr(X), _ptr(xq), _ptr(GW)))
 
     def conv_fwd(self, stream, desc, X, xq, pw: PreparedWeights, w_scale, Y, yq):
         self._check(lib().hq_conv_fwd(self.handle, _stream(stream), C.byref(desc), _ptr(X), _ptr(xq), pw.handle, _ptr(w_scale), _ptr(Y),

@@ -88,3 +88,40 @@ def test_linear_wgrad_bench_size_sampled_rows(ctx):
                            O.acc_scale(dy.scale, x.scale))
     assert np.array_equal(got[rows].view(np.uint32), want.view(np.uint32))
     assert np.isfinite(got).all()
+
+
+CONV_WGRAD_CASES = {
+    "3x3_c64_k64": dict(N=3, H=12, W=20, Cin=64, K=64, R=3, S=3, stride=1, pad=1),
+    "3x3_c16_k32_odd": dict(N=2, H=9, W=11, Cin=16, K=32, R=3, S=3, stride=1, pad=1),
+    "3x3_s2_c32_k48": dict(N=2, H=15, W=13, Cin=32, K=48, R=3, S=3, stride=2, pad=1),
+    "1x1_c144_k24": dict(N=2, H=10, W=13, Cin=144, K=24, R=1, S=1, stride=1, pad=0),
+    "1x1_s2_c64_k128": dict(N=2, H=14, W=14, Cin=64, K=128, R=1, S=1, stride=2, pad=0),
+    "5x5_c3_k20": dict(N=1, H=11, W=11, Cin=3, K=20, R=5, S=5, stride=1, pad=2),
+    "3x3_c128_k256_big": dict(N=8, H=28, W=28, Cin=128, K=256, R=3, S=3, stride=1, pad=1),
+    "7x7_s2_c3_k64_stem": dict(N=2, H=30, W=26, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
+    "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
+}
+
+
+@pytest.mark.parametrize("name", list(CONV_WGRAD_CASES))
+def test_conv_wgrad_matches_oracle(ctx, name):
+    c = CONV_WGRAD_CASES[name]
+    dev = torch.device("cuda", ctx.device)
+    r = synth.rng(303, len(name), c["H"], c["Cin"])
+    desc = hq.conv_desc(c["N"], c["H"], c["W"], c["Cin"], c["K"], c["R"], c["S"], stride=c["stride"], pad=c["pad"])
+    od = O.conv_desc(c["N"], c["H"], c["W"], c["Cin"], c["K"], c["R"], c["S"], stride=c["stride"], pad=c["pad"])
+    Ho, Wo = O.out_hw(od)
+    dy = synth.gradients(r, (c["N"], Ho, Wo, c["K"]))
+    x = synth.relu_activations(r, (c["N"], c["H"], c["W"], c["Cin"]))
+    dy_d, x_d = torch.from_numpy(dy.q).to(dev), torch.from_numpy(x.q).to(dev)
+    dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
+    xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
+    want = O.scale_to_real(O.conv_wgrad_acc(od, dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
+    for _ in range(2):
+        gw = torch.full((c["K"], c["R"], c["S"], c["Cin"]), float("nan"), dtype=torch.float32, device=dev)
+        ctx.conv_wgrad(None, desc, dy_d, dyq, x_d, xq, gw)
+        torch.cuda.synchronize(dev)
+        got = gw.cpu().numpy()
+        bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
+        assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
+    assert ctx.get_async_error() == 0
