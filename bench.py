@@ -485,7 +485,8 @@ WGRAD_SHAPE = dict(M=256, N=4096, K=4096)   # VGG16-style classifier layer 4096 
 
 
 def run_wgrad(args):
-    """One step = one hq_linear_wgrad call.  Algorithmic bytes: int8 dY and X in, binary32 G_W out."""
+    """One step = one hq_linear_wgrad call (wgrad) or one hq_conv_wgrad call on the 3x3 64 -> 64 layer of cfg2 (wgrad_conv).
+    Algorithmic bytes: int8 dY and X in, binary32 G_W out."""
     import torch
     from paper_2105_04246_b200 import hq
     if not torch.cuda.is_available():
@@ -494,22 +495,43 @@ def run_wgrad(args):
     torch.cuda.set_device(dev)
     ctx = hq.Context(0)
     peaks, peak_kind = load_peaks()
-    M, N, K = WGRAD_SHAPE["M"], WGRAD_SHAPE["N"], WGRAD_SHAPE["K"]
-    pool, Ksteps, W = 3, args.steps, max(3, args.warmup)
+    conv = args.workload == "wgrad_conv"
     g = synth.rng(4242)
-    dy, x = synth.gradients(g, (M, N)), synth.relu_activations(g, (M, K))
-    dys = [torch.from_numpy(np.roll(dy.q.reshape(-1), 7919 * j).reshape(M, N).copy()).to(dev) for j in range(pool)]
-    xs = [torch.from_numpy(np.roll(x.q.reshape(-1), 104729 * j).reshape(M, K).copy()).to(dev) for j in range(pool)]
-    gws = [torch.empty((N, K), dtype=torch.float32, device=dev) for _ in range(pool)]
+    if conv:
+        cs = wl.CFG2_CONV
+        desc = hq.conv_desc(cs.N, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad)
+        dy_shape, x_shape, gw_shape = (cs.N, cs.Ho, cs.Wo, cs.K), (cs.N, cs.H, cs.W, cs.C), (cs.K, cs.R, cs.S, cs.C)
+        M, N, K = cs.N * cs.Ho * cs.Wo, cs.K, cs.R * cs.S * cs.C
+        pool = 6
+        dy, x = synth.tiled(synth.gradients, g, dy_shape), synth.tiled(synth.relu_activations, g, x_shape)
+        label = f"wgrad_conv: weight gradient of conv3x3 {cs.C}->{cs.K} @{cs.H}x{cs.W}, batch {cs.N} -> FP32 G_W[{cs.K}x{cs.R}x{cs.S}x{cs.C}]"
+        path = "transposed filter windows, sliced reduction on the tensor-core layer kernel (int32 slabs), slab sum + conversion"
+    else:
+        M, N, K = WGRAD_SHAPE["M"], WGRAD_SHAPE["N"], WGRAD_SHAPE["K"]
+        dy_shape, x_shape, gw_shape = (M, N), (M, K), (N, K)
+        pool = 3
+        dy, x = synth.gradients(g, dy_shape), synth.relu_activations(g, x_shape)
+        label = f"wgrad: weight gradient of a linear layer, dY[{M}x{N}]^T X[{M}x{K}] -> FP32 G_W[{N}x{K}]"
+        path = "operand transposition, tensor-core layer kernel with binary32 epilogue"
+    Ksteps, W = args.steps, max(3, args.warmup)
+    dys = [torch.from_numpy(np.roll(dy.q.reshape(-1), 7919 * j).reshape(dy_shape).copy()).to(dev) for j in range(pool)]
+    xs = [torch.from_numpy(np.roll(x.q.reshape(-1), 104729 * j).reshape(x_shape).copy()).to(dev) for j in range(pool)]
+    gws = [torch.empty(gw_shape, dtype=torch.float32, device=dev) for _ in range(pool)]
+
+    def call(s_, j):
+        if conv:
+            ctx.conv_wgrad(s_, desc, dys[j], dyq, xs[j], xq, gws[j])
+        else:
+            ctx.linear_wgrad(s_, M, N, K, dys[j], dyq, xs[j], xq, gws[j])
     dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
     xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
     stream = torch.cuda.current_stream(dev)
     l0 = ctx.launch_count()
-    ctx.linear_wgrad(stream, M, N, K, dys[0], dyq, xs[0], xq, gws[0])      # also sizes the context's scratch before any capture
+    call(stream, 0)      # also sizes the context's scratch before any capture
     launches = ctx.launch_count() - l0
     torch.cuda.synchronize()
-    g_full = capture(torch, lambda s_, j: ctx.linear_wgrad(s_, M, N, K, dys[j], dyq, xs[j], xq, gws[j]), pool)
-    g_single = [capture(torch, lambda s_, _j, jj=j: ctx.linear_wgrad(s_, M, N, K, dys[jj], dyq, xs[jj], xq, gws[jj]), 1) for j in range(pool)]
+    g_full = capture(torch, call, pool)
+    g_single = [capture(torch, lambda s_, _j, jj=j: call(s_, jj), 1) for j in range(pool)]
     for _ in range(-(-W // pool)):
         g_full.replay()
     torch.cuda.synchronize()
@@ -521,7 +543,7 @@ def run_wgrad(args):
     sampler.join(timeout=2)
     # end to end with host buffers: both operands in from pinned memory, the gradient out to pinned memory
     h_dy, h_x = [t.cpu().pin_memory() for t in dys], [t.cpu().pin_memory() for t in xs]
-    h_gw = [torch.empty((N, K), dtype=torch.float32).pin_memory() for _ in range(pool)]
+    h_gw = [torch.empty(gw_shape, dtype=torch.float32).pin_memory() for _ in range(pool)]
     e2e_steps = min(Ksteps, 30)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -529,7 +551,7 @@ def run_wgrad(args):
         j = k % pool
         dys[j].copy_(h_dy[j], non_blocking=True)
         xs[j].copy_(h_x[j], non_blocking=True)
-        ctx.linear_wgrad(stream, M, N, K, dys[j], dyq, xs[j], xq, gws[j])
+        call(stream, j)
         h_gw[j].copy_(gws[j], non_blocking=True)
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
@@ -542,13 +564,12 @@ def run_wgrad(args):
         "metric": METRIC, "value": round(ops / (ms_step * 1e-3) / 1e12, 3), "unit": "TOPS", "n_gpus": 1, "steps": Ksteps, "warmup": W,
         "ms_per_step": round(ms_step, 6), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "impl": "hq",
-        "config": {"workload": f"wgrad: weight gradient of a linear layer, dY[{M}x{N}]^T X[{M}x{K}] -> FP32 G_W[{N}x{K}]",
-                   "path": "operand transposition, tensor-core layer kernel with binary32 epilogue",
+        "config": {"workload": label, "path": path,
                    "l2": f"operands and results rotate over a pool of {pool} buffer sets (> L2) inside CUDA graphs", "parallelism": "dp1"},
         "gpu_launches": int(launches * Ksteps), "launches_per_step": int(launches),
         "hbm_bytes_per_step": {"algorithmic": int(nbytes)},
         "roofline": {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                     "kernel": "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
+                     "kernel": "im2col_t_kernel + hq_gemm_kernel (int32 slabs) + wgrad_reduce_kernel" if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
                      "peak_source": peak_kind, "frac_of": f"of {peak_kind}"},
         "e2e": {"value": round(ops / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
                 "h2d_bytes_per_step": int(M * N + M * K), "d2h_bytes_per_step": int(4 * N * K), "steps": e2e_steps},
@@ -557,13 +578,20 @@ def run_wgrad(args):
     if not args.no_cpu_baseline:
         import oracle as O
         O.build()
-        Ns = N // 8                                   # bounded sample: one eighth of the output rows
         t0 = time.perf_counter()
-        acc = O.linear_wgrad_acc(dy.q[:, :Ns], dy.zero_point, x.q, x.zero_point)
+        if conv:                                      # bounded sample: the first 4 images of the batch
+            nb = 4
+            od = O.conv_desc(nb, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad)
+            acc = O.conv_wgrad_acc(od, dy.q[:nb], dy.zero_point, x.q[:nb], x.zero_point)
+            sample_ops, sample = ops * nb / cs.N, f"the first {nb} of {cs.N} images, one call"
+        else:
+            Ns = N // 8                               # bounded sample: one eighth of the output rows
+            acc = O.linear_wgrad_acc(dy.q[:, :Ns], dy.zero_point, x.q, x.zero_point)
+            sample_ops, sample = 2.0 * M * Ns * K, f"the first {Ns} of {N} output rows, one call"
         O.scale_to_real(acc, O.acc_scale(dy.scale, x.scale))
         dt = time.perf_counter() - t0
-        out["cpu_baseline"] = {"value": round(2.0 * M * Ns * K / dt / 1e12, 5), "unit": "TOPS", "cores": os.cpu_count() or 1, "kind": "oracle",
-                               "sample": f"the first {Ns} of {N} output rows, one call"}
+        out["cpu_baseline"] = {"value": round(sample_ops / dt / 1e12, 5), "unit": "TOPS", "cores": os.cpu_count() or 1, "kind": "oracle",
+                               "sample": sample}
     print(json.dumps(out))
 
 
@@ -614,7 +642,7 @@ def main():
     ap.add_argument("--steps", type=int, default=600)
     ap.add_argument("--warmup", type=int, default=24)
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad", "wgrad_conv"],
                     help="cfg1..cfg5: the five layer workloads; cfg4b: backward data through cfg4's block; wgrad: the weight gradient "
                          "of a linear layer (a later row of the scope)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -628,7 +656,7 @@ def main():
                     help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
                          "then --steps in-hindsight steps, then --steps dynamic steps")
     args = ap.parse_args()
-    if args.workload == "wgrad" and args.impl == "hq" and not args.profile:
+    if args.workload in ("wgrad", "wgrad_conv") and args.impl == "hq" and not args.profile:
         run_wgrad(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -1225,12 +1225,12 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   int32_t* colsum = rowsum + rows;
   hq_range_state* tmp = reinterpret_cast<hq_range_state*>(ctx->d_wgrad + a_bytes + b_bytes + slab_bytes + sum_bytes);
   if (Mp > INT32_MAX) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels");
+  // row sums of both operands (for the zero points), accumulated with integer atomics by the kernels that read the data anyway
+  HQ_CUDA(ctx, cudaMemsetAsync(rowsum, 0, ((size_t)rows + cols) * sizeof(int32_t), s));
   HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, rows, (int)Mp, 0, s));
-  HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, s));
-  const uint32_t one = 1u;
-  HQ_CUDA(ctx, launch_corr(At, rowsum, rows, 1, (int)Mp, 1, 1, &one, 1, &one, 1, rows, s));
-  HQ_CUDA(ctx, launch_corr(Bt, colsum, cols, 1, (int)Mp, 1, 1, &one, 1, &one, 1, cols, s));
-  ctx->launches += 4;
+  HQ_CUDA(ctx, launch_column_sums(dY, M, rows, rowsum, s));
+  HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, colsum, s));
+  ctx->launches += 3;
   SubSpec sp{};
   sp.n_img = slices; sp.TH = 1; sp.TW = rows; sp.in_mul_h = 1; sp.in_mul_w = 1;
   sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = rows; sp.Cin = slice_len; sp.Nout = cols;

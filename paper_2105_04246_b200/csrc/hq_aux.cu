@@ -425,36 +425,82 @@ __global__ void __launch_bounds__(256) transpose_rows_kernel(const int8_t* __res
 // Weight gradient of a convolution: the second GEMM operand, transposed.  Bt[(r*S + s)*C + c][m] = x(n, hi, wi, c) for
 // output pixel m = (n, ho, wo) and hi = ho*stride_h - pad_h + r (wi alike); the input zero point where (hi, wi) lies
 // outside the image (real zero, which the zero-point correction then turns into no contribution); 0 for m >= M.
-// One block: 32 output pixels x 32 channels of one filter tap, transposed through shared memory.
+// One block: 128 output pixels x 32 channels of one filter tap, transposed through shared memory (reads of four
+// channels per thread, writes of whole 128-byte runs); it also adds its part of the row sums of Bt (colsum, zeroed by
+// the caller), which the zero point of dY needs.
 __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict__ X, int8_t* __restrict__ Bt, const hq_range_state* __restrict__ xq,
-                                                        hq_conv_desc d, int Ho, int Wo, int64_t M, int64_t Mp) {
-  __shared__ int8_t tile[32][33];
-  const int64_t m0 = (int64_t)blockIdx.x * 32;
+                                                        hq_conv_desc d, int Ho, int Wo, int M, int Mp, int tiles_per_block,
+                                                        int32_t* __restrict__ colsum) {
+  __shared__ __align__(16) int8_t tile[32][128 + 16];
   const int c0 = blockIdx.y * 32;
+  int acc[4] = {0, 0, 0, 0};   // this lane's part of the row sums of its warp's four channel rows
   const int tap = blockIdx.z, r = tap / d.S, s = tap - r * d.S;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
   const int8_t zx = (int8_t)xq->zero_point;
+  const bool vec = (d.C & 3) == 0;   // four channels of a pixel are one aligned word
+  const int cg = threadIdx.x & 7, pl = threadIdx.x >> 3;   // channel group (4 channels) and pixel within a pass of 32
+  for (int mt = 0; mt < tiles_per_block; ++mt) {
+  const int m0 = (blockIdx.x * tiles_per_block + mt) * 128;
+  if (m0 >= Mp) break;   // the same for every thread of the block
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int64_t m = m0 + ty + 8 * j;
-    const int c = c0 + tx;
-    int8_t v = 0;
-    if (m < M && c < d.C) {
-      const int wo = (int)(m % Wo);
-      const int64_t t = m / Wo;
-      const int ho = (int)(t % Ho);
+  for (int pass = 0; pass < 4; ++pass) {
+    const int px = pass * 32 + pl;
+    const int m = m0 + px;
+    const int c = c0 + cg * 4;
+    int8_t v[4] = {0, 0, 0, 0};
+    if (m < M) {
+      const int wo = m % Wo;
+      const int t = m / Wo;
+      const int ho = t % Ho;
       const int64_t n = t / Ho;
       const int hi = ho * d.stride_h - d.pad_h + r, wi = wo * d.stride_w - d.pad_w + s;
-      v = (hi >= 0 && hi < d.H && wi >= 0 && wi < d.W) ? X[((n * d.H + hi) * d.W + wi) * d.C + c] : zx;
+      const bool inside = hi >= 0 && hi < d.H && wi >= 0 && wi < d.W;
+      const int8_t* src = X + ((n * d.H + hi) * d.W + wi) * d.C + c;
+      if (inside && vec && c + 3 < d.C) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(src);
+        v[0] = (int8_t)(w & 0xff); v[1] = (int8_t)((w >> 8) & 0xff); v[2] = (int8_t)((w >> 16) & 0xff); v[3] = (int8_t)(w >> 24);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (c + k < d.C) v[k] = inside ? src[k] : zx;
+      }
     }
-    tile[ty + 8 * j][tx] = v;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tile[cg * 4 + k][px] = v[k];
   }
   __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int c = c0 + ty + 8 * j;
-    const int64_t m = m0 + tx;
-    if (c < d.C && m < Mp) Bt[((int64_t)tap * d.C + c) * Mp + m] = tile[tx][ty + 8 * j];
+  for (int pass = 0; pass < 4; ++pass) {
+    const int cl = pass * 8 + warp;   // channel row of the tile
+    const int c = c0 + cl;
+    const uint32_t w = *reinterpret_cast<const uint32_t*>(&tile[cl][lane * 4]);
+    acc[pass] = __dp4a((int)w, 0x01010101, acc[pass]);
+    if (c < d.C) {
+      const int m = m0 + lane * 4;
+      if (m < Mp) *reinterpret_cast<uint32_t*>(Bt + ((int64_t)tap * d.C + c) * Mp + m) = w;   // Mp is a multiple of 128
+    }
+  }
+  __syncthreads();   // the tile is rewritten by the next round
+  }
+  const int lane2 = threadIdx.x & 31, warp2 = threadIdx.x >> 5;
+#pragma unroll
+  for (int pass = 0; pass < 4; ++pass) {
+    const int c = c0 + pass * 8 + warp2;
+    const int part = __reduce_add_sync(0xffffffffu, acc[pass]);
+    if (lane2 == 0 && c < d.C) atomicAdd(&colsum[tap * d.C + c], part);
+  }
+}
+// sums[k] += sum of dY[m][k] over this block's rows (the row sums of the first GEMM operand; zeroed by the caller)
+__global__ void __launch_bounds__(256) column_sums_kernel(const int8_t* __restrict__ dY, int64_t M, int K, int rows_per_block, int32_t* __restrict__ sums) {
+  const int64_t m_begin = (int64_t)blockIdx.x * rows_per_block;
+  const int64_t m_end = m_begin + rows_per_block < M ? m_begin + rows_per_block : M;
+  const int lanes = K >= (int)blockDim.x ? 1 : (int)blockDim.x / K;   // threads that share a column, on different rows
+  if ((int)threadIdx.x >= lanes * K && K < (int)blockDim.x) return;
+  const int rl = K >= (int)blockDim.x ? 0 : (int)threadIdx.x / K;
+  for (int k = K >= (int)blockDim.x ? (int)threadIdx.x : (int)threadIdx.x % K; k < K; k += blockDim.x) {
+    int sum = 0;
+    for (int64_t m = m_begin + rl; m < m_end; m += lanes) sum += dY[m * K + k];
+    atomicAdd(&sums[k], sum);
   }
 }
 // The reduction was cut into slices that accumulated into slabs of their own: sum them (modulo 2^32, like everything
@@ -997,10 +1043,17 @@ cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, i
   transpose_rows_kernel<<<grid, 256, 0, s>>>(in, out, R, C, Rp, ones_row);
   return cudaGetLastError();
 }
-cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, cudaStream_t s) {
+cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, int32_t* colsum,
+                            cudaStream_t s) {
   const int64_t M = (int64_t)d.N * Ho * Wo;
-  dim3 grid((unsigned)((Mp + 31) / 32), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
-  im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, M, Mp);
+  const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 4 : 1);
+  dim3 grid((unsigned)((tiles + tiles_per_block - 1) / tiles_per_block), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
+  im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, colsum);
+  return cudaGetLastError();
+}
+cudaError_t launch_column_sums(const int8_t* dY, int64_t M, int K, int32_t* sums, cudaStream_t s) {
+  const int rows_per_block = 1024;
+  column_sums_kernel<<<(unsigned)((M + rows_per_block - 1) / rows_per_block), 256, 0, s>>>(dY, M, K, rows_per_block, sums);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
