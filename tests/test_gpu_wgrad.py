@@ -125,3 +125,28 @@ def test_conv_wgrad_matches_oracle(ctx, name):
         bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
         assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
     assert ctx.get_async_error() == 0
+
+
+def test_conv_wgrad_bench_size_sampled_channels(ctx):
+    """The benchmark's layer (3x3, 64 -> 64, 56x56, batch 64: 200704 output pixels, 98 reduction slices): four output
+    channels compared in full with the oracle, which computes them from the matching channels of dY."""
+    from paper_2105_04246_b200 import workloads as wl
+    cs = wl.CFG2_CONV
+    dev = torch.device("cuda", ctx.device)
+    r = synth.rng(304)
+    dy = synth.tiled(synth.gradients, r, (cs.N, cs.Ho, cs.Wo, cs.K))
+    x = synth.tiled(synth.relu_activations, r, (cs.N, cs.H, cs.W, cs.C))
+    desc = hq.conv_desc(cs.N, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad)
+    dy_d, x_d = torch.from_numpy(dy.q).to(dev), torch.from_numpy(x.q).to(dev)
+    dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
+    xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
+    gw = torch.empty((cs.K, cs.R, cs.S, cs.C), dtype=torch.float32, device=dev)
+    ctx.conv_wgrad(None, desc, dy_d, dyq, x_d, xq, gw)
+    torch.cuda.synchronize(dev)
+    got = gw.cpu().numpy()
+    ks = [0, 17, 40, 63]
+    od = O.conv_desc(cs.N, cs.H, cs.W, cs.C, len(ks), cs.R, cs.S, cs.stride, cs.pad)
+    want = O.scale_to_real(O.conv_wgrad_acc(od, np.ascontiguousarray(dy.q[..., ks]), dy.zero_point, x.q, x.zero_point),
+                           O.acc_scale(dy.scale, x.scale))
+    assert np.array_equal(got[ks].view(np.uint32), want.view(np.uint32))
+    assert np.isfinite(got).all() and ctx.get_async_error() == 0
