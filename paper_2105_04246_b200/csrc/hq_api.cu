@@ -1229,7 +1229,7 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   HQ_CUDA(ctx, cudaMemsetAsync(rowsum, 0, ((size_t)rows + cols) * sizeof(int32_t), s));
   HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, rows, (int)Mp, 0, s));
   HQ_CUDA(ctx, launch_column_sums(dY, M, rows, rowsum, s));
-  HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, colsum, s));
+  HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, colsum, make_fastdiv(Wo), make_fastdiv(Ho), s));
   ctx->launches += 3;
   SubSpec sp{};
   sp.n_img = slices; sp.TH = 1; sp.TW = rows; sp.in_mul_h = 1; sp.in_mul_w = 1;

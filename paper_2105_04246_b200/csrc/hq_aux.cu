@@ -430,64 +430,84 @@ __global__ void __launch_bounds__(256) transpose_rows_kernel(const int8_t* __res
 // the caller), which the zero point of dY needs.
 __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict__ X, int8_t* __restrict__ Bt, const hq_range_state* __restrict__ xq,
                                                         hq_conv_desc d, int Ho, int Wo, int M, int Mp, int tiles_per_block,
-                                                        int32_t* __restrict__ colsum) {
-  __shared__ __align__(16) int8_t tile[32][128 + 16];
+                                                        FastDiv fd_wo, FastDiv fd_ho, int32_t* __restrict__ colsum) {
+  __shared__ __align__(16) uint32_t tile[32][33];   // [channel][4-pixel word]; 33: both phases hit 32 different banks
   const int c0 = blockIdx.y * 32;
   int acc[4] = {0, 0, 0, 0};   // this lane's part of the row sums of its warp's four channel rows
   const int tap = blockIdx.z, r = tap / d.S, s = tap - r * d.S;
-  const int8_t zx = (int8_t)xq->zero_point;
+  const uint32_t zx = (uint32_t)(uint8_t)(int8_t)xq->zero_point;
   const bool vec = (d.C & 3) == 0;   // four channels of a pixel are one aligned word
-  const int cg = threadIdx.x & 7, pl = threadIdx.x >> 3;   // channel group (4 channels) and pixel within a pass of 32
+  const int cg = threadIdx.x & 7, pg = threadIdx.x >> 3;   // channel group (4 channels) and pixel group (4 pixels)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int c = c0 + cg * 4;
   for (int mt = 0; mt < tiles_per_block; ++mt) {
-  const int m0 = (blockIdx.x * tiles_per_block + mt) * 128;
-  if (m0 >= Mp) break;   // the same for every thread of the block
+    const int m0 = (blockIdx.x * tiles_per_block + mt) * 128;
+    if (m0 >= Mp) break;   // the same for every thread of the block
+    // read: four consecutive output pixels x four channels, one word per pixel
+    uint32_t w[4];
+    // output pixel of the first of the four, then stepped (divisions by multiplication: the divisors are launch constants)
+    int wo, ho, n;
+    {
+      const int m = m0 + pg * 4;
+      const int t = fdiv(m, fd_wo);
+      wo = m - t * Wo;
+      n = fdiv(t, fd_ho);
+      ho = t - n * Ho;
+    }
 #pragma unroll
-  for (int pass = 0; pass < 4; ++pass) {
-    const int px = pass * 32 + pl;
-    const int m = m0 + px;
-    const int c = c0 + cg * 4;
-    int8_t v[4] = {0, 0, 0, 0};
-    if (m < M) {
-      const int wo = m % Wo;
-      const int t = m / Wo;
-      const int ho = t % Ho;
-      const int64_t n = t / Ho;
-      const int hi = ho * d.stride_h - d.pad_h + r, wi = wo * d.stride_w - d.pad_w + s;
-      const bool inside = hi >= 0 && hi < d.H && wi >= 0 && wi < d.W;
-      const int8_t* src = X + ((n * d.H + hi) * d.W + wi) * d.C + c;
-      if (inside && vec && c + 3 < d.C) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(src);
-        v[0] = (int8_t)(w & 0xff); v[1] = (int8_t)((w >> 8) & 0xff); v[2] = (int8_t)((w >> 16) & 0xff); v[3] = (int8_t)(w >> 24);
-      } else {
+    for (int j = 0; j < 4; ++j) {
+      const int m = m0 + pg * 4 + j;
+      uint32_t v = 0;
+      if (m < M && c < d.C) {
+        const int hi = ho * d.stride_h - d.pad_h + r, wi = wo * d.stride_w - d.pad_w + s;
+        const bool inside = hi >= 0 && hi < d.H && wi >= 0 && wi < d.W;
+        if (inside) {
+          const int8_t* src = X + (((int64_t)n * d.H + hi) * d.W + wi) * d.C + c;
+          if (vec) {
+            v = *reinterpret_cast<const uint32_t*>(src);
+          } else {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (c + k < d.C) v[k] = inside ? src[k] : zx;
+            for (int k = 0; k < 4; ++k)
+              if (c + k < d.C) v |= (uint32_t)(uint8_t)src[k] << (8 * k);
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (c + k < d.C) v |= zx << (8 * k);
+        }
+      }
+      w[j] = v;
+      if (++wo == Wo) {
+        wo = 0;
+        if (++ho == Ho) {
+          ho = 0;
+          ++n;
+        }
       }
     }
+    // 4x4 byte transposition in registers: t[k] = channel k of pixels 0..3
+    const uint32_t a0 = __byte_perm(w[0], w[1], 0x5140), a1 = __byte_perm(w[0], w[1], 0x7362);   // ch0|ch1 and ch2|ch3 of pixels 0,1
+    const uint32_t b0 = __byte_perm(w[2], w[3], 0x5140), b1 = __byte_perm(w[2], w[3], 0x7362);   // the same of pixels 2,3
+    tile[cg * 4 + 0][pg] = __byte_perm(a0, b0, 0x5410);
+    tile[cg * 4 + 1][pg] = __byte_perm(a0, b0, 0x7632);
+    tile[cg * 4 + 2][pg] = __byte_perm(a1, b1, 0x5410);
+    tile[cg * 4 + 3][pg] = __byte_perm(a1, b1, 0x7632);
+    __syncthreads();
 #pragma unroll
-    for (int k = 0; k < 4; ++k) tile[cg * 4 + k][px] = v[k];
-  }
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int pass = 0; pass < 4; ++pass) {
-    const int cl = pass * 8 + warp;   // channel row of the tile
-    const int c = c0 + cl;
-    const uint32_t w = *reinterpret_cast<const uint32_t*>(&tile[cl][lane * 4]);
-    acc[pass] = __dp4a((int)w, 0x01010101, acc[pass]);
-    if (c < d.C) {
+    for (int pass = 0; pass < 4; ++pass) {
+      const int cl = pass * 8 + warp;   // channel row of the tile
+      const uint32_t v = tile[cl][lane];
+      acc[pass] = __dp4a((int)v, 0x01010101, acc[pass]);
       const int m = m0 + lane * 4;
-      if (m < Mp) *reinterpret_cast<uint32_t*>(Bt + ((int64_t)tap * d.C + c) * Mp + m) = w;   // Mp is a multiple of 128
+      if (c0 + cl < d.C && m < Mp) *reinterpret_cast<uint32_t*>(Bt + ((int64_t)tap * d.C + c0 + cl) * Mp + m) = v;   // Mp is a multiple of 128
     }
+    __syncthreads();   // the tile is rewritten by the next round
   }
-  __syncthreads();   // the tile is rewritten by the next round
-  }
-  const int lane2 = threadIdx.x & 31, warp2 = threadIdx.x >> 5;
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
-    const int c = c0 + pass * 8 + warp2;
+    const int cc = c0 + pass * 8 + warp;
     const int part = __reduce_add_sync(0xffffffffu, acc[pass]);
-    if (lane2 == 0 && c < d.C) atomicAdd(&colsum[tap * d.C + c], part);
+    if (lane == 0 && cc < d.C) atomicAdd(&colsum[tap * d.C + cc], part);
   }
 }
 // sums[k] += sum of dY[m][k] over this block's rows (the row sums of the first GEMM operand; zeroed by the caller)
@@ -1044,11 +1064,11 @@ cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, i
   return cudaGetLastError();
 }
 cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, int32_t* colsum,
-                            cudaStream_t s) {
+                            FastDiv fd_wo, FastDiv fd_ho, cudaStream_t s) {
   const int64_t M = (int64_t)d.N * Ho * Wo;
   const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 4 : 1);
   dim3 grid((unsigned)((tiles + tiles_per_block - 1) / tiles_per_block), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
-  im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, colsum);
+  im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, fd_wo, fd_ho, colsum);
   return cudaGetLastError();
 }
 cudaError_t launch_column_sums(const int8_t* dY, int64_t M, int K, int32_t* sums, cudaStream_t s) {
