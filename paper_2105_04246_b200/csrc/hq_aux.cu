@@ -554,6 +554,37 @@ __global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int
   terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
 }
 
+// the same for K a multiple of 16 (at most 4096): 16-byte loads, one thread per 16 columns of a row, sums gathered in
+// shared memory before they go out
+__global__ void __launch_bounds__(256) column_sums16_kernel(const int8_t* __restrict__ dY, int64_t M, int K, int rows_per_block,
+                                                             int32_t* __restrict__ sums) {
+  extern __shared__ int32_t ssum[];
+  for (int k = threadIdx.x; k < K; k += blockDim.x) ssum[k] = 0;
+  __syncthreads();
+  const int groups = K / 16;                                   // threads per row (at most 256)
+  const int rows_per_pass = (int)blockDim.x / groups;
+  const int64_t m_begin = (int64_t)blockIdx.x * rows_per_block;
+  const int64_t m_end = m_begin + rows_per_block < M ? m_begin + rows_per_block : M;
+  const int g = (int)threadIdx.x % groups, rl = (int)threadIdx.x / groups;
+  if (rl < rows_per_pass) {
+    int acc[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = 0;
+    for (int64_t m = m_begin + rl; m < m_end; m += rows_per_pass) {
+      const uint4 v = *reinterpret_cast<const uint4*>(dY + m * K + g * 16);
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[4 * q + b] = __dp4a((int)w[q], 1 << (8 * b), acc[4 * q + b]);
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) atomicAdd(&ssum[g * 16 + i], acc[i]);
+  }
+  __syncthreads();
+  for (int k = threadIdx.x; k < K; k += blockDim.x) atomicAdd(&sums[k], ssum[k]);
+}
+
 // ---- depthwise convolution on CUDA cores --------------------------------------------------------
 // One thread: one output pixel x 16 consecutive channels.  Same epilogue as the tensor-core kernel.
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xffu); }
@@ -1073,7 +1104,11 @@ cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* x
 }
 cudaError_t launch_column_sums(const int8_t* dY, int64_t M, int K, int32_t* sums, cudaStream_t s) {
   const int rows_per_block = 1024;
-  column_sums_kernel<<<(unsigned)((M + rows_per_block - 1) / rows_per_block), 256, 0, s>>>(dY, M, K, rows_per_block, sums);
+  const unsigned blocks = (unsigned)((M + rows_per_block - 1) / rows_per_block);
+  if (K % 16 == 0 && K <= 4096 && (reinterpret_cast<uintptr_t>(dY) & 15u) == 0)
+    column_sums16_kernel<<<blocks, 256, (size_t)K * sizeof(int32_t), s>>>(dY, M, K, rows_per_block, sums);
+  else
+    column_sums_kernel<<<blocks, 256, 0, s>>>(dY, M, K, rows_per_block, sums);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
