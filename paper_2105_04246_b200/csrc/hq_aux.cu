@@ -431,7 +431,9 @@ __global__ void __launch_bounds__(256) transpose_rows_kernel(const int8_t* __res
 __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict__ X, int8_t* __restrict__ Bt, const hq_range_state* __restrict__ xq,
                                                         hq_conv_desc d, int Ho, int Wo, int M, int Mp, int tiles_per_block,
                                                         FastDiv fd_wo, FastDiv fd_ho, int32_t* __restrict__ colsum) {
-  __shared__ __align__(16) uint32_t tile[32][33];   // [channel][4-pixel word]; 33: both phases hit 32 different banks
+  // [round parity][channel][4-pixel word]; 33: both phases hit 32 different banks.  Two tiles: a round writes the one the
+  // round before last read, which every thread has left once it reaches this round's barrier -- one barrier per round.
+  __shared__ __align__(16) uint32_t tiles[2][32][33];
   const int c0 = blockIdx.y * 32;
   int acc[4] = {0, 0, 0, 0};   // this lane's part of the row sums of its warp's four channel rows
   const int tap = blockIdx.z, r = tap / d.S, s = tap - r * d.S;
@@ -443,6 +445,7 @@ __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict_
   for (int mt = 0; mt < tiles_per_block; ++mt) {
     const int m0 = (blockIdx.x * tiles_per_block + mt) * 128;
     if (m0 >= Mp) break;   // the same for every thread of the block
+    uint32_t (*tile)[33] = tiles[mt & 1];
     // read: four consecutive output pixels x four channels, one word per pixel
     uint32_t w[4];
     // output pixel of the first of the four, then stepped (divisions by multiplication: the divisors are launch constants)
@@ -501,7 +504,6 @@ __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict_
       const int m = m0 + lane * 4;
       if (c0 + cl < d.C && m < Mp) *reinterpret_cast<uint32_t*>(Bt + ((int64_t)tap * d.C + c0 + cl) * Mp + m) = v;   // Mp is a multiple of 128
     }
-    __syncthreads();   // the tile is rewritten by the next round
   }
 #pragma unroll
   for (int pass = 0; pass < 4; ++pass) {
@@ -1097,7 +1099,7 @@ cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, i
 cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, int32_t* colsum,
                             FastDiv fd_wo, FastDiv fd_ho, cudaStream_t s) {
   const int64_t M = (int64_t)d.N * Ho * Wo;
-  const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 4 : 1);
+  const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 8 : 1);
   dim3 grid((unsigned)((tiles + tiles_per_block - 1) / tiles_per_block), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
   im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, fd_wo, fd_ho, colsum);
   return cudaGetLastError();
