@@ -1227,10 +1227,13 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   if (Mp > INT32_MAX) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels");
   // row sums of both operands (for the zero points), accumulated with integer atomics by the kernels that read the data anyway
   HQ_CUDA(ctx, cudaMemsetAsync(rowsum, 0, ((size_t)rows + cols) * sizeof(int32_t), s));
-  HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, rows, (int)Mp, 0, s));
-  HQ_CUDA(ctx, launch_column_sums(dY, M, rows, rowsum, s));
+  {   // dY^T and its row sums: the same kernel, dY taken as the input of a 1x1 stride-1 layer (no padding, so no zero point is used)
+    hq_conv_desc t{};
+    t.N = d.N; t.H = Ho; t.W = Wo; t.C = d.K; t.K = d.K; t.R = 1; t.S = 1; t.stride_h = 1; t.stride_w = 1; t.pad_h = 0; t.pad_w = 0; t.groups = 1;
+    HQ_CUDA(ctx, launch_im2col_t(dY, At, dyq, t, Ho, Wo, Mp, rowsum, make_fastdiv(Wo), make_fastdiv(Ho), s));
+  }
   HQ_CUDA(ctx, launch_im2col_t(X, Bt, xq, d, Ho, Wo, Mp, colsum, make_fastdiv(Wo), make_fastdiv(Ho), s));
-  ctx->launches += 3;
+  ctx->launches += 2;
   SubSpec sp{};
   sp.n_img = slices; sp.TH = 1; sp.TW = rows; sp.in_mul_h = 1; sp.in_mul_w = 1;
   sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = rows; sp.Cin = slice_len; sp.Nout = cols;

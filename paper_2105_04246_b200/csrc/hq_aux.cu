@@ -512,19 +512,6 @@ __global__ void __launch_bounds__(256) im2col_t_kernel(const int8_t* __restrict_
     if (lane == 0 && cc < d.C) atomicAdd(&colsum[tap * d.C + cc], part);
   }
 }
-// sums[k] += sum of dY[m][k] over this block's rows (the row sums of the first GEMM operand; zeroed by the caller)
-__global__ void __launch_bounds__(256) column_sums_kernel(const int8_t* __restrict__ dY, int64_t M, int K, int rows_per_block, int32_t* __restrict__ sums) {
-  const int64_t m_begin = (int64_t)blockIdx.x * rows_per_block;
-  const int64_t m_end = m_begin + rows_per_block < M ? m_begin + rows_per_block : M;
-  const int lanes = K >= (int)blockDim.x ? 1 : (int)blockDim.x / K;   // threads that share a column, on different rows
-  if ((int)threadIdx.x >= lanes * K && K < (int)blockDim.x) return;
-  const int rl = K >= (int)blockDim.x ? 0 : (int)threadIdx.x / K;
-  for (int k = K >= (int)blockDim.x ? (int)threadIdx.x : (int)threadIdx.x % K; k < K; k += blockDim.x) {
-    int sum = 0;
-    for (int64_t m = m_begin + rl; m < m_end; m += lanes) sum += dY[m * K + k];
-    atomicAdd(&sums[k], sum);
-  }
-}
 // The reduction was cut into slices that accumulated into slabs of their own: sum them (modulo 2^32, like everything
 // before), take out both zero points -- sum (a - za)(b - zb) = sum a b - za * sum b - zb * (sum a - za * M), with sum b
 // the row sums of the second operand (colsum) and sum a those of the first (rowsum) -- and convert:
@@ -554,37 +541,6 @@ __global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int
   int sum = 0;
   for (int m = 0; m < M; ++m) sum += dY[(int64_t)m * N + n];
   terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
-}
-
-// the same for K a multiple of 16 (at most 4096): 16-byte loads, one thread per 16 columns of a row, sums gathered in
-// shared memory before they go out
-__global__ void __launch_bounds__(256) column_sums16_kernel(const int8_t* __restrict__ dY, int64_t M, int K, int rows_per_block,
-                                                             int32_t* __restrict__ sums) {
-  extern __shared__ int32_t ssum[];
-  for (int k = threadIdx.x; k < K; k += blockDim.x) ssum[k] = 0;
-  __syncthreads();
-  const int groups = K / 16;                                   // threads per row (at most 256)
-  const int rows_per_pass = (int)blockDim.x / groups;
-  const int64_t m_begin = (int64_t)blockIdx.x * rows_per_block;
-  const int64_t m_end = m_begin + rows_per_block < M ? m_begin + rows_per_block : M;
-  const int g = (int)threadIdx.x % groups, rl = (int)threadIdx.x / groups;
-  if (rl < rows_per_pass) {
-    int acc[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = 0;
-    for (int64_t m = m_begin + rl; m < m_end; m += rows_per_pass) {
-      const uint4 v = *reinterpret_cast<const uint4*>(dY + m * K + g * 16);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[4 * q + b] = __dp4a((int)w[q], 1 << (8 * b), acc[4 * q + b]);
-    }
-#pragma unroll
-    for (int i = 0; i < 16; ++i) atomicAdd(&ssum[g * 16 + i], acc[i]);
-  }
-  __syncthreads();
-  for (int k = threadIdx.x; k < K; k += blockDim.x) atomicAdd(&sums[k], ssum[k]);
 }
 
 // ---- depthwise convolution on CUDA cores --------------------------------------------------------
@@ -1102,15 +1058,6 @@ cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* x
   const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 8 : 1);
   dim3 grid((unsigned)((tiles + tiles_per_block - 1) / tiles_per_block), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
   im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, fd_wo, fd_ho, colsum);
-  return cudaGetLastError();
-}
-cudaError_t launch_column_sums(const int8_t* dY, int64_t M, int K, int32_t* sums, cudaStream_t s) {
-  const int rows_per_block = 1024;
-  const unsigned blocks = (unsigned)((M + rows_per_block - 1) / rows_per_block);
-  if (K % 16 == 0 && K <= 4096 && (reinterpret_cast<uintptr_t>(dY) & 15u) == 0)
-    column_sums16_kernel<<<blocks, 256, (size_t)K * sizeof(int32_t), s>>>(dY, M, K, rows_per_block, sums);
-  else
-    column_sums_kernel<<<blocks, 256, 0, s>>>(dY, M, K, rows_per_block, sums);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
