@@ -2,11 +2,12 @@
 // operands staged by TMA, with the requantization + min/max epilogue of the in-hindsight
 // scheme (arxiv 2105.04246, Sec. 3.1, Sec. 3.2 "static quantization", Sec. 4 steps 1 and 2).
 //
-// One persistent CTA per SM walks over 128-row output tiles.  Roles: warp 0 feeds operand A
-// (kModeTap: one box of A and one of B per filter tap and channel chunk; kModeHalo: the padded
-// input rows of the tile, once), warp 2 streams the weights in kModeHalo, warp 1 issues the MMAs,
-// eight epilogue warps drain a double-buffered TMEM accumulator, so the epilogue of tile i
-// overlaps the MAC loop of tile i+1.  Every wait is bounded (see mbar_wait).
+// One persistent CTA per SM walks over 128-row output tiles (or a pair of CTAs on neighbouring SMs over 256-row tiles:
+// the kPairK instantiation).  Roles: warp 0 feeds operand A (kModeTap: one box of A and one of B per filter tap and
+// channel chunk; kModeHalo: the padded input rows of the tile, once), warp 2 feeds the weights (streamed in kModeHalo,
+// or once when they stay resident), warp 1 -- and warps 3 and 2 where the planner says so -- issue the MMAs, sixteen
+// epilogue warps in 1, 2 or 4 groups drain 2 to 8 accumulator buffers in TMEM, so the epilogue of a tile overlaps
+// the MAC loops of the following ones.  Every wait is bounded (see mbar_wait).
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
