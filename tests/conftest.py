@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _native_code_is_built():
+    """The C-ABI library and the oracle are compiled in-tree once per run if their sources are newer than the binaries
+    (a no-op otherwise).  There is no other implementation to fall back to: a failed build fails the run."""
+    from paper_2105_04246_b200 import build as hq_build
+    import oracle
+    hq_build.build()
+    oracle.build()
