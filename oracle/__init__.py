@@ -127,12 +127,12 @@ def linear_wgrad_acc(dY, zdy, X, zx) -> np.ndarray:
 
 
 def conv_wgrad_acc(d: Conv, dY, zdy, X, zx) -> np.ndarray:
-    """int32 g[k,r,s,c] = sum over output pixels of (dy - z_dy) * (x - z_x), padded taps skipped (dense layers)."""
-    assert d.groups == 1
+    """int32 g[k,r,s,c] = sum over output pixels of (dy - z_dy) * (x - z_x), padded taps skipped; depthwise: g[c,r,s]."""
+    assert d.groups == 1 or (d.groups == d.C and d.K == d.C)
     dY, X = _i8(dY), _i8(X)
     Ho, Wo = out_hw(d)
     assert dY.shape == (d.N, Ho, Wo, d.K) and X.shape == (d.N, d.H, d.W, d.C)
-    g = np.empty((d.K, d.R, d.S, d.C), np.int32)
+    g = np.empty((d.K, d.R, d.S, d.C) if d.groups == 1 else (d.C, d.R, d.S), np.int32)
     ovf = lib().hqo_conv_wgrad_acc(C.byref(d), _p(dY, C.c_int8), int(zdy), _p(X, C.c_int8), int(zx), _p(g, C.c_int32))
     assert ovf == 0, "int32 accumulator overflow"
     return g

@@ -148,10 +148,32 @@ int hqo_linear_wgrad_acc(int M, int N, int K, const int8_t* dY, int zdy, const i
 // weight gradient of a convolution (Sec. 3.1, backward pass), W layout [K][R][S][C]:
 //   g(k,r,s,c) = sum over n,ho,wo of (dy(n,ho,wo,k) - z_dy) * (x(n,hi,wi,c) - z_x),  hi = ho*stride_h - pad_h + r (wi alike),
 //   over those output pixels whose (hi,wi) lies inside the image: padding is zero in the real domain (R-8), so a padded
-//   tap contributes nothing.  G_W = fl(float(g) * fl(s_dy * s_x)).  Dense layers only (groups == 1).
+//   tap contributes nothing.  G_W = fl(float(g) * fl(s_dy * s_x)).  Dense layers, or depthwise (groups == C == K).
 int hqo_conv_wgrad_acc(const hqo_conv* d, const int8_t* dY, int zdy, const int8_t* X, int zx, int32_t* g) {
   const int Ho = hqo_out_h(d), Wo = hqo_out_w(d);
   int ovf = 0;
+  if (d->groups != 1) {   // depthwise (K == C), W layout [C][R][S]: the same sum with k == c and no sum over channels
+#pragma omp parallel for collapse(2) reduction(| : ovf)
+    for (int c = 0; c < d->C; ++c)
+      for (int r = 0; r < d->R; ++r)
+        for (int s = 0; s < d->S; ++s) {
+          int64_t a = 0;
+          for (int n = 0; n < d->N; ++n)
+            for (int ho = 0; ho < Ho; ++ho) {
+              const int hi = ho * d->stride_h - d->pad_h + r;
+              if (hi < 0 || hi >= d->H) continue;
+              for (int wo = 0; wo < Wo; ++wo) {
+                const int wi = wo * d->stride_w - d->pad_w + s;
+                if (wi < 0 || wi >= d->W) continue;
+                a += (int64_t)((int)dY[(((int64_t)n * Ho + ho) * Wo + wo) * d->K + c] - zdy) *
+                     ((int)X[(((int64_t)n * d->H + hi) * d->W + wi) * d->C + c] - zx);
+              }
+            }
+          if (a > INT32_MAX || a < INT32_MIN) ovf |= 1;
+          g[((int64_t)c * d->R + r) * d->S + s] = (int32_t)a;
+        }
+    return ovf;
+  }
 #pragma omp parallel for collapse(2) reduction(| : ovf)
   for (int k = 0; k < d->K; ++k)
     for (int r = 0; r < d->R; ++r)

@@ -103,3 +103,25 @@ def test_conv_wgrad_against_library_convolution():
         gw = torch.nn.grad.conv2d_weight(xt, (c["K"], c["C"], c["R"], c["S"]), gt, stride=c["stride"], padding=c["pad"])
         want = gw.numpy().transpose(0, 2, 3, 1).round().astype(np.int64)
         assert np.array_equal(O.conv_wgrad_acc(d, dy, zdy, x, zx).astype(np.int64), want), c
+
+
+def test_depthwise_wgrad_trace_identity_and_library():
+    """Depthwise weight gradient: adjoint of the depthwise forward convolution with respect to the filter, and torch's
+    grouped conv2d weight gradient in float64."""
+    import torch
+    r = np.random.default_rng(24)
+    for c in [dict(N=2, H=6, W=7, C=4, R=3, S=3, stride=1, pad=1), dict(N=1, H=9, W=8, C=3, R=3, S=3, stride=2, pad=1),
+              dict(N=2, H=7, W=7, C=2, R=5, S=5, stride=1, pad=2)]:
+        d = O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["C"], c["R"], c["S"], stride=c["stride"], pad=c["pad"], groups=c["C"])
+        Ho, Wo = O.out_hw(d)
+        dy, x = _rand(r, (c["N"], Ho, Wo, c["C"])), _rand(r, (c["N"], c["H"], c["W"], c["C"]))
+        w = _rand(r, (c["C"], c["R"], c["S"]))
+        zdy, zx = 6, -9
+        g = O.conv_wgrad_acc(d, dy, zdy, x, zx)
+        assert g.shape == (c["C"], c["R"], c["S"])
+        y = O.conv_fwd_acc(d, x, zx, w).astype(np.int64)
+        assert int(((dy.astype(np.int64) - zdy) * y).sum()) == int((g.astype(np.int64) * w.astype(np.int64)).sum()), c
+        xt = torch.from_numpy((x.astype(np.float64) - zx).transpose(0, 3, 1, 2).copy())
+        gt = torch.from_numpy((dy.astype(np.float64) - zdy).transpose(0, 3, 1, 2).copy())
+        gw = torch.nn.grad.conv2d_weight(xt, (c["C"], 1, c["R"], c["S"]), gt, stride=c["stride"], padding=c["pad"], groups=c["C"])
+        assert np.array_equal(g.astype(np.int64), gw.numpy()[:, 0].round().astype(np.int64)), c
