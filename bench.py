@@ -495,17 +495,21 @@ def run_wgrad(args):
     torch.cuda.set_device(dev)
     ctx = hq.Context(0)
     peaks, peak_kind = load_peaks()
-    conv = args.workload == "wgrad_conv"
+    conv = args.workload in ("wgrad_conv", "wgrad_dw")
     g = synth.rng(4242)
     if conv:
-        cs = wl.CFG2_CONV
-        desc = hq.conv_desc(cs.N, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad)
-        dy_shape, x_shape, gw_shape = (cs.N, cs.Ho, cs.Wo, cs.K), (cs.N, cs.H, cs.W, cs.C), (cs.K, cs.R, cs.S, cs.C)
-        M, N, K = cs.N * cs.Ho * cs.Wo, cs.K, cs.R * cs.S * cs.C
-        pool = 6
+        cs = wl.CFG2_CONV if args.workload == "wgrad_conv" else wl.CFG4_DW
+        desc = hq.conv_desc(cs.N, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad, cs.groups)
+        dy_shape, x_shape = (cs.N, cs.Ho, cs.Wo, cs.K), (cs.N, cs.H, cs.W, cs.C)
+        gw_shape = (cs.K, cs.R, cs.S) if cs.depthwise else (cs.K, cs.R, cs.S, cs.C)
+        # (M, N, K) of the equivalent matrix product; depthwise: one output row, R*S*C independent sums over the pixels
+        M, N, K = cs.N * cs.Ho * cs.Wo, (1 if cs.depthwise else cs.K), cs.R * cs.S * cs.C
+        pool = 6 if not cs.depthwise else 2
         dy, x = synth.tiled(synth.gradients, g, dy_shape), synth.tiled(synth.relu_activations, g, x_shape)
-        label = f"wgrad_conv: weight gradient of conv3x3 {cs.C}->{cs.K} @{cs.H}x{cs.W}, batch {cs.N} -> FP32 G_W[{cs.K}x{cs.R}x{cs.S}x{cs.C}]"
-        path = "transposed filter windows, sliced reduction on the tensor-core layer kernel (int32 slabs), slab sum + conversion"
+        label = (f"{args.workload}: weight gradient of {'depthwise ' if cs.depthwise else ''}conv3x3 {cs.C}->{cs.K} @{cs.H}x{cs.W}, batch {cs.N} "
+                 f"-> FP32 G_W{list(gw_shape)}")
+        path = ("CUDA-core kernel, integer atomics, conversion" if cs.depthwise else
+                "transposed filter windows, sliced reduction on the tensor-core layer kernel (int32 slabs), slab sum + conversion")
     else:
         M, N, K = WGRAD_SHAPE["M"], WGRAD_SHAPE["N"], WGRAD_SHAPE["K"]
         dy_shape, x_shape, gw_shape = (M, N), (M, K), (N, K)
@@ -557,7 +561,7 @@ def run_wgrad(args):
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     assert ctx.get_async_error() == 0
     ops = 2.0 * M * N * K
-    nbytes = M * N + M * K + 4 * N * K
+    nbytes = int(np.prod(dy_shape)) + int(np.prod(x_shape)) + 4 * int(np.prod(gw_shape))   # int8 dY and X in, binary32 G_W out
     ms_step = ms_total / Ksteps
     ach = nbytes / (ms_step * 1e-3) / 1e9
     out = {
@@ -569,7 +573,7 @@ def run_wgrad(args):
         "gpu_launches": int(launches * Ksteps), "launches_per_step": int(launches),
         "hbm_bytes_per_step": {"algorithmic": int(nbytes)},
         "roofline": {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                     "kernel": "im2col_t_kernel + hq_gemm_kernel (int32 slabs) + wgrad_reduce_kernel" if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
+                     "kernel": ("dw_wgrad_kernel" if cs.depthwise else "im2col_t_kernel + hq_gemm_kernel (int32 slabs) + wgrad_reduce_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
                      "peak_source": peak_kind, "frac_of": f"of {peak_kind}"},
         "e2e": {"value": round(ops / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
                 "h2d_bytes_per_step": int(M * N + M * K), "d2h_bytes_per_step": int(4 * N * K), "steps": e2e_steps},
@@ -581,7 +585,7 @@ def run_wgrad(args):
         t0 = time.perf_counter()
         if conv:                                      # bounded sample: the first 4 images of the batch
             nb = 4
-            od = O.conv_desc(nb, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad)
+            od = O.conv_desc(nb, cs.H, cs.W, cs.C, cs.K, cs.R, cs.S, cs.stride, cs.pad, cs.groups)
             acc = O.conv_wgrad_acc(od, dy.q[:nb], dy.zero_point, x.q[:nb], x.zero_point)
             sample_ops, sample = ops * nb / cs.N, f"the first {nb} of {cs.N} images, one call"
         else:
@@ -642,7 +646,7 @@ def main():
     ap.add_argument("--steps", type=int, default=600)
     ap.add_argument("--warmup", type=int, default=24)
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad", "wgrad_conv"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad", "wgrad_conv", "wgrad_dw"],
                     help="cfg1..cfg5: the five layer workloads; cfg4b: backward data through cfg4's block; wgrad: the weight gradient "
                          "of a linear layer (a later row of the scope)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -656,7 +660,7 @@ def main():
                     help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
                          "then --steps in-hindsight steps, then --steps dynamic steps")
     args = ap.parse_args()
-    if args.workload in ("wgrad", "wgrad_conv") and args.impl == "hq" and not args.profile:
+    if args.workload in ("wgrad", "wgrad_conv", "wgrad_dw") and args.impl == "hq" and not args.profile:
         run_wgrad(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -233,7 +233,9 @@ hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32
  *   GW[k][r][s][c] = fl( float( sum over n,ho,wo of (dY[n][ho][wo][k] - z_dy) * (X[n][hi][wi][c] - z_x) ) * fl(s_dy * s_x) ),
  * hi = ho*stride_h - pad_h + r (wi alike), output pixels whose (hi,wi) lies outside the image contributing nothing (padding
  * is zero in the real domain).  dY is N x Ho x Wo x K, X is N x H x W x C, GW has the layout of the weights, binary32.
- * The sum is formed modulo 2^32: exact whenever the true sum fits in int32.  groups must be 1; at most 2^24 output pixels.
+ * The sum is formed modulo 2^32: exact whenever the true sum fits in int32.  At most 2^24 output pixels.  Depthwise layers
+ * (groups == C == K; 3x3 or 5x5 filters, C a multiple of 4, at most 1024): GW is [C][R][S], the sum runs with k == c, on a
+ * CUDA-core kernel with integer atomics.
  * How it runs: the filter windows of X and dY are written transposed (pixels innermost) into context-owned scratch (grown
  * with cudaMalloc when a larger layer is first seen: R*S times the size of X; calls on one context must not overlap);
  * the reduction over the pixels is cut into slices that the tensor-core layer kernel multiplies side by side, and a last

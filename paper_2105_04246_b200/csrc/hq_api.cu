@@ -1190,10 +1190,28 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   if (!aligned16(dY) || !aligned16(X) || !aligned16(GW) || !aligned16(dyq) || !aligned16(xq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
   const hq_conv_desc& d = *desc;
-  if (d.groups != 1) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient of grouped convolutions is not implemented");
   cudaStream_t s = (cudaStream_t)stream;
   const int Ho = out_dim(d.H, d.pad_h, d.R, d.stride_h), Wo = out_dim(d.W, d.pad_w, d.S, d.stride_w);
   const int64_t M64 = (int64_t)d.N * Ho * Wo;
+  if (d.groups != 1) {   // depthwise (check_desc admits groups == C == K only): a CUDA-core kernel, GW is [C][R][S]
+    if (!(d.R == d.S && (d.R == 3 || d.R == 5))) return fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise weight gradient: 3x3 and 5x5 filters only");
+    if (d.C % 4 != 0 || d.C > 1024 || (size_t)d.C * d.R * d.S * sizeof(int32_t) > 48u * 1024u)
+      return fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise weight gradient needs C %% 4 == 0, C <= 1024 and C * R * S <= 12288");
+    if (M64 > (1 << 30)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels");
+    const size_t need = (size_t)d.C * d.R * d.S * sizeof(int32_t) + 256;
+    if (need > ctx->wgrad_bytes) {
+      if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));
+      ctx->d_wgrad = nullptr;
+      ctx->wgrad_bytes = 0;
+      HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_wgrad, need));
+      ctx->wgrad_bytes = need;
+    }
+    int32_t* acc = reinterpret_cast<int32_t*>(ctx->d_wgrad);
+    HQ_CUDA(ctx, cudaMemsetAsync(acc, 0, (size_t)d.C * d.R * d.S * sizeof(int32_t), s));
+    HQ_CUDA(ctx, launch_dw_wgrad(dY, X, dyq, xq, d, Ho, Wo, ctx->num_sms, make_fastdiv(Wo), make_fastdiv(Ho), acc, GW, s));
+    ctx->launches += 2;
+    return HQ_OK;
+  }
   const int64_t cols64 = (int64_t)d.R * d.S * d.C;
   if (M64 > (1 << 24) || cols64 > (1 << 20)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels or filter elements");
   const int M = (int)M64, rows = d.K, cols = (int)cols64;

@@ -543,6 +543,70 @@ __global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int
   terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
 }
 
+// ---- weight gradient of a depthwise layer (CUDA cores) -----------------------------------------------------------
+// g[c][r][s] = sum over output pixels of (dy(.., c) - z_dy) * (x(hi, wi, c) - z_x), padded taps skipped.  A thread owns
+// four channels (one word) and every `lanes`-th output pixel of its block's range; its RS*RS*4 sums stay in registers,
+// are gathered per block in shared memory and leave as integer atomics on acc[c][tap] (zeroed by the caller).
+template <int RS>
+__global__ void __launch_bounds__(256) dw_wgrad_kernel(const int8_t* __restrict__ dY, const int8_t* __restrict__ X, const hq_range_state* __restrict__ dyq,
+                                                        const hq_range_state* __restrict__ xq, hq_conv_desc d, int Ho, int Wo, int M,
+                                                        int pixels_per_block, FastDiv fd_wo, FastDiv fd_ho, int32_t* __restrict__ acc_out) {
+  extern __shared__ int32_t sacc[];   // [C][RS*RS]
+  constexpr int T = RS * RS;
+  const int CW = d.C / 4;
+  for (int i = threadIdx.x; i < d.C * T; i += blockDim.x) sacc[i] = 0;
+  __syncthreads();
+  const int lanes = (int)blockDim.x / CW;   // C <= 1024
+  const int cw = (int)threadIdx.x % CW, pl = (int)threadIdx.x / CW;
+  const int zdy = dyq->zero_point, zx = xq->zero_point;
+  if (pl < lanes) {
+    int acc[T][4];
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[t][k] = 0;
+    const int m_begin = blockIdx.x * pixels_per_block;
+    const int m_end = min(M, m_begin + pixels_per_block);
+    for (int m = m_begin + pl; m < m_end; m += lanes) {
+      const int t0 = fdiv(m, fd_wo);
+      const int wo = m - t0 * Wo;
+      const int n = fdiv(t0, fd_ho);
+      const int ho = t0 - n * Ho;
+      const uint32_t gw = *reinterpret_cast<const uint32_t*>(dY + (int64_t)m * d.C + cw * 4);
+      int g[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) g[k] = (int)(int8_t)((gw >> (8 * k)) & 0xffu) - zdy;
+#pragma unroll
+      for (int r = 0; r < RS; ++r) {
+        const int hi = ho * d.stride_h - d.pad_h + r;
+        if (hi < 0 || hi >= d.H) continue;
+#pragma unroll
+        for (int s = 0; s < RS; ++s) {
+          const int wi = wo * d.stride_w - d.pad_w + s;
+          if (wi < 0 || wi >= d.W) continue;
+          const uint32_t xw = *reinterpret_cast<const uint32_t*>(X + (((int64_t)n * d.H + hi) * d.W + wi) * d.C + cw * 4);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) acc[r * RS + s][k] += g[k] * ((int)(int8_t)((xw >> (8 * k)) & 0xffu) - zx);
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) atomicAdd(&sacc[(cw * 4 + k) * T + t], acc[t][k]);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < d.C * T; i += blockDim.x) {
+    const int v = sacc[i];
+    if (v != 0) atomicAdd(&acc_out[i], v);
+  }
+}
+__global__ void scale_to_real_kernel(const int32_t* __restrict__ acc, int count, const hq_range_state* __restrict__ dyq,
+                                     const hq_range_state* __restrict__ xq, float* __restrict__ G) {
+  const float sc = __fmul_rn(dyq->scale, xq->scale);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x) G[i] = __fmul_rn(__int2float_rn(acc[i]), sc);
+}
+
 // ---- depthwise convolution on CUDA cores --------------------------------------------------------
 // One thread: one output pixel x 16 consecutive channels.  Same epilogue as the tensor-core kernel.
 __device__ __forceinline__ int sx8(uint32_t w, int k) { return (int)(int8_t)((w >> (8 * k)) & 0xffu); }
@@ -1058,6 +1122,22 @@ cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* x
   const int tiles = (int)((Mp + 127) / 128), tiles_per_block = tiles >= 4096 ? 16 : (tiles >= 256 ? 8 : 1);
   dim3 grid((unsigned)((tiles + tiles_per_block - 1) / tiles_per_block), (unsigned)((d.C + 31) / 32), (unsigned)(d.R * d.S));
   im2col_t_kernel<<<grid, 256, 0, s>>>(X, Bt, xq, d, Ho, Wo, (int)M, (int)Mp, tiles_per_block, fd_wo, fd_ho, colsum);
+  return cudaGetLastError();
+}
+cudaError_t launch_dw_wgrad(const int8_t* dY, const int8_t* X, const hq_range_state* dyq, const hq_range_state* xq, const hq_conv_desc& d, int Ho,
+                            int Wo, int num_sms, FastDiv fd_wo, FastDiv fd_ho, int32_t* acc, float* G, cudaStream_t s) {
+  const int M = d.N * Ho * Wo, T = d.R * d.S;
+  int blocks = std::max(1, std::min(num_sms * 4, (M + 255) / 256));
+  const int pixels_per_block = (M + blocks - 1) / blocks;
+  blocks = (M + pixels_per_block - 1) / pixels_per_block;
+  const size_t smem = (size_t)d.C * T * sizeof(int32_t);
+  if (d.R == 3)
+    dw_wgrad_kernel<3><<<blocks, 256, smem, s>>>(dY, X, dyq, xq, d, Ho, Wo, M, pixels_per_block, fd_wo, fd_ho, acc);
+  else
+    dw_wgrad_kernel<5><<<blocks, 256, smem, s>>>(dY, X, dyq, xq, d, Ho, Wo, M, pixels_per_block, fd_wo, fd_ho, acc);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  scale_to_real_kernel<<<std::max(1, std::min(64, (d.C * T + 255) / 256)), 256, 0, s>>>(acc, d.C * T, dyq, xq, G);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,

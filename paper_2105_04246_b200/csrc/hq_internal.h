@@ -203,6 +203,9 @@ cudaError_t launch_pad_rows(const int8_t* src, int8_t* dst, int rows, int K, int
 cudaError_t launch_transpose_rows(const int8_t* in, int8_t* out, int R, int C, int Rp, int ones_row, cudaStream_t s);
 cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* xq, const hq_conv_desc& d, int Ho, int Wo, int64_t Mp, int32_t* colsum,
                             FastDiv fd_wo, FastDiv fd_ho, cudaStream_t s);
+// depthwise weight gradient, 3x3 or 5x5 filters, C a multiple of 4 and at most 1024; acc: C*R*S zeroed int32
+cudaError_t launch_dw_wgrad(const int8_t* dY, const int8_t* X, const hq_range_state* dyq, const hq_range_state* xq, const hq_conv_desc& d, int Ho,
+                            int Wo, int num_sms, FastDiv fd_wo, FastDiv fd_ho, int32_t* acc, float* G, cudaStream_t s);
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
                                 const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,

@@ -150,3 +150,49 @@ def test_conv_wgrad_bench_size_sampled_channels(ctx):
                            O.acc_scale(dy.scale, x.scale))
     assert np.array_equal(got[ks].view(np.uint32), want.view(np.uint32))
     assert np.isfinite(got).all() and ctx.get_async_error() == 0
+
+
+DW_WGRAD_CASES = {
+    "dw3x3_c144": dict(N=2, H=10, W=12, C=144, R=3, stride=1, pad=1),
+    "dw3x3_s2_c32": dict(N=2, H=11, W=11, C=32, R=3, stride=2, pad=1),
+    "dw3x3_c32_ragged": dict(N=3, H=13, W=21, C=32, R=3, stride=1, pad=1),
+    "dw3x3_c256_nopad": dict(N=1, H=11, W=12, C=256, R=3, stride=1, pad=0),
+    "dw5x5_c48": dict(N=1, H=13, W=9, C=48, R=5, stride=1, pad=2),
+    "dw3x3_c320": dict(N=2, H=7, W=7, C=320, R=3, stride=1, pad=1),
+    "dw3x3_c144_56": dict(N=4, H=56, W=56, C=144, R=3, stride=1, pad=1),
+}
+
+
+@pytest.mark.parametrize("name", list(DW_WGRAD_CASES))
+def test_depthwise_wgrad_matches_oracle(ctx, name):
+    c = DW_WGRAD_CASES[name]
+    dev = torch.device("cuda", ctx.device)
+    r = synth.rng(305, len(name), c["H"], c["C"])
+    desc = hq.conv_desc(c["N"], c["H"], c["W"], c["C"], c["C"], c["R"], c["R"], stride=c["stride"], pad=c["pad"], groups=c["C"])
+    od = O.conv_desc(c["N"], c["H"], c["W"], c["C"], c["C"], c["R"], c["R"], stride=c["stride"], pad=c["pad"], groups=c["C"])
+    Ho, Wo = O.out_hw(od)
+    dy = synth.gradients(r, (c["N"], Ho, Wo, c["C"]))
+    x = synth.relu_activations(r, (c["N"], c["H"], c["W"], c["C"]))
+    dy_d, x_d = torch.from_numpy(dy.q).to(dev), torch.from_numpy(x.q).to(dev)
+    dyq = hq.states_to_device(hq.input_state(dy.scale, dy.zero_point), dev)
+    xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
+    want = O.scale_to_real(O.conv_wgrad_acc(od, dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
+    for _ in range(2):
+        gw = torch.full((c["C"], c["R"], c["R"]), float("nan"), dtype=torch.float32, device=dev)
+        ctx.conv_wgrad(None, desc, dy_d, dyq, x_d, xq, gw)
+        torch.cuda.synchronize(dev)
+        got = gw.cpu().numpy()
+        bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
+        assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
+    assert ctx.get_async_error() == 0
+
+
+def test_depthwise_wgrad_refuses_other_filters(ctx):
+    dev = torch.device("cuda", ctx.device)
+    t = torch.zeros(4096, dtype=torch.int8, device=dev)
+    st = hq.states_to_device(hq.input_state(0.1, 0), dev)
+    g = torch.zeros(4096, dtype=torch.float32, device=dev)
+    n0 = ctx.launch_count()
+    with pytest.raises(hq.HqError) as e:
+        ctx.conv_wgrad(None, hq.conv_desc(1, 8, 8, 16, 16, 7, 7, stride=1, pad=3, groups=16), t, st, t, st, g)
+    assert e.value.status == 2 and ctx.launch_count() == n0
