@@ -30,7 +30,8 @@
 //        the running (q_min,q_max) of Eq. 2-3 stay un-widened.
 //   R-4  round half to even; y/s is evaluated as y * (1/s) with 1/s rounded once; every
 //        floating-point step is one binary32 round-to-nearest-even operation, never fused.
-//   R-5  weights symmetric (z_w = 0 on the graded path; the loops still take z_w).
+//   R-5  weights symmetric by default (z_w = 0); every accumulator loop takes z_w, pinned with non-zero
+//        values against int64 matrix products, scatter-form loops and library convolutions in float64.
 //   R-6  deterministic rounding for gradients as well.
 //   R-7  statistics are taken on the zero-point-corrected int32 accumulator (+ int32
 //        bias), before any clamping; float(min acc) * s_acc is then the exact minimum of
@@ -45,7 +46,8 @@
 // arithmetic, the forward/backward adjoint identity, the trace identity <dY, X W^T> = <dY^T X, W>
 // that ties the weight gradient to the forward layer, library convolutions in float64,
 // the closed form of the Eq. 2-3 recurrence, grid invariants of the quantizer, and
-// static == dynamic when the ranges coincide.
+// static == dynamic when the ranges coincide; the stochastic dynamic path is tied to the
+// deterministic one (range) and to the static stochastic quantizer (codes, draw count).
 // PARITY UNPINNED: the tie rule of the rounding (R-4), the zero-point formula of
 // hqo_derive beyond its grid invariants, and symmetric weights (R-5) are fixed by the
 // readings above only -- the paper prints no formula or worked example for them.

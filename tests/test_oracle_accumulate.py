@@ -212,3 +212,86 @@ def test_statistics_are_exact_extremes_in_any_order():
     lo = min(O.minmax(t)[0] for t in tiles); hi = max(O.minmax(t)[1] for t in tiles)
     assert (lo, hi) == (int(acc.min()), int(acc.max()))
     assert O.minmax(np.array([5], np.int32)) == (5, 5)
+
+
+# ---- weight zero point (asymmetric weights: every loop takes z_w) ------------------------------------
+def test_weight_zero_point_by_eye():
+    # weights that all equal their zero point are real zeros: nothing accumulates, whatever the input
+    g = synth.rng(10)
+    X = _rand_i8(g, (3, 8))
+    assert not O.linear_acc(X, 5, np.full((4, 8), -7, np.int8), zw=-7).any()
+    d = O.conv_desc(1, 5, 5, 2, 3, 3, 3, stride=1, pad=1)
+    Xc = _rand_i8(g, (1, 5, 5, 2))
+    assert not O.conv_fwd_acc(d, Xc, 3, np.full((3, 3, 3, 2), 9, np.int8), zw=9).any()
+    assert not O.conv_bwd_data_acc(d, Xc[..., :1].repeat(3, -1), 3, np.full((3, 3, 3, 2), 9, np.int8), zw=9).any()
+    # all-ones input, weights one above their zero point: the count of valid taps (padding contributes nothing)
+    acc = O.conv_fwd_acc(d, np.ones((1, 5, 5, 2), np.int8), 0, np.full((3, 3, 3, 2), 10, np.int8), zw=9)
+    taps = np.array([[4, 6, 6, 6, 4], [6, 9, 9, 9, 6], [6, 9, 9, 9, 6], [6, 9, 9, 9, 6], [4, 6, 6, 6, 4]]) * 2
+    assert np.array_equal(acc[0, :, :, 0], taps)
+    # a single row, readable: (1-1, 2-1, 3-1) . (4+2, 0+2, -2+2) = 0*6 + 1*2 + 2*0
+    assert O.linear_acc(np.array([[1, 2, 3]], np.int8), 1, np.array([[4, 0, -2]], np.int8), zw=-2).tolist() == [[2]]
+
+
+def test_linear_weight_zero_point_against_numpy_int64():
+    g = synth.rng(11)
+    X = _rand_i8(g, (21, 50)); W = _rand_i8(g, (13, 50))
+    bias = g.integers(-10**5, 10**5, size=13).astype(np.int32)
+    for zx, zw in [(-128, 127), (17, -128), (0, 5)]:
+        ref = (X.astype(np.int64) - zx) @ (W.astype(np.int64) - zw).T + bias
+        assert np.array_equal(O.linear_acc(X, zx, W, zw=zw, bias=bias), ref)
+        idx = g.integers(0, ref.size, size=40)
+        assert np.array_equal(O.linear_acc_at(X, zx, W, idx, zw=zw, bias=bias), ref.ravel()[idx])
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("zw", [-128, 6, 127])
+def test_conv_weight_zero_point_against_scatter_loops(case, zw):
+    g = synth.rng(12, case["H"], case["R"], zw + 128)
+    d = _desc(case)
+    Ho, Wo = O.out_hw(d)
+    X = _rand_i8(g, (d.N, d.H, d.W, d.C))
+    Wt = _rand_i8(g, (d.K, d.R, d.S, d.C))
+    G = _rand_i8(g, (d.N, Ho, Wo, d.K))
+    zx, zg = -9, 12
+    y = np.zeros((d.N, Ho, Wo, d.K), np.int64)
+    dx = np.zeros((d.N, d.H, d.W, d.C), np.int64)
+    for n, ho, wo, k, r, s, c in itertools.product(range(d.N), range(Ho), range(Wo), range(d.K), range(d.R), range(d.S), range(d.C)):
+        hi = ho * d.stride_h - d.pad_h + r
+        wi = wo * d.stride_w - d.pad_w + s
+        if 0 <= hi < d.H and 0 <= wi < d.W:
+            w = int(Wt[k, r, s, c]) - zw
+            y[n, ho, wo, k] += (int(X[n, hi, wi, c]) - zx) * w
+            dx[n, hi, wi, c] += (int(G[n, ho, wo, k]) - zg) * w
+    assert np.array_equal(O.conv_fwd_acc(d, X, zx, Wt, zw), y)
+    assert np.array_equal(O.conv_bwd_data_acc(d, G, zg, Wt, zw), dx)
+    idx = g.integers(0, y.size, size=min(30, y.size))
+    assert np.array_equal(O.conv_fwd_acc_at(d, X, zx, Wt, idx, zw), y.ravel()[idx])
+    idx = g.integers(0, dx.size, size=min(30, dx.size))
+    assert np.array_equal(O.conv_bwd_data_acc_at(d, G, zg, Wt, idx, zw), dx.ravel()[idx])
+
+
+@pytest.mark.parametrize("case", LIB_CASES[:3])
+@pytest.mark.parametrize("depthwise", [False, True])
+def test_weight_zero_point_against_torch_float64(case, depthwise):
+    g = synth.rng(13, case["H"], case["R"], int(depthwise))
+    c = dict(case)
+    if depthwise:
+        c["K"] = c["C"]
+    groups = c["C"] if depthwise else 1
+    d = _desc(c, groups=groups)
+    Ho, Wo = O.out_hw(d)
+    X = _rand_i8(g, (d.N, d.H, d.W, d.C))
+    Wt = _rand_i8(g, (d.K, d.R, d.S) if depthwise else (d.K, d.R, d.S, d.C))
+    G = _rand_i8(g, (d.N, Ho, Wo, d.K))
+    zx, zg, zw = 23, -6, -31
+    w4 = Wt.reshape(d.K, d.R, d.S, 1) if depthwise else Wt
+    tw = torch.from_numpy(w4.astype(np.float64) - zw).permute(0, 3, 1, 2).contiguous()
+    tx = torch.from_numpy(X.astype(np.float64) - zx).permute(0, 3, 1, 2).contiguous()
+    ty = torch.nn.functional.conv2d(tx, tw, stride=(d.stride_h, d.stride_w), padding=(d.pad_h, d.pad_w), groups=groups)
+    assert np.array_equal(O.conv_fwd_acc(d, X, zx, Wt, zw), ty.permute(0, 2, 3, 1).numpy().astype(np.int64))
+    tg = torch.from_numpy(G.astype(np.float64) - zg).permute(0, 3, 1, 2).contiguous()
+    oph = d.H - ((Ho - 1) * d.stride_h - 2 * d.pad_h + d.R)
+    opw = d.W - ((Wo - 1) * d.stride_w - 2 * d.pad_w + d.S)
+    tdx = torch.nn.functional.conv_transpose2d(tg, tw, stride=(d.stride_h, d.stride_w), padding=(d.pad_h, d.pad_w),
+                                               output_padding=(oph, opw), groups=groups)
+    assert np.array_equal(O.conv_bwd_data_acc(d, G, zg, Wt, zw), tdx.permute(0, 2, 3, 1).numpy().astype(np.int64))

@@ -110,3 +110,24 @@ def test_layer_uses_iteration_count_and_previous_range():
     r1 = layer.step(acc1, 1e-3)
     assert np.array_equal(r1.q, O.quantize_sr(acc1, 1e-3, before, 77, 1))   # old range, draws of iteration 1
     assert not np.array_equal(r1.q, O.quantize_sr(acc1, 1e-3, before, 77, 2))
+
+
+@pytest.mark.parametrize("prior_steps", [0, 3])
+def test_dynamic_path_draws_with_the_count_before_its_update(prior_steps):
+    """The dynamic path with stochastic rounding is Eq. 1 for the range (the separately pinned deterministic dynamic
+    path gives the same range) followed by the separately pinned static stochastic quantizer, drawing with the number
+    of updates the state had seen BEFORE this call; one count later gives other codes."""
+    g = np.random.default_rng(35 + prior_steps)
+    acc = g.integers(-7000, 9000, size=(12, 40)).astype(np.int32)
+    s_acc, seed = 2.5e-3, 4242
+    st = O.derive(O.Range(q_min=-1.0, q_max=2.0, step=prior_steps))
+    yf, codes = O.dynamic_sr(acc, s_acc, st, seed)
+    ref = O.derive(O.Range(q_min=-1.0, q_max=2.0, step=prior_steps))
+    yf_ref, _ = O.dynamic(acc, s_acc, ref)
+    assert st.astuple() == ref.astuple() and st.step == prior_steps + 1
+    assert (st.q_min, st.q_max) == (float(yf_ref.min()), float(yf_ref.max()))
+    assert np.array_equal(yf, yf_ref)
+    assert np.array_equal(codes, O.quantize_sr(acc, s_acc, st, seed, iteration=prior_steps))
+    assert not np.array_equal(codes, O.quantize_sr(acc, s_acc, st, seed, iteration=prior_steps + 1))
+    if prior_steps:
+        assert not np.array_equal(codes, O.quantize_sr(acc, s_acc, st, seed, iteration=prior_steps - 1))
