@@ -17,6 +17,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -39,8 +40,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the named layer's kernel, from the ncu captures
 # summarised under profiles/ (taken with the kernels as committed; set an entry to None when its kernel changes).
 # Output lines still dirty in L2 when the kernel ends are not in these counters.
-NCU_TRAFFIC = {"resnet_conv3x3_64": 12992000, "resnet_conv3x3_256_bwd": 13547776, "mbv2_dw3x3": 182444800,
-               "mbv2_expand": 81283328, "mbv2_project": 121651200}
+NCU_TRAFFIC = {}
+# kernels other than the tensor-core layer kernel, by layer name
+KERNEL_OF = {"mbv2_dw3x3": "depthwise3x3_tiled_kernel"}
 
 
 def load_peaks():
@@ -154,7 +156,13 @@ def run_oracle(workload: str, steps: int, warmup: int, budget_s: float):
 
 
 # ---- GPU arm ---------------------------------------------------------------------------------------
+L2_ROTATE_BYTES = 192 << 20           # per-layer buffer pools are sized so that one cycle through them moves more than L2 (126 MB)
+MAX_POOL = 64
+
+
 class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons with nvidia-smi every 50 ms while timed regions run."""
+
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.samples, self.stop_flag = index, [], False
@@ -167,24 +175,29 @@ class ClockSampler(threading.Thread):
                 out = subprocess.run(["nvidia-smi", f"--id={self.index}", f"--query-gpu={q}", "--format=csv,noheader,nounits"],
                                      capture_output=True, text=True, timeout=5).stdout.strip()
                 if out:
-                    self.samples.append([v.strip() for v in out.split(",")])
+                    self.samples.append((time.perf_counter(), [v.strip() for v in out.split(",")]))
             except Exception:
                 pass
             time.sleep(0.05)
 
-    def summary(self):
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
+    def summary(self, t0: float | None = None, t1: float | None = None):
+        rows = [s for (t, s) in self.samples if (t0 is None or t >= t0) and (t1 is None or t <= t1)]
+        sm = [float(s[0]) for s in rows if s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in rows if s[1].replace(".", "").isdigit()]
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        reasons = sorted({names[i] for s in self.samples for i in range(4) if len(s) >= 6 and s[2 + i].lower().startswith("active")})
+        reasons = sorted({names[i] for s in rows for i in range(4) if len(s) >= 6 and s[2 + i].lower().startswith("active")})
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None, "reasons": reasons,
-                "samples": len(self.samples)}
+                "samples": len(rows)}
 
 
 class GpuWorkload:
-    """All device buffers of one workload plus the calls of one step (hindsight or dynamic)."""
+    """All device buffers of one workload plus the calls of one step (hindsight or dynamic).
 
-    def __init__(self, name: str, ctx, dev, pool: int, seed_key: int, stochastic: bool = False):
+    Every layer has its own pool of input / output / workspace buffer sets, sized so that one cycle through the pool
+    moves more bytes than the L2 holds: back-to-back launches of ONE layer then meet cold operands, as they do inside a
+    whole step (where the other layers' traffic flushes the cache)."""
+
+    def __init__(self, name: str, ctx, dev, seed_key: int, stochastic: bool = False, pool_cap: int = MAX_POOL):
         import torch
         from paper_2105_04246_b200 import hq
         self.hq, self.torch, self.ctx, self.dev, self.name = hq, torch, ctx, dev, name
@@ -198,10 +211,13 @@ class GpuWorkload:
                     st[i]["rounding"], st[i]["seed"] = hq.ROUND_STOCHASTIC, 0x2105 + i
         self.states = hq.states_to_device(st, dev)
         self.state_ptr = [self.states.data_ptr() + 48 * i for i in range(n)]
-        self.W, self.w_scale, self.pw, self.desc, self.x_pool, self.xq_pool, self.y_pool, self.ws = [], [], [], [], [], [], [], []
+        self.W, self.w_scale, self.pw, self.desc, self.x_pool, self.xq_pool, self.y_pool, self.ws_pool, self.pool = [], [], [], [], [], [], [], [], []
         stream = torch.cuda.current_stream(dev)
         for i, (kind, s, recipe) in enumerate(self.layers):
             xsh, ysh, wsh = layer_shapes(kind, s)
+            xb, yb = int(np.prod(xsh)), int(np.prod(ysh))
+            pool = 2 if self.chained else int(min(pool_cap, max(2, -(-L2_ROTATE_BYTES // (xb + yb)))))
+            self.pool.append(pool)
             w = synth.weights(g, wsh) if kind != "linear" else synth.uniform_int8(g, wsh, scale=0.01)
             self.W.append(torch.from_numpy(w.q).to(dev))
             self.w_scale.append(torch.tensor([w.scale], dtype=torch.float32, device=dev))
@@ -215,10 +231,10 @@ class GpuWorkload:
             if recipe is not None:
                 xs, xqs = [], []
                 base = make_input(recipe, g, xsh)
+                base_d = torch.from_numpy(np.ascontiguousarray(base.q)).to(dev)
                 for j in range(pool):
                     # pool members: the same samples rolled by a prime offset (distinct bytes at every address)
-                    q = base.q if j == 0 else np.roll(base.q.reshape(-1), 104729 * j).reshape(xsh)
-                    xs.append(torch.from_numpy(np.ascontiguousarray(q)).to(dev))
+                    xs.append(base_d if j == 0 else torch.roll(base_d.reshape(-1), 104729 * j).reshape(xsh).contiguous())
                     xqs.append(hq.states_to_device(hq.input_state(base.scale * (1.0 + 0.05 * (j % 3)), base.zero_point), dev))
                 self.x_pool.append(xs)
                 self.xq_pool.append(xqs)
@@ -226,32 +242,34 @@ class GpuWorkload:
                 self.x_pool.append(None)
                 self.xq_pool.append(None)
             self.y_pool.append([torch.empty(ysh, dtype=torch.int8, device=dev) for _ in range(pool)])
-            self.ws.append(None)
-        self.pool = pool
+            self.ws_pool.append(None)
         self.ops = sum(s.ops for _, s, _ in self.layers)
-        self.static_bytes = [wl.layer_static_bytes(s, kind == "conv_bwd") for kind, s, _ in self.layers]
-        self.dynamic_bytes = [wl.layer_dynamic_bytes(s, kind == "conv_bwd") for kind, s, _ in self.layers]
+        self.static_bytes = [wl.layer_static_bytes(s, kind == "conv_bwd" or s.name.endswith(".bwd")) for kind, s, _ in self.layers]
+        self.dynamic_bytes = [wl.layer_dynamic_bytes(s, kind == "conv_bwd" or s.name.endswith(".bwd")) for kind, s, _ in self.layers]
         self.h2d_bytes = sum(int(np.prod(layer_shapes(k, s)[0])) for (k, s, r) in self.layers if r is not None)
         self.d2h_bytes = int(np.prod(layer_shapes(*self.layers[-1][:2])[1]))
 
     def _inputs(self, i, j):
         if self.x_pool[i] is not None:
-            return self.x_pool[i][j], self.xq_pool[i][j].data_ptr()
-        return self.y_pool[i - 1][j], self.state_ptr[i - 1]
+            jj = j % self.pool[i]
+            return self.x_pool[i][jj], self.xq_pool[i][jj].data_ptr()
+        return self.y_pool[i - 1][j % self.pool[i - 1]], self.state_ptr[i - 1]
 
     def layer_call(self, stream, i, j, dynamic=False):
         hq, ctx = self.hq, self.ctx
         kind, s, _ = self.layers[i]
         x, xq = self._inputs(i, j)
-        y = self.y_pool[i][j]
+        y = self.y_pool[i][j % self.pool[i]]
         if dynamic:
-            if self.ws[i] is None:
-                self.ws[i] = self.torch.empty(y.shape, dtype=self.torch.float32, device=self.dev)
+            if self.ws_pool[i] is None:   # the binary32 intermediate of Eq. 5 rotates like the other buffers
+                nws = int(min(self.pool[i], max(2, -(-L2_ROTATE_BYTES // (4 * y.numel())))))
+                self.ws_pool[i] = [self.torch.empty(y.shape, dtype=self.torch.float32, device=self.dev) for _ in range(nws)]
+            ws = self.ws_pool[i][j % len(self.ws_pool[i])]
             if kind == "linear":
                 op = hq.linear_op(s.M, s.N, s.K, x, xq, self.W[i], self.w_scale[i])
             else:
                 op = hq.conv_op(hq.OP_CONV_FWD if kind == "conv_fwd" else hq.OP_CONV_BWD_DATA, self.desc[i], x, xq, self.pw[i], self.w_scale[i])
-            ctx.dynamic_quant(stream, op, self.ws[i], y, self.state_ptr[i])
+            ctx.dynamic_quant(stream, op, ws, y, self.state_ptr[i])
         elif kind == "linear":
             ctx.linear_fwd(stream, s.M, s.N, s.K, x, xq, self.W[i], self.w_scale[i], None, y, self.state_ptr[i])
         elif kind == "conv_fwd":
@@ -265,12 +283,18 @@ class GpuWorkload:
                 self.layer_call(stream, i, j, dynamic)
         if update and not dynamic:
             if exchange is not None:      # batch shards: min/max over all ranks before Eq. 2-3
-                exchange(self.states)
+                exchange(stream, self.states)
             self.ctx.range_update(stream, self.states, len(self.layers), 0.9)
+
+    def release(self):
+        for pw in self.pw:
+            if pw is not None:
+                pw.release()
+        self.x_pool = self.y_pool = self.ws_pool = self.W = None
 
 
 def capture(torch, stream_fn, reps: int):
-    """Captures `reps` consecutive steps (pool member j = rep index) into one CUDA graph."""
+    """Captures `reps` consecutive steps (pool slot = rep index) into one CUDA graph."""
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
         s = torch.cuda.current_stream()
@@ -279,23 +303,125 @@ def capture(torch, stream_fn, reps: int):
     return g
 
 
-def time_graph(torch, graph_full, graphs_single, steps: int, pool: int, dist=None):
-    """Times exactly `steps` steps: whole-pool graphs, then single-step graphs for the remainder."""
-    full, rem = divmod(steps, pool)
-    if dist is not None:
-        dist.barrier()
+def timed_repeats(torch, run_once, units: int, min_time_s: float, min_repeats: int, dist=None, max_repeats: int = 4000):
+    """Runs `run_once` (which enqueues `units` steps or launches) as often as it takes to fill `min_time_s`, at least
+    `min_repeats` times, each repeat between its own pair of CUDA events on the launching stream (with more than one rank:
+    a barrier and a device synchronisation on both sides of every repeat, and the maximum over the ranks).
+    Returns per-unit times in ms: (median, min, max, repeats)."""
+    def one():
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run_once()
+        e1.record()
+        if dist is not None:
+            torch.cuda.synchronize()
+            dist.barrier()
+            t = torch.tensor([e0.elapsed_time(e1)], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return (e0, e1)
     torch.cuda.synchronize()
+    first = one()
+    if dist is None:
+        torch.cuda.synchronize()
+        first = first[0].elapsed_time(first[1])
+    reps = int(min(max_repeats, max(min_repeats, -(-min_time_s * 1e3 // max(first, 1e-3)))))
+    if dist is not None:    # every rank must run the same number of repeats
+        t = torch.tensor([reps], device="cuda", dtype=torch.int64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        reps = int(t.item())
+    got = [one() for _ in range(reps)]
+    if dist is None:
+        torch.cuda.synchronize()
+        got = [a.elapsed_time(b) for (a, b) in got]
+    per = sorted(x / units for x in got)
+    return statistics.median(per), per[0], per[-1], reps
+
+
+def measure_mma_peak(torch, ctx, sampler, sustained_s: float = 4.0):
+    """int8 MMA-only throughput of this GPU: best of 10 launches (burst) and back-to-back launches for `sustained_s`."""
+    out = {}
+    chunks = 512                                             # 512 x 32 instructions per SM: about a millisecond
+    for pair in (0, 1):
+        ops = ctx.mma_peak_probe(None, pair, 256, chunks)    # warm-up
+        torch.cuda.synchronize()
+        best = None
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.mma_peak_probe(None, pair, 256, chunks)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+        out["pair" if pair else "single"] = {"burst_tops": round(ops / (best * 1e-3) / 1e12, 1)}
+    pair = 1 if out["pair"]["burst_tops"] >= out["single"]["burst_tops"] else 0
+    n = max(1, int(sustained_s * 1e3 / max(best, 1e-3)))
+    t0 = time.perf_counter()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
-    for _ in range(full):
-        graph_full.replay()
-    for j in range(rem):
-        graphs_single[j].replay()
+    for _ in range(n):
+        ops = ctx.mma_peak_probe(None, pair, 256, chunks)
     e1.record()
     torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    return e0.elapsed_time(e1)
+    t1 = time.perf_counter()
+    sus = ops * n / (e0.elapsed_time(e1) * 1e-3) / 1e12
+    clk = sampler.summary(t0 + 0.5, t1)
+    assert ctx.get_async_error() == 0, "a device-side wait expired in the MMA probe"
+    return {"burst_tops": max(out["pair"]["burst_tops"], out["single"]["burst_tops"]), "single_cta_burst_tops": out["single"]["burst_tops"],
+            "cta_pair_burst_tops": out["pair"]["burst_tops"], "sustained_tops": round(sus, 1), "sustained_s": round(t1 - t0, 2),
+            "sustained_sm_mhz": clk["sm_mhz"], "sustained_reasons": clk["reasons"],
+            "what": "tcgen05.mma kind::i8 128x256x32 (pair: 256x256x32) issued back to back on operand tiles resident in shared memory, every SM, no loads, no epilogue"}
+
+
+def layer_rows(torch, wk, cfg_name, peaks, probe_peak, min_time_s, min_repeats):
+    """Per-layer rows of one workload: each layer's launches alone (no update kernel), replayed from a CUDA graph that
+    cycles through the layer's whole buffer pool; hindsight and dynamic path."""
+    int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
+    hbm_peak = peaks["hbm_gbs"]
+    rows = []
+    for i, (kind, s, _) in enumerate(wk.layers):
+        reps = wk.pool[i] if not wk.chained else 2
+        if wk.chained:
+            # a chained layer reads the previous layer's output: make sure every pool slot of that output exists
+            g_h = capture(torch, lambda st, j, ii=i: wk.step(st, j, only_layer=ii, update=False), reps)
+            g_d = capture(torch, lambda st, j, ii=i: wk.step(st, j, dynamic=True, only_layer=ii), reps)
+        else:
+            g_h = capture(torch, lambda st, j, ii=i: wk.layer_call(st, ii, j), reps)
+            g_d = capture(torch, lambda st, j, ii=i: wk.layer_call(st, ii, j, dynamic=True), reps)
+        ms, lo, hi, r = timed_repeats(torch, g_h.replay, reps, min_time_s, min_repeats)
+        msd, lod, hid, rd = timed_repeats(torch, g_d.replay, reps, min_time_s, min_repeats)
+        del g_h, g_d
+        us, usd = ms * 1e3, msd * 1e3
+        dw = getattr(s, "depthwise", False)
+        t_tensor = s.ops / (int8_peak * 1e12) * 1e6
+        t_hbm = wk.static_bytes[i] / (hbm_peak * 1e9) * 1e6
+        rows.append({
+            "config": cfg_name, "layer": s.name, "kind": kind, "us": round(us, 3), "us_min": round(lo * 1e3, 3), "us_max": round(hi * 1e3, 3),
+            "repeats": r, "launches_per_repeat": reps, "us_dynamic": round(usd, 3),
+            "tops": round(s.ops / us / 1e6, 2), "gbs": round(wk.static_bytes[i] / us / 1e3, 1),
+            "gbs_dynamic": round(wk.dynamic_bytes[i] / usd / 1e3, 1),
+            "hbm_bytes_hindsight": int(wk.static_bytes[i]), "hbm_bytes_dynamic": int(wk.dynamic_bytes[i]),
+            "bound": "alu-or-hbm" if dw else ("tensor" if t_tensor >= t_hbm else "hbm"),
+            "frac_tensor": None if dw else round(t_tensor / us, 4),
+            "frac_tensor_probe": None if (dw or not probe_peak) else round(s.ops / (probe_peak * 1e12) * 1e6 / us, 4),
+            "frac_hbm": round(t_hbm / us, 4),
+        })
+    return rows
+
+
+def spawn_ranks(args) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) the way torchrun would."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def run_gpu(args):
@@ -320,157 +446,196 @@ def run_gpu(args):
     ctx.set_option("depthwise", args.depthwise)
     peaks, peak_kind = load_peaks()
     name = args.workload
-    pool = {"cfg1": 16, "cfg2": 12, "cfg3": 12, "cfg4": 2, "cfg4b": 2, "cfg5": 2}[name]
-    wk = GpuWorkload(name, ctx, dev, pool, seed_key=rank, stochastic=args.rounding == "stochastic")
     K, W = args.steps, max(3, args.warmup)
     stream = torch.cuda.current_stream(dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+
+    # what the tensor cores of this GPU sustain on int8 with nothing else in the way (second denominator of the tensor roofline)
+    probe = None
+    if not args.no_probe and rank == 0:
+        probe = measure_mma_peak(torch, ctx, sampler, sustained_s=args.probe_seconds)
+    probe_peak = probe["burst_tops"] if probe else None
+
+    wk = GpuWorkload(name, ctx, dev, seed_key=rank, stochastic=args.rounding == "stochastic")
     n_layers = len(wk.layers)
+    cyc = 2                                   # steps per captured graph; a whole step moves far more than L2 by itself
 
     # iteration 0 of the scheme: the dynamic path initialises every range (also warms the dynamic kernels up)
-    for j in range(pool):
+    for j in range(cyc):
         wk.step(stream, j, dynamic=True)
     torch.cuda.synchronize()
+    exchange = None
+    if dist is not None:
+        from paper_2105_04246_b200 import parallel
+        exchange = parallel.StatsExchange(ctx, n_layers, dev)
     l0 = ctx.launch_count()
-    wk.step(stream, 0)
+    wk.step(stream, 0, exchange=exchange)
     launches_per_step = ctx.launch_count() - l0
     torch.cuda.synchronize()
 
-    # graphs: the launch-bound loop is replayed from CUDA graphs (all parameters live in device memory)
-    g_full = capture(torch, lambda s, j: wk.step(s, j), pool)
-    g_single = [capture(torch, lambda s, _j, jj=j: wk.step(s, jj), 1) for j in range(pool)]
-    g_dyn = capture(torch, lambda s, j: wk.step(s, j, dynamic=True), pool)
-    g_dyn_single = [capture(torch, lambda s, _j, jj=j: wk.step(s, jj, dynamic=True), 1) for j in range(pool)]
-    g_layer = [capture(torch, lambda s, j, ii=i: wk.step(s, j, only_layer=ii, update=False), pool) for i in range(n_layers)]
-    g_layer_dyn = [capture(torch, lambda s, j, ii=i: wk.step(s, j, dynamic=True, only_layer=ii), pool) for i in range(n_layers)]
+    # graphs: the launch-bound loop is replayed from CUDA graphs (all parameters live in device memory); with several
+    # ranks the statistics exchange (pack kernel, NCCL all-reduce, unpack kernel) is part of the captured step
+    g_full = capture(torch, lambda s, j: wk.step(s, j, exchange=exchange), cyc)
+    g_single = capture(torch, lambda s, j: wk.step(s, j, exchange=exchange), 1)
+    g_dyn = capture(torch, lambda s, j: wk.step(s, j, dynamic=True), cyc)
+    g_dyn_single = capture(torch, lambda s, j: wk.step(s, j, dynamic=True), 1)
 
-    for _ in range(-(-W // pool)):
+    def k_steps(gf, g1):
+        def run():
+            for _ in range(K // cyc):
+                gf.replay()
+            for _ in range(K % cyc):
+                g1.replay()
+        return run
+
+    for _ in range(-(-W // cyc)):
         g_full.replay()
         g_dyn.replay()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.15)
-    if dist is None:
-        ms_total = time_graph(torch, g_full, g_single, K, pool, dist)
-    else:
-        # more than one rank: eager steps with the statistics all-reduce between the layers and the update
-        from paper_2105_04246_b200 import parallel
-        for k in range(W):
-            wk.step(stream, k % pool, exchange=parallel.allreduce_stats)
-        dist.barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for k in range(K):
-            wk.step(stream, k % pool, exchange=parallel.allreduce_stats)
-        e1.record()
-        torch.cuda.synchronize()
-        dist.barrier()
-        ms_total = e0.elapsed_time(e1)
-    # per-layer kernel durations: the same launches replayed back to back without the update kernel
-    reps = max(1, K // pool)
-    layer_us, layer_dyn_us = [], []
-    for i in range(n_layers):
-        layer_us.append(time_graph(torch, g_layer[i], None, reps * pool, pool) * 1e3 / (reps * pool))
-    ms_dyn = time_graph(torch, g_dyn, g_dyn_single, K, pool, dist)
-    for i in range(n_layers):
-        layer_dyn_us.append(time_graph(torch, g_layer_dyn[i], None, reps * pool, pool) * 1e3 / (reps * pool))
-    sampler.stop_flag = True
-    sampler.join(timeout=2)
+    t_sec0 = time.perf_counter()
+    ms_step, ms_lo, ms_hi, repeats = timed_repeats(torch, k_steps(g_full, g_single), K, args.min_time, args.min_repeats, dist)
+    t_sec1 = time.perf_counter()
+    step_clocks = sampler.summary(t_sec0, t_sec1)
+    ms_dyn, _, _, _ = timed_repeats(torch, k_steps(g_dyn, g_dyn_single), K, args.min_time, args.min_repeats, dist)
+
+    # per-layer kernel durations of this workload, then of the other configurations (rows only)
+    per_layer = layer_rows(torch, wk, name, peaks, probe_peak, args.min_time, args.min_repeats)
+    layer_us = [r["us"] for r in per_layer]
 
     # end to end through the binding with host buffers: every step copies its inputs from pinned host memory, runs, and
     # copies its result back to pinned host memory.  Copies run on their own streams, ordered against the compute stream
-    # with events per pool slot, so the H2D of step k+1 and the D2H of step k-1 overlap step k (as a serving loop would).
-    e2e_steps = min(K, 50)
-    host_in = [[x.cpu().pin_memory() for x in xs] if xs is not None else None for xs in wk.x_pool]
-    host_out = [torch.empty(wk.y_pool[-1][0].shape, dtype=torch.int8).pin_memory() for _ in range(pool)]
+    # with events per slot, so the H2D of step k+1 and the D2H of step k-1 overlap step k (as a serving loop would).
+    e2e_steps = max(4, min(K, 50))
+    host_in = [[xs[j % len(xs)].cpu().pin_memory() for j in range(cyc)] if xs is not None else None for xs in wk.x_pool]
+    host_out = [torch.empty(wk.y_pool[-1][0].shape, dtype=torch.int8).pin_memory() for _ in range(cyc)]
     s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-    ev_in = [torch.cuda.Event() for _ in range(pool)]
-    ev_done = [torch.cuda.Event() for _ in range(pool)]
-    ev_out = [torch.cuda.Event() for _ in range(pool)]
+    ev_in = [torch.cuda.Event() for _ in range(cyc)]
+    ev_done = [torch.cuda.Event() for _ in range(cyc)]
+    ev_out = [torch.cuda.Event() for _ in range(cyc)]
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     t0 = time.perf_counter()
     for k in range(e2e_steps):
-        j = k % pool
+        j = k % cyc
         with torch.cuda.stream(s_in):
-            if k >= pool:
+            if k >= cyc:
                 s_in.wait_event(ev_done[j])          # the step that last read this slot's inputs has finished
             for i in range(n_layers):
                 if host_in[i] is not None:
                     wk.x_pool[i][j].copy_(host_in[i][j], non_blocking=True)
             ev_in[j].record(s_in)
         stream.wait_event(ev_in[j])
-        if k >= pool:
+        if k >= cyc:
             stream.wait_event(ev_out[j])             # the slot's previous result has left the device
-        wk.step(stream, j)
+        wk.step(stream, j, exchange=exchange)
         ev_done[j].record(stream)
         with torch.cuda.stream(s_out):
             s_out.wait_event(ev_done[j])
-            host_out[j].copy_(wk.y_pool[-1][j], non_blocking=True)
+            host_out[j].copy_(wk.y_pool[-1][j % wk.pool[-1]], non_blocking=True)
             ev_out[j].record(s_out)
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+    del host_in, host_out
     assert ctx.get_async_error() == 0, "a device-side wait expired during the benchmark"
-
     if dist is not None:
-        t = torch.tensor([ms_total, ms_dyn, e2e_ms], device=dev, dtype=torch.float64)
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_dyn, e2e_ms = t.tolist()
+        e2e_ms = float(t.item())
 
-    ms_step = ms_total / K
-    tops = wk.ops * world / (ms_step * 1e-3) / 1e12
+    # the other configurations: per-layer rows and a step value each (rank 0 of a single-GPU run only)
+    other = {}
+    if args.all_configs and world == 1:
+        ops_main, static_main, dyn_main = wk.ops, list(wk.static_bytes), list(wk.dynamic_bytes)
+        layers_main = list(wk.layers)
+        wk.release()
+        del g_full, g_single, g_dyn, g_dyn_single
+        torch.cuda.empty_cache()
+        for cfg in [c for c in ("cfg1", "cfg2", "cfg3", "cfg4") if c != name]:
+            w2 = GpuWorkload(cfg, ctx, dev, seed_key=rank)
+            for j in range(2):
+                w2.step(stream, j, dynamic=True)
+            torch.cuda.synchronize()
+            w2.step(stream, 0)
+            torch.cuda.synchronize()
+            cyc2 = 2 if w2.chained else max(w2.pool)
+            gs = capture(torch, lambda s, j: w2.step(s, j), cyc2)
+            gd = capture(torch, lambda s, j: w2.step(s, j, dynamic=True), cyc2)
+            for _ in range(3):
+                gs.replay(); gd.replay()
+            ms2, lo2, hi2, r2 = timed_repeats(torch, gs.replay, cyc2, args.min_time, args.min_repeats)
+            msd2, _, _, _ = timed_repeats(torch, gd.replay, cyc2, args.min_time, args.min_repeats)
+            del gs, gd
+            per_layer += layer_rows(torch, w2, cfg, peaks, probe_peak, args.min_time, args.min_repeats)
+            other[cfg] = {"workload": f"{cfg}: " + ", ".join(s.name for _, s, _ in w2.layers), "value": round(w2.ops / (ms2 * 1e-3) / 1e12, 3),
+                          "unit": "TOPS", "ms_per_step": round(ms2, 6), "ms_per_step_min": round(lo2, 6), "ms_per_step_max": round(hi2, 6),
+                          "repeats": r2, "steps_per_repeat": cyc2,
+                          "dynamic": {"value": round(w2.ops / (msd2 * 1e-3) / 1e12, 3), "ms_per_step": round(msd2, 6)},
+                          "hbm_bytes_per_step": {"hindsight": int(sum(w2.static_bytes)), "dynamic": int(sum(w2.dynamic_bytes))}}
+            assert ctx.get_async_error() == 0, f"a device-side wait expired during {cfg}"
+            w2.release()
+            del w2
+            torch.cuda.empty_cache()
+        wk_ops, wk_static, wk_dynamic, wk_layers = ops_main, static_main, dyn_main, layers_main
+    else:
+        wk_ops, wk_static, wk_dynamic, wk_layers = wk.ops, wk.static_bytes, wk.dynamic_bytes, wk.layers
+    sampler.stop_flag = True
+    sampler.join(timeout=2)
+
+    tops = wk_ops * world / (ms_step * 1e-3) / 1e12
     int8_peak = peaks["bf16_tflops"] * NOMINAL_INT8_OVER_BF16
     hbm_peak = peaks["hbm_gbs"]
-    per_layer = []
-    for i, (kind, s, _) in enumerate(wk.layers):
-        us, usd = layer_us[i], layer_dyn_us[i]
-        t_tensor = s.ops / (int8_peak * 1e12) * 1e6
-        t_hbm = wk.static_bytes[i] / (hbm_peak * 1e9) * 1e6
-        per_layer.append({
-            "layer": s.name, "kind": kind, "us": round(us, 3), "us_dynamic": round(usd, 3),
-            "tops": round(s.ops / us / 1e6, 2), "gbs": round(wk.static_bytes[i] / us / 1e3, 1),
-            "gbs_dynamic": round(wk.dynamic_bytes[i] / usd / 1e3, 1),
-            "hbm_bytes_hindsight": int(wk.static_bytes[i]), "hbm_bytes_dynamic": int(wk.dynamic_bytes[i]),
-            "bound": "alu-or-hbm" if getattr(s, "depthwise", False) else ("tensor" if t_tensor >= t_hbm else "hbm"),
-            "frac_tensor": None if getattr(s, "depthwise", False) else round(t_tensor / us, 4), "frac_hbm": round(t_hbm / us, 4),
-        })
-    # dominant kernel of the step = the layer with the longest measured duration
+    # dominant kernel of the step = the layer with the longest measured launch
     dom = max(range(n_layers), key=lambda i: layer_us[i])
-    kind, s, _ = wk.layers[dom]
+    kind, s, _ = wk_layers[dom]
     t_tensor = s.ops / (int8_peak * 1e12) * 1e6
-    t_hbm = wk.static_bytes[dom] / (hbm_peak * 1e9) * 1e6
-    if getattr(s, "depthwise", False) or t_hbm > t_tensor:
-        ach = wk.static_bytes[dom] / layer_us[dom] / 1e3
-        roof = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s", "frac": round(ach / hbm_peak, 4)}
+    t_hbm = wk_static[dom] / (hbm_peak * 1e9) * 1e6
+    dw = getattr(s, "depthwise", False)
+    if dw or t_hbm > t_tensor:
+        ach = wk_static[dom] / layer_us[dom] / 1e3
+        roof = {"bound": "hbm", "achieved": round(ach, 1), "peak": hbm_peak, "unit": "GB/s", "frac": round(ach / hbm_peak, 4),
+                "peak_source": f"{peak_kind} copy bandwidth"}
     else:
         ach = s.ops / layer_us[dom] / 1e6
-        roof = {"bound": "tensor", "achieved": round(ach, 1), "peak": round(int8_peak, 1), "unit": "TOP/s", "frac": round(ach / int8_peak, 4)}
-    roof.update({"kernel": "depthwise_kernel" if getattr(s, "depthwise", False) else "hq_gemm_kernel", "layer": s.name,
-                 "launch_us": round(layer_us[dom], 3), "traffic": NCU_TRAFFIC.get(s.name), "peak_source": f"{peak_kind} (int8 = bf16 burst x {NOMINAL_INT8_OVER_BF16})",
+        roof = {"bound": "tensor", "achieved": round(ach, 1), "peak": round(int8_peak, 1), "unit": "TOP/s", "frac": round(ach / int8_peak, 4),
+                "peak_source": f"{peak_kind} bf16 burst x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)",
+                "frac_of_mma_probe": None if not probe_peak else round(ach / probe_peak, 4)}
+    tr = NCU_TRAFFIC.get(s.name)
+    roof.update({"kernel": KERNEL_OF.get(s.name, "depthwise3x3_tiled_kernel" if dw else "hq_gemm_kernel"), "layer": s.name,
+                 "launch_us": round(layer_us[dom], 3), "algorithmic_bytes": int(wk_static[dom]), "traffic": tr,
                  "frac_of": f"of {peak_kind}"})
 
     out = {
         "metric": METRIC, "value": round(tops, 3), "unit": "TOPS", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": round(ms_step, 6), "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
         "data": "synthetic", "impl": "hq",
-        "config": {"workload": f"{name}: " + ", ".join(s.name for _, s, _ in wk.layers), "path": "in-hindsight (static requant in the epilogue + min/max)",
-                   "l2": f"inputs and outputs rotate over a pool of {pool} buffer sets (> L2) inside CUDA graphs", "eta": 0.9,
+        "config": {"workload": f"{name}: " + ", ".join(s.name for _, s, _ in wk_layers), "path": "in-hindsight (static requant in the epilogue + min/max)",
+                   "l2": "every layer's inputs, outputs and workspaces rotate over a pool of buffer sets whose cycle moves more than L2 (192 MB); "
+                         "a whole step moves about 1 GB",
+                   "eta": 0.9,
                    "launch": "ordinary" if args.no_overlap else "programmatic stream serialization",
                    "rounding": "nearest even" if args.rounding == "nearest" else "stochastic for gradient layers, nearest even otherwise",
-                   "parallelism": f"dp{world} (batch shards; one int32 min/max all-reduce per step before the range update)" if world > 1 else "dp1"},
-        "gpu_launches": int(launches_per_step * K),
+                   "parallelism": f"dp{world} (batch shards; one int32 min/max all-reduce per step before the range update, inside the captured step)" if world > 1 else "dp1"},
+        "timing": {"repeats": repeats, "steps_per_repeat": K, "ms_per_step_min": round(ms_lo, 6), "ms_per_step_max": round(ms_hi, 6),
+                   "min_time_s": args.min_time, "statistic": "median over repeats; each repeat is exactly `steps` steps between its own CUDA events",
+                   "sm_mhz_during_steps": step_clocks["sm_mhz"],
+                   "ms_per_step_x_sm_mhz": None if not step_clocks["sm_mhz"] else round(ms_step * step_clocks["sm_mhz"], 3)},
+        "gpu_launches": int(launches_per_step * K * repeats),
         "launches_per_step": int(launches_per_step),
-        "dynamic": {"value": round(wk.ops * world / (ms_dyn / K * 1e-3) / 1e12, 3), "unit": "TOPS", "ms_per_step": round(ms_dyn / K, 6)},
-        "hbm_bytes_per_step": {"hindsight": int(sum(wk.static_bytes)), "dynamic": int(sum(wk.dynamic_bytes))},
+        "dynamic": {"value": round(wk_ops * world / (ms_dyn * 1e-3) / 1e12, 3), "unit": "TOPS", "ms_per_step": round(ms_dyn, 6)},
+        "hbm_bytes_per_step": {"hindsight": int(sum(wk_static)), "dynamic": int(sum(wk_dynamic))},
         "layers": per_layer,
         "roofline": roof,
-        "e2e": {"value": round(wk.ops * world / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
+        "e2e": {"value": round(wk_ops * world / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
                 "h2d_bytes_per_step": int(wk.h2d_bytes), "d2h_bytes_per_step": int(wk.d2h_bytes), "steps": e2e_steps},
         "clocks": sampler.summary(),
     }
+    if other:
+        out["configs"] = other
+    if probe:
+        out["int8_mma_probe"] = probe
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, ms, cores, sample = run_oracle(name, steps=3, warmup=1, budget_s=12.0)
         out["cpu_baseline"] = {"value": round(v, 5), "unit": "TOPS", "cores": cores, "kind": "oracle", "sample": sample}
@@ -535,14 +700,13 @@ def run_wgrad(args):
     launches = ctx.launch_count() - l0
     torch.cuda.synchronize()
     g_full = capture(torch, call, pool)
-    g_single = [capture(torch, lambda s_, _j, jj=j: call(s_, jj), 1) for j in range(pool)]
     for _ in range(-(-W // pool)):
         g_full.replay()
     torch.cuda.synchronize()
     sampler = ClockSampler(0)
     sampler.start()
     time.sleep(0.15)
-    ms_total = time_graph(torch, g_full, g_single, Ksteps, pool)
+    ms_step, ms_lo, ms_hi, repeats = timed_repeats(torch, g_full.replay, pool, args.min_time, args.min_repeats)
     sampler.stop_flag = True
     sampler.join(timeout=2)
     # end to end with host buffers: both operands in from pinned memory, the gradient out to pinned memory
@@ -562,7 +726,6 @@ def run_wgrad(args):
     assert ctx.get_async_error() == 0
     ops = 2.0 * M * N * K
     nbytes = int(np.prod(dy_shape)) + int(np.prod(x_shape)) + 4 * int(np.prod(gw_shape))   # int8 dY and X in, binary32 G_W out
-    ms_step = ms_total / Ksteps
     ach = nbytes / (ms_step * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": round(ops / (ms_step * 1e-3) / 1e12, 3), "unit": "TOPS", "n_gpus": 1, "steps": Ksteps, "warmup": W,
@@ -570,7 +733,9 @@ def run_wgrad(args):
         "impl": "hq",
         "config": {"workload": label, "path": path,
                    "l2": f"operands and results rotate over a pool of {pool} buffer sets (> L2) inside CUDA graphs", "parallelism": "dp1"},
-        "gpu_launches": int(launches * Ksteps), "launches_per_step": int(launches),
+        "timing": {"repeats": repeats, "steps_per_repeat": pool, "ms_per_step_min": round(ms_lo, 6), "ms_per_step_max": round(ms_hi, 6),
+                   "statistic": "median over repeats of one cycle through the buffer pool"},
+        "gpu_launches": int(launches * pool * repeats), "launches_per_step": int(launches),
         "hbm_bytes_per_step": {"algorithmic": int(nbytes)},
         "roofline": {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
                      "kernel": ("dw_wgrad_kernel" if cs.depthwise else "im2col_t_kernel + hq_gemm_kernel (int32 slabs) + wgrad_reduce_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
@@ -600,6 +765,9 @@ def run_wgrad(args):
 
 
 def run_profile(args):
+    """Eager launches only, for a profiler.  The ranges are initialised by one dynamic step per pool slot; then, for the
+    chosen layer (--layer NAME; all layers when absent), --steps in-hindsight launches rotate through the layer's buffer
+    pool (more than L2, so that earlier outputs are evicted to DRAM while later launches run), then --steps dynamic ones."""
     import torch
     from paper_2105_04246_b200 import hq
     dev = torch.device("cuda", 0)
@@ -608,19 +776,25 @@ def run_profile(args):
     if args.no_overlap:
         ctx.set_option("overlap_launches", 0)
     ctx.set_option("depthwise", args.depthwise)
-    wk = GpuWorkload(args.workload, ctx, dev, 2, seed_key=0, stochastic=args.rounding == "stochastic")
+    wk = GpuWorkload(args.workload, ctx, dev, seed_key=0, stochastic=args.rounding == "stochastic", pool_cap=args.pool_cap)
     stream = torch.cuda.current_stream(dev)
-    for j in range(2):
+    names = [s.name for _, s, _ in wk.layers]
+    sel = [i for i, n in enumerate(names) if args.layer in (None, n)]
+    if not sel:
+        raise SystemExit(f"no layer named {args.layer} in {args.workload}: {names}")
+    for j in range(max(wk.pool[i] for i in sel) if not wk.chained else 2):
         wk.step(stream, j, dynamic=True)
     torch.cuda.synchronize()
     for k in range(args.steps):
-        wk.step(stream, k % 2)
+        wk.step(stream, k, update=False) if args.layer is None else [wk.layer_call(stream, i, k) for i in sel]
     torch.cuda.synchronize()
-    for k in range(args.steps):
-        wk.step(stream, k % 2, dynamic=True)
-    torch.cuda.synchronize()
+    if not args.no_dynamic:
+        for k in range(args.steps):
+            wk.step(stream, k, dynamic=True) if args.layer is None else [wk.layer_call(stream, i, k, dynamic=True) for i in sel]
+        torch.cuda.synchronize()
     assert ctx.get_async_error() == 0
-    print(json.dumps({"profile": args.workload, "steps": args.steps, "launches": ctx.launch_count()}))
+    print(json.dumps({"profile": args.workload, "layer": args.layer, "steps": args.steps, "pool": [wk.pool[i] for i in sel],
+                      "launches": ctx.launch_count()}))
 
 
 def run_reference(args):
@@ -643,10 +817,10 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=600)
-    ap.add_argument("--warmup", type=int, default=24)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="hq", choices=["hq", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad", "wgrad_conv", "wgrad_dw"],
+    ap.add_argument("--workload", default="cfg5", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg4b", "cfg5", "wgrad", "wgrad_conv", "wgrad_dw"],
                     help="cfg1..cfg5: the five layer workloads; cfg4b: backward data through cfg4's block; wgrad: the weight gradient "
                          "of a linear layer (a later row of the scope)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -657,9 +831,20 @@ def main():
     ap.add_argument("--no-overlap", action="store_true",
                     help="ordinary launches instead of programmatic stream serialization (set-up of a kernel overlapping its predecessor's tail)")
     ap.add_argument("--profile", action="store_true",
-                    help="eager launches only, for a profiler: pool of 2; one dynamic step per pool member (initialises the ranges), "
-                         "then --steps in-hindsight steps, then --steps dynamic steps")
+                    help="eager launches only, for a profiler: one dynamic step per pool slot (initialises the ranges), then --steps "
+                         "in-hindsight launches of --layer (or whole steps), then as many dynamic ones")
+    ap.add_argument("--layer", default=None, help="--profile: only this layer of the workload")
+    ap.add_argument("--no-dynamic", action="store_true", help="--profile: leave the dynamic launches out")
+    ap.add_argument("--pool-cap", type=int, default=MAX_POOL, help="--profile: at most this many buffer sets per layer")
+    ap.add_argument("--min-time", type=float, default=0.2, help="every measurement repeats until this many seconds have been timed")
+    ap.add_argument("--min-repeats", type=int, default=5, help="and at least this often; the median over the repeats is reported")
+    ap.add_argument("--no-probe", action="store_true", help="skip the int8 MMA-only throughput probe")
+    ap.add_argument("--probe-seconds", type=float, default=4.0, help="length of the probe's sustained run")
+    ap.add_argument("--only", dest="all_configs", action="store_false",
+                    help="time --workload alone; by default the per-layer rows and step values of the other four configurations are appended")
     args = ap.parse_args()
+    if args.impl == "hq" and args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.profile:
+        sys.exit(spawn_ranks(args))
     if args.workload in ("wgrad", "wgrad_conv", "wgrad_dw") and args.impl == "hq" and not args.profile:
         run_wgrad(args)
     elif args.impl == "reference":

@@ -21,7 +21,16 @@
  *     context, prepared weights and their internal tables.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Layer,
  *     update and dynamic calls only enqueue work: they do not synchronise and read every
- *     quantization parameter from device memory.
+ *     quantization parameter from device memory.  The exceptions are spelled out at the calls
+ *     concerned: a call that first meets a shape needing more context-owned scratch than the
+ *     context holds grows it with cudaFree + cudaMalloc (which synchronise the device), so make
+ *     the first call of each such shape outside stream capture and timed regions.
+ *   - The context's device must be the current device for every call that launches work
+ *     (HQ_ERR_INVALID_ARG otherwise).
+ *   - Context-owned scratch is shared by the calls of one context: the column sums of
+ *     hq_linear_fwd / hq_dynamic_quant(linear), the padded copies for K % 16 != 0, and the
+ *     weight-gradient scratch.  Calls of ONE context that use the same scratch must not overlap
+ *     on the GPU (different streams); use one context per stream for that.
  *   - Arguments are validated before anything is launched; a rejected call launches
  *     nothing and hq_last_error() holds a HOST string describing the reason.
  *   - Every device-side wait is bounded.  If one expires the kernel records a code in the
@@ -252,6 +261,16 @@ hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
  * A state whose slot is empty is left untouched. */
 hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, float eta);
 
+/* Batch-sharded data parallelism (each GPU runs the layer calls on its slice of the batch with the same weights and
+ * the same range states): Sec. 4.1 takes min/max over the WHOLE tensor, so the statistics slots are merged over the
+ * ranks before hq_range_update.  hq_stats_pack writes acc_min of the `count` states to buf[0 .. count) and the bitwise
+ * complement of acc_max to buf[count .. 2*count) (DEVICE, int32); one element-wise MIN all-reduce of buf over the ranks
+ * (NCCL, on the same stream) then merges both columns, the complement turning max into min without overflow and an
+ * empty slot being the identity; hq_stats_unpack writes the merged pair back.  Every rank then applies Eq. 2-3 to the
+ * same numbers, so the replicated states stay bit-identical.  Both calls only enqueue one small kernel. */
+hq_status hq_stats_pack(hq_ctx* ctx, void* stream, const hq_range_state* states, int32_t count, int32_t* buf);
+hq_status hq_stats_unpack(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, const int32_t* buf);
+
 /* Dynamic quantization of the same layer (Sec. 3.2, Eq. 1; traffic of Eq. 5): kernel 1 runs the
  * layer's MAC loop and writes y = float(acc) * s_acc as binary32 to `workspace` (caller-owned,
  * one float per output element) while reducing min/max; kernel 2 sets q_min/q_max of *yq to the
@@ -271,12 +290,15 @@ hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op,
  * process whose device memory was handed out in full at start-up -- and that therefore cannot
  * provide the one-float-per-output workspace of hq_dynamic_quant.  Here the workspace is a fixed device array that is part of the library image:
  * every GPU that loads the library sets aside HQ_STATIC_WORKSPACE_ELEMS floats (16 MiB) for it until
- * the process exits.  The call itself allocates and frees nothing, neither through CUDA nor through
- * any other library.
+ * the process exits.  The call itself allocates and frees nothing: no device memory, through CUDA or any other
+ * library, and no host memory either (its launch planning uses fixed-size tables, and a rejected call writes its
+ * reason into a fixed buffer of the context).
  *   - Same operands, results and status codes as hq_dynamic_quant; Y and *yq are still the caller's.
  *   - Outputs of more than HQ_STATIC_WORKSPACE_ELEMS elements are rejected with HQ_ERR_UNSUPPORTED
- *     before anything is launched; so is a linear layer whose N exceeds the column-sum scratch the
- *     context allocated when it was created (4096 columns).
+ *     before anything is launched.  So is a linear layer that needs more context scratch than the context
+ *     holds at the time of the call: column sums for more than 4096 output columns (unless an earlier
+ *     hq_linear_fwd / hq_dynamic_quant on this context already grew that scratch), or K that is not a multiple
+ *     of 16 (padded operand copies, unless an earlier call already made room for this size).
  *   - The context's device must be the current device.  The first call on a device looks up the
  *     array's device address (a host-side query, no launch); make that first call before starting
  *     any stream capture.
@@ -285,6 +307,14 @@ hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op,
  *     calls that overlap on the GPU -- different streams, or different contexts on the same device --
  *     race on it.  Serialise them. */
 hq_status hq_dynamic_quant_static(hq_ctx* ctx, void* stream, const hq_op_desc* op, int8_t* Y, hq_range_state* yq);
+
+/* Measurement hook (the paper has no counterpart): enqueues one kernel in which every SM -- pair = 0: one CTA per SM,
+ * 128 x bn x 32 per instruction; pair = 1: one CTA pair per two SMs, 256 x bn x 32 -- issues `chunks` x 32 int8
+ * tensor-core instructions (the MAC of Sec. 3.1 and nothing else) on operand tiles that stay in shared memory: no loads,
+ * no epilogue.  *ops (HOST, may be NULL) receives the 2 x MAC count of the launch; the caller times the launch with
+ * events.  This is the "int8 MMA peak as measured on this GPU" that the layer kernels' tensor roofline is quoted against.
+ * bn: a multiple of 32, at most 256. */
+hq_status hq_mma_peak_probe(hq_ctx* ctx, void* stream, int32_t pair, int32_t bn, int32_t chunks, uint64_t* ops);
 
 /* Test hook: writes the zero-point-corrected int32 accumulator (+bias) of the layer to `acc`
  * (one int32 per output element) and merges its min/max into *yq.  The hot path never

@@ -6,6 +6,7 @@
 #include <stddef.h>
 #include <stdint.h>
 #include <stdio.h>
+#include <string.h>
 
 #include <algorithm>
 #include <functional>
@@ -22,12 +23,10 @@ namespace {
 
 hq_status fail(hq_ctx* ctx, hq_status s, const char* fmt, ...) {
   if (ctx) {
-    char buf[512];
     va_list ap;
     va_start(ap, fmt);
-    vsnprintf(buf, sizeof(buf), fmt, ap);
+    vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
     va_end(ap);
-    ctx->err = buf;
   }
   return s;
 }
@@ -37,6 +36,15 @@ hq_status fail(hq_ctx* ctx, hq_status s, const char* fmt, ...) {
     cudaError_t e__ = (expr);                                                                                \
     if (e__ != cudaSuccess) return fail(ctx, HQ_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e__)); \
   } while (0)
+
+// Every launching entry point runs on the context's device: with another device current the kernels would be launched
+// there, against pointers that device may not even map.  A host-side query, no launch.
+hq_status check_device(hq_ctx* ctx) {
+  int cur = -1;
+  HQ_CUDA(ctx, cudaGetDevice(&cur));
+  if (cur != ctx->device) return fail(ctx, HQ_ERR_INVALID_ARG, "device %d must be current (device %d is)", ctx->device, cur);
+  return HQ_OK;
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -62,7 +70,7 @@ bool same_desc(const hq_conv_desc& a, const hq_conv_desc& b) {
 }
 
 // border classes of one tile-space axis: which taps of `d` fall inside [0, a_dim) at position i
-void border_classes(int T, int in_mul, const std::vector<int>& d, int a_dim, std::vector<uint8_t>& cls, std::vector<uint32_t>& masks) {
+void border_classes(int T, int in_mul, const TapVec& d, int a_dim, std::vector<uint8_t>& cls, MaskVec& masks) {
   cls.assign(T, 0);
   masks.clear();
   for (int i = 0; i < T; ++i) {
@@ -110,7 +118,7 @@ FastDiv make_fastdiv(int d) {
 struct SubSpec {            // geometry of one launch, before tiling
   int n_img, TH, TW;
   int in_mul_h, in_mul_w;
-  std::vector<int> dh, dw;  // tap offsets per axis (taps = product, row-major)
+  TapVec dh, dw;            // tap offsets per axis (taps = product, row-major)
   int a_H, a_W;             // image size of operand A (for border classes)
   int Cin;                  // reduction length per tap
   int Nout;
@@ -125,7 +133,7 @@ struct SubSpec {            // geometry of one launch, before tiling
 // fills everything in sub.p that does not depend on per-call pointers, for a given number of column tiles
 // (ncol_req = 0: as few as the MMA allows) and a given answer to "CTA pairs?" (pair_req: 0 no, 1 where the layer allows)
 hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
-                         std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks, int ncol_req, int pair_req) {
+                         MaskVec& rowmasks, MaskVec& colmasks, int ncol_req, int pair_req) {
   GemmParams& p = sub.p;
   p.n_img = sp.n_img;
   p.TH = sp.TH;
@@ -341,14 +349,14 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
 //    as many column tiles as still fit in one round, none narrower than 64 columns.  Everywhere else splitting the
 //    columns multiplies the traffic of operand A and is much slower.
 hq_status plan_sub(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, std::vector<uint8_t>& rowcls, std::vector<uint8_t>& colcls,
-                   std::vector<uint32_t>& rowmasks, std::vector<uint32_t>& colmasks) {
+                   MaskVec& rowmasks, MaskVec& colmasks) {
   if (sp.flat) return plan_sub_fixed(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks, std::max(0, ctx->force_cols), 0);
   int ncol = std::max(0, ctx->force_cols);
   int pair = ctx->force_pair;
   if (ctx->force_cols < 0 || ctx->force_pair < 0) {
     hq_sub_problem trial = sub;
     std::vector<uint8_t> rc, cc;
-    std::vector<uint32_t> rm, cm;
+    MaskVec rm, cm;
     hq_status st = plan_sub_fixed(ctx, sp, trial, rc, cc, rm, cm, ncol, 0);
     if (st != HQ_OK) return st;
     const GemmParams& t = trial.p;
@@ -445,7 +453,7 @@ hq_status build_sub(hq_ctx* ctx, hq_prepared_weights* pw, cudaStream_t s, const 
   hq_sub_problem& sub = pw->subs.back();
   sub.gfold = gfold;
   std::vector<uint8_t> rowcls, colcls;
-  std::vector<uint32_t> rowmasks, colmasks;
+  MaskVec rowmasks, colmasks;
   hq_status st = plan_sub(ctx, sp, sub, rowcls, colcls, rowmasks, colmasks);
   if (st != HQ_OK) return st;
   GemmParams& p = sub.p;
@@ -611,20 +619,35 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     HQ_CUDA(ctx, cudaEventRecord(ctx->ev_fork, s));
   }
   int sub_index = -1;
+  int forked = 0;   // side streams that wait on the fork event so far
   auto join = [&]() -> hq_status {
     if (!side_by_side) return HQ_OK;
-    for (int k = 0; k < std::min(nsub - 1, 3); ++k) {
+    for (int k = 0; k < forked; ++k) {
       HQ_CUDA(ctx, cudaEventRecord(ctx->ev_join[k], ctx->side[k]));
       HQ_CUDA(ctx, cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
     }
     return HQ_OK;
+  };
+  // A failure after the fork still joins the side streams first: what they already run is then ordered before the
+  // caller's later work on `stream`, and a stream capture is not left with an unjoined branch.  The first error is
+  // the one reported (its text is kept across the join).
+  auto join_after = [&](hq_status e) -> hq_status {
+    char keep[sizeof(ctx->err)];
+    memcpy(keep, ctx->err, sizeof(keep));
+    (void)join();
+    memcpy(ctx->err, keep, sizeof(keep));
+    return e;
   };
   for (const hq_sub_problem& sub : pw->subs) {
     ++sub_index;
     cudaStream_t ss = s;
     if (side_by_side && sub_index > 0) {
       ss = ctx->side[(sub_index - 1) % 3];
-      if (sub_index <= 3) HQ_CUDA(ctx, cudaStreamWaitEvent(ss, ctx->ev_fork, 0));
+      if (sub_index <= 3) {
+        const cudaError_t we = cudaStreamWaitEvent(ss, ctx->ev_fork, 0);
+        if (we != cudaSuccess) return join_after(fail(ctx, HQ_ERR_CUDA, "cudaStreamWaitEvent failed: %s", cudaGetErrorString(we)));
+        ++forked;
+      }
     }
     const int max_ctas = side_by_side ? share[sub_index] : 0;
     CUtensorMap ta;
@@ -632,22 +655,24 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       ta = CUtensorMap{};
     } else if (sub.patch_matrix != nullptr) {
       // channel counts that no TMA box can address (C = 3): gather the filter windows into rows first
-      HQ_CUDA(ctx, launch_patch_matrix(in, sub.patch_matrix, inq, desc->N, desc->H, desc->W, desc->C, Ho, Wo, desc->R, desc->S, desc->stride_h,
-                                       desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, sub.patch_RP, s));
+      const cudaError_t pe = launch_patch_matrix(in, sub.patch_matrix, inq, desc->N, desc->H, desc->W, desc->C, Ho, Wo, desc->R, desc->S,
+                                                 desc->stride_h, desc->stride_w, desc->pad_h, desc->pad_w, sub.patch_K, sub.patch_RP, s);
+      if (pe != cudaSuccess) return join_after(fail(ctx, HQ_ERR_CUDA, "patch gather launch failed: %s", cudaGetErrorString(pe)));
       ctx->launches += 1;
       st = encode_a(ctx, sub, sub.patch_matrix, sub.patch_K, desc->N * Ho * Wo, 1, 1, &ta);
     } else if (sub.window != nullptr) {
-      HQ_CUDA(ctx, launch_row_window(in, sub.window, inq, desc->N, desc->H, desc->W, desc->C, sub.win_Hg, Wo, desc->S, sub.win_sh,
-                                     desc->stride_w, desc->pad_w, sub.win_SB, s));
+      const cudaError_t we = launch_row_window(in, sub.window, inq, desc->N, desc->H, desc->W, desc->C, sub.win_Hg, Wo, desc->S, sub.win_sh,
+                                               desc->stride_w, desc->pad_w, sub.win_SB, s);
+      if (we != cudaSuccess) return join_after(fail(ctx, HQ_ERR_CUDA, "window gather launch failed: %s", cudaGetErrorString(we)));
       ctx->launches += 1;
       st = encode_a(ctx, sub, sub.window, sub.win_sh * sub.win_SB, Wo, sub.win_Hg, desc->N, &ta);
     } else if (sub.chans > 0) {
       // depthwise: this launch is the dense layer over the channel slice [chan0, chan0 + chans) of input and output
       st = encode_a(ctx, sub, in + sub.chan0, sub.chans, aW, aH, desc->N, &ta, desc->C);
-      if (st != HQ_OK) return st;
+      if (st != HQ_OK) return join_after(st);
       void* o = out_mode == kOutInt8 ? (void*)((int8_t*)out + sub.chan0) : (void*)((uint32_t*)out + sub.chan0);
       st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas, weights_early);
-      if (st != HQ_OK) return st;
+      if (st != HQ_OK) return join_after(st);
       continue;
     } else if (sub.a_flat) {
       const int64_t rows = (int64_t)desc->N * aH * aW / sub.gfold;
@@ -655,15 +680,16 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     } else {
       st = encode_a(ctx, sub, in, aC, aW, aH, desc->N, &ta);
     }
-    if (st != HQ_OK) return st;
-    st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas, weights_early);
-    if (st != HQ_OK) return st;
+    if (st == HQ_OK) st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas, weights_early);
+    if (st != HQ_OK) return join_after(st);
   }
   return join();
 }
 
 hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
-                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, const int32_t* row_term = nullptr) {
+                     const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, const int32_t* row_term = nullptr,
+                     bool no_grow = false) {
+  // no_grow: the call may not allocate; shapes that would need larger context scratch are refused instead
   if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
   if (!X || !xq || !W || !w_scale || !out || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(X) || !aligned16(W) || !aligned16(out) || !aligned16(xq) || !aligned16(yq))
@@ -672,6 +698,8 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
     // rows whose length no TMA box can address: zero-padded copies of both operands in context-owned scratch
     const int Kp = round_up(K, 16);
     const size_t need = ((size_t)M + (size_t)N) * Kp;
+    if (need > ctx->pad_bytes && no_grow)
+      return fail(ctx, HQ_ERR_UNSUPPORTED, "K = %d: rows that are not a multiple of 16 bytes need %zu bytes of padded copies; the context holds %zu and this call may not allocate", K, need, ctx->pad_bytes);
     if (need > ctx->pad_bytes) {
       if (ctx->d_pad) HQ_CUDA(ctx, cudaFree(ctx->d_pad));
       ctx->d_pad = nullptr;
@@ -694,9 +722,12 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
   sp.out_H = 1; sp.out_W = M; sp.os_h = 1; sp.os_w = 1; sp.oa_h = 0; sp.oa_w = 0; sp.ldY = N; sp.flat = true;
   hq_sub_problem sub;
   std::vector<uint8_t> rc, cc;
-  std::vector<uint32_t> rm, cm;
+  MaskVec rm, cm;
   hq_status st = plan_sub(ctx, sp, sub, rc, cc, rm, cm);
   if (st != HQ_OK) return st;
+  if ((size_t)sub.p.corr_ld > ctx->scratch_elems && no_grow)
+    return fail(ctx, HQ_ERR_UNSUPPORTED, "N = %d needs %d column sums; the context holds %zu and this call may not allocate", N, sub.p.corr_ld,
+                ctx->scratch_elems);
   if ((size_t)sub.p.corr_ld > ctx->scratch_elems) {
     if (ctx->d_scratch) HQ_CUDA(ctx, cudaFree(ctx->d_scratch));
     ctx->d_scratch = nullptr;
@@ -718,10 +749,11 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
   return launch_sub(ctx, s, sub, ta, tb, xq, w_scale, bias, out, yq, out_mode, 0, false, row_term);
 }
 
-hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, hq_range_state* yq, int out_mode) {
+hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, hq_range_state* yq, int out_mode, bool no_grow = false) {
   if (!op) return fail(ctx, HQ_ERR_INVALID_ARG, "operation descriptor is null");
   switch (op->kind) {
-    case HQ_OP_LINEAR: return run_linear(ctx, s, op->M, op->N, op->K, op->x, op->xq, op->w, op->w_scale, op->bias, out, yq, out_mode);
+    case HQ_OP_LINEAR:
+      return run_linear(ctx, s, op->M, op->N, op->K, op->x, op->xq, op->w, op->w_scale, op->bias, out, yq, out_mode, nullptr, no_grow);
     case HQ_OP_CONV_FWD: return run_conv(ctx, s, op->conv, HQ_DIR_FWD, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
     case HQ_OP_CONV_BWD_DATA: return run_conv(ctx, s, op->conv, HQ_DIR_BWD_DATA, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
     default: return fail(ctx, HQ_ERR_INVALID_ARG, "unknown operation kind %d", op->kind);
@@ -819,7 +851,7 @@ __attribute__((visibility("default"))) hq_status hq_destroy(hq_ctx* ctx) {
   return HQ_OK;
 }
 
-__attribute__((visibility("default"))) const char* hq_last_error(const hq_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+__attribute__((visibility("default"))) const char* hq_last_error(const hq_ctx* ctx) { return ctx ? ctx->err : "null context"; }
 
 __attribute__((visibility("default"))) uint64_t hq_launch_count(const hq_ctx* ctx) { return ctx ? ctx->launches : 0; }
 __attribute__((visibility("default"))) uint64_t hq_pair_launch_count(const hq_ctx* ctx) { return ctx ? ctx->pair_launches : 0; }
@@ -888,6 +920,7 @@ __attribute__((visibility("default"))) hq_status hq_get_async_error(hq_ctx* ctx,
 
 __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W, hq_prepared_weights** out) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (!out) return fail(ctx, HQ_ERR_INVALID_ARG, "out is null");
   *out = nullptr;
   hq_status st = check_desc(ctx, desc);
@@ -955,11 +988,11 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   }
   if (d.groups != 1 && !dw_dense) {
     pw->depthwise = true;
-    std::vector<int> dh, dw;
+    TapVec dh, dw;
     for (int r = 0; r < d.R; ++r) dh.push_back(r - dwd.pad_h);
     for (int q = 0; q < d.S; ++q) dw.push_back(q - dwd.pad_w);
     std::vector<uint8_t> rowcls, colcls;
-    std::vector<uint32_t> rm, cm;
+    MaskVec rm, cm;
     // output rows / columns of the layer the kernel runs (backward data: the input image of the original layer)
     const int run_Ho = out_dim(dwd.H, dwd.pad_h, dwd.R, dwd.stride_h), run_Wo = out_dim(dwd.W, dwd.pad_w, dwd.S, dwd.stride_w);
     border_classes(run_Ho, dwd.stride_h, dh, dwd.H, rowcls, rm);
@@ -1104,23 +1137,27 @@ __attribute__((visibility("default"))) hq_status hq_weights_release(hq_ctx* ctx,
 __attribute__((visibility("default"))) hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
                         const float* w_scale, const int32_t* bias, int8_t* Y, hq_range_state* yq) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   return run_linear(ctx, (cudaStream_t)stream, M, N, K, X, xq, W, w_scale, bias, Y, yq, kOutInt8);
 }
 
 __attribute__((visibility("default"))) hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* X, const hq_range_state* xq,
                       const hq_prepared_weights* pw, const float* w_scale, int8_t* Y, hq_range_state* yq) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   return run_conv(ctx, (cudaStream_t)stream, desc, HQ_DIR_FWD, X, xq, pw, w_scale, Y, yq, kOutInt8);
 }
 
 __attribute__((visibility("default"))) hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* dY, const hq_range_state* dyq,
                            const hq_prepared_weights* pw, const float* w_scale, int8_t* dX, hq_range_state* dxq) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   return run_conv(ctx, (cudaStream_t)stream, desc, HQ_DIR_BWD_DATA, dY, dyq, pw, w_scale, dX, dxq, kOutInt8);
 }
 
 __attribute__((visibility("default"))) hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, float eta) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (!states || count <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "states is null or count is not positive");
   if (!aligned16(states)) return fail(ctx, HQ_ERR_ALIGNMENT, "range states must be 16-byte aligned");
   if (!(eta >= 0.0f && eta <= 1.0f)) return fail(ctx, HQ_ERR_INVALID_ARG, "eta must lie in [0, 1]");
@@ -1129,8 +1166,39 @@ __attribute__((visibility("default"))) hq_status hq_range_update(hq_ctx* ctx, vo
   return HQ_OK;
 }
 
+__attribute__((visibility("default"))) hq_status hq_stats_pack(hq_ctx* ctx, void* stream, const hq_range_state* states, int32_t count, int32_t* buf) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
+  if (!states || !buf || count <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "states or buf is null, or count is not positive");
+  if (!aligned16(states)) return fail(ctx, HQ_ERR_ALIGNMENT, "range states must be 16-byte aligned");
+  HQ_CUDA(ctx, launch_stats_pack(states, count, buf, (cudaStream_t)stream));
+  ctx->launches += 1;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_stats_unpack(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, const int32_t* buf) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
+  if (!states || !buf || count <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "states or buf is null, or count is not positive");
+  if (!aligned16(states)) return fail(ctx, HQ_ERR_ALIGNMENT, "range states must be 16-byte aligned");
+  HQ_CUDA(ctx, launch_stats_unpack(states, count, buf, (cudaStream_t)stream));
+  ctx->launches += 1;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_mma_peak_probe(hq_ctx* ctx, void* stream, int32_t pair, int32_t bn, int32_t chunks, uint64_t* ops) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
+  if (pair < 0 || pair > 1 || chunks <= 0 || chunks > (1 << 20)) return fail(ctx, HQ_ERR_INVALID_ARG, "pair must be 0 or 1, chunks in [1, 2^20]");
+  if (bn < 32 || bn > 256 || bn % 32 != 0) return fail(ctx, HQ_ERR_INVALID_ARG, "bn must be a multiple of 32 in [32, 256]");
+  HQ_CUDA(ctx, launch_mma_peak(pair, bn, chunks, ctx->num_sms, ctx->d_status, (cudaStream_t)stream, ops));
+  ctx->launches += 1;
+  return HQ_OK;
+}
+
 __attribute__((visibility("default"))) hq_status hq_dynamic_quant(hq_ctx* ctx, void* stream, const hq_op_desc* op, float* workspace, int8_t* Y, hq_range_state* yq) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (!op || !workspace || !Y || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(workspace) || !aligned16(Y)) return fail(ctx, HQ_ERR_ALIGNMENT, "workspace and Y must be 16-byte aligned");
   cudaStream_t s = (cudaStream_t)stream;
@@ -1145,6 +1213,7 @@ __attribute__((visibility("default"))) hq_status hq_dynamic_quant(hq_ctx* ctx, v
 __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t K, const int8_t* dY,
                                                                  const hq_range_state* dyq, const int8_t* X, const hq_range_state* xq, float* GW) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
   if (!dY || !dyq || !X || !xq || !GW) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(dY) || !aligned16(X) || !aligned16(GW) || !aligned16(dyq) || !aligned16(xq))
@@ -1184,6 +1253,7 @@ __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, vo
 __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* dY,
                                                                const hq_range_state* dyq, const int8_t* X, const hq_range_state* xq, float* GW) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   hq_status st = check_desc(ctx, desc);
   if (st != HQ_OK) return st;
   if (!dY || !dyq || !X || !xq || !GW) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
@@ -1259,7 +1329,7 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   sp.slices = slices; sp.slice_len = slice_len;
   hq_sub_problem sub;
   std::vector<uint8_t> rc, cc;
-  std::vector<uint32_t> rm, cm;
+  MaskVec rm, cm;
   st = plan_sub(ctx, sp, sub, rc, cc, rm, cm);
   if (st != HQ_OK) return st;
   sub.p.corr = nullptr;       // both zero points are taken out after the slabs are summed
@@ -1287,6 +1357,7 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
 
 __attribute__((visibility("default"))) hq_status hq_debug_accumulate(hq_ctx* ctx, void* stream, const hq_op_desc* op, int32_t* acc, hq_range_state* yq) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (!op || !acc || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   return run_op(ctx, (cudaStream_t)stream, op, acc, yq, kOutAcc);
 }
@@ -1303,6 +1374,8 @@ static __device__ __align__(256) float hq_static_workspace[HQ_STATIC_WORKSPACE_E
 
 namespace {
 constexpr int kMaxDevices = 64;
+// Written without a lock: two host threads that make the first call on a device at the same time both store the same
+// address (the symbol's address on that device never changes), so the race is benign.
 float* g_static_ws[kMaxDevices] = {};
 
 hq_status static_workspace(hq_ctx* ctx, float** out) {
@@ -1331,27 +1404,19 @@ extern "C" __attribute__((visibility("default"))) hq_status hq_dynamic_quant_sta
     if (st != HQ_OK) return st;
   } else if (op->M <= 0 || op->N <= 0 || op->K <= 0) {
     return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
-  } else if (op->K % 16 != 0) {
-    return fail(ctx, HQ_ERR_UNSUPPORTED, "K = %d: rows that are not a multiple of 16 bytes need padded copies, which this call may not allocate",
-                op->K);
   }
   const int64_t elems = op_out_elems(op);
   if (elems > (int64_t)HQ_STATIC_WORKSPACE_ELEMS)
     return fail(ctx, HQ_ERR_UNSUPPORTED, "output has %lld elements; the built-in workspace holds at most %lld", (long long)elems,
                 (long long)HQ_STATIC_WORKSPACE_ELEMS);
-  if (op->kind == HQ_OP_LINEAR) {
-    // the column-sum scratch of the context is fixed here: it is never grown on this path
-    const int ncol = ceil_div(op->N, 256);
-    const int bn = round_up(ceil_div(op->N, ncol), 16);
-    if ((size_t)(ceil_div(op->N, bn) * bn) > ctx->scratch_elems)
-      return fail(ctx, HQ_ERR_UNSUPPORTED, "N = %d needs more column-sum scratch than the context holds (%zu)", op->N, ctx->scratch_elems);
-  }
   if (!aligned16(Y)) return fail(ctx, HQ_ERR_ALIGNMENT, "Y must be 16-byte aligned");
   float* ws = nullptr;
   hq_status st = static_workspace(ctx, &ws);
   if (st != HQ_OK) return st;
   cudaStream_t s = (cudaStream_t)stream;
-  st = run_op(ctx, s, op, ws, yq, kOutF32);
+  // the planner decides what the layer needs; with no_grow it refuses, before any launch, whatever the context's scratch
+  // (column sums of a linear layer's weights, padded operand copies) cannot hold as it stands
+  st = run_op(ctx, s, op, ws, yq, kOutF32, true);
   if (st != HQ_OK) return st;
   HQ_CUDA(ctx, launch_dynamic_derive(yq, s, ctx->overlap));
   HQ_CUDA(ctx, launch_quantize_pass(ws, Y, elems, yq, ctx->num_sms, s, false));

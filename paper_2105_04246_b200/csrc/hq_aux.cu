@@ -51,6 +51,23 @@ __global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
   s->acc_max = INT32_MIN;
 }
 
+// Batch-sharded data parallelism: the only exchange of the method is the statistics.  pack writes {acc_min, ~acc_max}
+// of every state into one int32 array (the complement reverses the order without overflow, so ONE element-wise MIN
+// all-reduce over the ranks serves both columns; an empty slot {INT32_MAX, INT32_MIN} is its identity); unpack puts the
+// reduced pair back, after which every rank applies Eq. 2-3 to identical numbers.
+__global__ void stats_pack_kernel(const hq_range_state* st, int count, int32_t* buf) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  buf[i] = st[i].acc_min;
+  buf[count + i] = ~st[i].acc_max;
+}
+__global__ void stats_unpack_kernel(hq_range_state* st, int count, const int32_t* buf) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  st[i].acc_min = buf[i];
+  st[i].acc_max = ~buf[count + i];
+}
+
 // Eq. 1: the range is the min/max of the tensor that was just written; with dynamic_eta > 0, its moving average.
 __global__ void dynamic_derive_kernel(hq_range_state* s) {
   grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
@@ -1009,6 +1026,15 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
 
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap) {
   return launch_overlapped(range_update_kernel, (count + 127) / 128, 128, 0, s, overlap, st, count, eta);
+}
+
+cudaError_t launch_stats_pack(const hq_range_state* st, int count, int32_t* buf, cudaStream_t s) {
+  stats_pack_kernel<<<(count + 127) / 128, 128, 0, s>>>(st, count, buf);
+  return cudaGetLastError();
+}
+cudaError_t launch_stats_unpack(hq_range_state* st, int count, const int32_t* buf, cudaStream_t s) {
+  stats_unpack_kernel<<<(count + 127) / 128, 128, 0, s>>>(st, count, buf);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overlap) {

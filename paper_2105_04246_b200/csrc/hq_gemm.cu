@@ -922,6 +922,90 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   }
 }
 
+
+// ---- measurement: what the tensor cores sustain on kind::i8 with nothing else in the way ---------------------------
+// One CTA (or CTA pair) per SM issues the same 128 x BN x 32 (pair: 256 x BN x 32) MMA on operand tiles that sit in
+// shared memory for the whole kernel: no loads, no epilogue.  MMAs go out in chunks of kProbeChunk, each chunk followed
+// by a commit; the issuer waits for the chunk before the previous one, so one to two chunks are always in flight.
+// Operand bytes are pseudo-random (the data pattern moves power and thus clocks).  Gives the denominator "int8 MMA peak
+// as measured on this GPU" for the tensor roofline of the layer kernels.
+constexpr int kProbeChunk = 32;
+template <bool kPairK>
+__global__ void __launch_bounds__(128, 1) mma_peak_kernel(int bn, int chunks, uint32_t idesc, int32_t* status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+  const int warp = threadIdx.x >> 5;
+  const uint32_t tile_a = (smem_u32(smem_raw) + 1023u) & ~1023u;   // 128 rows x 128 bytes, 128-byte swizzle
+  const uint32_t tile_b = tile_a + 128u * 128u;                     // bn (pair: bn / 2) rows x 128 bytes
+  const uint32_t bar0 = smem_u32(bars);
+  uint32_t crank = 0u;
+  if constexpr (kPairK) crank = cluster_cta_rank();
+  {
+    uint32_t* w = reinterpret_cast<uint32_t*>(smem_raw + (tile_a - smem_u32(smem_raw)));
+    const int words = (128 * 128 + (kPairK ? bn / 2 : bn) * 128) / 4;
+    for (int i = threadIdx.x; i < words; i += blockDim.x) {
+      uint32_t h = (uint32_t)i * 2654435761u + blockIdx.x * 40503u;
+      h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+      w[i] = h;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    mbar_init(bar0, 1);
+    mbar_init(bar0 + 8u, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  const uint32_t cols = 512;
+  if (warp == 0) {
+    if constexpr (kPairK) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(cols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+  }
+  tc_fence_before();
+  if constexpr (kPairK) cluster_sync_all();
+  else __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  if (warp == 1) {   // in a pair rank 0 issues for both tensor cores; the peer follows the same barriers (its copies of the arrivals)
+    const uint64_t adesc = make_smem_desc(tile_a, false), bdesc = make_smem_desc(tile_b, false);
+    const uint32_t buf_stride = bn <= 256 ? 256u : 512u;
+    bool ok = true;
+    for (int c = 0; c < chunks && ok; ++c) {
+      if (c >= 2) ok = warp_wait(bar0 + 8u * (c & 1), (uint32_t)((c >> 1) - 1) & 1u, abort_flag, status, kAsyncMmaTmemEmptyWait, 200u);
+      if (!ok) break;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(c & 1) * buf_stride;
+      if (crank == 0 && elect_one()) {
+#pragma unroll
+        for (int i = 0; i < kProbeChunk / 4; ++i)
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mma_any<kPairK>(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (i | k) ? 1u : 0u);
+        commit_any<kPairK>(bar0 + 8u * (c & 1));   // arrives (in both CTAs of a pair) once every MMA issued so far has finished
+      }
+      __syncwarp();
+    }
+    // drain: the last two chunks
+    for (int c = (chunks >= 2 ? chunks - 2 : 0); c < chunks && ok; ++c)
+      ok = warp_wait(bar0 + 8u * (c & 1), (uint32_t)(c >> 1) & 1u, abort_flag, status, kAsyncMmaTmemEmptyWait, 200u);
+  }
+  tc_fence_before();
+  if constexpr (kPairK) cluster_sync_all();
+  else __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    if constexpr (kPairK) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(cols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(cols) : "memory");
+  }
+}
+
 }  // namespace
 
 template <int kOut, bool kPairK>
@@ -965,4 +1049,26 @@ cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtens
   }
 }
 
+}  // namespace hq
+
+namespace hq {
+cudaError_t launch_mma_peak(int pair, int bn, int chunks, int num_sms, int32_t* status, cudaStream_t s, uint64_t* ops) {
+  // instruction descriptor as for the layer kernel: D = s32, A = B = signed 8-bit, K-major, N = bn, M = 128 (256 across a pair)
+  const int m = pair ? 256 : 128;
+  const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+  const uint32_t smem = 1024u + 128u * 128u + (uint32_t)(pair ? bn / 2 : bn) * 128u;
+  const int grid = pair ? (num_sms / 2) * 2 : num_sms;
+  cudaError_t e;
+  if (pair) {
+    e = cudaFuncSetAttribute(mma_peak_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = launch_overlapped_cluster(mma_peak_kernel<true>, grid, 128, smem, s, false, 2u, bn, chunks, idesc, status);
+  } else {
+    e = cudaFuncSetAttribute(mma_peak_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = launch_overlapped(mma_peak_kernel<false>, grid, 128, smem, s, false, bn, chunks, idesc, status);
+  }
+  if (ops) *ops = 2ull * (uint64_t)m * (uint64_t)bn * 32ull * (uint64_t)kProbeChunk * (uint64_t)chunks * (uint64_t)(pair ? grid / 2 : grid);
+  return e;
+}
 }  // namespace hq

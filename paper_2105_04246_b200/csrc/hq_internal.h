@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <initializer_list>
 #include <string>
 #include <utility>
 #include <vector>
@@ -36,6 +37,31 @@ enum AsyncCode : int32_t {
   kAsyncMmaBFullWait = 6,
   kAsyncDepthwiseFullWait = 7,
 };
+
+// Fixed-capacity list for the planner's small tables (tap offsets, border-class masks): planning a layer call makes no
+// host heap allocation, so the calls that promise to allocate nothing may plan too.
+template <typename T, int kCap>
+struct SmallVec {
+  T v[kCap];
+  int n = 0;
+  SmallVec() = default;
+  SmallVec(std::initializer_list<T> il) { for (const T& x : il) push_back(x); }
+  void push_back(const T& x) { if (n < kCap) v[n++] = x; }
+  void clear() { n = 0; }
+  void assign(int count, const T& x) { n = 0; for (int i = 0; i < count; ++i) push_back(x); }
+  size_t size() const { return (size_t)n; }
+  bool empty() const { return n == 0; }
+  T& operator[](size_t i) { return v[i]; }
+  const T& operator[](size_t i) const { return v[i]; }
+  T* begin() { return v; }
+  T* end() { return v + n; }
+  const T* begin() const { return v; }
+  const T* end() const { return v + n; }
+  T* data() { return v; }
+  const T* data() const { return v; }
+};
+using TapVec = SmallVec<int, 8>;          // tap offsets of one axis (filters up to 7 wide)
+using MaskVec = SmallVec<uint32_t, 64>;   // border-class masks of one axis (more than 16 are refused)
 
 struct FastDiv {                      // n / d == (umulhi(m, n) + n) >> l for 0 <= n < 2^31
   uint32_t m, l;
@@ -186,6 +212,10 @@ cudaError_t depthwise_tiled_set_smem_attr(uint32_t smem_bytes);
 uint32_t depthwise_tiled_smem_bytes(const DwParams& p);
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap);
 cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overlap);
+cudaError_t launch_stats_pack(const hq_range_state* st, int count, int32_t* buf, cudaStream_t s);
+cudaError_t launch_stats_unpack(hq_range_state* st, int count, const int32_t* buf, cudaStream_t s);
+// MMA-only throughput probe (measurement): one CTA or CTA pair per SM, `chunks` x 32 MMAs of 128 (pair: 256) x bn x 32 each
+cudaError_t launch_mma_peak(int pair, int bn, int chunks, int num_sms, int32_t* status, cudaStream_t s, uint64_t* ops);
 cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
                                  bool overlap);
 cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
@@ -240,7 +270,7 @@ struct hq_ctx {
   cudaEvent_t ev_fork = nullptr, ev_join[3] = {nullptr, nullptr, nullptr};
   bool parallel_subs = true;
   bool overlap = true;                // launch the hot-path kernels with programmatic stream serialization
-  std::string err;
+  char err[512] = {0};               // HOST text of the last rejected call (fixed storage: rejecting a call allocates nothing)
 };
 
 struct hq_sub_problem {               // one kernel launch of a prepared convolution

@@ -25,7 +25,8 @@ OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_pair_launch_count",
            "hq_set_option",
            "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
-           "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate", "hq_linear_wgrad", "hq_conv_wgrad"]
+           "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate", "hq_linear_wgrad", "hq_conv_wgrad",
+           "hq_stats_pack", "hq_stats_unpack", "hq_mma_peak_probe"]
 
 # numpy view of hq_range_state (48 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
@@ -80,6 +81,9 @@ def lib():
         L.hq_dynamic_quant.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp, vp]
         L.hq_debug_accumulate.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
         L.hq_dynamic_quant_static.argtypes = [vp, vp, C.POINTER(OpDesc), vp, vp]
+        L.hq_stats_pack.argtypes = [vp, vp, vp, i32, vp]
+        L.hq_stats_unpack.argtypes = [vp, vp, vp, i32, vp]
+        L.hq_mma_peak_probe.argtypes = [vp, vp, i32, i32, i32, C.POINTER(C.c_uint64)]
         for name in EXPORTS:
             if name not in ("hq_status_string", "hq_last_error", "hq_launch_count", "hq_pair_launch_count"):
                 getattr(L, name).restype = C.c_int
@@ -185,6 +189,18 @@ class Context:
         """hq_dynamic_quant with the library's built-in workspace: for callers that cannot allocate
         device memory (see include/hq.h).  Shares one array per device; do not overlap calls."""
         self._check(lib().hq_dynamic_quant_static(self.handle, _stream(stream), C.byref(op), _ptr(Y), _ptr(yq)))
+
+    def stats_pack(self, stream, states, count: int, buf):
+        self._check(lib().hq_stats_pack(self.handle, _stream(stream), _ptr(states), int(count), _ptr(buf)))
+
+    def stats_unpack(self, stream, states, count: int, buf):
+        self._check(lib().hq_stats_unpack(self.handle, _stream(stream), _ptr(states), int(count), _ptr(buf)))
+
+    def mma_peak_probe(self, stream, pair: int, bn: int, chunks: int) -> int:
+        """Enqueues the MMA-only probe kernel; returns the 2 x MAC count of the launch."""
+        ops = C.c_uint64(0)
+        self._check(lib().hq_mma_peak_probe(self.handle, _stream(stream), int(pair), int(bn), int(chunks), C.byref(ops)))
+        return int(ops.value)
 
     def debug_accumulate(self, stream, op: OpDesc, acc, yq):
         self._check(lib().hq_debug_accumulate(self.handle, _stream(stream), C.byref(op), _ptr(acc), _ptr(yq)))

@@ -10,6 +10,32 @@ from paper_2105_04246_b200 import hq
 from paper_2105_04246_b200.synth import QTensor
 
 
+GUARD_BYTES = 4096            # sentinel band on both sides of every output the kernels write
+GUARD_BYTE = 0xA5
+
+
+class Guarded:
+    """An output tensor carved out of a larger byte buffer with GUARD_BYTES of a sentinel value before and after it.
+    check() fails if a kernel wrote outside the tensor (the memory checker of the toolkit is not available on the
+    machines these tests run on, so stores past the end of ragged tiles would otherwise go unseen)."""
+
+    def __init__(self, shape, dtype, dev, fill=None):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.nbytes = n
+        self.buf = torch.full((2 * GUARD_BYTES + ((n + 15) // 16) * 16,), GUARD_BYTE, dtype=torch.uint8, device=dev)
+        self.t = self.buf[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)     # 16-byte aligned like a fresh allocation
+        assert self.t.data_ptr() % 16 == 0
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self):
+        lo = self.buf[:GUARD_BYTES]
+        hi = self.buf[GUARD_BYTES + self.nbytes:]
+        assert bool((lo == GUARD_BYTE).all()), "a kernel wrote BEFORE the start of its output tensor"
+        assert bool((hi == GUARD_BYTE).all()), "a kernel wrote PAST the end of its output tensor"
+        return self.t
+
+
 class GpuLayer:
     """kind: 'linear' | 'conv_fwd' | 'conv_bwd'.  For conv kinds `shape` is a dict of conv_desc arguments."""
 
@@ -60,24 +86,29 @@ class GpuLayer:
     def accumulate(self, x: QTensor):
         """Debug hook: int32 accumulator and its min/max (does not disturb the layer's own state)."""
         xd, xq, out_shape = self._put(x)
-        acc = torch.empty(out_shape, dtype=torch.int32, device=self.dev)
+        g_acc = Guarded(out_shape, torch.int32, self.dev)
+        acc = g_acc.t
         tmp = hq.states_to_device(hq.new_states(1), self.dev)
         self.ctx.debug_accumulate(self.stream, self._op(xd, xq), acc, tmp)
         torch.cuda.synchronize(self.dev)
+        g_acc.check()
         st = hq.states_from_device(tmp)[0]
         return acc.cpu().numpy(), int(st["acc_min"]), int(st["acc_max"]), float(st["acc_scale"])
 
     def dynamic(self, x: QTensor):
         xd, xq, out_shape = self._put(x)
-        ws = torch.empty(out_shape, dtype=torch.float32, device=self.dev)
-        y = torch.full(out_shape, 99, dtype=torch.int8, device=self.dev)
+        g_ws, g_y = Guarded(out_shape, torch.float32, self.dev), Guarded(out_shape, torch.int8, self.dev, fill=99)
+        ws, y = g_ws.t, g_y.t
         self.ctx.dynamic_quant(self.stream, self._op(xd, xq), ws, y, self.yq)
         torch.cuda.synchronize(self.dev)
+        g_ws.check()
+        g_y.check()
         return y.cpu().numpy(), ws.cpu().numpy()
 
     def hindsight(self, x: QTensor, update: bool = True):
         xd, xq, out_shape = self._put(x)
-        y = torch.full(out_shape, 99, dtype=torch.int8, device=self.dev)
+        g_y = Guarded(out_shape, torch.int8, self.dev, fill=99)
+        y = g_y.t
         if self.kind == "linear":
             self.ctx.linear_fwd(self.stream, xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias, y, self.yq)
         elif self.kind == "conv_fwd":
@@ -85,6 +116,7 @@ class GpuLayer:
         else:
             self.ctx.conv_bwd_data(self.stream, self.desc, xd, xq, self.pw, self.w_scale, y, self.yq)
         torch.cuda.synchronize(self.dev)
+        g_y.check()
         stats = self.state()
         if update:
             self.ctx.range_update(self.stream, self.yq, 1, self.eta)

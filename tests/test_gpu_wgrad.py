@@ -6,6 +6,7 @@ import torch
 
 import oracle as O
 from paper_2105_04246_b200 import hq, synth
+from tests.harness import Guarded
 
 pytestmark = pytest.mark.gpu
 
@@ -29,9 +30,10 @@ def test_linear_wgrad_matches_oracle(ctx, M, N, K):
     xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
     want = O.scale_to_real(O.linear_wgrad_acc(dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
     for _ in range(2):    # the second call reuses the context's scratch with stale contents
-        gw = torch.full((N, K), float("nan"), dtype=torch.float32, device=dev)
+        g_gw = Guarded((N, K), torch.float32, dev, fill=float("nan")); gw = g_gw.t
         ctx.linear_wgrad(None, M, N, K, dy_d, dyq, x_d, xq, gw)
         torch.cuda.synchronize(dev)
+        g_gw.check()
         got = gw.cpu().numpy()
         bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
         assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
@@ -49,9 +51,10 @@ def test_linear_wgrad_partial_sums_may_leave_int32(ctx):
     dy_d, x_d = torch.from_numpy(dy).to(dev), torch.from_numpy(x).to(dev)
     dyq = hq.states_to_device(hq.input_state(0.5, -128), dev)
     xq = hq.states_to_device(hq.input_state(0.25, 127), dev)
-    gw = torch.full((N, K), float("nan"), dtype=torch.float32, device=dev)
+    g_gw = Guarded((N, K), torch.float32, dev, fill=float("nan")); gw = g_gw.t
     ctx.linear_wgrad(None, M, N, K, dy_d, dyq, x_d, xq, gw)
     torch.cuda.synchronize(dev)
+    g_gw.check()
     want = O.scale_to_real(O.linear_wgrad_acc(dy, -128, x, 127), O.acc_scale(0.5, 0.25))
     assert want[0, 0] == 0.0 and want[0, 1] == np.float32(-255 * M) * np.float32(0.125)
     assert np.array_equal(gw.cpu().numpy().view(np.uint32), want.view(np.uint32))
@@ -118,9 +121,10 @@ def test_conv_wgrad_matches_oracle(ctx, name):
     xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
     want = O.scale_to_real(O.conv_wgrad_acc(od, dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
     for _ in range(2):
-        gw = torch.full((c["K"], c["R"], c["S"], c["Cin"]), float("nan"), dtype=torch.float32, device=dev)
+        g_gw = Guarded((c["K"], c["R"], c["S"], c["Cin"]), torch.float32, dev, fill=float("nan")); gw = g_gw.t
         ctx.conv_wgrad(None, desc, dy_d, dyq, x_d, xq, gw)
         torch.cuda.synchronize(dev)
+        g_gw.check()
         got = gw.cpu().numpy()
         bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
         assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"
@@ -178,9 +182,10 @@ def test_depthwise_wgrad_matches_oracle(ctx, name):
     xq = hq.states_to_device(hq.input_state(x.scale, x.zero_point), dev)
     want = O.scale_to_real(O.conv_wgrad_acc(od, dy.q, dy.zero_point, x.q, x.zero_point), O.acc_scale(dy.scale, x.scale))
     for _ in range(2):
-        gw = torch.full((c["C"], c["R"], c["R"]), float("nan"), dtype=torch.float32, device=dev)
+        g_gw = Guarded((c["C"], c["R"], c["R"]), torch.float32, dev, fill=float("nan")); gw = g_gw.t
         ctx.conv_wgrad(None, desc, dy_d, dyq, x_d, xq, gw)
         torch.cuda.synchronize(dev)
+        g_gw.check()
         got = gw.cpu().numpy()
         bad = np.argwhere(got.view(np.uint32) != want.view(np.uint32))
         assert bad.size == 0, f"{len(bad)} mismatches, first {bad[:5]}: gpu {got[tuple(bad[0])]} oracle {want[tuple(bad[0])]}"

@@ -51,3 +51,38 @@ def test_sharded_statistics_equal_whole_tensor_statistics():
     acc = r.integers(-10**6, 10**6, size=(8, 50)).astype(np.int32)
     shards = [O.minmax(acc[:4]), O.minmax(acc[4:])]
     assert (min(s[0] for s in shards), max(s[1] for s in shards)) == O.minmax(acc)
+
+
+def _train_worker(rank, world, port, accs, s_acc, eta, out):
+    """Each rank sees its half of every iteration's accumulator tensor; statistics are merged, then Eq. 2-3 is applied locally."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    q = O.Range()
+    st = hq.new_states(1)
+    for acc in accs:
+        shard = np.array_split(acc, world, axis=0)[rank]
+        st["acc_min"][0], st["acc_max"][0] = O.minmax(shard)
+        t = torch.from_numpy(st.view(np.uint8).reshape(-1).copy())
+        parallel.allreduce_stats(t)
+        merged = t.numpy().view(hq.RANGE_STATE_DTYPE)
+        O.range_update(q, int(merged["acc_min"][0]), int(merged["acc_max"][0]), s_acc, eta)
+        st["acc_min"][0], st["acc_max"][0] = hq.INT32_MAX, hq.INT32_MIN       # the update empties the slot
+    out[rank] = q.astuple()
+    dist.destroy_process_group()
+
+
+def test_replicated_range_state_stays_identical_over_iterations():
+    """Five iterations on two ranks: after every exchange both ranks apply the moving average of Eq. 2-3 to the same
+    pair, so their range states stay bit-identical and equal the state of one process that saw the whole batch."""
+    r = synth.rng(301)
+    accs = [(r.integers(-10**5, 10**5, size=(16, 40)) * (1.0 + 0.3 * t)).astype(np.int32) for t in range(5)]
+    s_acc, eta = 3.0e-4, 0.9
+    mgr = mp.Manager()
+    out = mgr.dict()
+    mp.spawn(_train_worker, args=(2, _free_port(), accs, s_acc, eta, out), nprocs=2, join=True)
+    whole = O.Range()
+    for acc in accs:
+        O.range_update(whole, *O.minmax(acc), s_acc, eta)
+    assert out[0] == out[1] == whole.astuple()
+    assert whole.step == 5

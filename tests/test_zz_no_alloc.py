@@ -11,12 +11,14 @@ import pytest
 import torch
 
 from paper_2105_04246_b200 import hq, synth
+from tests.harness import Guarded
 
 pytestmark = pytest.mark.gpu
 
 
 def _run(ctx, dev, op_maker, out_shape, static):
-    y = torch.full(out_shape, 77, dtype=torch.int8, device=dev)
+    g_y = Guarded(out_shape, torch.int8, dev, fill=77)      # sentinel bands around the output: nothing may be written outside it
+    y = g_y.t
     yq = hq.states_to_device(hq.new_states(1), dev)
     op = op_maker()
     if static:
@@ -25,6 +27,7 @@ def _run(ctx, dev, op_maker, out_shape, static):
         ws = torch.empty(out_shape, dtype=torch.float32, device=dev)
         ctx.dynamic_quant(None, op, ws, y, yq)
     torch.cuda.synchronize(dev)
+    g_y.check()
     return y.cpu().numpy(), hq.states_from_device(yq)[0]
 
 
@@ -63,6 +66,16 @@ def test_static_workspace_matches_caller_workspace_twice_in_a_row():
     with pytest.raises(hq.HqError) as e:
         ctx.dynamic_quant_static(None, hq.linear_op(8192, 1024, 64, xl_d, xlq, Wl_d, wsl), xl_d, xlq)
     assert e.value.status == 2 and "workspace" in str(e.value)
+    assert ctx.launch_count() == n1
+    # scratch the context does not hold is not grown by this call: refused, nothing launched
+    big_w = torch.zeros((5000, 64), dtype=torch.int8, device=dev)
+    with pytest.raises(hq.HqError) as e:
+        ctx.dynamic_quant_static(None, hq.linear_op(64, 5000, 64, xl_d, xlq, big_w, wsl), xl_d, xlq)
+    assert e.value.status == 2 and "may not allocate" in str(e.value)
+    odd_w = torch.zeros((40, 24), dtype=torch.int8, device=dev)
+    with pytest.raises(hq.HqError) as e:
+        ctx.dynamic_quant_static(None, hq.linear_op(100, 40, 24, xl_d, xlq, odd_w, wsl), xl_d, xlq)
+    assert e.value.status == 2 and "may not allocate" in str(e.value)
     assert ctx.launch_count() == n1
     assert ctx.get_async_error() == 0
     pw.release()
