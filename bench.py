@@ -210,7 +210,7 @@ class GpuWorkload:
                 if kind == "conv_bwd" or _s.name.endswith(".bwd"):
                     st[i]["rounding"], st[i]["seed"] = hq.ROUND_STOCHASTIC, 0x2105 + i
         self.states = hq.states_to_device(st, dev)
-        self.state_ptr = [self.states.data_ptr() + 48 * i for i in range(n)]
+        self.state_ptr = [self.states.data_ptr() + hq.STATE_BYTES * i for i in range(n)]
         self.W, self.w_scale, self.pw, self.desc, self.x_pool, self.xq_pool, self.y_pool, self.ws_pool, self.pool = [], [], [], [], [], [], [], [], []
         stream = torch.cuda.current_stream(dev)
         for i, (kind, s, recipe) in enumerate(self.layers):

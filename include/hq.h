@@ -59,7 +59,7 @@ typedef enum {
   HQ_ERR_TIMEOUT = 6          /* a bounded device-side wait expired (hq_get_async_error)       */
 } hq_status;
 
-/* Per-tensor quantizer state, device resident, 48 bytes, 16-byte aligned, plain data:
+/* Per-tensor quantizer state, device resident, 64 bytes, 16-byte aligned, plain data:
  * a checkpoint of the method's whole state is a copy of the array of these.
  *   acc_min/acc_max  statistics slot (Sec. 4 step 2): min and max of the zero-point-corrected
  *                    int32 accumulator of the tensor, merged by the layer kernels with atomics.
@@ -80,9 +80,18 @@ typedef enum {
  *   dynamic_eta      read by hq_dynamic_quant only: 0 (default) = current min-max (Eq. 1); eta in (0,1) =
  *                    running min-max (Sec. 4.1): the range that quantizes the tensor is
  *                    (1-eta) * its own min/max + eta * the previous range (first tensor: its min/max).
+ *   sat_below, sat_above   the saturation statistic of Sec. 4 ("the proportion of values that lie outside the
+ *                    quantization grid"), as counts: a layer call that writes this tensor with HQ_COUNT_SATURATION set in
+ *                    `rounding` adds the number of outputs whose grid coordinate u = fl(fl(float(acc) * s_acc) * inv_scale)
+ *                    lies below the lowest grid point (u < -128 - zero_point) or above the highest (u > 127 - zero_point),
+ *                    taken before rounding, so the counts do not depend on the rounding mode.  Dividing by the tensor's
+ *                    element count gives the ratio.
+ *   last_sat_below, last_sat_above   hq_range_update / hq_dynamic_quant move the counts here and clear the running pair.
  * For a layer INPUT only scale and zero_point are read.                                      */
 #define HQ_ROUND_NEAREST_EVEN 0u
 #define HQ_ROUND_STOCHASTIC 1u
+#define HQ_ROUND_MODE_MASK 0xFFu     /* low byte of `rounding`: the rounding mode */
+#define HQ_COUNT_SATURATION 0x100u   /* flag in `rounding`: count the outputs that lie outside the grid */
 typedef struct {
   int32_t acc_min, acc_max;
   float acc_scale;
@@ -93,6 +102,8 @@ typedef struct {
   uint32_t rounding;
   uint32_t seed;
   float dynamic_eta;
+  uint32_t sat_below, sat_above;
+  uint32_t last_sat_below, last_sat_above;
 } hq_range_state;
 
 /* Forward-convolution geometry.  Input N x H x W x C, output N x Ho x Wo x K with
@@ -122,7 +133,7 @@ typedef struct {
   const hq_range_state* xq;      /* its scale / zero_point */
   const int8_t* w;               /* linear only: W[N][K] */
   const int32_t* bias;           /* linear only, may be NULL */
-  const hq_prepared_weights* pw; /* conv kinds only */
+  const hq_prepared_weights* pw; /* conv kinds; linear: NULL, or a handle from hq_linear_prepare (N, K, w then ignored) */
   const float* w_scale;          /* one float: the weights' scale s_w (zero point 0) */
 } hq_op_desc;
 
@@ -185,6 +196,22 @@ hq_status hq_set_option(hq_ctx* ctx, const char* key, int32_t value);
  * The handle is valid for this geometry (including N, H, W) only. */
 hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir,
                              const int8_t* W, hq_prepared_weights** out);
+/* The same for asymmetric weights (Sec. 5.2: the weights are quantized with the current min-max method; with an
+ * asymmetric grid they carry a zero point): W holds codes whose real value is s_w * (code - w_zero_point), and every layer
+ * call with the handle forms sum (x - z_x) * (w - z_w).  How: sum (x - z_x)(w - z_w) = [sum (x - z_x) w] - z_w * sum (x - z_x);
+ * the bracket is what the layer kernels compute for symmetric weights, the second term is one number per output pixel
+ * (the sum of the pixel's in-image input window), written by a small kernel at the head of every layer call into scratch
+ * the handle owns, and subtracted in the epilogue before statistics and requantization.  w_zero_point in -128..127;
+ * 0 gives exactly hq_weights_prepare.  Depthwise layers with a zero point run a direct CUDA-core kernel. */
+hq_status hq_weights_prepare_zp(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir,
+                                const int8_t* W, int32_t w_zero_point, hq_prepared_weights** out);
+/* Prepared weights of a LINEAR layer, once per weight update: copies W[N][K] (zero-padding K to a multiple of 16) and caches
+ * the column sums that remove the input zero point, so that hq_linear_fwd_prepared launches the layer kernel alone and
+ * never touches context scratch.  w_zero_point as for hq_weights_prepare_zp.  max_M: the largest row count the handle
+ * will be used with; needed (> 0) when K is not a multiple of 16 (room for the padded copy of X) or w_zero_point != 0
+ * (room for the per-row term), ignored otherwise.  Release with hq_weights_release. */
+hq_status hq_linear_prepare(hq_ctx* ctx, void* stream, int32_t N, int32_t K, const int8_t* W, int32_t w_zero_point,
+                            int32_t max_M, hq_prepared_weights** out);
 hq_status hq_weights_release(hq_ctx* ctx, hq_prepared_weights* pw);
 
 /* ---- the hot path --------------------------------------------------------------------------- */
@@ -203,6 +230,13 @@ hq_status hq_linear_fwd(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32_t
                         const int8_t* W, const float* w_scale, const int32_t* bias,
                         int8_t* Y, hq_range_state* yq);
 
+/* hq_linear_fwd with weights from hq_linear_prepare: same arithmetic (with the handle's weight zero point), no per-call
+ * column sums, no context scratch, nothing allocated.  Two calls with different handles may overlap on the GPU; two calls
+ * with the SAME handle may not when the handle owns scratch (K not a multiple of 16, or a weight zero point). */
+hq_status hq_linear_fwd_prepared(hq_ctx* ctx, void* stream, int32_t M, const int8_t* X, const hq_range_state* xq,
+                                 const hq_prepared_weights* pw, const float* w_scale, const int32_t* bias,
+                                 int8_t* Y, hq_range_state* yq);
+
 /* Forward convolution as an implicit GEMM (Sec. 3.1), same epilogue as hq_linear_fwd.
  * Padding is zero in the real domain.  pw must come from hq_weights_prepare(.., HQ_DIR_FWD, ..)
  * with the same descriptor.  groups == C selects the depthwise kernel.  Spatial filters over a channel
@@ -218,8 +252,8 @@ hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
  *   dX[n][hi][wi][c] = Q_G( sum over (r,s,k) with ho*stride_h - pad_h + r == hi (wo alike)
  *                           of (dY[n][ho][wo][k] - z_dy) * W[k][r][s][c] ).
  * dY is N x Ho x Wo x K, dX is N x H x W x C.  pw from hq_weights_prepare(.., HQ_DIR_BWD_DATA, ..).
- * Depthwise layers (groups == C): stride 1 and pad <= filter size - 1 only (HQ_ERR_UNSUPPORTED otherwise, from
- * hq_weights_prepare); the sum then runs over (r,s) alone with k == c. */
+ * Depthwise layers (groups == C): the sum runs over (r,s) alone with k == c; stride-1 layers run the forward depthwise
+ * kernels over the output gradient with the filter turned by 180 degrees, strided layers a direct kernel. */
 hq_status hq_conv_bwd_data(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                            const int8_t* dY, const hq_range_state* dyq,
                            const hq_prepared_weights* pw, const float* w_scale,
@@ -257,8 +291,8 @@ hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
  *   m_lo = float(acc_min) * acc_scale, m_hi alike;
  *   step == 0:  q_min = m_lo, q_max = m_hi                      (initialisation, Sec. 4.1)
  *   else:       q_min = (1-eta)*m_lo + eta*q_min, q_max alike    (Eq. 2-3)
- * then derives scale / inv_scale / zero_point, increments step and empties the statistics slot.
- * A state whose slot is empty is left untouched. */
+ * then derives scale / inv_scale / zero_point, increments step, empties the statistics slot and moves the saturation
+ * counts to last_sat_below / last_sat_above.  A state whose slot is empty is left untouched. */
 hq_status hq_range_update(hq_ctx* ctx, void* stream, hq_range_state* states, int32_t count, float eta);
 
 /* Batch-sharded data parallelism (each GPU runs the layer calls on its slice of the batch with the same weights and

@@ -69,6 +69,7 @@ def lib():
         L.hqo_conv_bwd_data_acc_at.argtypes = [cp, i8p, C.c_int, i8p, C.c_int, i64p, C.c_int64, i64p]; L.hqo_conv_bwd_data_acc_at.restype = None
         L.hqo_minmax.argtypes = [i32p, C.c_int64, i32p, i32p]; L.hqo_minmax.restype = None
         L.hqo_quantize.argtypes = [i32p, C.c_int64, C.c_float, rp, i8p]; L.hqo_quantize.restype = None
+        L.hqo_saturation.argtypes = [i32p, C.c_int64, C.c_float, rp, C.c_int, C.c_uint32, C.c_uint32, C.c_int64, i64p, i64p]; L.hqo_saturation.restype = None
         L.hqo_range_update.argtypes = [rp, C.c_int32, C.c_int32, C.c_float, C.c_float]; L.hqo_range_update.restype = None
         L.hqo_dynamic.argtypes = [i32p, C.c_int64, C.c_float, rp, f32p, i8p]; L.hqo_dynamic.restype = None
         L.hqo_acc_scale.argtypes = [C.c_float, C.c_float]; L.hqo_acc_scale.restype = C.c_float
@@ -200,6 +201,16 @@ def quantize(acc: np.ndarray, s_acc: float, q: Range) -> np.ndarray:
     out = np.empty(acc.shape, np.int8)
     lib().hqo_quantize(_p(acc, C.c_int32), acc.size, C.c_float(s_acc), C.byref(q), _p(out, C.c_int8))
     return out
+
+
+def saturation(acc: np.ndarray, s_acc: float, q: Range, sr_seed: int | None = None, iteration: int = 0, first: int = 0):
+    """(below, above): how many outputs the quantizer clips to the lowest / highest level (rounded grid coordinate + zero
+    point outside -128..127).  sr_seed: None = round half to even, else stochastic rounding with that seed and iteration."""
+    acc = np.ascontiguousarray(acc, dtype=np.int32)
+    b, a = C.c_int64(), C.c_int64()
+    lib().hqo_saturation(_p(acc, C.c_int32), acc.size, C.c_float(s_acc), C.byref(q), 0 if sr_seed is None else 1,
+                         C.c_uint32(0 if sr_seed is None else sr_seed), C.c_uint32(iteration), C.c_int64(first), C.byref(b), C.byref(a))
+    return b.value, a.value
 
 
 def range_update(q: Range, mn: int, mx: int, s_acc: float, eta: float) -> Range:

@@ -41,6 +41,7 @@
 //   R-13 a degenerate range (hi - lo not > 0) gives s = 1.
 //   R-15 the dynamic path materialises binary32 y = fl(float(acc) * s_acc).
 //   R-18..R-20 stochastic rounding for gradients: see the section further down.
+//   R-22 saturation statistic: see hqo_saturation.
 //
 // Pins (tests/ -m "not gpu"): brute-force and readable-by-eye cases for the index
 // arithmetic, the forward/backward adjoint identity, the trace identity <dY, X W^T> = <dY^T X, W>
@@ -456,6 +457,36 @@ static inline int8_t quantize_real_sr(float y, const hqo_range* q, uint32_t seed
 void hqo_quantize_sr(const int32_t* acc, int64_t count, float s_acc, const hqo_range* q, uint32_t seed, uint32_t iteration, int64_t first,
                      int8_t* out) {
   for (int64_t i = 0; i < count; ++i) out[i] = quantize_real_sr((float)acc[i] * s_acc, q, seed, iteration, first + i);
+}
+
+// ------------------------------------------------------------------------------------
+// Saturation statistic (Sec. 4: besides min and max the statistic may be "the saturation ratio", the proportion
+// of values that lie outside the quantization grid).  The final text of the paper gives no formula; the reading taken
+// (R-22) is "clipped by the quantization operation": an output is counted when its rounded grid coordinate plus the zero
+// point falls outside the 2^8 levels, i.e. when the clamp of O4 changes it:
+//   c = rint(u) + z   (stochastic rounding: floor(fl(u + r)) + z),   below: c < -128,   above: c > 127,
+// with u = fl(fl(float(acc) * s_acc) * inv_scale) as in O4.  Counts, not the ratio: the caller divides by the element
+// count.  sr = 0: round half to even; sr = 1: stochastic rounding with (seed, iteration), element i having index first + i.
+// ------------------------------------------------------------------------------------
+void hqo_saturation(const int32_t* acc, int64_t count, float s_acc, const hqo_range* q, int sr, uint32_t seed, uint32_t iteration, int64_t first,
+                    int64_t* below, int64_t* above) {
+  int64_t b = 0, a = 0;
+  for (int64_t i = 0; i < count; ++i) {
+    float y = (float)acc[i] * s_acc;
+    float u = y * q->inv_scale;
+    int64_t c;
+    if (sr) {
+      float r = (float)hqo_draw16(seed, iteration, first + i) * (1.0f / 65536.0f);
+      float t = u + r;
+      c = (int64_t)floor_to_i32(t) + q->zero_point;
+    } else {
+      c = (int64_t)round_half_even_to_i32(u) + q->zero_point;
+    }
+    if (c < -128) ++b;
+    if (c > 127) ++a;
+  }
+  *below = b;
+  *above = a;
 }
 
 // dynamic path with stochastic rounding: as hqo_dynamic; the draws use the iteration count before this call

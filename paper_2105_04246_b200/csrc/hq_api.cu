@@ -169,6 +169,8 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
   p.Cpad = round_up(sp.Cin, p.BK);
   p.chunks_per_tap = p.Cpad / p.BK;
   p.Nout = sp.Nout;
+  p.rt_fold = 1;
+  p.rt_cols = sp.Nout;
   // column tiles: as wide as the MMA allows, except for very short reductions, where the epilogue is the bottleneck and
   // narrower tiles give it four or more accumulator buffers to work on
   const int ncol = std::max(ncol_req, ceil_div(sp.Nout, p.ntaps * p.Cpad <= 128 ? 128 : 256));
@@ -499,6 +501,10 @@ hq_status launch_sub(hq_ctx* ctx, cudaStream_t s, const hq_sub_problem& sub, con
                      bool weights_early = false, const int32_t* row_term = nullptr) {
   GemmParams p = sub.p;
   p.row_term = row_term;
+  if (row_term != nullptr && sub.gfold > 1) {   // a GEMM row of a folded 1x1 layer holds gfold pixels side by side
+    p.rt_fold = sub.gfold;
+    p.rt_cols = p.Nout / sub.gfold;
+  }
   p.out_col0 = sub.chan0;
   p.weights_early = weights_early ? 1 : 0;
   p.xq = xq;
@@ -532,12 +538,11 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
   if (!in || !inq || !pw || !w_scale || !out || !outq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(in) || !aligned16(out) || !aligned16(inq) || !aligned16(outq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
-  if (pw->dir != dir || !same_desc(pw->desc, *desc)) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights were built for another layer");
+  if (pw->linear || pw->dir != dir || !same_desc(pw->desc, *desc)) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights were built for another layer");
   if (pw->depthwise) {
     // the geometry the kernel runs (see hq_weights_prepare): for backward data the forward layer over the output gradient
     const hq_conv_desc* const caller_desc = desc;
     desc = &pw->dw_run;
-    (void)caller_desc;
     const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
     DwParams p{};
     p.N = desc->N; p.H = desc->H; p.W = desc->W; p.C = desc->C; p.Ho = Ho; p.Wo = Wo; p.R = desc->R; p.S = desc->S;
@@ -545,8 +550,19 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     p.x = in; p.w = pw->dw_w; p.corr = pw->dw_corr; p.rowcls = pw->dw_rowcls; p.colcls = pw->dw_colcls; p.ncolcls = pw->dw_ncolcls;
     p.xq = inq; p.w_scale = w_scale; p.yq = outq; p.out = out;
     p.status = ctx->d_status;
+    p.w_zp = pw->w_zp;
+    if (pw->dw_bwd_direct) {   // backward data by the definition (strided layers, asymmetric weights): the forward geometry, dY in p.x
+      const hq_conv_desc* f = caller_desc;
+      p.N = f->N; p.H = f->H; p.W = f->W; p.C = f->C; p.R = f->R; p.S = f->S;
+      p.Ho = out_dim(f->H, f->pad_h, f->R, f->stride_h); p.Wo = out_dim(f->W, f->pad_w, f->S, f->stride_w);
+      p.stride_h = f->stride_h; p.stride_w = f->stride_w; p.pad_h = f->pad_h; p.pad_w = f->pad_w;
+      p.w = pw->dw_w_plain;
+      HQ_CUDA(ctx, launch_depthwise_bwd(p, out_mode, ctx->num_sms, s));
+      ctx->launches += 1;
+      return HQ_OK;
+    }
     // 3x3 stride 1 with at most 256 channels: output tiles of 4 rows whose input patch one TMA box stages in shared memory
-    if (desc->R == 3 && desc->S == 3 && desc->stride_h == 1 && desc->stride_w == 1 && desc->C <= 256 && ctx->force_dw_tiled != 0) {
+    if (desc->R == 3 && desc->S == 3 && desc->stride_h == 1 && desc->stride_w == 1 && desc->C <= 256 && ctx->force_dw_tiled != 0 && pw->w_zp == 0) {
       p.TR = 4;
       const int budget = 50 * 1024;   // two patches + tables per CTA, two CTAs per SM
       int twt = (budget / (desc->C * (p.TR + 2)) - 2) / 8 * 8;
@@ -598,6 +614,13 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
   // joined back into the caller's stream with events.
   const bool weights_early = ctx->overlap && pw->used;
   pw->used = true;
+  // asymmetric weights: z_w times the input sum of every output pixel, subtracted by the layer kernels' epilogue
+  const int32_t* row_term = nullptr;
+  if (pw->w_zp != 0) {
+    HQ_CUDA(ctx, launch_rowsum(in, inq, *desc, Ho, Wo, dir == HQ_DIR_BWD_DATA ? 1 : 0, pw->w_zp, pw->row_term, s));
+    ctx->launches += 1;
+    row_term = pw->row_term;
+  }
   const int nsub = (int)pw->subs.size();
   constexpr int kMaxSideBySide = 64;
   bool side_by_side = nsub > 1 && nsub <= kMaxSideBySide && ctx->parallel_subs;
@@ -671,7 +694,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       st = encode_a(ctx, sub, in + sub.chan0, sub.chans, aW, aH, desc->N, &ta, desc->C);
       if (st != HQ_OK) return join_after(st);
       void* o = out_mode == kOutInt8 ? (void*)((int8_t*)out + sub.chan0) : (void*)((uint32_t*)out + sub.chan0);
-      st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas, weights_early);
+      st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, o, outq, out_mode, max_ctas, weights_early, row_term);
       if (st != HQ_OK) return join_after(st);
       continue;
     } else if (sub.a_flat) {
@@ -680,7 +703,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     } else {
       st = encode_a(ctx, sub, in, aC, aW, aH, desc->N, &ta);
     }
-    if (st == HQ_OK) st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas, weights_early);
+    if (st == HQ_OK) st = launch_sub(ctx, ss, sub, ta, sub.tmap_b, inq, w_scale, nullptr, out, outq, out_mode, max_ctas, weights_early, row_term);
     if (st != HQ_OK) return join_after(st);
   }
   return join();
@@ -688,13 +711,36 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
 
 hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int8_t* X, const hq_range_state* xq, const int8_t* W,
                      const float* w_scale, const int32_t* bias, void* out, hq_range_state* yq, int out_mode, const int32_t* row_term = nullptr,
-                     bool no_grow = false) {
+                     bool no_grow = false, const hq_prepared_weights* lpw = nullptr) {
   // no_grow: the call may not allocate; shapes that would need larger context scratch are refused instead
+  // lpw: weights prepared by hq_linear_prepare (padded copy, cached column sums, weight zero point); N, K and W then come from it
+  if (lpw != nullptr) {
+    if (!lpw->linear) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights do not belong to a linear layer");
+    N = lpw->lin_N;
+    K = lpw->lin_K;
+    W = lpw->lin_w;
+  }
   if (M <= 0 || N <= 0 || K <= 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
   if (!X || !xq || !W || !w_scale || !out || !yq) return fail(ctx, HQ_ERR_INVALID_ARG, "null pointer argument");
   if (!aligned16(X) || !aligned16(W) || !aligned16(out) || !aligned16(xq) || !aligned16(yq))
     return fail(ctx, HQ_ERR_ALIGNMENT, "tensors and range states must be 16-byte aligned");
-  if (K % 16 != 0) {
+  if (lpw != nullptr) {
+    if ((lpw->lin_Kp != K || lpw->w_zp != 0) && M > lpw->lin_maxM)
+      return fail(ctx, HQ_ERR_UNSUPPORTED, "M = %d exceeds the max_M = %d these weights were prepared for", M, lpw->lin_maxM);
+    if (lpw->w_zp != 0) {   // z_w times the row sums of the (unpadded) input
+      hq_conv_desc rd{};
+      rd.N = 1; rd.H = 1; rd.W = M; rd.C = K; rd.K = N; rd.R = 1; rd.S = 1; rd.stride_h = rd.stride_w = 1; rd.groups = 1;
+      HQ_CUDA(ctx, launch_rowsum(X, xq, rd, 1, M, 0, lpw->w_zp, lpw->row_term, s));
+      ctx->launches += 1;
+      row_term = lpw->row_term;
+    }
+    if (lpw->lin_Kp != K) {
+      HQ_CUDA(ctx, launch_pad_rows(X, lpw->lin_xpad, M, K, lpw->lin_Kp, s));
+      ctx->launches += 1;
+      X = lpw->lin_xpad;
+      K = lpw->lin_Kp;
+    }
+  } else if (K % 16 != 0) {
     // rows whose length no TMA box can address: zero-padded copies of both operands in context-owned scratch
     const int Kp = round_up(K, 16);
     const size_t need = ((size_t)M + (size_t)N) * Kp;
@@ -725,6 +771,18 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
   MaskVec rm, cm;
   hq_status st = plan_sub(ctx, sp, sub, rc, cc, rm, cm);
   if (st != HQ_OK) return st;
+  if (lpw != nullptr) {   // column sums cached with the weights (zero padded well beyond the widest column tiling)
+    sub.p.corr = lpw->lin_corr;
+    sub.p.Cpad = K;
+    CUtensorMap pta, ptb;
+    st = encode_a(ctx, sub, X, K, M, 1, 1, &pta);
+    if (st != HQ_OK) return st;
+    st = encode_b(ctx, sub, W, K, &ptb);
+    if (st != HQ_OK) return st;
+    const bool weights_early = ctx->overlap && lpw->used;   // the library's copy of the weights is older than any kernel in flight
+    lpw->used = true;
+    return launch_sub(ctx, s, sub, pta, ptb, xq, w_scale, bias, out, yq, out_mode, 0, weights_early, row_term);
+  }
   if ((size_t)sub.p.corr_ld > ctx->scratch_elems && no_grow)
     return fail(ctx, HQ_ERR_UNSUPPORTED, "N = %d needs %d column sums; the context holds %zu and this call may not allocate", N, sub.p.corr_ld,
                 ctx->scratch_elems);
@@ -752,8 +810,8 @@ hq_status run_linear(hq_ctx* ctx, cudaStream_t s, int M, int N, int K, const int
 hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, hq_range_state* yq, int out_mode, bool no_grow = false) {
   if (!op) return fail(ctx, HQ_ERR_INVALID_ARG, "operation descriptor is null");
   switch (op->kind) {
-    case HQ_OP_LINEAR:
-      return run_linear(ctx, s, op->M, op->N, op->K, op->x, op->xq, op->w, op->w_scale, op->bias, out, yq, out_mode, nullptr, no_grow);
+    case HQ_OP_LINEAR:   // pw set: weights prepared by hq_linear_prepare (N, K and w of the descriptor are then ignored)
+      return run_linear(ctx, s, op->M, op->N, op->K, op->x, op->xq, op->w, op->w_scale, op->bias, out, yq, out_mode, nullptr, no_grow, op->pw);
     case HQ_OP_CONV_FWD: return run_conv(ctx, s, op->conv, HQ_DIR_FWD, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
     case HQ_OP_CONV_BWD_DATA: return run_conv(ctx, s, op->conv, HQ_DIR_BWD_DATA, op->x, op->xq, op->pw, op->w_scale, out, yq, out_mode);
     default: return fail(ctx, HQ_ERR_INVALID_ARG, "unknown operation kind %d", op->kind);
@@ -761,7 +819,7 @@ hq_status run_op(hq_ctx* ctx, cudaStream_t s, const hq_op_desc* op, void* out, h
 }
 
 int64_t op_out_elems(const hq_op_desc* op) {
-  if (op->kind == HQ_OP_LINEAR) return (int64_t)op->M * op->N;
+  if (op->kind == HQ_OP_LINEAR) return (int64_t)op->M * (op->pw ? op->pw->lin_N : op->N);
   const hq_conv_desc* d = op->conv;
   if (op->kind == HQ_OP_CONV_FWD)
     return (int64_t)d->N * out_dim(d->H, d->pad_h, d->R, d->stride_h) * out_dim(d->W, d->pad_w, d->S, d->stride_w) * d->K;
@@ -918,11 +976,16 @@ __attribute__((visibility("default"))) hq_status hq_get_async_error(hq_ctx* ctx,
   return HQ_OK;
 }
 
-__attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W, hq_prepared_weights** out) {
+}  // extern "C"
+
+namespace {
+hq_status prepare_conv_body(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W, int32_t w_zero_point,
+                            hq_prepared_weights** out) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
   if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
   if (!out) return fail(ctx, HQ_ERR_INVALID_ARG, "out is null");
   *out = nullptr;
+  if (w_zero_point < -128 || w_zero_point > 127) return fail(ctx, HQ_ERR_INVALID_ARG, "weight zero point %d is not an int8 code", w_zero_point);
   hq_status st = check_desc(ctx, desc);
   if (st != HQ_OK) return st;
   if (!W) return fail(ctx, HQ_ERR_INVALID_ARG, "W is null");
@@ -934,6 +997,7 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   if (!pw) return fail(ctx, HQ_ERR_CUDA, "out of host memory");
   pw->desc = d;
   pw->dir = dir;
+  pw->w_zp = w_zero_point;
   auto bail = [&](hq_status e) {
     for (void* p : pw->allocs) cudaFree(p);
     delete pw;
@@ -942,13 +1006,28 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
 
   // Backward data of a stride-1 depthwise layer is a forward depthwise layer over the output gradient (Ho x Wo) with the
   // filter turned by 180 degrees and padding R-1-pad: dx(hi) = sum_r dy(hi + pad - r) w(r) = sum_r' dy(hi - (R-1-pad) + r') w(R-1-r').
+  // Strided depthwise layers, and any depthwise layer with a non-zero weight zero point, run backward data by the
+  // definition instead (depthwise_bwd_kernel).
   const bool dw_bwd = d.groups != 1 && dir == HQ_DIR_BWD_DATA;
+  const bool dw_bwd_direct = dw_bwd && (d.stride_h != 1 || d.stride_w != 1 || w_zero_point != 0);
   hq_conv_desc dwd = d;
   if (d.groups != 1) {
     if (d.C % 16 != 0) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise needs C %% 16 == 0"));
+    if (dw_bwd_direct) {
+      pw->depthwise = true;
+      pw->dw_bwd_direct = true;
+      pw->dw_run = d;
+      int32_t* unused_corr = nullptr;
+      const uint32_t all = 0xFFFFFFFFu;
+      if ((st = dev_alloc(ctx, pw, (void**)&pw->dw_w_plain, (size_t)d.C * d.R * d.S)) != HQ_OK) return bail(st);
+      if ((st = dev_alloc(ctx, pw, (void**)&unused_corr, (size_t)d.C * sizeof(int32_t))) != HQ_OK) return bail(st);
+      cudaError_t e = launch_dw_prep(W, pw->dw_w_plain, unused_corr, d.C, d.R, d.S, &all, 1, &all, 1, 0, s);   // tap-major copy, not turned
+      if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "depthwise weight preparation failed: %s", cudaGetErrorString(e)));
+      ctx->launches += 1;
+      *out = pw;
+      return HQ_OK;
+    }
     if (dw_bwd) {
-      if (d.stride_h != 1 || d.stride_w != 1) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data needs stride 1"));
-      if (d.pad_h > d.R - 1 || d.pad_w > d.S - 1) return bail(fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise backward data needs pad <= filter size - 1"));
       dwd.H = Ho;
       dwd.W = Wo;
       dwd.pad_h = d.R - 1 - d.pad_h;
@@ -960,7 +1039,7 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   // input and output, each with a weight matrix that is zero off the channel diagonal (the int32 sums are the same).
   // Measured on the 56x56x144 layer it is only on a par with the CUDA-core kernel (N = 64 MMAs are bound by
   // shared-memory reads of the pixel operand), so it is not chosen by default.
-  const bool dw_dense = d.groups != 1 && ctx->force_depthwise == 1 && !dw_bwd;
+  const bool dw_dense = d.groups != 1 && ctx->force_depthwise == 1 && !dw_bwd && w_zero_point == 0;
   if (dw_dense) {
     for (int c0 = 0; c0 < d.C; c0 += 64) {
       const int cw = std::min(64, d.C - c0);
@@ -1125,6 +1204,91 @@ __attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx,
   }
   *out = pw;
   return HQ_OK;
+}
+
+hq_status prepare_conv(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W, int32_t w_zero_point,
+                       hq_prepared_weights** out) {
+  hq_status st = prepare_conv_body(ctx, stream, desc, dir, W, w_zero_point, out);
+  if (st != HQ_OK) return st;
+  hq_prepared_weights* pw = *out;
+  if (w_zero_point != 0 && !pw->depthwise) {
+    // room for the weight-zero-point term of every output pixel (forward: N x Ho x Wo, backward data: N x H x W)
+    const hq_conv_desc& d = pw->desc;
+    const int Ho = out_dim(d.H, d.pad_h, d.R, d.stride_h), Wo = out_dim(d.W, d.pad_w, d.S, d.stride_w);
+    pw->row_term_elems = dir == HQ_DIR_FWD ? (size_t)d.N * Ho * Wo : (size_t)d.N * d.H * d.W;
+    st = dev_alloc(ctx, pw, (void**)&pw->row_term, pw->row_term_elems * sizeof(int32_t));
+    if (st != HQ_OK) {
+      for (void* p : pw->allocs) cudaFree(p);
+      delete pw;
+      *out = nullptr;
+      return st;
+    }
+  }
+  return HQ_OK;
+}
+}  // namespace
+
+extern "C" {
+
+__attribute__((visibility("default"))) hq_status hq_weights_prepare(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W,
+                                                                    hq_prepared_weights** out) {
+  return prepare_conv(ctx, stream, desc, dir, W, 0, out);
+}
+
+__attribute__((visibility("default"))) hq_status hq_weights_prepare_zp(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, hq_direction dir, const int8_t* W,
+                                                                       int32_t w_zero_point, hq_prepared_weights** out) {
+  return prepare_conv(ctx, stream, desc, dir, W, w_zero_point, out);
+}
+
+__attribute__((visibility("default"))) hq_status hq_linear_prepare(hq_ctx* ctx, void* stream, int32_t N, int32_t K, const int8_t* W, int32_t w_zero_point,
+                                                                   int32_t max_M, hq_prepared_weights** out) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
+  if (!out) return fail(ctx, HQ_ERR_INVALID_ARG, "out is null");
+  *out = nullptr;
+  if (N <= 0 || K <= 0 || max_M < 0) return fail(ctx, HQ_ERR_INVALID_ARG, "linear sizes must be positive");
+  if (!W || !aligned16(W)) return fail(ctx, W ? HQ_ERR_ALIGNMENT : HQ_ERR_INVALID_ARG, "W is null or not 16-byte aligned");
+  if (w_zero_point < -128 || w_zero_point > 127) return fail(ctx, HQ_ERR_INVALID_ARG, "weight zero point %d is not an int8 code", w_zero_point);
+  const int Kp = round_up(K, 16);
+  if ((Kp != K || w_zero_point != 0) && max_M <= 0)
+    return fail(ctx, HQ_ERR_INVALID_ARG, "max_M must be given when K is not a multiple of 16 or the weights have a zero point");
+  cudaStream_t s = (cudaStream_t)stream;
+  hq_prepared_weights* pw = new (std::nothrow) hq_prepared_weights();
+  if (!pw) return fail(ctx, HQ_ERR_CUDA, "out of host memory");
+  auto bail = [&](hq_status e) {
+    for (void* p : pw->allocs) cudaFree(p);
+    delete pw;
+    return e;
+  };
+  pw->linear = true;
+  pw->lin_N = N; pw->lin_K = K; pw->lin_Kp = Kp; pw->lin_maxM = max_M;
+  pw->w_zp = w_zero_point;
+  hq_status st;
+  if ((st = dev_alloc(ctx, pw, (void**)&pw->lin_w, (size_t)N * Kp)) != HQ_OK) return bail(st);
+  const size_t corr_elems = (size_t)N + 512;   // every column tiling pads N by less than this
+  if ((st = dev_alloc(ctx, pw, (void**)&pw->lin_corr, corr_elems * sizeof(int32_t))) != HQ_OK) return bail(st);
+  cudaError_t e = cudaMemsetAsync(pw->lin_corr, 0, corr_elems * sizeof(int32_t), s);
+  if (e == cudaSuccess) e = launch_pad_rows(W, pw->lin_w, N, K, Kp, s);
+  const uint32_t one = 1u;
+  if (e == cudaSuccess) e = launch_corr(pw->lin_w, pw->lin_corr, N, 1, Kp, 1, 1, &one, 1, &one, 1, (int)corr_elems, s);
+  if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "linear weight preparation failed: %s", cudaGetErrorString(e)));
+  ctx->launches += 2;
+  if (Kp != K && (st = dev_alloc(ctx, pw, (void**)&pw->lin_xpad, (size_t)max_M * Kp)) != HQ_OK) return bail(st);
+  if (w_zero_point != 0) {
+    pw->row_term_elems = (size_t)max_M;
+    if ((st = dev_alloc(ctx, pw, (void**)&pw->row_term, pw->row_term_elems * sizeof(int32_t))) != HQ_OK) return bail(st);
+  }
+  *out = pw;
+  return HQ_OK;
+}
+
+__attribute__((visibility("default"))) hq_status hq_linear_fwd_prepared(hq_ctx* ctx, void* stream, int32_t M, const int8_t* X, const hq_range_state* xq,
+                                                                        const hq_prepared_weights* pw, const float* w_scale, const int32_t* bias,
+                                                                        int8_t* Y, hq_range_state* yq) {
+  if (!ctx) return HQ_ERR_INVALID_ARG;
+  if (hq_status ds = check_device(ctx); ds != HQ_OK) return ds;
+  if (!pw) return fail(ctx, HQ_ERR_INVALID_ARG, "prepared weights are null");
+  return run_linear(ctx, (cudaStream_t)stream, M, 0, 0, X, xq, nullptr, w_scale, bias, Y, yq, kOutInt8, nullptr, false, pw);
 }
 
 __attribute__((visibility("default"))) hq_status hq_weights_release(hq_ctx* ctx, hq_prepared_weights* pw) {

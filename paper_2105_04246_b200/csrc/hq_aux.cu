@@ -49,6 +49,10 @@ __global__ void range_update_kernel(hq_range_state* st, int count, float eta) {
   derive_grid(s);
   s->acc_min = INT32_MAX;
   s->acc_max = INT32_MIN;
+  s->last_sat_below = s->sat_below;   // the saturation counts of the tensor just finished
+  s->last_sat_above = s->sat_above;
+  s->sat_below = 0u;
+  s->sat_above = 0u;
 }
 
 // Batch-sharded data parallelism: the only exchange of the method is the statistics.  pack writes {acc_min, ~acc_max}
@@ -89,10 +93,14 @@ __global__ void dynamic_derive_kernel(hq_range_state* s) {
   derive_grid(s);
   s->acc_min = INT32_MAX;
   s->acc_max = INT32_MIN;
+  s->last_sat_below = 0u;   // the quantize pass that follows counts this tensor's clipped outputs straight into these
+  s->last_sat_above = 0u;
+  s->sat_below = 0u;
+  s->sat_above = 0u;
 }
 
 // second pass of the dynamic path: read the binary32 output back and quantize it
-__global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __restrict__ out, int64_t count, const hq_range_state* st) {
+__global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __restrict__ out, int64_t count, hq_range_state* st) {
   grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
   QParams q;
   q.s_acc = 1.0f;
@@ -100,11 +108,8 @@ __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __rest
   q.inv_scale = st->inv_scale;
   q.zp = st->zero_point;
   qparams_finish(q);
-  if (st->rounding == HQ_ROUND_STOCHASTIC) {   // the derive kernel has already counted this iteration
-    q.sr = 1;
-    q.sr_seed = st->seed;
-    q.sr_iter = st->step - 1u;
-  }
+  qparams_output_mode(q, st->rounding, st->seed, st->step - 1u);   // the derive kernel has already counted this iteration
+  int sat_below = 0, sat_above = 0;
   const int64_t groups = count / 16;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < groups; g += stride) {
@@ -116,29 +121,42 @@ __global__ void quantize_pass_kernel(const float* __restrict__ y, int8_t* __rest
         uint32_t h[8];
         sr_draws8(q, (uint64_t)(2 * g + b), h);
         const float4 f0 = __ldcs(src + 2 * b), f1 = __ldcs(src + 2 * b + 1);
-        w[2 * b] = q.fast ? pack_sat4(requant_real_sr<true>(f0.x, h[0], q), requant_real_sr<true>(f0.y, h[1], q),
-                                      requant_real_sr<true>(f0.z, h[2], q), requant_real_sr<true>(f0.w, h[3], q))
-                          : pack_sat4(requant_real_sr<false>(f0.x, h[0], q), requant_real_sr<false>(f0.y, h[1], q),
-                                      requant_real_sr<false>(f0.z, h[2], q), requant_real_sr<false>(f0.w, h[3], q));
-        w[2 * b + 1] = q.fast ? pack_sat4(requant_real_sr<true>(f1.x, h[4], q), requant_real_sr<true>(f1.y, h[5], q),
-                                          requant_real_sr<true>(f1.z, h[6], q), requant_real_sr<true>(f1.w, h[7], q))
-                              : pack_sat4(requant_real_sr<false>(f1.x, h[4], q), requant_real_sr<false>(f1.y, h[5], q),
-                                          requant_real_sr<false>(f1.z, h[6], q), requant_real_sr<false>(f1.w, h[7], q));
+        w[2 * b] = q.fast ? finish4(requant_real_sr<true>(f0.x, h[0], q), requant_real_sr<true>(f0.y, h[1], q),
+                                    requant_real_sr<true>(f0.z, h[2], q), requant_real_sr<true>(f0.w, h[3], q), q, sat_below, sat_above)
+                          : finish4(requant_real_sr<false>(f0.x, h[0], q), requant_real_sr<false>(f0.y, h[1], q),
+                                    requant_real_sr<false>(f0.z, h[2], q), requant_real_sr<false>(f0.w, h[3], q), q, sat_below, sat_above);
+        w[2 * b + 1] = q.fast ? finish4(requant_real_sr<true>(f1.x, h[4], q), requant_real_sr<true>(f1.y, h[5], q),
+                                        requant_real_sr<true>(f1.z, h[6], q), requant_real_sr<true>(f1.w, h[7], q), q, sat_below, sat_above)
+                              : finish4(requant_real_sr<false>(f1.x, h[4], q), requant_real_sr<false>(f1.y, h[5], q),
+                                        requant_real_sr<false>(f1.z, h[6], q), requant_real_sr<false>(f1.w, h[7], q), q, sat_below, sat_above);
       }
     } else {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float4 f = __ldcs(src + e);
-        w[e] = q.fast ? pack_sat4(requant_real<true>(f.x, q), requant_real<true>(f.y, q), requant_real<true>(f.z, q), requant_real<true>(f.w, q))
-                      : pack_sat4(requant_real<false>(f.x, q), requant_real<false>(f.y, q), requant_real<false>(f.z, q), requant_real<false>(f.w, q));
+        w[e] = q.fast ? finish4(requant_real<true>(f.x, q), requant_real<true>(f.y, q), requant_real<true>(f.z, q), requant_real<true>(f.w, q), q,
+                                sat_below, sat_above)
+                      : finish4(requant_real<false>(f.x, q), requant_real<false>(f.y, q), requant_real<false>(f.z, q), requant_real<false>(f.w, q), q,
+                                sat_below, sat_above);
       }
     }
     reinterpret_cast<uint4*>(out)[g] = make_uint4(w[0], w[1], w[2], w[3]);
   }
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
   if (blockIdx.x == 0) {
-    for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x)
-      out[i] = (int8_t)min(max(q.sr ? requant_real_sr<false>(y[i], sr_draw1(q, i), q) : requant_real<false>(y[i], q), -128), 127);
+    for (int64_t i = groups * 16 + threadIdx.x; i < count; i += blockDim.x) {
+      const int r = q.sr ? requant_real_sr<false>(y[i], sr_draw1(q, i), q) : requant_real<false>(y[i], q);
+      if (q.count_sat) count_clipped(r, sat_below, sat_above);
+      out[i] = (int8_t)min(max(r, -128), 127);
+    }
+  }
+  if (q.count_sat) {   // this tensor's clipped outputs (the derive kernel cleared the pair)
+    sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+    sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    if ((threadIdx.x & 31) == 0) {
+      if (sat_below) atomicAdd(&st->last_sat_below, (uint32_t)sat_below);
+      if (sat_above) atomicAdd(&st->last_sat_above, (uint32_t)sat_above);
+    }
   }
 }
 
@@ -638,11 +656,8 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
-  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
-    q.sr = 1;
-    q.sr_seed = p.yq->seed;
-    q.sr_iter = p.yq->step;
-  }
+  if (kOut == kOutInt8) qparams_output_mode(q, p.yq->rounding, p.yq->seed, p.yq->step);
+  int sat_below = 0, sat_above = 0;
   const float s_acc = q.s_acc;
   const int zx = q.zx;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = s_acc;
@@ -669,11 +684,16 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
         const uint4 wv = *reinterpret_cast<const uint4*>(p.w + (int64_t)(r * p.S + s) * p.C + cg * 16);
         const uint32_t xa[4] = {xv.x, xv.y, xv.z, xv.w};
         const uint32_t wa[4] = {wv.x, wv.y, wv.z, wv.w};
+        if (p.w_zp != 0) {   // asymmetric weights: both zero points taken out term by term (padded taps were skipped above)
 #pragma unroll
-        for (int e = 0; e < 16; ++e) acc[e] += sx8(xa[e >> 2], e & 3) * sx8(wa[e >> 2], e & 3);
+          for (int e = 0; e < 16; ++e) acc[e] += (sx8(xa[e >> 2], e & 3) - zx) * (sx8(wa[e >> 2], e & 3) - p.w_zp);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) acc[e] += sx8(xa[e >> 2], e & 3) * sx8(wa[e >> 2], e & 3);
+        }
       }
     }
-    if (zx != 0) {
+    if (zx != 0 && p.w_zp == 0) {
       const int cls = p.rowcls[ho] * p.ncolcls + p.colcls[wo];
       const int32_t* cr = p.corr + (int64_t)cls * p.C + cg * 16;
 #pragma unroll
@@ -688,12 +708,7 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
     if constexpr (kOut == kOutInt8) {
       uint32_t w[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        int c[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) c[k] = q.fast ? requant_acc<true>(acc[4 * e + k], q) : requant_acc<false>(acc[4 * e + k], q);
-        w[e] = q.sr ? pack4_sr(acc[4 * e], acc[4 * e + 1], acc[4 * e + 2], acc[4 * e + 3], o + 4 * e, q) : pack_sat4(c[0], c[1], c[2], c[3]);
-      }
+      for (int e = 0; e < 4; ++e) w[e] = quant4_acc(acc[4 * e], acc[4 * e + 1], acc[4 * e + 2], acc[4 * e + 3], o + 4 * e, q, sat_below, sat_above);
       *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
     } else {
       uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + o;
@@ -708,6 +723,14 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
     }
   }
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
+  if (q.count_sat) {   // clipped outputs: one atomic pair per warp that saw any
+    sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+    sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    if ((threadIdx.x & 31) == 0) {
+      if (sat_below) atomicAdd(&p.yq->sat_below, (uint32_t)sat_below);
+      if (sat_above) atomicAdd(&p.yq->sat_above, (uint32_t)sat_above);
+    }
+  }
   mn = __reduce_min_sync(0xffffffffu, mn);
   mx = __reduce_max_sync(0xffffffffu, mx);
   const int warp = threadIdx.x >> 5;
@@ -729,6 +752,155 @@ __global__ void __launch_bounds__(256) depthwise_kernel(const DwParams p) {
 }
 
 
+// Backward data of a depthwise layer, any stride (Sec. 3.1, backward pass), by the definition:
+//   dx(n,hi,wi,c) = sum over (r,s) with ho = (hi + pad_h - r) / stride_h, wo = (wi + pad_w - s) / stride_w integral and
+//   inside the output image of (dy(n,ho,wo,c) - z_dy) * (w(c,r,s) - z_w).
+// One thread: one input pixel x 16 channels; p describes the FORWARD layer (H x W input, Ho x Wo output), p.x is dY,
+// p.w the weights tap-major [R*S][C] (not turned).  Same epilogue as every other kernel.
+template <int kOut>
+__global__ void __launch_bounds__(256) depthwise_bwd_kernel(const DwParams p) {
+  __shared__ int red_min[8], red_max[8];
+  QParams q;
+  q.s_acc = __fmul_rn(p.xq->scale, *p.w_scale);
+  q.zx = p.xq->zero_point;
+  q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
+  q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
+  qparams_finish(q);
+  if (kOut == kOutInt8) qparams_output_mode(q, p.yq->rounding, p.yq->seed, p.yq->step);
+  int sat_below = 0, sat_above = 0;
+  const int zdy = q.zx;
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
+  const int cgs = p.C / 16;
+  const int64_t total = (int64_t)p.N * p.H * p.W * cgs;
+  int mn = INT32_MAX, mx = INT32_MIN;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int cg = (int)(idx % cgs);
+    int64_t t = idx / cgs;
+    const int wi = (int)(t % p.W);
+    t /= p.W;
+    const int hi = (int)(t % p.H);
+    const int n = (int)(t / p.H);
+    int acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0;
+    for (int r = 0; r < p.R; ++r) {
+      const int th = hi + p.pad_h - r;
+      if (th < 0 || th % p.stride_h != 0) continue;
+      const int ho = th / p.stride_h;
+      if (ho >= p.Ho) continue;
+      for (int s = 0; s < p.S; ++s) {
+        const int tw = wi + p.pad_w - s;
+        if (tw < 0 || tw % p.stride_w != 0) continue;
+        const int wo = tw / p.stride_w;
+        if (wo >= p.Wo) continue;
+        const uint4 gv = *reinterpret_cast<const uint4*>(p.x + (((int64_t)n * p.Ho + ho) * p.Wo + wo) * p.C + cg * 16);
+        const uint4 wv = *reinterpret_cast<const uint4*>(p.w + (int64_t)(r * p.S + s) * p.C + cg * 16);
+        const uint32_t ga[4] = {gv.x, gv.y, gv.z, gv.w};
+        const uint32_t wa[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] += (sx8(ga[e >> 2], e & 3) - zdy) * (sx8(wa[e >> 2], e & 3) - p.w_zp);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      mn = min(mn, acc[e]);
+      mx = max(mx, acc[e]);
+    }
+    const int64_t o = (((int64_t)n * p.H + hi) * p.W + wi) * p.C + cg * 16;
+    if constexpr (kOut == kOutInt8) {
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) w[e] = quant4_acc(acc[4 * e], acc[4 * e + 1], acc[4 * e + 2], acc[4 * e + 3], o + 4 * e, q, sat_below, sat_above);
+      *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + o) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + o;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        uint32_t w[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(acc[4 * e + k]), q.s_acc)) : (uint32_t)acc[4 * e + k];
+        *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+  if (q.count_sat) {
+    sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+    sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    if ((threadIdx.x & 31) == 0) {
+      if (sat_below) atomicAdd(&p.yq->sat_below, (uint32_t)sat_below);
+      if (sat_above) atomicAdd(&p.yq->sat_above, (uint32_t)sat_above);
+    }
+  }
+  mn = __reduce_min_sync(0xffffffffu, mn);
+  mx = __reduce_max_sync(0xffffffffu, mx);
+  const int warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) {
+    red_min[warp] = mn;
+    red_max[warp] = mx;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int e = 1; e < (int)(blockDim.x >> 5); ++e) {
+      mn = min(mn, red_min[e]);
+      mx = max(mx, red_max[e]);
+    }
+    if (mn <= mx) {
+      atomicMin(&p.yq->acc_min, mn);
+      atomicMax(&p.yq->acc_max, mx);
+    }
+  }
+}
+
+// Asymmetric weights (z_w != 0): sum (a - z_a)(w - z_w) = [sum (a - z_a) w] - z_w * sum (a - z_a), the sums over the taps
+// inside the image and all channels.  The bracket is what the layer kernels form; this pre-pass writes the second term,
+// one number per output pixel, which their epilogue subtracts.  bwd = 0: pixel (n,ho,wo) of the forward output, sum
+// over its input window; bwd = 1: pixel (n,hi,wi) of the input gradient, sum over the output-gradient pixels that reach it.
+__global__ void __launch_bounds__(256) rowsum_kernel(const int8_t* __restrict__ a, const hq_range_state* __restrict__ aq, hq_conv_desc d, int Ho, int Wo,
+                                                     int bwd, int zw, int32_t* __restrict__ out, int64_t total) {
+  const int za = aq->zero_point;
+  const int Ca = bwd ? d.K : d.C;                 // channels of the operand that is summed
+  const int Ha = bwd ? Ho : d.H, Wa = bwd ? Wo : d.W;
+  const int PH = bwd ? d.H : Ho, PW = bwd ? d.W : Wo;   // image of the pixels the sums are for
+  const bool vec = (Ca & 3) == 0;
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+    const int pw_ = (int)(idx % PW);
+    const int ph_ = (int)((idx / PW) % PH);
+    const int n = (int)(idx / ((int64_t)PW * PH));
+    int sum = 0, cnt = 0;
+    for (int r = 0; r < d.R; ++r) {
+      int ah;
+      if (bwd) {
+        const int th = ph_ + d.pad_h - r;
+        if (th < 0 || th % d.stride_h != 0) continue;
+        ah = th / d.stride_h;
+      } else {
+        ah = ph_ * d.stride_h - d.pad_h + r;
+      }
+      if (ah < 0 || ah >= Ha) continue;
+      for (int s = 0; s < d.S; ++s) {
+        int aw;
+        if (bwd) {
+          const int tw = pw_ + d.pad_w - s;
+          if (tw < 0 || tw % d.stride_w != 0) continue;
+          aw = tw / d.stride_w;
+        } else {
+          aw = pw_ * d.stride_w - d.pad_w + s;
+        }
+        if (aw < 0 || aw >= Wa) continue;
+        const int8_t* src = a + (((int64_t)n * Ha + ah) * Wa + aw) * Ca;
+        if (vec) {
+          for (int c = 0; c < Ca; c += 4) sum = __dp4a(*reinterpret_cast<const int*>(src + c), 0x01010101, sum);
+        } else {
+          for (int c = 0; c < Ca; ++c) sum += src[c];
+        }
+        ++cnt;
+      }
+    }
+    out[idx] = zw * (sum - za * cnt * Ca);
+  }
+}
+
 // 3x3, stride 1: thread = one 32-bit word of channels (4 channels) x 8 consecutive output pixels of a row.
 // The 36 weights of its channels stay in registers, each already shifted into its byte lane so that one dp4a
 // against the input word multiplies exactly one channel (the other three lanes meet zeros).  Input words are
@@ -746,11 +918,8 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
-  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
-    q.sr = 1;
-    q.sr_seed = p.yq->seed;
-    q.sr_iter = p.yq->step;
-  }
+  if (kOut == kOutInt8) qparams_output_mode(q, p.yq->rounding, p.yq->seed, p.yq->step);
+  int sat_below = 0, sat_above = 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
   const int CW = p.C / 4;
   const int cw = threadIdx.x % CW, slot = threadIdx.x / CW;
@@ -819,11 +988,7 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
         mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
         const int64_t o = (((int64_t)n * p.Ho + ho) * p.Wo + wo) * p.C + cw * 4;
         if constexpr (kOut == kOutInt8) {
-          const uint32_t w = q.sr     ? pack4_sr(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q)
-                             : q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q), requant_acc<true>(acc[j][2], q),
-                                                  requant_acc<true>(acc[j][3], q))
-                                      : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
-                                                  requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+          const uint32_t w = quant4_acc(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q, sat_below, sat_above);
           *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
         } else {
           uint32_t w[4];
@@ -836,6 +1001,14 @@ __global__ void __launch_bounds__(256) depthwise3x3_kernel(const DwParams p, int
     }
   }
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
+  if (q.count_sat) {   // clipped outputs: one atomic pair per warp that saw any
+    sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+    sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    if ((threadIdx.x & 31) == 0) {
+      if (sat_below) atomicAdd(&p.yq->sat_below, (uint32_t)sat_below);
+      if (sat_above) atomicAdd(&p.yq->sat_above, (uint32_t)sat_above);
+    }
+  }
   mn = __reduce_min_sync(0xffffffffu, mn);
   mx = __reduce_max_sync(0xffffffffu, mx);
   const int warp = threadIdx.x >> 5;
@@ -907,11 +1080,8 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
   q.inv_scale = (kOut == kOutInt8) ? p.yq->inv_scale : 1.0f;
   q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
   qparams_finish(q);
-  if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
-    q.sr = 1;
-    q.sr_seed = p.yq->seed;
-    q.sr_iter = p.yq->step;
-  }
+  if (kOut == kOutInt8) qparams_output_mode(q, p.yq->rounding, p.yq->seed, p.yq->step);
+  int sat_below = 0, sat_above = 0;
   if (blockIdx.x == 0 && threadIdx.x == 0) p.yq->acc_scale = q.s_acc;
   for (int i = threadIdx.x; i < p.ncls * p.C; i += blockDim.x) zc_s[i] = q.zx * p.corr[i];
   for (int i = threadIdx.x; i < p.Ho; i += blockDim.x) rcls_s[i] = p.rowcls[i];
@@ -981,11 +1151,7 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
             mx = max(__vimax3_s32(mx, acc[j][0], acc[j][1]), max(acc[j][2], acc[j][3]));
             const int64_t o = o0 + (int64_t)j * p.C;
             if constexpr (kOut == kOutInt8) {
-              const uint32_t w = q.sr     ? pack4_sr(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q)
-                                 : q.fast ? pack_sat4(requant_acc<true>(acc[j][0], q), requant_acc<true>(acc[j][1], q),
-                                                      requant_acc<true>(acc[j][2], q), requant_acc<true>(acc[j][3], q))
-                                          : pack_sat4(requant_acc<false>(acc[j][0], q), requant_acc<false>(acc[j][1], q),
-                                                      requant_acc<false>(acc[j][2], q), requant_acc<false>(acc[j][3], q));
+              const uint32_t w = quant4_acc(acc[j][0], acc[j][1], acc[j][2], acc[j][3], o, q, sat_below, sat_above);
               *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(p.out) + o) = w;
             } else {
               uint32_t w[4];
@@ -1002,6 +1168,14 @@ __global__ void __launch_bounds__(512) depthwise3x3_tiled_kernel(const DwParams 
     if (threadIdx.x == 0 && tile + 2 * (int)gridDim.x < total) issue(tile + 2 * gridDim.x, buf);
   }
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
+  if (q.count_sat) {   // clipped outputs: one atomic pair per warp that saw any
+    sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+    sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    if ((threadIdx.x & 31) == 0) {
+      if (sat_below) atomicAdd(&p.yq->sat_below, (uint32_t)sat_below);
+      if (sat_above) atomicAdd(&p.yq->sat_above, (uint32_t)sat_above);
+    }
+  }
   mn = __reduce_min_sync(0xffffffffu, mn);
   mx = __reduce_max_sync(0xffffffffu, mx);
   const int warp = threadIdx.x >> 5;
@@ -1041,7 +1215,7 @@ cudaError_t launch_dynamic_derive(hq_range_state* st, cudaStream_t s, bool overl
   return launch_overlapped(dynamic_derive_kernel, 1, 1, 0, s, overlap, st);
 }
 
-cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, hq_range_state* st, int num_sms, cudaStream_t s,
                                  bool overlap) {
   const int threads = 256;
   int64_t want = (count / 16 + threads - 1) / threads;
@@ -1179,6 +1353,27 @@ cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_rang
   return cudaGetLastError();
 }
 
+cudaError_t launch_rowsum(const int8_t* a, const hq_range_state* aq, const hq_conv_desc& d, int Ho, int Wo, int bwd, int zw, int32_t* out,
+                          cudaStream_t s) {
+  const int64_t total = bwd ? (int64_t)d.N * d.H * d.W : (int64_t)d.N * Ho * Wo;
+  const int blocks = (int)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 16));
+  rowsum_kernel<<<blocks, 256, 0, s>>>(a, aq, d, Ho, Wo, bwd, zw, out, total);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_depthwise_bwd(const DwParams& p, int out_mode, int num_sms, cudaStream_t s) {
+  const int64_t total = (int64_t)p.N * p.H * p.W * (p.C / 16);
+  int64_t want = (total + 255) / 256;
+  int blocks = (int)(want > (int64_t)num_sms * 8 ? (int64_t)num_sms * 8 : want);
+  if (blocks < 1) blocks = 1;
+  switch (out_mode) {
+    case kOutInt8: depthwise_bwd_kernel<kOutInt8><<<blocks, 256, 0, s>>>(p); break;
+    case kOutF32: depthwise_bwd_kernel<kOutF32><<<blocks, 256, 0, s>>>(p); break;
+    default: depthwise_bwd_kernel<kOutAcc><<<blocks, 256, 0, s>>>(p); break;
+  }
+  return cudaGetLastError();
+}
+
 uint32_t depthwise_tiled_smem_bytes(const DwParams& p) {
   return 2u * p.patch_stride + (uint32_t)p.ncls * p.C * 4u + (uint32_t)p.Ho + (uint32_t)p.Wo + 256u;
 }
@@ -1207,7 +1402,7 @@ cudaError_t launch_depthwise_tiled(const DwParams& p, const CUtensorMap& tmap, i
 
 cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s, bool overlap) {
   const int CW = p.C / 4;
-  if (p.R == 3 && p.S == 3 && p.stride_h == 1 && p.stride_w == 1 && CW <= 256) {
+  if (p.R == 3 && p.S == 3 && p.stride_h == 1 && p.stride_w == 1 && CW <= 256 && p.w_zp == 0) {
     const int slots = 256 / CW;                           // pixel groups per block
     const int threads = ((slots * CW + 31) / 32) * 32;
     const int groups_w = (p.Wo + kDwPix - 1) / kDwPix;

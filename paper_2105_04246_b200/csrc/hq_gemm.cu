@@ -128,6 +128,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int red_min[kEpilogueWarps], red_max[kEpilogueWarps];
+  __shared__ int red_below[kEpilogueWarps], red_above[kEpilogueWarps];   // saturation counts (tensors that ask for them)
   __shared__ uint32_t tapoff_s[kMaxTaps];      // kModeHalo: start shift of tap t in 16-byte units
   __shared__ uint8_t cls_s[1024];              // border classes of rows [0,512) and columns [512,1024) when they fit
 
@@ -614,11 +615,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       q.zp = (kOut == kOutInt8) ? p.yq->zero_point : 0;
       qparams_finish(q);
       qparams_bound(q, p.acc_bound);
-      if (kOut == kOutInt8 && p.yq->rounding == HQ_ROUND_STOCHASTIC) {
-        q.sr = 1;
-        q.sr_seed = p.yq->seed;
-        q.sr_iter = p.yq->step;
-      }
+      if (kOut == kOutInt8) qparams_output_mode(q, p.yq->rounding, p.yq->seed, p.yq->step);
     }
     if (blockIdx.x == 0 && ew == 0 && lane == 0) p.yq->acc_scale = q.s_acc;
     // The epilogue's tables are filled here, by the epilogue warps alone, while the first operand tiles are in flight:
@@ -640,6 +637,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       asm volatile("bar.sync 1, %0;" ::"r"(kEpiThreads) : "memory");
     }
     int mn = INT32_MAX, mx = INT32_MIN;
+    int sat_below = 0, sat_above = 0;
     const int rn = row / (p.Ht * p.Wt);
     const int rh = (row / p.Wt) % p.Ht;
     const int rw = row % p.Wt;
@@ -649,7 +647,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const bool has_corr = p.corr != nullptr;
     // per-layer part of the condition for the straight-line pass (see below)
     const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.row_term == nullptr &&
-                            p.zc_in_smem && has_corr;
+                            p.zc_in_smem && has_corr && !q.count_sat;
     for (int local_tile = group; ; local_tile += ngroups) {
       const int tile = own_tile(local_tile);
       if (tile < 0) break;
@@ -723,10 +721,16 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           for (int e = 0; e < CW; ++e)
             if (e < nvalid) v[e] += p.bias[col0 + c0 + e];
         }
-        if (p.row_term != nullptr && row_valid) {   // flat layers: the output row is the pixel index
-          const int rt = p.row_term[pix];
+        if (p.row_term != nullptr && row_valid) {   // one number per output pixel
+          if (p.rt_fold == 1) {
+            const int rt = p.row_term[pix];
 #pragma unroll
-          for (int e = 0; e < CW; ++e) v[e] -= rt;
+            for (int e = 0; e < CW; ++e) v[e] -= rt;
+          } else {   // the GEMM row holds rt_fold pixels side by side
+#pragma unroll
+            for (int e = 0; e < CW; ++e)
+              if (e < nvalid) v[e] -= p.row_term[pix * p.rt_fold + (col0 + c0 + e) / p.rt_cols];
+          }
         }
         if (nvalid == CW) {   // two independent chains, then merged: short dependency depth
           int lo[2], hi[2];
@@ -750,9 +754,9 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         if (nvalid > 0) {
           if constexpr (kOut == kOutInt8) {
             uint32_t w[CW / 4];
+            int r[CW];   // rounded grid coordinate + zero point, before saturation
             if (q.sr) {   // stochastic rounding, one draw per element (shapes that miss the straight-line pass)
               const int64_t e0 = pix * p.ldY + p.out_col0 + col0 + c0;
-              int r[CW];
               if (nvalid == CW && (e0 & 7) == 0) {   // two aligned blocks of eight elements: one generator call each
 #pragma unroll
                 for (int b = 0; b < 2; ++b) {
@@ -769,19 +773,20 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                              ? (q.fast ? requant_acc_sr<true>(v[e], sr_draw1(q, e0 + e), q) : requant_acc_sr<false>(v[e], sr_draw1(q, e0 + e), q))
                              : 0;
               }
-#pragma unroll
-              for (int e = 0; e < CW / 4; ++e) w[e] = pack_sat4(r[4 * e + 0], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
             } else if (q.fast) {
 #pragma unroll
-              for (int e = 0; e < CW / 4; ++e)
-                w[e] = pack_sat4(requant_acc<true>(v[4 * e + 0], q), requant_acc<true>(v[4 * e + 1], q), requant_acc<true>(v[4 * e + 2], q),
-                                 requant_acc<true>(v[4 * e + 3], q));
+              for (int e = 0; e < CW; ++e) r[e] = requant_acc<true>(v[e], q);
             } else {
 #pragma unroll
-              for (int e = 0; e < CW / 4; ++e)
-                w[e] = pack_sat4(requant_acc<false>(v[4 * e + 0], q), requant_acc<false>(v[4 * e + 1], q), requant_acc<false>(v[4 * e + 2], q),
-                                 requant_acc<false>(v[4 * e + 3], q));
+              for (int e = 0; e < CW; ++e) r[e] = requant_acc<false>(v[e], q);
             }
+            if (q.count_sat) {
+#pragma unroll
+              for (int e = 0; e < CW; ++e)
+                if (e < nvalid) count_clipped(r[e], sat_below, sat_above);
+            }
+#pragma unroll
+            for (int e = 0; e < CW / 4; ++e) w[e] = pack_sat4(r[4 * e + 0], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0 + c0;
             if (out_vec == 16) store_bytes16<16>(dst, w, nvalid);
             else if (out_vec == 8) store_bytes16<8>(dst, w, nvalid);
@@ -895,19 +900,31 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     // statistics: registers -> warp -> CTA -> one atomic pair per CTA
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);
+    if (q.count_sat) {
+      sat_below = __reduce_add_sync(0xffffffffu, sat_below);
+      sat_above = __reduce_add_sync(0xffffffffu, sat_above);
+    }
     if (lane == 0) {
       red_min[ew] = mn;
       red_max[ew] = mx;
+      red_below[ew] = sat_below;
+      red_above[ew] = sat_above;
     }
     asm volatile("bar.sync 1, %0;" ::"r"(kEpilogueWarps * 32) : "memory");
     if (ew == 0 && lane == 0) {
       for (int e = 1; e < kEpilogueWarps; ++e) {
         mn = min(mn, red_min[e]);
         mx = max(mx, red_max[e]);
+        sat_below += red_below[e];
+        sat_above += red_above[e];
       }
       if (mn <= mx) {
         atomicMin(&p.yq->acc_min, mn);
         atomicMax(&p.yq->acc_max, mx);
+      }
+      if (q.count_sat) {
+        if (sat_below) atomicAdd(&p.yq->sat_below, (uint32_t)sat_below);
+        if (sat_above) atomicAdd(&p.yq->sat_above, (uint32_t)sat_above);
       }
     }
   }

@@ -109,7 +109,9 @@ struct GemmParams {
   const int32_t* bias;                // [Nout] or null
   int32_t b_slice;                    // kModeTap, streamed weights: image n of the tile space reads operand B at reduction offset n * b_slice
                                       // (the reduction of one GEMM cut into slices that run as "images"; 0 otherwise)
-  const int32_t* row_term;            // [output rows] or null: subtracted from every accumulator of the row (flat layers only)
+  const int32_t* row_term;            // [output pixels] or null: subtracted from every accumulator of the pixel (weight zero point times
+                                      // the pixel's input sum; the weight gradient's input-zero-point term)
+  int32_t rt_fold, rt_cols;           // a GEMM row holds rt_fold pixels of rt_cols columns each (folded 1x1 layers; else 1, Nout)
   float acc_bound;                    // upper bound of |accumulator| before the bias: reduction length x 255 x 128
   const hq_range_state* xq;
   const float* w_scale;
@@ -145,6 +147,7 @@ struct DwParams {                     // depthwise (CUDA cores)
   const float* w_scale;
   hq_range_state* yq;
   void* out;
+  int32_t w_zp;                       // weight zero point; non-zero layers run the generic kernel with (x - z_x) * (w - z_w) formed directly
   // tiled 3x3 kernel: output tile of TR rows x TWt columns, input patch of (TR + 2) x (TWt + 2) pixels in shared memory
   int32_t TR, TWt, tiles_h, tiles_w, slots, ncls;
   uint32_t patch_bytes;               // bytes one TMA box delivers
@@ -216,7 +219,7 @@ cudaError_t launch_stats_pack(const hq_range_state* st, int count, int32_t* buf,
 cudaError_t launch_stats_unpack(hq_range_state* st, int count, const int32_t* buf, cudaStream_t s);
 // MMA-only throughput probe (measurement): one CTA or CTA pair per SM, `chunks` x 32 MMAs of 128 (pair: 256) x bn x 32 each
 cudaError_t launch_mma_peak(int pair, int bn, int chunks, int num_sms, int32_t* status, cudaStream_t s, uint64_t* ops);
-cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, const hq_range_state* st, int num_sms, cudaStream_t s,
+cudaError_t launch_quantize_pass(const float* y, int8_t* out, int64_t count, hq_range_state* st, int num_sms, cudaStream_t s,
                                  bool overlap);
 cudaError_t launch_prep_weights(const int8_t* W, int8_t* Wmat, int Nout, int ntaps, int Cpad, int Ksrc, int R, int S, int Csrc,
                                 const int8_t* tap_r, const int8_t* tap_s, int transposed, int blockdiag_g, cudaStream_t s);
@@ -240,6 +243,12 @@ cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int 
                                 const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
                                    cudaStream_t s);
+// sum over the in-image taps and the channels of (a - z_a), times zw, per output pixel of the layer (forward: over the
+// input windows; backward data: over the output-gradient pixels that reach the input pixel): the weight-zero-point term
+cudaError_t launch_rowsum(const int8_t* a, const hq_range_state* aq, const hq_conv_desc& d, int Ho, int Wo, int bwd, int zw, int32_t* out,
+                          cudaStream_t s);
+// backward data of a depthwise layer with any stride, direct arithmetic (one input pixel x 16 channels per thread)
+cudaError_t launch_depthwise_bwd(const DwParams& p, int out_mode, int num_sms, cudaStream_t s);
 cudaError_t launch_dw_dense(const int8_t* W, int8_t* Wd, int taps, int c0, int cw, cudaStream_t s);
 cudaError_t launch_dw_prep(const int8_t* W, int8_t* Wt, int32_t* corr, int C, int R, int S, const uint32_t* rowmasks, int nrowcls,
                            const uint32_t* colmasks, int ncolcls, int flip, cudaStream_t s);
@@ -296,6 +305,17 @@ struct hq_prepared_weights {
   hq_conv_desc desc{};
   hq_direction dir = HQ_DIR_FWD;
   bool depthwise = false;
+  bool dw_bwd_direct = false;         // depthwise backward data that runs the direct kernel (strided layers, non-zero weight zero point)
+  int8_t* dw_w_plain = nullptr;       // its weights, tap-major [R*S][C], not turned
+  int32_t w_zp = 0;                   // weight zero point (asymmetric weights); 0: symmetric
+  int32_t* row_term = nullptr;        // w_zp != 0: scratch for w_zp * (input sum of every output pixel), written by each call
+  size_t row_term_elems = 0;
+  // prepared weights of a linear layer (hq_linear_prepare)
+  bool linear = false;
+  int lin_N = 0, lin_K = 0, lin_Kp = 0, lin_maxM = 0;
+  int8_t* lin_w = nullptr;            // [N][Kp], zero padded to a multiple of 16 columns
+  int32_t* lin_corr = nullptr;        // column sums of the weights (zero padded), for the input zero point
+  int8_t* lin_xpad = nullptr;         // Kp != K: room for the padded copy of the input, lin_maxM rows
   hq_conv_desc dw_run{};              // geometry the depthwise kernel runs: desc itself (forward) or, for backward data of a stride-1
                                       // layer, the forward layer over the output gradient with the turned filter
   mutable bool used = false;          // set by the first layer call: later calls know that the tables were complete long before

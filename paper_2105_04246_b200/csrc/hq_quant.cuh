@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "hq.h"
+
 namespace hq {
 
 struct QParams {
@@ -16,11 +18,13 @@ struct QParams {
   int noclamp;     // fast, and |u| < 2^22 for every accumulator the layer can produce: the lower clamp is not needed
   int sr;          // stochastic rounding (the output state's `rounding`); draws keyed on (sr_seed, sr_iter, element index)
   uint32_t sr_seed, sr_iter;
+  int count_sat;   // count the outputs the clamp changes (the output state's HQ_COUNT_SATURATION flag)
 };
 
 __device__ __forceinline__ void qparams_finish(QParams& q) {
   q.sr = 0;
   q.sr_seed = q.sr_iter = 0u;
+  q.count_sat = 0;
   q.magic_sub = 0x4B400000 - q.zp;
   q.fast = (isfinite(q.inv_scale) && q.inv_scale != 0.0f && isfinite(q.s_acc)) ? 1 : 0;
   q.noclamp = 0;
@@ -170,12 +174,62 @@ __device__ __forceinline__ uint32_t pack_sat4(int q0, int q1, int q2, int q3) {
   return d;
 }
 
+// rounding mode and statistics flags of the tensor a kernel writes (`rounding` word of its range state; `step` = the
+// state's update count at the time the draws are taken)
+__device__ __forceinline__ void qparams_output_mode(QParams& q, uint32_t rounding, uint32_t seed, uint32_t step) {
+  if ((rounding & HQ_ROUND_MODE_MASK) == HQ_ROUND_STOCHASTIC) {
+    q.sr = 1;
+    q.sr_seed = seed;
+    q.sr_iter = step;
+  }
+  q.count_sat = (rounding & HQ_COUNT_SATURATION) ? 1 : 0;
+}
+
+// Saturation statistic (Sec. 4: "the proportion of values that lie outside the quantization grid", as counts): r is the
+// rounded grid coordinate plus the zero point, before the saturating pack; counted when the pack changes it.
+__device__ __forceinline__ void count_clipped(int r, int& below, int& above) {
+  below += r < -128 ? 1 : 0;
+  above += r > 127 ? 1 : 0;
+}
+// four rounded values -> four codes; counts the clipped ones when the tensor asks for it
+__device__ __forceinline__ uint32_t finish4(int r0, int r1, int r2, int r3, const QParams& q, int& below, int& above) {
+  if (q.count_sat) {
+    count_clipped(r0, below, above);
+    count_clipped(r1, below, above);
+    count_clipped(r2, below, above);
+    count_clipped(r3, below, above);
+  }
+  return pack_sat4(r0, r1, r2, r3);
+}
+
 template <bool kClamp>
 __device__ __forceinline__ uint32_t requant_pack4(int a0, int a1, int a2, int a3, const QParams& q, const QPacked& k) {
   int r0, r1, r2, r3;
   requant_acc2<kClamp>(a0, a1, q, k, r0, r1);
   requant_acc2<kClamp>(a2, a3, q, k, r2, r3);
   return pack_sat4(r0, r1, r2, r3);
+}
+
+// four accumulators whose first element has linear index e (a multiple of 4) -> four codes, whatever the rounding mode
+__device__ __forceinline__ uint32_t quant4_acc(int a0, int a1, int a2, int a3, int64_t e, const QParams& q, int& below, int& above) {
+  int r0, r1, r2, r3;
+  if (q.sr) {
+    uint32_t h[8];
+    sr_draws8(q, (uint64_t)e >> 3, h);
+    const int o = (int)(e & 4);
+    if (q.fast) {
+      r0 = requant_acc_sr<true>(a0, h[o], q); r1 = requant_acc_sr<true>(a1, h[o + 1], q);
+      r2 = requant_acc_sr<true>(a2, h[o + 2], q); r3 = requant_acc_sr<true>(a3, h[o + 3], q);
+    } else {
+      r0 = requant_acc_sr<false>(a0, h[o], q); r1 = requant_acc_sr<false>(a1, h[o + 1], q);
+      r2 = requant_acc_sr<false>(a2, h[o + 2], q); r3 = requant_acc_sr<false>(a3, h[o + 3], q);
+    }
+  } else if (q.fast) {
+    r0 = requant_acc<true>(a0, q); r1 = requant_acc<true>(a1, q); r2 = requant_acc<true>(a2, q); r3 = requant_acc<true>(a3, q);
+  } else {
+    r0 = requant_acc<false>(a0, q); r1 = requant_acc<false>(a1, q); r2 = requant_acc<false>(a2, q); r3 = requant_acc<false>(a3, q);
+  }
+  return finish4(r0, r1, r2, r3, q, below, above);
 }
 
 // four accumulators whose first element has linear index e (a multiple of 4) -> four codes with stochastic rounding

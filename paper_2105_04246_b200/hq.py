@@ -24,14 +24,16 @@ OP_LINEAR, OP_CONV_FWD, OP_CONV_BWD_DATA = 0, 1, 2
 # every extern "C" symbol include/hq.h declares
 EXPORTS = ["hq_create", "hq_destroy", "hq_status_string", "hq_last_error", "hq_get_async_error", "hq_launch_count", "hq_pair_launch_count",
            "hq_set_option",
-           "hq_weights_prepare", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
+           "hq_weights_prepare", "hq_weights_prepare_zp", "hq_linear_prepare", "hq_linear_fwd_prepared", "hq_weights_release", "hq_linear_fwd", "hq_conv_fwd", "hq_conv_bwd_data", "hq_range_update",
            "hq_dynamic_quant", "hq_dynamic_quant_static", "hq_debug_accumulate", "hq_linear_wgrad", "hq_conv_wgrad",
            "hq_stats_pack", "hq_stats_unpack", "hq_mma_peak_probe"]
 
-# numpy view of hq_range_state (48 bytes)
+# numpy view of hq_range_state (64 bytes)
 RANGE_STATE_DTYPE = np.dtype([("acc_min", "<i4"), ("acc_max", "<i4"), ("acc_scale", "<f4"), ("step", "<u4"), ("q_min", "<f4"),
-                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("rounding", "<u4"), ("seed", "<u4"), ("dynamic_eta", "<f4")])
-assert RANGE_STATE_DTYPE.itemsize == 48
+                              ("q_max", "<f4"), ("scale", "<f4"), ("inv_scale", "<f4"), ("zero_point", "<i4"), ("rounding", "<u4"), ("seed", "<u4"), ("dynamic_eta", "<f4"),
+                              ("sat_below", "<u4"), ("sat_above", "<u4"), ("last_sat_below", "<u4"), ("last_sat_above", "<u4")])
+assert RANGE_STATE_DTYPE.itemsize == 64
+STATE_BYTES = RANGE_STATE_DTYPE.itemsize
 INT32_MAX, INT32_MIN = 2**31 - 1, -2**31
 
 
@@ -71,6 +73,9 @@ def lib():
         L.hq_pair_launch_count.argtypes = [vp]; L.hq_pair_launch_count.restype = C.c_uint64
         L.hq_set_option.argtypes = [vp, C.c_char_p, i32]
         L.hq_weights_prepare.argtypes = [vp, vp, C.POINTER(ConvDesc), C.c_int, vp, C.POINTER(vp)]
+        L.hq_weights_prepare_zp.argtypes = [vp, vp, C.POINTER(ConvDesc), C.c_int, vp, i32, C.POINTER(vp)]
+        L.hq_linear_prepare.argtypes = [vp, vp, i32, i32, vp, i32, i32, C.POINTER(vp)]
+        L.hq_linear_fwd_prepared.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp, vp, vp]
         L.hq_weights_release.argtypes = [vp, vp]
         L.hq_linear_fwd.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp]
         L.hq_conv_fwd.argtypes = [vp, vp, C.POINTER(ConvDesc), vp, vp, vp, vp, vp, vp]
@@ -156,10 +161,23 @@ class Context:
             raise HqError(st, lib().hq_last_error(self.handle).decode())
 
     # ---- calls, named as in include/hq.h ------------------------------------------------------
-    def weights_prepare(self, stream, desc: ConvDesc, direction: int, W) -> PreparedWeights:
+    def weights_prepare(self, stream, desc: ConvDesc, direction: int, W, w_zero_point: int = 0) -> PreparedWeights:
         out = C.c_void_p()
-        self._check(lib().hq_weights_prepare(self.handle, _stream(stream), C.byref(desc), int(direction), _ptr(W), C.byref(out)))
+        if w_zero_point:
+            self._check(lib().hq_weights_prepare_zp(self.handle, _stream(stream), C.byref(desc), int(direction), _ptr(W), int(w_zero_point),
+                                                    C.byref(out)))
+        else:
+            self._check(lib().hq_weights_prepare(self.handle, _stream(stream), C.byref(desc), int(direction), _ptr(W), C.byref(out)))
         return PreparedWeights(self, out.value, desc, int(direction))
+
+    def linear_prepare(self, stream, N: int, K: int, W, w_zero_point: int = 0, max_M: int = 0) -> PreparedWeights:
+        out = C.c_void_p()
+        self._check(lib().hq_linear_prepare(self.handle, _stream(stream), int(N), int(K), _ptr(W), int(w_zero_point), int(max_M), C.byref(out)))
+        return PreparedWeights(self, out.value, None, DIR_FWD)
+
+    def linear_fwd_prepared(self, stream, M, X, xq, pw: PreparedWeights, w_scale, bias, Y, yq):
+        self._check(lib().hq_linear_fwd_prepared(self.handle, _stream(stream), int(M), _ptr(X), _ptr(xq), pw.handle, _ptr(w_scale), _ptr(bias),
+                                                 _ptr(Y), _ptr(yq)))
 
     def linear_fwd(self, stream, M, N, K, X, xq, W, w_scale, bias, Y, yq):
         self._check(lib().hq_linear_fwd(self.handle, _stream(stream), M, N, K, _ptr(X), _ptr(xq), _ptr(W), _ptr(w_scale), _ptr(bias),
@@ -222,8 +240,11 @@ class Context:
         return int(lib().hq_pair_launch_count(self.handle))
 
 
-def linear_op(M, N, K, X, xq, W, w_scale, bias=None) -> OpDesc:
-    return OpDesc(OP_LINEAR, M, N, K, None, _ptr(X), _ptr(xq), _ptr(W), _ptr(bias), None, _ptr(w_scale))
+def linear_op(M, N, K, X, xq, W, w_scale, bias=None, pw: PreparedWeights | None = None) -> OpDesc:
+    """pw: weights from linear_prepare (N, K and W are then taken from the handle)."""
+    op = OpDesc(OP_LINEAR, M, N, K, None, _ptr(X), _ptr(xq), _ptr(W), _ptr(bias), None if pw is None else pw.handle, _ptr(w_scale))
+    op._keep = (pw,)
+    return op
 
 
 def conv_op(kind: int, desc: ConvDesc, X, xq, pw: PreparedWeights, w_scale) -> OpDesc:
@@ -234,6 +255,7 @@ def conv_op(kind: int, desc: ConvDesc, X, xq, pw: PreparedWeights, w_scale) -> O
 
 # ---- range-state helpers (host-side packing of the plain-data struct) -------------------------------
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
+COUNT_SATURATION = 0x100      # flag in `rounding`: count the outputs outside the grid (sat_below / sat_above)
 
 
 def new_states(count: int, sr_seed: int | None = None) -> np.ndarray:

@@ -15,7 +15,7 @@ from __future__ import annotations
 import torch
 import torch.distributed as dist
 
-STATE_WORDS = 12          # hq_range_state is 12 x 32-bit words; words 0 and 1 are acc_min and acc_max
+STATE_WORDS = 16          # hq_range_state is 16 x 32-bit words; words 0 and 1 are acc_min and acc_max
 
 
 def allreduce_stats(states: torch.Tensor, group=None) -> None:

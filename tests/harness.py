@@ -40,20 +40,27 @@ class GpuLayer:
     """kind: 'linear' | 'conv_fwd' | 'conv_bwd'.  For conv kinds `shape` is a dict of conv_desc arguments."""
 
     def __init__(self, ctx: hq.Context, kind: str, W: QTensor, shape: dict | None = None, bias: np.ndarray | None = None, eta: float = 0.9,
-                 sr_seed: int | None = None):
+                 sr_seed: int | None = None, count_sat: bool = False, prepared: bool = False, max_M: int = 0):
+        """W.zero_point != 0: asymmetric weights (prepared with their zero point).  count_sat: the output state asks for the
+        saturation counts.  prepared (linear): weights go through hq_linear_prepare / hq_linear_fwd_prepared."""
         self.ctx, self.kind, self.eta = ctx, kind, eta
         self.dev = torch.device("cuda", ctx.device)
         self.W = torch.from_numpy(np.ascontiguousarray(W.q)).to(self.dev)
         self.w_scale = torch.tensor([W.scale], dtype=torch.float32, device=self.dev)
         self.bias = None if bias is None else torch.from_numpy(np.ascontiguousarray(bias, dtype=np.int32)).to(self.dev)
-        self.yq = hq.states_to_device(hq.new_states(1, sr_seed), self.dev)   # sr_seed: stochastic rounding of this layer's output
+        st = hq.new_states(1, sr_seed)                                        # sr_seed: stochastic rounding of this layer's output
+        if count_sat:
+            st["rounding"] |= hq.COUNT_SATURATION
+        self.yq = hq.states_to_device(st, self.dev)
         self.stream = torch.cuda.current_stream(self.dev)
         if kind == "linear":
             self.N, self.K = W.q.shape
             self.pw = None
+            if prepared or W.zero_point != 0:
+                self.pw = ctx.linear_prepare(self.stream, self.N, self.K, self.W, W.zero_point, max_M)
         else:
             self.desc = hq.conv_desc(**shape)
-            self.pw = ctx.weights_prepare(self.stream, self.desc, hq.DIR_FWD if kind == "conv_fwd" else hq.DIR_BWD_DATA, self.W)
+            self.pw = ctx.weights_prepare(self.stream, self.desc, hq.DIR_FWD if kind == "conv_fwd" else hq.DIR_BWD_DATA, self.W, W.zero_point)
             d = self.desc
             Ho = (d.H + 2 * d.pad_h - d.R) // d.stride_h + 1
             Wo = (d.W + 2 * d.pad_w - d.S) // d.stride_w + 1
@@ -73,7 +80,7 @@ class GpuLayer:
 
     def _op(self, xd, xq):
         if self.kind == "linear":
-            return hq.linear_op(xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias)
+            return hq.linear_op(xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias, pw=self.pw)
         return hq.conv_op(hq.OP_CONV_FWD if self.kind == "conv_fwd" else hq.OP_CONV_BWD_DATA, self.desc, xd, xq, self.pw, self.w_scale)
 
     def state(self) -> np.ndarray:
@@ -109,7 +116,9 @@ class GpuLayer:
         xd, xq, out_shape = self._put(x)
         g_y = Guarded(out_shape, torch.int8, self.dev, fill=99)
         y = g_y.t
-        if self.kind == "linear":
+        if self.kind == "linear" and self.pw is not None:
+            self.ctx.linear_fwd_prepared(self.stream, xd.shape[0], xd, xq, self.pw, self.w_scale, self.bias, y, self.yq)
+        elif self.kind == "linear":
             self.ctx.linear_fwd(self.stream, xd.shape[0], self.N, self.K, xd, xq, self.W, self.w_scale, self.bias, y, self.yq)
         elif self.kind == "conv_fwd":
             self.ctx.conv_fwd(self.stream, self.desc, xd, xq, self.pw, self.w_scale, y, self.yq)
@@ -141,10 +150,10 @@ class OracleLayer:
 
     def accumulate(self, x: QTensor) -> np.ndarray:
         if self.kind == "linear":
-            return O.linear_acc(x.q, x.zero_point, self.W.q, 0, self.bias)
+            return O.linear_acc(x.q, x.zero_point, self.W.q, self.W.zero_point, self.bias)
         if self.kind == "conv_fwd":
-            return O.conv_fwd_acc(self.desc, x.q, x.zero_point, self.W.q, 0)
-        return O.conv_bwd_data_acc(self.desc, x.q, x.zero_point, self.W.q, 0)
+            return O.conv_fwd_acc(self.desc, x.q, x.zero_point, self.W.q, self.W.zero_point)
+        return O.conv_bwd_data_acc(self.desc, x.q, x.zero_point, self.W.q, self.W.zero_point)
 
     def s_acc(self, x: QTensor) -> float:
         return O.acc_scale(x.scale, self.W.scale)

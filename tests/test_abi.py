@@ -39,4 +39,4 @@ def test_range_state_layout_matches_header():
         if decl:
             names += [re.sub(r"\[.*\]", "", n).strip() for n in decl.split(None, 1)[1].split(",")]
     assert names == list(hq.RANGE_STATE_DTYPE.names)
-    assert hq.RANGE_STATE_DTYPE.itemsize == 48
+    assert hq.RANGE_STATE_DTYPE.itemsize == 64

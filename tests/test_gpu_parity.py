@@ -25,21 +25,24 @@ def ctx():
     c.close()
 
 
-def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1, sr_seed=None, pair=-1):
+def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, staging=-1, repack=-1, depthwise=-1, sr_seed=None, pair=-1,
+                    count_sat=False, prepared=False, max_M=0):
     ctx.set_option("staging", staging)      # how the input reaches shared memory; results must not depend on it
     ctx.set_option("pair", pair)            # one CTA per 128-row tile or CTA pairs on 256-row tiles; likewise
     ctx.set_option("repack", repack)        # how few-channel inputs are repacked; likewise
     ctx.set_option("depthwise", depthwise)  # CUDA-core kernel or dense expansion on the tensor cores; likewise
     try:
-        g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
+        g = GpuLayer(ctx, kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed, count_sat=count_sat, prepared=prepared, max_M=max_M)
     finally:
         ctx.set_option("staging", -1)
         ctx.set_option("pair", -1)
         ctx.set_option("repack", -1)
         ctx.set_option("depthwise", -1)
     o = OracleLayer(kind, W, shape, bias=bias, eta=eta, sr_seed=sr_seed)
+    clipped_total = 0
     for t in range(iters):
         x = make_x(t)
+        before = o.layer.state.copy()
         if t == 0:
             acc, mn, mx, s_acc = g.accumulate(x)
             ref = o.accumulate(x)
@@ -60,7 +63,17 @@ def _run_iterations(ctx, kind, W, shape, make_x, iters, bias=None, eta=0.9, stag
         st = g.state()
         assert_state_close(st, o.layer.state)
         assert (int(st["acc_min"]), int(st["acc_max"])) == (hq.INT32_MAX, hq.INT32_MIN)   # slot emptied by the update
+        assert (int(st["sat_below"]), int(st["sat_above"])) == (0, 0)
+        if count_sat:
+            # what the quantizer clipped: with the range that quantized this tensor (dynamic: its own; hindsight: the previous one)
+            used = o.layer.state if res.mode == "dynamic" else before
+            want = O.saturation(res.acc, res.s_acc, used, sr_seed, iteration=before.step)
+            assert (int(st["last_sat_below"]), int(st["last_sat_above"])) == want, (t, res.mode, want)
+            clipped_total += sum(want)
+        else:
+            assert (int(st["last_sat_below"]), int(st["last_sat_above"])) == (0, 0)
     assert ctx.get_async_error() == 0
+    g.clipped_total = clipped_total
     return g, o
 
 
@@ -290,14 +303,6 @@ def test_depthwise_bwd_data(ctx, name, dw_staging):
         ctx.set_option("depthwise_staging", -1)
 
 
-def test_depthwise_bwd_data_strided_is_refused(ctx):
-    dev = torch.device("cuda", ctx.device)
-    W = torch.zeros((32, 3, 3), dtype=torch.int8, device=dev)
-    with pytest.raises(hq.HqError) as e:
-        ctx.weights_prepare(None, hq.conv_desc(2, 11, 11, 32, 32, 3, 3, stride=2, pad=1, groups=32), hq.DIR_BWD_DATA, W)
-    assert e.value.status == 2
-
-
 # ---- protocol and edge cases ---------------------------------------------------------------------
 def test_teacher_forced_state_and_saturation(ctx):
     """The oracle is fed the GPU's own state before each step: isolates the layer kernel from the
@@ -357,13 +362,13 @@ def test_rejected_calls_launch_nothing(ctx):
     ws = torch.ones(1, dtype=torch.float32, device=dev)
     n0 = ctx.launch_count()
     with pytest.raises(hq.HqError) as e:
-        ctx.linear_fwd(None, 64, 64, 64, x[1:], st, x, ws, None, x, st[48:])      # misaligned X
+        ctx.linear_fwd(None, 64, 64, 64, x[1:], st, x, ws, None, x, st[hq.STATE_BYTES:])      # misaligned X
     assert e.value.status == 3
     with pytest.raises(hq.HqError) as e:
-        ctx.linear_fwd(None, 0, 64, 64, x, st, x, ws, None, x, st[48:])
+        ctx.linear_fwd(None, 0, 64, 64, x, st, x, ws, None, x, st[hq.STATE_BYTES:])
     assert e.value.status == 1
     with pytest.raises(hq.HqError) as e:
-        ctx.linear_fwd(None, 64, 64, 64, x, None, x, ws, None, x, st[48:])
+        ctx.linear_fwd(None, 64, 64, 64, x, None, x, ws, None, x, st[hq.STATE_BYTES:])
     assert e.value.status == 1
     with pytest.raises(hq.HqError) as e:
         ctx.weights_prepare(None, hq.conv_desc(1, 8, 8, 16, 3, 3, 3, 1, 1), hq.DIR_BWD_DATA, x)   # backward data with K = 3

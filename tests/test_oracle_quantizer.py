@@ -217,3 +217,69 @@ def test_running_minmax_recurrence_and_use_of_the_current_tensor(eta):
     _, run_codes = O.dynamic_running(big, 1.0, run, eta)
     assert not np.array_equal(res.q, run_codes)
     assert (run.q_min, run.q_max) == (layer.state.q_min, layer.state.q_max)    # same Eq. 2-3 numbers, used one step earlier
+
+
+# ---- saturation statistic (Sec. 4: "the proportion of values that lie outside the quantization grid") ----------------
+def test_saturation_counts_by_eye():
+    q = O.derive(O.Range(q_min=0.0, q_max=2.55, step=1))             # 255 steps of 0.01 from 0: zero point -128
+    assert q.zero_point == -128 and abs(q.scale - 0.01) < 1e-8
+    s_acc = 1e-3
+    #            -0.6 steps: clipped   -0.4: rounds to 0   0   2.554: level 255   2.556: level 256, clipped   far out
+    acc = np.array([-6, -4, 0, 2554, 2556, 9000, -9000, 1270], np.int32)
+    assert O.saturation(acc, s_acc, q) == (2, 2)
+    codes = O.quantize(acc, s_acc, q)
+    assert codes.tolist() == [-128, -128, -128, 127, 127, 127, -128, -1]
+    assert O.saturation(np.zeros(7, np.int32), s_acc, q) == (0, 0)   # real zero is always on the grid
+
+
+def test_saturation_counts_against_float64_comparison():
+    g = np.random.default_rng(41)
+    for lo, hi in [(-0.7, 2.3), (0.0, 5.0), (-3.0, 0.0), (-1e-3, 1e-3)]:
+        q = O.derive(O.Range(q_min=lo, q_max=hi, step=1))
+        s_acc = (hi - lo) / 50000.0
+        acc = g.integers(-60000, 60000, size=20000).astype(np.int32)
+        below, above = O.saturation(acc, s_acc, q)
+        # the definition in float64: the level a value rounds to, compared with the end levels
+        u = acc.astype(np.float64) * np.float64(np.float32(s_acc)) / np.float64(q.scale) + q.zero_point
+        near_tie = (np.abs(u - (-128.5)) < 1e-3) | (np.abs(u - 127.5) < 1e-3)
+        b64, a64 = int((np.rint(u[~near_tie]) < -128).sum()), int((np.rint(u[~near_tie]) > 127).sum())
+        n_tie = int(near_tie.sum())
+        assert n_tie < 20 and b64 <= below <= b64 + n_tie and a64 <= above <= a64 + n_tie
+        assert below + above > 0
+        # counted elements are a subset of those that carry an end code, and codes strictly inside are never counted
+        codes = O.quantize(acc, s_acc, q).astype(np.int64)
+        assert below <= int((codes == -128).sum()) and above <= int((codes == 127).sum())
+        # the first and last level stand for themselves: a value exactly on an end level is not clipped
+        s = np.float64(q.scale)
+        for level, want in ((-128, (0, 0)), (127, (0, 0)), (-129, (1, 0)), (128, (0, 1))):
+            on = np.array([int(np.rint((level - q.zero_point) * s / np.float64(np.float32(s_acc))))], np.int32)
+            u_on = on[0] * np.float64(np.float32(s_acc)) / s + q.zero_point
+            if abs(u_on - level) < 0.4:                                  # the accumulator grid is fine enough to hit the level
+                assert O.saturation(on, s_acc, q) == want, (level, u_on)
+
+
+def test_saturation_independent_of_order_and_additive_over_shards():
+    g = np.random.default_rng(42)
+    q = O.derive(O.Range(q_min=-1.0, q_max=0.5, step=3))
+    acc = g.integers(-3000, 3000, size=5001).astype(np.int32)
+    whole = O.saturation(acc, 1e-3, q)
+    assert whole[0] > 0 and whole[1] > 0
+    parts = [O.saturation(p, 1e-3, q) for p in np.array_split(g.permutation(acc), 7)]
+    assert whole == (sum(p[0] for p in parts), sum(p[1] for p in parts))
+
+
+def test_saturation_with_stochastic_rounding_counts_what_the_quantizer_clips():
+    g = np.random.default_rng(43)
+    q = O.derive(O.Range(q_min=-0.4, q_max=1.1, step=5))
+    acc = g.integers(-1500, 2000, size=4000).astype(np.int32)
+    s_acc, seed, it, first = 1e-3, 99, 5, 64
+    below, above = O.saturation(acc, s_acc, q, sr_seed=seed, iteration=it, first=first)
+    # the same draws as the (separately pinned) stochastic quantizer: floor(u + r) + z outside the levels
+    y = (acc.astype(np.float32) * np.float32(s_acc)).astype(np.float32)
+    u = (y * np.float32(q.inv_scale)).astype(np.float32)
+    r = (np.array([O.draw16(seed, it, first + i) for i in range(acc.size)], np.float32) / np.float32(65536.0)).astype(np.float32)
+    c = np.floor((u + r).astype(np.float32)).astype(np.int64) + q.zero_point
+    assert (below, above) == (int((c < -128).sum()), int((c > 127).sum()))
+    assert below > 0 and above > 0
+    det = O.saturation(acc, s_acc, q)
+    assert abs(det[0] - below) <= 0.02 * acc.size and abs(det[1] - above) <= 0.02 * acc.size   # differs only within one level of the ends
