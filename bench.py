@@ -539,7 +539,8 @@ def run_gpu(args):
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
     del host_in, host_out
-    assert ctx.get_async_error() == 0, "a device-side wait expired during the benchmark"
+    code = ctx.get_async_error()
+    assert code == 0, f"a device-side wait expired during the benchmark (code {code})"
     if dist is not None:
         t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -574,7 +575,8 @@ def run_gpu(args):
                           "repeats": r2, "steps_per_repeat": cyc2,
                           "dynamic": {"value": round(w2.ops / (msd2 * 1e-3) / 1e12, 3), "ms_per_step": round(msd2, 6)},
                           "hbm_bytes_per_step": {"hindsight": int(sum(w2.static_bytes)), "dynamic": int(sum(w2.dynamic_bytes))}}
-            assert ctx.get_async_error() == 0, f"a device-side wait expired during {cfg}"
+            code = ctx.get_async_error()
+            assert code == 0, f"a device-side wait expired during {cfg} (code {code})"
             w2.release()
             del w2
             torch.cuda.empty_cache()

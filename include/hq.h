@@ -167,9 +167,11 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              choice (default), 0 = direct global loads, 1 = input patches staged in shared memory by TMA
  *              where the shape allows.
  *   "repack":  how spatial filters over a channel count that is not a multiple of 16 (the RGB stem),
- *              prepared AFTER this call, are repacked for the tensor cores: -1 = chosen per layer
- *              (default), 0 = whole filter patches per output pixel, 1 = horizontal filter windows
- *              per input row where the shape allows.
+ *              prepared AFTER this call, are brought to the tensor cores: -1 = chosen per layer
+ *              (default), 0 = whole filter patches per output pixel gathered into a library-owned matrix,
+ *              1 = horizontal filter windows per input row gathered into a library-owned tensor where the
+ *              shape allows, 2 = the fused kernel that gathers the filter windows in shared memory (nothing
+ *              repacked in global memory) where the shape allows, else as -1.
  *   "epilogue_groups": layers prepared AFTER this call: -1 = chosen per layer (default); g = 0, 1, 2: the sixteen
  *              epilogue warps form 2^g groups that drain alternate tiles (at most one group per accumulator buffer).
  *   "col_tiles": into how many column tiles (each a multiple of 16 columns, at most 256) the output channels of
@@ -240,8 +242,10 @@ hq_status hq_linear_fwd_prepared(hq_ctx* ctx, void* stream, int32_t M, const int
 /* Forward convolution as an implicit GEMM (Sec. 3.1), same epilogue as hq_linear_fwd.
  * Padding is zero in the real domain.  pw must come from hq_weights_prepare(.., HQ_DIR_FWD, ..)
  * with the same descriptor.  groups == C selects the depthwise kernel.  Spatial filters over a channel
- * count that is not a multiple of 16 (an RGB stem) run a gather pre-pass into a library-owned
- * [pixels][R*S*C] matrix that the handle allocates at preparation time. */
+ * count that is not a multiple of 16 (an RGB stem) run a fused kernel that gathers the filter windows in shared
+ * memory when W * C is a multiple of 16, K a multiple of 16 of at most 256 and the filter is one of the built sizes
+ * (7x7x3, 5x5x3, 5x5x4, 3x3x3, 3x3x4, 3x3x5); other such shapes run a gather pre-pass into a library-owned tensor
+ * that the handle allocates at preparation time. */
 hq_status hq_conv_fwd(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                       const int8_t* X, const hq_range_state* xq,
                       const hq_prepared_weights* pw, const float* w_scale,

@@ -605,6 +605,25 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     return HQ_OK;
   }
   const int Ho = out_dim(desc->H, desc->pad_h, desc->R, desc->stride_h), Wo = out_dim(desc->W, desc->pad_w, desc->S, desc->stride_w);
+  if (pw->gather) {   // few input channels: the fused kernel; the image as {W*C/4 words, H, N}, one box of R rows per tile
+    GatherParams g = pw->gp;
+    g.xq = inq; g.w_scale = w_scale; g.yq = outq; g.out = out;
+    g.weights_early = (ctx->overlap && pw->used) ? 1 : 0;
+    pw->used = true;
+    CUtensorMap tm;
+    const uint64_t row_bytes = (uint64_t)desc->W * desc->C;
+    uint64_t dims[3] = {row_bytes / 4, (uint64_t)desc->H, (uint64_t)desc->N};
+    uint64_t strides[2] = {row_bytes, row_bytes * desc->H};
+    uint32_t box[3] = {g.raw_pitch / 4, (uint32_t)desc->R, 1u};
+    uint32_t es[3] = {1, 1, 1};
+    CUresult r = ctx->encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<int8_t*>(in), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(ctx, HQ_ERR_CUDA, "tensor map encoding failed (CUresult %d)", (int)r);
+    const int grid = std::max(1, std::min(g.num_tiles, ctx->num_sms));
+    HQ_CUDA(ctx, launch_gather_conv(g, tm, out_mode, grid, pw->gather_smem, s, ctx->overlap));
+    ctx->launches += 1;
+    return HQ_OK;
+  }
   // operand A is the forward input (fwd) or the output gradient (bwd data)
   const int aC = dir == HQ_DIR_FWD ? desc->C : desc->K;
   const int aH = dir == HQ_DIR_FWD ? desc->H : Ho;
@@ -937,7 +956,7 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     return HQ_OK;
   }
   if (std::string(key) == "repack") {
-    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "repack must be -1, 0 or 1");
+    if (value < -1 || value > 2) return fail(ctx, HQ_ERR_INVALID_ARG, "repack must be -1, 0, 1 or 2");
     ctx->force_repack = value;
     return HQ_OK;
   }
@@ -1109,6 +1128,82 @@ hq_status prepare_conv_body(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
         // Channel counts no TMA box can address (the RGB stem).  Preferred: a pre-pass gathers, per output column, the
         // horizontal filter windows of stride_h consecutive input rows into a library-owned tensor X2 of
         // Cg = stride_h * SB bytes per pixel; over X2 the layer is a stride-1 convolution with vertical taps only.
+        // Preferred where the shape allows: the fused kernel that gathers the filter windows in shared memory (no repacked
+        // copy of the input in global memory).  Needs image rows that a TMA box can address (W*C a multiple of 16), one
+        // column tile (K a multiple of 16, at most 256), an instantiated (R, S*C) and symmetric weights.
+        {
+          const int SC = d.S * d.C, Kp = round_up(d.R * SC, 32);
+          const uint32_t pitch = (uint32_t)round_up((127 * d.stride_w + d.S) * d.C + 15 + 8, 16);
+          std::vector<uint8_t> grc, gcc;
+          MaskVec grm, gcm;
+          TapVec gdh, gdw;
+          for (int r = 0; r < d.R; ++r) gdh.push_back(r - d.pad_h);
+          for (int q = 0; q < d.S; ++q) gdw.push_back(q - d.pad_w);
+          border_classes(Ho, d.stride_h, gdh, d.H, grc, grm);
+          border_classes(Wo, d.stride_w, gdw, d.W, gcc, gcm);
+          const int corr_ld = round_up(d.K, 16);
+          const size_t zc_bytes = grm.size() * gcm.size() * (size_t)corr_ld * 4;
+          if (gather_conv_supported(d.R, SC) && (d.W * d.C) % 16 == 0 && d.K % 16 == 0 && d.K <= 256 && pitch <= 1024 && grm.size() <= 16 &&
+              gcm.size() <= 16 && zc_bytes <= kMaxZcBytes && w_zero_point == 0 && (ctx->force_repack < 0 || ctx->force_repack == 2) &&
+              (int64_t)d.N * Ho * ceil_div(Wo, kTileM) < INT32_MAX) {
+            GatherParams& g = pw->gp;
+            g.N = d.N; g.H = d.H; g.W = d.W; g.C = d.C; g.Ho = Ho; g.Wo = Wo; g.R = d.R; g.S = d.S;
+            g.stride_h = d.stride_h; g.stride_w = d.stride_w; g.pad_h = d.pad_h; g.pad_w = d.pad_w;
+            g.BN = d.K;
+            g.tiles_w = ceil_div(Wo, kTileM);
+            g.num_tiles = d.N * Ho * g.tiles_w;
+            g.raw_pitch = pitch;
+            g.raw_box_bytes = pitch * (uint32_t)d.R;
+            g.raw_stage_stride = (g.raw_box_bytes + 127u) & ~127u;
+            g.a_stage_bytes = (uint32_t)kTileM * (uint32_t)Kp;
+            g.stages_raw = 4;
+            g.off_w = 0;
+            g.off_zc = (uint32_t)round_up(d.K * Kp, 128);
+            g.off_raw = (uint32_t)round_up((int)(g.off_zc + zc_bytes), 1024);
+            g.off_a = (uint32_t)round_up((int)(g.off_raw + g.stages_raw * g.raw_stage_stride + 64), 1024);
+            const uint32_t budget = 200u * 1024u;
+            g.stages_a = (int)std::min<uint32_t>(8u, (budget - g.off_a) / g.a_stage_bytes);
+            if (g.stages_a >= 2) {
+              pw->gather_smem = g.off_a + (uint32_t)g.stages_a * g.a_stage_bytes + 1024u;
+              g.corr_ld = corr_ld;
+              g.ncolcls = (int)gcm.size();
+              g.zc_elems = (int)(grm.size() * gcm.size()) * corr_ld;
+              g.cls_in_smem = (Ho <= 512 && Wo <= 512) ? 1 : 0;
+              g.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(d.K >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+              uint32_t stride = 32;
+              while ((int)stride < d.K) stride <<= 1;
+              g.tmem_buf_stride = stride;
+              g.tmem_bufs = (int)std::min<uint32_t>(8, 512 / stride);
+              g.tmem_cols = (uint32_t)g.tmem_bufs * stride;
+              g.epi_groups = std::min(3, g.tmem_bufs);
+              g.tmem_bufs_log2 = g.tmem_bufs == 8 ? 3 : (g.tmem_bufs == 4 ? 2 : 1);
+              g.epi_groups_log2 = g.epi_groups == 4 ? 2 : 1;
+              g.fd_tiles_w = make_fastdiv(g.tiles_w);
+              g.fd_Ho = make_fastdiv(Ho);
+              g.status = ctx->d_status;
+              g.acc_bound = (float)(d.R * SC) * 255.0f * 128.0f;
+              int8_t* wm = nullptr;
+              int32_t* corr = nullptr;
+              if ((st = dev_alloc(ctx, pw, (void**)&wm, (size_t)d.K * Kp)) != HQ_OK) return bail(st);
+              if ((st = dev_alloc(ctx, pw, (void**)&corr, zc_bytes)) != HQ_OK) return bail(st);
+              cudaError_t e = cudaMemsetAsync(corr, 0, zc_bytes, s);
+              if (e == cudaSuccess) e = launch_pad_rows(W, wm, d.K, d.R * SC, Kp, s);   // the filter's own order, rows padded to Kp
+              if (e == cudaSuccess) e = launch_gather_corr(W, corr, d.K, d.R, d.S, d.C, grm.data(), (int)grm.size(), gcm.data(), (int)gcm.size(), corr_ld, s);
+              if (e != cudaSuccess) return bail(fail(ctx, HQ_ERR_CUDA, "weight preparation failed: %s", cudaGetErrorString(e)));
+              ctx->launches += 2;
+              g.wmat = wm;
+              g.corr = corr;
+              uint8_t *drc = nullptr, *dcc = nullptr;
+              if ((st = upload(ctx, pw, grc, &drc, s)) != HQ_OK) return bail(st);
+              if ((st = upload(ctx, pw, gcc, &dcc, s)) != HQ_OK) return bail(st);
+              g.rowcls = drc;
+              g.colcls = dcc;
+              pw->gather = true;
+              *out = pw;
+              return HQ_OK;
+            }
+          }
+        }
         const int sh = d.stride_h, sc = d.S * d.C;
         int SB = round_up(sc, 16), Cg = 0;
         if (64 % sh == 0 && sh * SB <= 64) { SB = 64 / sh; Cg = 64; }

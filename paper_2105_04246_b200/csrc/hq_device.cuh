@@ -36,12 +36,13 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
   return t;
 }
 
-// Bounded wait on an mbarrier phase.  Gives up when another role has already given up or
-// after kWaitLimitNs; the first to give up records `code` in the status word.
+// Bounded wait on an mbarrier phase.  Gives up when another role has already given up or after kWaitLimitCycles of this
+// SM's own cycle counter (monotonic and private to the SM; the global nanosecond timer is shared with the host side and
+// may be stepped while a kernel runs); the first to give up records `code` in the status word.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int code,
                                           uint32_t hint_ns = 200u) {
   if (mbar_try(bar, parity, hint_ns)) return true;
-  const uint64_t t0 = global_timer_ns();
+  const long long t0 = clock64();
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try(bar, parity, hint_ns)) return true;
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     __nanosleep(hint_ns >> 2);
     if ((++spins & 15u) == 0u) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) {
+      if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;

@@ -17,85 +17,10 @@
 #include "hq_device.cuh"
 #include "hq_internal.h"
 #include "hq_quant.cuh"
+#include "hq_tc.cuh"
 
 namespace hq {
 namespace {
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major operand whose rows are one swizzle span wide
-// (64 or 128 bytes) and contiguous: 8-row groups are 8 spans apart.  The swizzle is applied to the
-// absolute shared-memory address (the same function the TMA write used), so a start that is
-// shifted by whole rows -- a tile that begins at an arbitrary pixel of a resident patch -- reads
-// the right bytes with the base-offset field left at zero.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, bool sw64) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;
-  d |= (uint64_t)((sw64 ? 512u : 1024u) >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)(sw64 ? 4u : 2u) << 61;
-  return d;
-}
-
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// CTA pair: one instruction drives the tensor cores of both SMs (rows 0..127 of the 256-row tile come from this CTA's
-// operand A, rows 128..255 from the peer's at the same shared-memory offset; each CTA holds half of the rows of B);
-// the commit arrives on the barrier at the same offset in both CTAs.
-__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{ .reg .pred p; setp.ne.b32 p, %4, 0; tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-               "h"((uint16_t)3)
-               : "memory");
-}
-template <bool kPair>
-__device__ __forceinline__ void mma_any(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  if constexpr (kPair) umma_i8_pair(d_tmem, adesc, bdesc, idesc, accumulate);
-  else umma_i8(d_tmem, adesc, bdesc, idesc, accumulate);
-}
-template <bool kPair>
-__device__ __forceinline__ void commit_any(uint32_t bar) {
-  if constexpr (kPair) umma_commit_pair(bar);
-  else umma_commit(bar);
-}
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int* v) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
-        "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// eight columns; the matching wait names the registers, so that no use of them can be scheduled ahead of it while
-// another load is in flight
-__device__ __forceinline__ void tmem_ld8(uint32_t taddr, int (&v)[8]) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
-               : "r"(taddr)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait8(int (&v)[8]) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7])
-               :
-               : "memory");
-}
 
 template <int V>
 __device__ __forceinline__ void store_bytes16(int8_t* p, const uint32_t* w, int nvalid) {
@@ -648,6 +573,12 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     // per-layer part of the condition for the straight-line pass (see below)
     const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.row_term == nullptr &&
                             p.zc_in_smem && has_corr && !q.count_sat;
+    // The tile loop is instantiated once per epilogue variant (kLean >= 0: the straight-line int8 pass with that rounding
+    // for every tile whose columns all lie inside the layer; -1: the general pass only), so that the loop a warp runs holds
+    // one variant's code: fewer instruction-cache misses and branches in the hot loop.
+    auto run_tiles = [&](auto lean_tag) {
+    constexpr int kLean = decltype(lean_tag)::value;
+    const QPacked qk = qpacked(q);
     for (int local_tile = group; ; local_tile += ngroups) {
       const int tile = own_tile(local_tile);
       if (tile < 0) break;
@@ -815,36 +746,15 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       // parameters, no bias, every column of the pass inside the layer, correction table in shared memory (it holds
       // zeros when the input zero point is 0).  Rows outside the image (tile padding) are computed like the others
       // and only kept out of the statistics and the store.
-      const bool lean = lean_layer && col0 + c_end * CW <= p.Nout;
+      const bool lean = kLean >= 0 && col0 + c_end * CW <= p.Nout;
       if (lean) {
         const int32_t* zrow = zc_s + zoff;
         int8_t* dst_row = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0;
         const int64_t elem_row = pix * p.ldY + p.out_col0 + col0;   // linear index in the output tensor of this row's first column
         int tmn = INT32_MAX, tmx = INT32_MIN;
         // eight columns at a time, two register sets: the load of the next eight is in flight while these are processed
-        const QPacked qk = qpacked(q);
         auto half = [&](int (&x)[8], int c, uint32_t& w0, uint32_t& w1) {
-          const int4 ca = *reinterpret_cast<const int4*>(zrow + c), cb = *reinterpret_cast<const int4*>(zrow + c + 4);
-          x[0] -= ca.x; x[1] -= ca.y; x[2] -= ca.z; x[3] -= ca.w;
-          x[4] -= cb.x; x[5] -= cb.y; x[6] -= cb.z; x[7] -= cb.w;
-          tmn = __vimin3_s32(tmn, x[0], x[1]); tmx = __vimax3_s32(tmx, x[0], x[1]);
-          tmn = __vimin3_s32(tmn, x[2], x[3]); tmx = __vimax3_s32(tmx, x[2], x[3]);
-          tmn = __vimin3_s32(tmn, x[4], x[5]); tmx = __vimax3_s32(tmx, x[4], x[5]);
-          tmn = __vimin3_s32(tmn, x[6], x[7]); tmx = __vimax3_s32(tmx, x[6], x[7]);
-          if (q.sr) {   // stochastic rounding: one aligned block of eight elements, one generator call
-            uint32_t h[8];
-            sr_draws8(q, (uint64_t)(elem_row + c) >> 3, h);
-            w0 = pack_sat4(requant_acc_sr<true>(x[0], h[0], q), requant_acc_sr<true>(x[1], h[1], q), requant_acc_sr<true>(x[2], h[2], q),
-                           requant_acc_sr<true>(x[3], h[3], q));
-            w1 = pack_sat4(requant_acc_sr<true>(x[4], h[4], q), requant_acc_sr<true>(x[5], h[5], q), requant_acc_sr<true>(x[6], h[6], q),
-                           requant_acc_sr<true>(x[7], h[7], q));
-          } else if (q.noclamp) {
-            w0 = requant_pack4<false>(x[0], x[1], x[2], x[3], q, qk);
-            w1 = requant_pack4<false>(x[4], x[5], x[6], x[7], q, qk);
-          } else {
-            w0 = requant_pack4<true>(x[0], x[1], x[2], x[3], q, qk);
-            w1 = requant_pack4<true>(x[4], x[5], x[6], x[7], q, qk);
-          }
+          if constexpr (kLean >= 0) lean_half8m<kLean>(x, zrow + c, tmn, tmx, q, qk, elem_row + c, w0, w1);
         };
         int va[8], vb[8];
         tmem_ld8(taddr + c_begin * CW, va);
@@ -897,6 +807,11 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         }
       }
     }
+    };
+    if (!lean_layer) run_tiles(std::integral_constant<int, -1>{});
+    else if (q.sr) run_tiles(std::integral_constant<int, kLeanSr>{});
+    else if (q.noclamp) run_tiles(std::integral_constant<int, kLeanNoClamp>{});
+    else run_tiles(std::integral_constant<int, kLeanClamp>{});
     // statistics: registers -> warp -> CTA -> one atomic pair per CTA
     mn = __reduce_min_sync(0xffffffffu, mn);
     mx = __reduce_max_sync(0xffffffffu, mx);

@@ -24,7 +24,7 @@ constexpr int kMaxStagesA = 12;
 constexpr int kMaxStagesB = 32;
 constexpr uint32_t kSmemBudget = 212 * 1024;              // operand rings + correction table; barriers sit in static shared memory
 constexpr uint32_t kMaxZcBytes = 20 * 1024;               // largest correction table kept in shared memory
-constexpr uint64_t kWaitLimitNs = 2000000000ull;          // bound of every device-side wait
+constexpr long long kWaitLimitCycles = 4000000000ll;      // bound of every device-side wait, in SM cycles (2 to 4 seconds)
 
 // status-word codes written by kernels when a bounded wait expires
 enum AsyncCode : int32_t {
@@ -154,6 +154,42 @@ struct DwParams {                     // depthwise (CUDA cores)
   uint32_t patch_stride;              // patch_bytes rounded up to 128: distance of the two buffers (TMA destinations are 128-byte aligned)
   int32_t* status;                    // device status word (expired waits)
 };
+
+// Fused forward convolution over few input channels (hq_gather.cu): raw input rows by TMA, im2col rows gathered in shared memory
+struct GatherParams {
+  int32_t N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w;
+  int32_t BN;                          // output channels (a multiple of 16, at most 256): one column tile
+  int32_t tiles_w, num_tiles;          // tiles of up to 128 output pixels per output row; N * Ho * tiles_w
+  uint32_t raw_pitch;                  // bytes of one raw row in shared memory = width of the TMA box (a multiple of 16, at most 1024)
+  uint32_t raw_box_bytes, raw_stage_stride;   // raw_pitch * R, and that rounded up to 128
+  uint32_t a_stage_bytes;              // 128 * Kp
+  int32_t stages_raw, stages_a;
+  uint32_t off_w, off_zc, off_raw, off_a;   // byte offsets from the 1024-aligned base of dynamic shared memory
+  const int32_t* corr;                 // [ncls][corr_ld]
+  int32_t zc_elems, corr_ld, ncolcls;
+  const uint8_t* rowcls;               // [Ho]
+  const uint8_t* colcls;               // [Wo]
+  int32_t cls_in_smem;
+  const int8_t* wmat;                  // [BN][Kp]: the filter in its own (r, s, c) order, rows zero padded to Kp
+  const hq_range_state* xq;
+  const float* w_scale;
+  hq_range_state* yq;
+  void* out;
+  int32_t* status;
+  uint32_t idesc, tmem_cols, tmem_buf_stride;
+  int32_t tmem_bufs, epi_groups;       // powers of two
+  int32_t tmem_bufs_log2, epi_groups_log2;
+  FastDiv fd_tiles_w, fd_Ho;
+  int32_t weights_early;
+  float acc_bound;
+};
+struct ClassMasksG {
+  uint32_t row[16], col[16];
+};
+bool gather_conv_supported(int R, int SC);
+cudaError_t launch_gather_conv(const GatherParams& p, const CUtensorMap& tm, int out_mode, int grid, uint32_t smem, cudaStream_t s, bool overlap);
+cudaError_t launch_gather_corr(const int8_t* W, int32_t* corr, int K, int R, int S, int C, const uint32_t* rowmasks, int nrowcls,
+                               const uint32_t* colmasks, int ncolcls, int corr_ld, cudaStream_t s);
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -310,6 +346,10 @@ struct hq_prepared_weights {
   int32_t w_zp = 0;                   // weight zero point (asymmetric weights); 0: symmetric
   int32_t* row_term = nullptr;        // w_zp != 0: scratch for w_zp * (input sum of every output pixel), written by each call
   size_t row_term_elems = 0;
+  // few-channel spatial filter run by the fused gather kernel (hq_gather.cu)
+  bool gather = false;
+  hq::GatherParams gp{};
+  uint32_t gather_smem = 0;
   // prepared weights of a linear layer (hq_linear_prepare)
   bool linear = false;
   int lin_N = 0, lin_K = 0, lin_Kp = 0, lin_maxM = 0;

@@ -210,6 +210,55 @@ __device__ __forceinline__ uint32_t requant_pack4(int a0, int a1, int a2, int a3
   return pack_sat4(r0, r1, r2, r3);
 }
 
+// The straight-line epilogue pass over eight accumulators of one output row: zero-point correction from the shared
+// table (already multiplied by the input zero point), running min/max, requantization, two words of codes.
+// zrow: the eight corrections of these columns; elem: linear index of the first element in the output tensor (a multiple
+// of 8: one generator call covers the eight draws of stochastic rounding).  Requires q.fast.
+// kMode selects the rounding at compile time, so that a kernel's tile loop holds one variant only:
+//   kLeanNoClamp  nearest even, |u| < 2^22 guaranteed (QParams::noclamp)   kLeanClamp  nearest even   kLeanSr  stochastic
+enum LeanMode : int { kLeanNoClamp = 0, kLeanClamp = 1, kLeanSr = 2 };
+__device__ __forceinline__ int lean_mode(const QParams& q) { return q.sr ? kLeanSr : (q.noclamp ? kLeanNoClamp : kLeanClamp); }
+template <int kMode>
+__device__ __forceinline__ void lean_half8c(int (&x)[8], int4 ca, int4 cb, int& tmn, int& tmx, const QParams& q, const QPacked& qk, int64_t elem,
+                                            uint32_t& w0, uint32_t& w1);
+template <int kMode>
+__device__ __forceinline__ void lean_half8m(int (&x)[8], const int32_t* zrow, int& tmn, int& tmx, const QParams& q, const QPacked& qk, int64_t elem,
+                                            uint32_t& w0, uint32_t& w1) {
+  lean_half8c<kMode>(x, *reinterpret_cast<const int4*>(zrow), *reinterpret_cast<const int4*>(zrow + 4), tmn, tmx, q, qk, elem, w0, w1);
+}
+// the same with the eight corrections already in registers (callers that fetch them ahead of the accumulators)
+template <int kMode>
+__device__ __forceinline__ void lean_half8c(int (&x)[8], int4 ca, int4 cb, int& tmn, int& tmx, const QParams& q, const QPacked& qk, int64_t elem,
+                                            uint32_t& w0, uint32_t& w1) {
+  x[0] -= ca.x; x[1] -= ca.y; x[2] -= ca.z; x[3] -= ca.w;
+  x[4] -= cb.x; x[5] -= cb.y; x[6] -= cb.z; x[7] -= cb.w;
+  tmn = __vimin3_s32(tmn, x[0], x[1]); tmx = __vimax3_s32(tmx, x[0], x[1]);
+  tmn = __vimin3_s32(tmn, x[2], x[3]); tmx = __vimax3_s32(tmx, x[2], x[3]);
+  tmn = __vimin3_s32(tmn, x[4], x[5]); tmx = __vimax3_s32(tmx, x[4], x[5]);
+  tmn = __vimin3_s32(tmn, x[6], x[7]); tmx = __vimax3_s32(tmx, x[6], x[7]);
+  if constexpr (kMode == kLeanSr) {   // stochastic rounding: one aligned block of eight elements, one generator call
+    uint32_t h[8];
+    sr_draws8(q, (uint64_t)elem >> 3, h);
+    w0 = pack_sat4(requant_acc_sr<true>(x[0], h[0], q), requant_acc_sr<true>(x[1], h[1], q), requant_acc_sr<true>(x[2], h[2], q),
+                   requant_acc_sr<true>(x[3], h[3], q));
+    w1 = pack_sat4(requant_acc_sr<true>(x[4], h[4], q), requant_acc_sr<true>(x[5], h[5], q), requant_acc_sr<true>(x[6], h[6], q),
+                   requant_acc_sr<true>(x[7], h[7], q));
+  } else if constexpr (kMode == kLeanNoClamp) {
+    w0 = requant_pack4<false>(x[0], x[1], x[2], x[3], q, qk);
+    w1 = requant_pack4<false>(x[4], x[5], x[6], x[7], q, qk);
+  } else {
+    w0 = requant_pack4<true>(x[0], x[1], x[2], x[3], q, qk);
+    w1 = requant_pack4<true>(x[4], x[5], x[6], x[7], q, qk);
+  }
+}
+// the same with the rounding chosen at run time
+__device__ __forceinline__ void lean_half8(int (&x)[8], const int32_t* zrow, int& tmn, int& tmx, const QParams& q, const QPacked& qk, int64_t elem,
+                                           uint32_t& w0, uint32_t& w1) {
+  if (q.sr) lean_half8m<kLeanSr>(x, zrow, tmn, tmx, q, qk, elem, w0, w1);
+  else if (q.noclamp) lean_half8m<kLeanNoClamp>(x, zrow, tmn, tmx, q, qk, elem, w0, w1);
+  else lean_half8m<kLeanClamp>(x, zrow, tmn, tmx, q, qk, elem, w0, w1);
+}
+
 // four accumulators whose first element has linear index e (a multiple of 4) -> four codes, whatever the rounding mode
 __device__ __forceinline__ uint32_t quant4_acc(int a0, int a1, int a2, int a3, int64_t e, const QParams& q, int& below, int& above) {
   int r0, r1, r2, r3;

@@ -128,6 +128,14 @@ FWD_CASES = {
     "3x3_s4_c3": dict(N=2, H=21, W=19, Cin=3, K=16, R=3, S=3, stride=4, pad=1),
     "5x5_s3_c3": dict(N=1, H=20, W=20, Cin=3, K=16, R=5, S=5, stride=3, pad=2),
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
+    # few channels with image rows a TMA box can address (W * C a multiple of 16): the fused gather kernel
+    "7x7_s2_c3_w32_gather": dict(N=2, H=30, W=32, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
+    "7x7_s2_c3_w224_gather": dict(N=1, H=12, W=224, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
+    "3x3_c3_w320_gather": dict(N=2, H=6, W=320, Cin=3, K=32, R=3, S=3, stride=1, pad=1),
+    "5x5_s2_c4_w20_gather": dict(N=1, H=17, W=20, Cin=4, K=16, R=5, S=5, stride=2, pad=1),
+    "3x3_c5_w16_gather": dict(N=3, H=9, W=16, Cin=5, K=48, R=3, S=3, stride=1, pad=1),
+    "5x5_s3_c3_w32_gather": dict(N=2, H=20, W=32, Cin=3, K=16, R=5, S=5, stride=3, pad=2),
+    "3x3_c4_w64_k256_gather": dict(N=2, H=7, W=64, Cin=4, K=256, R=3, S=3, stride=1, pad=0),
     "dw3x3_c144": dict(N=2, H=10, W=12, Cin=144, K=144, R=3, S=3, stride=1, pad=1, groups=144),
     "dw3x3_s2_c32": dict(N=2, H=11, W=11, Cin=32, K=32, R=3, S=3, stride=2, pad=1, groups=32),
     "dw3x3_c64_wide": dict(N=2, H=9, W=150, Cin=64, K=64, R=3, S=3, stride=1, pad=1, groups=64),
@@ -184,10 +192,11 @@ def test_depthwise_cuda_core_staging(ctx, name, dw_staging):
         ctx.set_option("depthwise_staging", -1)
 
 
-@pytest.mark.parametrize("repack", [0, 1])
+@pytest.mark.parametrize("repack", [0, 1, 2])
 @pytest.mark.parametrize("name", [n for n, c in FWD_CASES.items() if c["Cin"] % 16 != 0 and c.get("R", 1) > 1])
 def test_conv_fwd_few_channels_repacking(ctx, name, repack):
-    """Both repackings of few-channel inputs (whole filter patches; horizontal windows per input row) give the oracle's bytes."""
+    """All three ways to bring few-channel inputs to the tensor cores (whole filter patches; horizontal windows per input
+    row; filter windows gathered in shared memory by the fused kernel, where the shape allows) give the oracle's bytes."""
     shape = dict(FWD_CASES[name])
     r = synth.rng(104, len(name), shape["H"], repack)
     W = _weights(r, shape)
