@@ -221,9 +221,9 @@ class GpuWorkload:
             w = synth.weights(g, wsh) if kind != "linear" else synth.uniform_int8(g, wsh, scale=0.01)
             self.W.append(torch.from_numpy(w.q).to(dev))
             self.w_scale.append(torch.tensor([w.scale], dtype=torch.float32, device=dev))
-            if kind == "linear":
+            if kind == "linear":          # weights prepared once: padded copy and column sums cached, one launch per call
                 self.desc.append(None)
-                self.pw.append(None)
+                self.pw.append(ctx.linear_prepare(stream, s.N, s.K, self.W[-1], 0, s.M))
             else:
                 d = hq.conv_desc(s.N, s.H, s.W, s.C, s.K, s.R, s.S, s.stride, s.pad, s.groups)
                 self.desc.append(d)
@@ -266,12 +266,12 @@ class GpuWorkload:
                 self.ws_pool[i] = [self.torch.empty(y.shape, dtype=self.torch.float32, device=self.dev) for _ in range(nws)]
             ws = self.ws_pool[i][j % len(self.ws_pool[i])]
             if kind == "linear":
-                op = hq.linear_op(s.M, s.N, s.K, x, xq, self.W[i], self.w_scale[i])
+                op = hq.linear_op(s.M, s.N, s.K, x, xq, self.W[i], self.w_scale[i], pw=self.pw[i])
             else:
                 op = hq.conv_op(hq.OP_CONV_FWD if kind == "conv_fwd" else hq.OP_CONV_BWD_DATA, self.desc[i], x, xq, self.pw[i], self.w_scale[i])
             ctx.dynamic_quant(stream, op, ws, y, self.state_ptr[i])
         elif kind == "linear":
-            ctx.linear_fwd(stream, s.M, s.N, s.K, x, xq, self.W[i], self.w_scale[i], None, y, self.state_ptr[i])
+            ctx.linear_fwd_prepared(stream, s.M, x, xq, self.pw[i], self.w_scale[i], None, y, self.state_ptr[i])
         elif kind == "conv_fwd":
             ctx.conv_fwd(stream, self.desc[i], x, xq, self.pw[i], self.w_scale[i], y, self.state_ptr[i])
         else:
@@ -377,6 +377,12 @@ def measure_mma_peak(torch, ctx, sampler, sustained_s: float = 4.0):
             "what": "tcgen05.mma kind::i8 128x256x32 (pair: 256x256x32) issued back to back on operand tiles resident in shared memory, every SM, no loads, no epilogue"}
 
 
+def check_waits(ctx, where: str):
+    """Every device-side wait of the kernels is bounded; one that expired leaves a code in the context's status word."""
+    code = ctx.get_async_error()
+    assert code == 0, f"a device-side wait expired (code {code}) during: {where}"
+
+
 def layer_rows(torch, wk, cfg_name, peaks, probe_peak, min_time_s, min_repeats):
     """Per-layer rows of one workload: each layer's launches alone (no update kernel), replayed from a CUDA graph that
     cycles through the layer's whole buffer pool; hindsight and dynamic path."""
@@ -393,7 +399,9 @@ def layer_rows(torch, wk, cfg_name, peaks, probe_peak, min_time_s, min_repeats):
             g_h = capture(torch, lambda st, j, ii=i: wk.layer_call(st, ii, j), reps)
             g_d = capture(torch, lambda st, j, ii=i: wk.layer_call(st, ii, j, dynamic=True), reps)
         ms, lo, hi, r = timed_repeats(torch, g_h.replay, reps, min_time_s, min_repeats)
+        check_waits(wk.ctx, f"{cfg_name} {s.name} in-hindsight")
         msd, lod, hid, rd = timed_repeats(torch, g_d.replay, reps, min_time_s, min_repeats)
+        check_waits(wk.ctx, f"{cfg_name} {s.name} dynamic")
         del g_h, g_d
         us, usd = ms * 1e3, msd * 1e3
         dw = getattr(s, "depthwise", False)
@@ -558,16 +566,19 @@ def run_gpu(args):
             w2 = GpuWorkload(cfg, ctx, dev, seed_key=rank)
             for j in range(2):
                 w2.step(stream, j, dynamic=True)
-            torch.cuda.synchronize()
+            check_waits(ctx, f"{cfg} first dynamic steps")
             w2.step(stream, 0)
-            torch.cuda.synchronize()
+            check_waits(ctx, f"{cfg} first in-hindsight step")
             cyc2 = 2 if w2.chained else max(w2.pool)
             gs = capture(torch, lambda s, j: w2.step(s, j), cyc2)
             gd = capture(torch, lambda s, j: w2.step(s, j, dynamic=True), cyc2)
             for _ in range(3):
                 gs.replay(); gd.replay()
+            check_waits(ctx, f"{cfg} warm-up replays")
             ms2, lo2, hi2, r2 = timed_repeats(torch, gs.replay, cyc2, args.min_time, args.min_repeats)
+            check_waits(ctx, f"{cfg} in-hindsight steps")
             msd2, _, _, _ = timed_repeats(torch, gd.replay, cyc2, args.min_time, args.min_repeats)
+            check_waits(ctx, f"{cfg} dynamic steps")
             del gs, gd
             per_layer += layer_rows(torch, w2, cfg, peaks, probe_peak, args.min_time, args.min_repeats)
             other[cfg] = {"workload": f"{cfg}: " + ", ".join(s.name for _, s, _ in w2.layers), "value": round(w2.ops / (ms2 * 1e-3) / 1e12, 3),
@@ -575,8 +586,7 @@ def run_gpu(args):
                           "repeats": r2, "steps_per_repeat": cyc2,
                           "dynamic": {"value": round(w2.ops / (msd2 * 1e-3) / 1e12, 3), "ms_per_step": round(msd2, 6)},
                           "hbm_bytes_per_step": {"hindsight": int(sum(w2.static_bytes)), "dynamic": int(sum(w2.dynamic_bytes))}}
-            code = ctx.get_async_error()
-            assert code == 0, f"a device-side wait expired during {cfg} (code {code})"
+            check_waits(ctx, f"{cfg} layer rows")
             w2.release()
             del w2
             torch.cuda.empty_cache()

@@ -181,6 +181,8 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              (default), 0 = every CTA works on its own 128-row tile, 1 = pairs of CTAs on neighbouring SMs share
  *              256-row tiles (one tensor-core instruction for both, each CTA holding half of the weight rows)
  *              wherever the layer allows.
+ *   "issuers": upper limit (1, 2 or 3; default 3) of the warps of a CTA that issue tensor-core instructions,
+ *              each for every n-th tile, in layers prepared AFTER this call.
  *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their
  *              set-up may run while the previous kernel in the stream drains; each waits for that
  *              kernel to finish before it reads memory, so stream order is unchanged.  0 = ordinary

@@ -325,9 +325,18 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
     p.mma_issuers = (rings_ok && kiters > 0 && p.num_tiles >= 2 * ctx->num_sms && !p.pair) ? 2 : 1;
     // narrow tiles (64 columns or fewer) keep the tensor core busy for so short a time per tile that a third issuer pays;
     // the weight producer's warp takes that part once resident weights are on their way
-    if (p.mma_issuers == 2 && p.b_resident && p.BN <= 64 && 3 * a_per_tile <= p.stages_a && p.num_tiles >= 3 * ctx->num_sms &&
-        p.tmem_bufs >= 4)
+    // Three issuers share the accumulator buffers unevenly (three does not divide their number), and an issuer's wait for
+    // a drained buffer is only sound when the buffer's previous tile has already been issued, possibly by another issuer.
+    // The kernel gets that from the operand ring (see its issuer loop), provided the ring holds no more than as many tiles
+    // as there are buffers: the ring is shortened to that where needed.
+    const int ring3 = std::min(p.stages_a, p.tmem_bufs * a_per_tile);
+    if (p.mma_issuers == 2 && ctx->max_issuers >= 3 && p.b_resident && p.BN <= 64 && 3 * a_per_tile <= ring3 && ring3 >= 6 &&
+        p.num_tiles >= 3 * ctx->num_sms && p.tmem_bufs >= 4) {
       p.mma_issuers = 3;
+      p.stages_a = ring3;
+      if (p.mode == kModeTap) p.producer_lanes = std::min(p.producer_lanes, p.stages_a);
+    }
+    p.mma_issuers = std::min(p.mma_issuers, ctx->max_issuers);
     // Several tiles per CTA: as many epilogue groups as there are accumulator buffers (at most four), so that a warp
     // pays its per-tile set-up once per several column passes; one or two tiles per CTA: all warps on every tile (the
     // epilogue of the last tile, which nothing overlaps, is then shortest).  Measured on the ResNet-18 shapes.
@@ -973,6 +982,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "pair") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "pair must be -1, 0 or 1");
     ctx->force_pair = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "issuers") {
+    if (value < 1 || value > 3) return fail(ctx, HQ_ERR_INVALID_ARG, "issuers must be 1, 2 or 3");
+    ctx->max_issuers = value;
     return HQ_OK;
   }
   if (std::string(key) == "overlap_launches") {

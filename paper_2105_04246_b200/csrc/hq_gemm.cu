@@ -235,6 +235,16 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         if (tile < 0) break;
         const int buf = local_tile & (nbuf - 1);
         const uint32_t tph = (uint32_t)(local_tile >> nbuf_log2) & 1u;
+        // A parity wait cannot tell "the previous use of this buffer was drained" from "the use before that was drained
+        // and the previous one has not even been issued": the wait below is only sound once tile local_tile - nbuf has
+        // passed this point.  With one or two issuers that tile is this issuer's own (nbuf is a multiple of two).  With
+        // three it belongs to another issuer, which may lag behind this one; then the tile's first operand stage has to be
+        // there first: the producer fills stages in order and reuses a stage only after the MMAs that read it, and the
+        // host keeps the ring no deeper than nbuf tiles, so a filled first stage means tile local_tile - nbuf was issued.
+        if (nissuers > 2) {
+          ok = warp_wait(a_full(stage), phase, abort_flag, p.status, kAsyncMmaFullWait, 200u);
+          if (!ok) break;
+        }
         ok = warp_wait(tempty_bar(buf), tph ^ 1u, abort_flag, p.status, kAsyncMmaTmemEmptyWait, 200u);
         if (!ok) break;
         tc_fence_after();

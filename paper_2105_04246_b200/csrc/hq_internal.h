@@ -311,6 +311,7 @@ struct hq_ctx {
   int force_epi_groups = -1;          // log2 of the epilogue warp groups: -1 chosen per layer, else min(value, log2 of the accumulator buffers)
   int force_cols = -1;                // column tiles: -1 chosen by estimated duration, 0 as wide as the MMA allows, n > 0 at least n
   int force_pair = -1;                // CTA pairs on 256-row tiles: -1 choose per layer, 0 never, 1 wherever the layer allows
+  int max_issuers = 3;                // upper limit of the warps that issue MMAs in one CTA (1, 2 or 3)
   cudaStream_t side[3] = {nullptr, nullptr, nullptr};   // independent launches of one call run side by side (see run_conv)
   cudaEvent_t ev_fork = nullptr, ev_join[3] = {nullptr, nullptr, nullptr};
   bool parallel_subs = true;
