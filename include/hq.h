@@ -165,7 +165,8 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              caller's stream; 0 = one after the other.
  *   "depthwise_staging": CUDA-core depthwise 3x3 stride-1 layers (read at every call): -1 = library's
  *              choice (default), 0 = direct global loads, 1 = input patches staged in shared memory by TMA
- *              where the shape allows.
+ *              where the shape allows, one multiply-accumulate per 4-way dot-product instruction, 2 = the same
+ *              staging with the patch transposed in registers so that one such instruction covers a filter row.
  *   "repack":  how spatial filters over a channel count that is not a multiple of 16 (the RGB stem),
  *              prepared AFTER this call, are brought to the tensor cores: -1 = chosen per layer
  *              (default), 0 = whole filter patches per output pixel gathered into a library-owned matrix,

@@ -570,7 +570,41 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
       ctx->launches += 1;
       return HQ_OK;
     }
-    // 3x3 stride 1 with at most 256 channels: output tiles of 4 rows whose input patch one TMA box stages in shared memory
+    // 3x3 stride 1 with at most 256 channels, transposing kernel: tiles of kDwColRows rows x up to 28 columns, one thread per
+    // channel word and group of 4 columns (see hq_dw3x3.cu)
+    if (desc->R == 3 && desc->S == 3 && desc->stride_h == 1 && desc->stride_w == 1 && desc->C <= 256 && desc->C % 16 == 0 &&
+        (ctx->force_dw_tiled < 0 || ctx->force_dw_tiled == 2) && pw->w_zp == 0) {
+      const int cwords = desc->C / 4;
+      const int groups = std::min(std::min(round_up(Wo, 4) / 4, 7), kDwColMaxThreads / cwords);
+      p.TR = kDwColRows;
+      p.TWt = 4 * groups;
+      p.tiles_h = ceil_div(Ho, p.TR);
+      p.tiles_w = ceil_div(Wo, p.TWt);
+      p.ncls = pw->dw_ncls;
+      p.patch_bytes = (uint32_t)desc->C * (uint32_t)(p.TWt + 2) * (uint32_t)(p.TR + 2);
+      p.patch_stride = (p.patch_bytes + 127u) & ~127u;
+      const int64_t n_tiles = (int64_t)desc->N * p.tiles_h * p.tiles_w;
+      const uint32_t smem = depthwise_col_smem_bytes(p);
+      if (groups >= 1 && groups * cwords >= 64 && n_tiles <= INT32_MAX && smem <= 200u * 1024u) {
+        CUtensorMap tm;
+        uint64_t dims[4] = {(uint64_t)desc->C, (uint64_t)desc->W, (uint64_t)desc->H, (uint64_t)desc->N};
+        uint64_t strides[3] = {(uint64_t)desc->C, (uint64_t)desc->C * desc->W, (uint64_t)desc->C * desc->W * desc->H};
+        uint32_t box[4] = {(uint32_t)desc->C, (uint32_t)(p.TWt + 2), (uint32_t)(p.TR + 2), 1u};
+        uint32_t es[4] = {1, 1, 1, 1};
+        CUresult r = ctx->encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(in), dims, strides, box, es,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return fail(ctx, HQ_ERR_CUDA, "tensor map encoding failed (CUresult %d)", (int)r);
+        // CTAs per SM: by registers (128 per thread, whole warps) and by shared memory (1 KB per CTA is the system's)
+        const int warps = ceil_div(groups * cwords, 32);
+        const int by_regs = 65536 / (warps * 32 * 128), by_smem = (int)((228u * 1024u) / (smem + 1024u));
+        const int per_sm = std::max(1, std::min(std::min(by_regs, by_smem), 8));
+        HQ_CUDA(ctx, launch_depthwise_col(p, tm, out_mode, ctx->num_sms, per_sm, s, false));
+        ctx->launches += 1;
+        return HQ_OK;
+      }
+    }
+    // the same shapes with strips of 8 pixels per thread and one multiply-accumulate per dp4a: output tiles of 4 rows
     if (desc->R == 3 && desc->S == 3 && desc->stride_h == 1 && desc->stride_w == 1 && desc->C <= 256 && ctx->force_dw_tiled != 0 && pw->w_zp == 0) {
       p.TR = 4;
       const int budget = 50 * 1024;   // two patches + tables per CTA, two CTAs per SM
@@ -914,7 +948,7 @@ __attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int dev
   ctx->scratch_elems = 4096;
   if (cudaMalloc((void**)&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc((void**)&ctx->d_scratch, ctx->scratch_elems * sizeof(int32_t)) != cudaSuccess ||
-      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess ||
+      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess || depthwise_col_set_smem_attr(200u * 1024u) != cudaSuccess ||
       !make_side_streams(ctx)) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_scratch) cudaFree(ctx->d_scratch);
@@ -955,7 +989,7 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     return HQ_OK;
   }
   if (std::string(key) == "depthwise_staging") {
-    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "depthwise_staging must be -1, 0 or 1");
+    if (value < -1 || value > 2) return fail(ctx, HQ_ERR_INVALID_ARG, "depthwise_staging must be -1, 0, 1 or 2");
     ctx->force_dw_tiled = value;
     return HQ_OK;
   }

@@ -247,6 +247,12 @@ cudaError_t gemm_set_smem_attr(uint32_t smem_bytes);
 cudaError_t launch_depthwise(const DwParams& p, int out_mode, int num_sms, cudaStream_t s, bool overlap);
 // 3x3 stride-1 depthwise with the input patch staged by TMA (p.TR ... p.status filled in); tmap covers the NHWC input
 cudaError_t launch_depthwise_tiled(const DwParams& p, const CUtensorMap& tmap, int out_mode, int num_sms, cudaStream_t s);
+// 3x3 stride-1 depthwise, columns of tiles of kDwColRows x 4 pixels per thread (hq_dw3x3.cu): TR = kDwColRows, TWt a multiple of 4
+constexpr int kDwColRows = 7;
+constexpr int kDwColMaxThreads = 448;
+cudaError_t launch_depthwise_col(const DwParams& p, const CUtensorMap& tmap, int out_mode, int num_sms, int ctas_per_sm, cudaStream_t s, bool overlap);
+cudaError_t depthwise_col_set_smem_attr(uint32_t smem_bytes);
+uint32_t depthwise_col_smem_bytes(const DwParams& p);
 cudaError_t depthwise_tiled_set_smem_attr(uint32_t smem_bytes);
 uint32_t depthwise_tiled_smem_bytes(const DwParams& p);
 cudaError_t launch_range_update(hq_range_state* st, int count, float eta, cudaStream_t s, bool overlap);

@@ -143,6 +143,7 @@ FWD_CASES = {
     "dw3x3_c256_nopad": dict(N=1, H=11, W=12, Cin=256, K=256, R=3, S=3, stride=1, pad=0, groups=256),
     "dw5x5_c48": dict(N=1, H=13, W=9, Cin=48, K=48, R=5, S=5, stride=1, pad=2, groups=48),
     "dw3x3_c320": dict(N=1, H=7, W=7, Cin=320, K=320, R=3, S=3, stride=1, pad=1, groups=320),
+    "dw3x3_c192_tiles": dict(N=2, H=16, W=61, Cin=192, K=192, R=3, S=3, stride=1, pad=1, groups=192),
 }
 
 
@@ -176,10 +177,11 @@ def test_depthwise_both_paths(ctx, name, depthwise):
     _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, depthwise=depthwise)
 
 
-@pytest.mark.parametrize("dw_staging", [0, 1])
-@pytest.mark.parametrize("name", ["dw3x3_c144", "dw3x3_c64_wide", "dw3x3_c32_ragged", "dw3x3_c256_nopad"])
+@pytest.mark.parametrize("dw_staging", [0, 1, 2])
+@pytest.mark.parametrize("name", ["dw3x3_c144", "dw3x3_c64_wide", "dw3x3_c32_ragged", "dw3x3_c256_nopad", "dw3x3_c192_tiles"])
 def test_depthwise_cuda_core_staging(ctx, name, dw_staging):
-    """CUDA-core depthwise 3x3: direct global loads and TMA-staged patches (several tiles, ragged edges) give the oracle's bytes."""
+    """CUDA-core depthwise 3x3: direct global loads, TMA-staged patches with one product per dot-product instruction, and
+    TMA-staged patches transposed in registers (several tiles in both directions, ragged edges) give the oracle's bytes."""
     shape = dict(FWD_CASES[name])
     r = synth.rng(106, len(name), shape["H"], dw_staging)
     W = _weights(r, shape)
@@ -294,7 +296,7 @@ DW_BWD_CASES = {
 }
 
 
-@pytest.mark.parametrize("dw_staging", [0, 1])
+@pytest.mark.parametrize("dw_staging", [0, 1, 2])
 @pytest.mark.parametrize("name", list(DW_BWD_CASES))
 def test_depthwise_bwd_data(ctx, name, dw_staging):
     """Input gradient of a stride-1 depthwise layer (run as a forward depthwise layer over the output gradient with the
