@@ -61,6 +61,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// one 32-byte store (dst 32-byte aligned): a whole sector per thread
+__device__ __forceinline__ void st_global_v8(uint32_t* dst, const uint32_t* w) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]),
+               "r"(w[6]), "r"(w[7])
+               : "memory");
+}
+
 // n / d for 0 <= n < 2^31 with the multiplier and shift prepared on the host (see make_fastdiv)
 __device__ __forceinline__ int fdiv(int n, FastDiv d) { return (int)((__umulhi(d.m, (uint32_t)n) + (uint32_t)n) >> d.l); }
 

@@ -581,7 +581,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     const int c_end = ((slice + 1) * nchunks) / slices;
     const bool has_corr = p.corr != nullptr;
     // per-layer part of the condition for the straight-line pass (see below)
-    const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec == 16 && q.fast && p.bias == nullptr && p.row_term == nullptr &&
+    const bool lean_layer = kOut == kOutInt8 && kiters > 0 && out_vec >= 16 && q.fast && p.bias == nullptr && p.row_term == nullptr &&
                             p.zc_in_smem && has_corr && !q.count_sat;
     // The tile loop is instantiated once per epilogue variant (kLean >= 0: the straight-line int8 pass with that rounding
     // for every tile whose columns all lie inside the layer; -1: the general pass only), so that the loop a warp runs holds
@@ -729,20 +729,22 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
 #pragma unroll
             for (int e = 0; e < CW / 4; ++e) w[e] = pack_sat4(r[4 * e + 0], r[4 * e + 1], r[4 * e + 2], r[4 * e + 3]);
             int8_t* dst = reinterpret_cast<int8_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16) store_bytes16<16>(dst, w, nvalid);
+            if (out_vec >= 16) store_bytes16<16>(dst, w, nvalid);
             else if (out_vec == 8) store_bytes16<8>(dst, w, nvalid);
             else if (out_vec == 4) store_bytes16<4>(dst, w, nvalid);
             else store_bytes16<1>(dst, w, nvalid);
           } else {
             uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + pix * p.ldY + col0 + c0;
-            if (out_vec == 16 && nvalid == CW) {
+            if (out_vec >= 16 && nvalid == CW) {
+              uint32_t w[CW];
 #pragma unroll
-              for (int e = 0; e < CW / 4; ++e) {
-                uint32_t w[4];
+              for (int e = 0; e < CW; ++e) w[e] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[e]), q.s_acc)) : (uint32_t)v[e];
+              if (out_vec == 32 && ((col0 + c0) & 7) == 0) {   // whole 32-byte sectors per thread: half the store instructions
+                st_global_v8(dst, w);
+                st_global_v8(dst + 8, w + 8);
+              } else {
 #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                  w[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[4 * e + k]), q.s_acc)) : (uint32_t)v[4 * e + k];
-                *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[0], w[1], w[2], w[3]);
+                for (int e = 0; e < CW / 4; ++e) *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(w[4 * e], w[4 * e + 1], w[4 * e + 2], w[4 * e + 3]);
               }
             } else {
 #pragma unroll
@@ -768,16 +770,29 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
         };
         int va[8], vb[8];
         tmem_ld8(taddr + c_begin * CW, va);
-        for (int ch = c_begin; ch < c_end; ++ch) {
+        auto pass16 = [&](int ch, uint32_t* w) {   // sixteen columns -> four words of codes
           const int c0 = ch * CW;
-          uint32_t w[4];
           tmem_ld_wait8(va);
           tmem_ld8(taddr + c0 + 8, vb);
           half(va, c0, w[0], w[1]);
           tmem_ld_wait8(vb);
           if (ch + 1 < c_end) tmem_ld8(taddr + c0 + CW, va);
           half(vb, c0 + 8, w[2], w[3]);
-          if (row_valid) *reinterpret_cast<uint4*>(dst_row + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+        };
+        if (out_vec == 32 && ((c_begin | c_end) & 1) == 0 && (col0 & 31) == 0) {
+          // 32 columns per store: every thread writes whole 32-byte sectors, in half as many store instructions
+          for (int ch = c_begin; ch < c_end; ch += 2) {
+            uint32_t w[8];
+            pass16(ch, w);
+            pass16(ch + 1, w + 4);
+            if (row_valid) st_global_v8(reinterpret_cast<uint32_t*>(dst_row + ch * CW), w);
+          }
+        } else {
+          for (int ch = c_begin; ch < c_end; ++ch) {
+            uint32_t w[4];
+            pass16(ch, w);
+            if (row_valid) *reinterpret_cast<uint4*>(dst_row + ch * CW) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
         }
         if (row_valid) {
           mn = min(mn, tmn);
@@ -790,7 +805,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           tmem_ld_wait();
           process(ch * CW, v);
         }
-      } else if (kOut == kOutInt8 && out_vec == 16 && q.fast && p.bias == nullptr && !has_corr && col0 + c_end * CW <= p.Nout) {
+      } else if (kOut == kOutInt8 && out_vec >= 16 && q.fast && p.bias == nullptr && !has_corr && col0 + c_end * CW <= p.Nout) {
         // no taps (a parity class of a strided backward pass that no filter position reaches): every accumulator is 0,
         // so every code is the zero point, whatever the rounding
         const uint32_t code = (uint32_t)(uint8_t)(int8_t)max(-128, min(127, q.zp)) * 0x01010101u;
@@ -966,16 +981,17 @@ cudaError_t gemm_set_smem_attr(uint32_t smem_bytes) {
 
 cudaError_t launch_gemm(const GemmParams& p, const CUtensorMap& ta, const CUtensorMap& tb, int out_mode, int grid, uint32_t smem_bytes,
                         cudaStream_t s, bool overlap) {
-  // widest aligned store the output rows allow
+  // widest aligned store the output rows allow (bytes; 32: every row starts on a 32-byte boundary, so a thread can write whole sectors)
   int out_vec;
   const uintptr_t addr = reinterpret_cast<uintptr_t>(p.out);
   if (out_mode == kOutInt8) {
-    if (p.ldY % 16 == 0 && addr % 16 == 0) out_vec = 16;
+    if (p.ldY % 32 == 0 && addr % 32 == 0) out_vec = 32;
+    else if (p.ldY % 16 == 0 && addr % 16 == 0) out_vec = 16;
     else if (p.ldY % 8 == 0 && addr % 8 == 0) out_vec = 8;
     else if (p.ldY % 4 == 0 && addr % 4 == 0) out_vec = 4;
     else out_vec = 1;
   } else {
-    out_vec = (p.ldY % 4 == 0 && addr % 16 == 0) ? 16 : 4;
+    out_vec = (p.ldY % 8 == 0 && addr % 32 == 0) ? 32 : ((p.ldY % 4 == 0 && addr % 16 == 0) ? 16 : 4);
   }
   if (p.pair) {   // grid is an even number of CTAs: clusters of two
     switch (out_mode) {
