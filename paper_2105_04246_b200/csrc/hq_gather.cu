@@ -323,6 +323,10 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
     const int c_begin = 0, c_end = p.BN / 16;   // a warp drains all columns of its 32 rows
     const QPacked qk = qpacked(q);
     const bool lean = kOut == kOutInt8 && q.fast && !q.count_sat;
+    // 32-byte stores where every output row starts on a 32-byte boundary (int8 rows of BN bytes; 4-byte rows of 4 BN)
+    const bool base32 = (reinterpret_cast<uintptr_t>(p.out) & 31u) == 0;
+    [[maybe_unused]] const bool wide = base32 && (p.BN & 31) == 0;
+    [[maybe_unused]] const bool wide32 = base32 && (p.BN & 7) == 0;
     // The tile loop, instantiated per epilogue variant (kMode >= 0: straight-line int8 pass with that rounding; -1: the
     // general pass), so that the loop a warp actually runs holds one variant's code only.
     auto run_tiles = [&](auto mode_tag) {
@@ -357,8 +361,7 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
           // sixteen columns per load, two register sets: the next load is in flight while a set is processed
           int va[16], vb[16];
           tmem_ld16r(taddr, va);
-          auto pass16 = [&](int (&v)[16], int c0) {
-            uint32_t wd[4];
+          auto pass16 = [&](int (&v)[16], int c0, uint32_t* wd) {
             int lo[8], hi[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
@@ -367,17 +370,25 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
             }
             lean_half8m<kMode>(lo, zrow + c0, tmn, tmx, q, qk, elem_row + c0, wd[0], wd[1]);
             lean_half8m<kMode>(hi, zrow + c0 + 8, tmn, tmx, q, qk, elem_row + c0 + 8, wd[2], wd[3]);
-            if (row_valid) *reinterpret_cast<uint4*>(dst_row + c0) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
           };
           for (int ch = 0; ch < c_end; ch += 2) {   // chunks ch (in va) and, if there is one, ch + 1 (in vb)
             const bool last = ch + 1 == c_end;
             tmem_ld_wait16(va);
             if (!last) tmem_ld16r(taddr + (ch + 1) * 16, vb);
-            pass16(va, ch * 16);
+            uint32_t wd[8];
+            pass16(va, ch * 16, wd);
             if (!last) {
               tmem_ld_wait16(vb);
               if (ch + 2 < c_end) tmem_ld16r(taddr + (ch + 2) * 16, va);
-              pass16(vb, (ch + 1) * 16);
+              pass16(vb, (ch + 1) * 16, wd + 4);
+            }
+            if (row_valid) {
+              if (!last && wide) {   // 32 columns in one store: a whole 32-byte sector per thread
+                st_global_v8(reinterpret_cast<uint32_t*>(dst_row + ch * 16), wd);
+              } else {
+                *reinterpret_cast<uint4*>(dst_row + ch * 16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                if (!last) *reinterpret_cast<uint4*>(dst_row + (ch + 1) * 16) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
+              }
             }
           }
           if (row_valid) {
@@ -405,13 +416,15 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
                 *reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(p.out) + pix * p.BN + c0) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
               } else {
                 uint32_t* dst = reinterpret_cast<uint32_t*>(p.out) + pix * p.BN + c0;
+                uint32_t wd[16];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                  uint32_t wd[4];
+                for (int e = 0; e < 16; ++e) wd[e] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[e]), q.s_acc)) : (uint32_t)v[e];
+                if (wide32) {   // rows of 4-byte values start on 32-byte boundaries
+                  st_global_v8(dst, wd);
+                  st_global_v8(dst + 8, wd + 8);
+                } else {
 #pragma unroll
-                  for (int k = 0; k < 4; ++k)
-                    wd[k] = (kOut == kOutF32) ? __float_as_uint(__fmul_rn(__int2float_rn(v[4 * e + k]), q.s_acc)) : (uint32_t)v[4 * e + k];
-                  *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+                  for (int e = 0; e < 4; ++e) *reinterpret_cast<uint4*>(dst + 4 * e) = make_uint4(wd[4 * e], wd[4 * e + 1], wd[4 * e + 2], wd[4 * e + 3]);
                 }
               }
             }
