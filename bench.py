@@ -37,12 +37,17 @@ from paper_2105_04246_b200 import workloads as wl
 METRIC = "int8 TOPS & HBM bytes/layer: hindsight-fused vs dynamic quant, % of roofline"
 NOMINAL_INT8_OVER_BF16 = 2.0          # dense int8 peak / dense bf16 peak on B200 (4.5 / 2.25 POPS)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the named layer's kernel, from the ncu captures
-# summarised under profiles/ (taken with the kernels as committed; set an entry to None when its kernel changes).
-# Output lines still dirty in L2 when the kernel ends are not in these counters.
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the named layer's kernel: mean over the last 16 of 24
+# launches that rotate over a buffer pool larger than L2, caches not flushed between launches, so that the output of
+# earlier launches is written back to DRAM while later ones run (ncu captures summarised under profiles/, taken with
+# the kernels as committed; set an entry to None when its kernel changes).
+NCU_TRAFFIC = {
+    "stem7x7": 122782496, "layer1.0": 51050416, "layer2.1": 25284896, "layer3.1": 12634112, "layer4.1": 6581504,
+    "resnet_conv3x3_64": 25393920, "resnet_conv3x3_256_bwd": 25511104,
+    "mbv2_expand": 134992112, "mbv2_dw3x3": 231284256, "mbv2_project": 135075152,
+}
 # kernels other than the tensor-core layer kernel, by layer name
-KERNEL_OF = {"mbv2_dw3x3": "depthwise3x3_tiled_kernel"}
+KERNEL_OF = {"mbv2_dw3x3": "depthwise3x3_col_kernel", "stem7x7": "hq_gather_conv_kernel"}
 
 
 def load_peaks():
@@ -417,6 +422,7 @@ def layer_rows(torch, wk, cfg_name, peaks, probe_peak, min_time_s, min_repeats):
             "frac_tensor": None if dw else round(t_tensor / us, 4),
             "frac_tensor_probe": None if (dw or not probe_peak) else round(s.ops / (probe_peak * 1e12) * 1e6 / us, 4),
             "frac_hbm": round(t_hbm / us, 4),
+            "traffic": NCU_TRAFFIC.get(s.name),
         })
     return rows
 
@@ -615,7 +621,7 @@ def run_gpu(args):
                 "peak_source": f"{peak_kind} bf16 burst x {NOMINAL_INT8_OVER_BF16} (nominal int8 / bf16 ratio)",
                 "frac_of_mma_probe": None if not probe_peak else round(ach / probe_peak, 4)}
     tr = NCU_TRAFFIC.get(s.name)
-    roof.update({"kernel": KERNEL_OF.get(s.name, "depthwise3x3_tiled_kernel" if dw else "hq_gemm_kernel"), "layer": s.name,
+    roof.update({"kernel": KERNEL_OF.get(s.name, "depthwise3x3_col_kernel" if dw else "hq_gemm_kernel"), "layer": s.name,
                  "launch_us": round(layer_us[dom], 3), "algorithmic_bytes": int(wk_static[dom]), "traffic": tr,
                  "frac_of": f"of {peak_kind}"})
 
@@ -750,7 +756,7 @@ def run_wgrad(args):
         "gpu_launches": int(launches * pool * repeats), "launches_per_step": int(launches),
         "hbm_bytes_per_step": {"algorithmic": int(nbytes)},
         "roofline": {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                     "kernel": ("dw_wgrad_kernel" if cs.depthwise else "im2col_t_kernel + hq_gemm_kernel (int32 slabs) + wgrad_reduce_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
+                     "kernel": ("dw_wgrad_kernel" if cs.depthwise else "wgrad_pack_kernel x 2 + hq_gemm_kernel (int32 slabs) + wgrad_reduce_taps_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
                      "peak_source": peak_kind, "frac_of": f"of {peak_kind}"},
         "e2e": {"value": round(ops / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
                 "h2d_bytes_per_step": int(M * N + M * K), "d2h_bytes_per_step": int(4 * N * K), "steps": e2e_steps},

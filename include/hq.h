@@ -182,6 +182,10 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              (default), 0 = every CTA works on its own 128-row tile, 1 = pairs of CTAs on neighbouring SMs share
  *              256-row tiles (one tensor-core instruction for both, each CTA holding half of the weight rows)
  *              wherever the layer allows.
+ *   "wgrad_windows": weight gradient of dense convolutions (read at every call): -1 = library's choice (default),
+ *              0 = stride-1 layers pack both tensors channel-major over a padded pixel index (one copy of dY, one
+ *              copy of X per horizontal filter offset) wherever the shape allows, 1 = always the general form
+ *              (one transposed copy of X per filter tap).
  *   "issuers": upper limit (1, 2 or 3; default 3) of the warps of a CTA that issue tensor-core instructions,
  *              each for every n-th tile, in layers prepared AFTER this call.
  *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their

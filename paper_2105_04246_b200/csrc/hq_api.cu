@@ -1018,6 +1018,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     ctx->force_pair = value;
     return HQ_OK;
   }
+  if (std::string(key) == "wgrad_windows") {
+    if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "wgrad_windows must be -1, 0 or 1");
+    ctx->wgrad_windows = value;
+    return HQ_OK;
+  }
   if (std::string(key) == "issuers") {
     if (value < 1 || value > 3) return fail(ctx, HQ_ERR_INVALID_ARG, "issuers must be 1, 2 or 3");
     ctx->max_issuers = value;
@@ -1557,6 +1562,127 @@ __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, vo
   return run_linear(ctx, s, N, K, Mp, At, dyq, Bt, x_scale, nullptr, GW, tmp, kOutF32, terms);
 }
 
+}  // extern "C"
+
+// Weight gradient of a dense stride-1 convolution without filter-window copies of the input.  Both tensors are packed
+// channel-major over one padded pixel index m = (n * Hp + pad_h + h) * P + w (Hp = Ho + R - 1 rows per image, P = Wo rounded
+// up to 16): dY once, X once per horizontal filter offset (shifted by it); a vertical offset is then a shift of the
+// reduction index by a multiple of P, which a TMA coordinate can carry, and padding is zeros in both.  The GEMM is the
+// layer kernel over slices of m (int32 slabs, as in the general form) with column tiles grouped by filter row: the tiles
+// of filter row r read the same rows of the packed input at reduction offset (r - pad_h) * P.  The zero-point terms need
+// sums over the output pixels whose tap lies inside the image; the packing kernels take them on the way.
+// *done = false (and HQ_OK) when the shape is left to the general form.
+static hq_status conv_wgrad_stride1(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc& d, int Ho, int Wo, const int8_t* dY, const hq_range_state* dyq,
+                                    const int8_t* X, const hq_range_state* xq, float* GW, bool* done) {
+  *done = false;
+  const int P = round_up(Wo, 16), Hp = Ho + d.R - 1, RS = d.R * d.S;
+  if (d.stride_h != 1 || d.stride_w != 1 || d.R > 8 || d.S > 8 || RS > kMaxTaps || d.C % 16 != 0 || d.K % 4 != 0 || P > 256 || d.W > 256 ||
+      d.pad_w > 16 || d.S - 1 - d.pad_w > 16 || d.pad_h >= d.R || d.pad_w >= d.S)
+    return HQ_OK;
+  const int brows = d.S * d.C;   // rows of the packed input: (horizontal offset, channel)
+  int per_row = 0;               // column tiles per filter row: the fewest that divide brows into multiples of 16 of at most 256
+  for (int t = 1; t <= brows / 16; ++t)
+    if (brows % t == 0 && (brows / t) % 16 == 0 && brows / t <= 256) {
+      per_row = t;
+      break;
+    }
+  if (per_row == 0) return HQ_OK;
+  const int rows = d.K, cols = RS * d.C;
+  const int64_t Mv = (int64_t)d.N * Hp * P;   // padded reduction length
+  if (Mv > (1 << 26)) return HQ_OK;
+  const int tiles_one = ceil_div(rows, kTileM) * d.R * per_row;
+  const int want_slices = std::max(1, (2 * ctx->num_sms + tiles_one - 1) / tiles_one);
+  const int slice_len = (int)std::max<int64_t>(128, round_up((int)ceil_div((int)Mv, want_slices), 128));
+  const int slices = ceil_div((int)Mv, slice_len);
+  const int64_t Mp = (int64_t)slices * slice_len;
+  const size_t a_bytes = (size_t)rows * Mp, b_bytes = (size_t)brows * Mp;
+  const size_t ab_bytes = (a_bytes + b_bytes + 255) & ~(size_t)255;
+  const size_t slab_bytes = ((size_t)slices * rows * cols * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t sum_bytes = ((size_t)RS * (rows + d.C) * sizeof(int32_t) + 255) & ~(size_t)255;
+  const size_t need = ab_bytes + slab_bytes + sum_bytes + 256;
+  if (need > ctx->wgrad_bytes) {
+    if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));
+    ctx->d_wgrad = nullptr;
+    ctx->wgrad_bytes = 0;
+    HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_wgrad, need));
+    ctx->wgrad_bytes = need;
+  }
+  int8_t* At = reinterpret_cast<int8_t*>(ctx->d_wgrad);
+  int8_t* Bs = At + a_bytes;   // the same pitch: the rows of both lie back to back
+  int32_t* slabs = reinterpret_cast<int32_t*>(ctx->d_wgrad + ab_bytes);
+  int32_t* rowsum = reinterpret_cast<int32_t*>(ctx->d_wgrad + ab_bytes + slab_bytes);   // [tap][K]
+  int32_t* colsum = rowsum + (size_t)RS * rows;                                         // [tap][C]
+  hq_range_state* tmp = reinterpret_cast<hq_range_state*>(ctx->d_wgrad + ab_bytes + slab_bytes + sum_bytes);
+  HQ_CUDA(ctx, cudaMemsetAsync(rowsum, 0, (size_t)RS * (rows + d.C) * sizeof(int32_t), s));
+  // output pixels whose tap (r, s) lies inside the image: rows [pad_h - r, H + pad_h - r) and columns alike, cut to the output
+  PackRanges ry{}, rx{};
+  TapCounts mvalid{};
+  ry.nr = rx.nr = d.R;
+  ry.ns = rx.ns = d.S;
+  for (int r = 0; r < d.R; ++r) {
+    ry.row_lo[r] = (int16_t)std::max(0, d.pad_h - r);
+    ry.row_hi[r] = (int16_t)std::min(Ho, d.H + d.pad_h - r);
+    rx.row_lo[r] = (int16_t)std::max(0, r - d.pad_h);            // the input rows those outputs read through filter row r
+    rx.row_hi[r] = (int16_t)std::min(d.H, Ho + r - d.pad_h);
+  }
+  for (int r = 0; r < d.R; ++r)
+    for (int c = 0; c < d.S; ++c) {
+      const int cols_in = std::max(0, std::min(Wo, d.W + d.pad_w - c) - std::max(0, d.pad_w - c));
+      mvalid.v[r * d.S + c] = d.N * std::max(0, ry.row_hi[r] - ry.row_lo[r]) * cols_in;
+    }
+  // dY: views shifted by pad_w - s, summed over the first W columns (the pixels of the input row they pair with); X: views
+  // shifted by s - pad_w, summed over the first Wo columns
+  HQ_CUDA(ctx, launch_wgrad_pack(dY, At, d.N, Ho, Wo, d.K, Hp, P, d.pad_h, -1, d.pad_w, d.W, Mp, ry, rowsum, s));
+  HQ_CUDA(ctx, launch_wgrad_pack(X, Bs, d.N, d.H, d.W, d.C, Hp, P, d.pad_h, +1, d.pad_w, Wo, Mp, rx, colsum, s));
+  HQ_CUDA(ctx, launch_zero_tail(At, rows + brows, Mp, Mv, s));
+  ctx->launches += Mp > Mv ? 3 : 2;
+  SubSpec sp{};
+  sp.n_img = slices; sp.TH = 1; sp.TW = rows; sp.in_mul_h = 1; sp.in_mul_w = 1;
+  sp.dh = {0}; sp.dw = {0}; sp.a_H = 1; sp.a_W = rows; sp.Cin = slice_len; sp.Nout = cols;
+  sp.out_H = 1; sp.out_W = rows; sp.os_h = 1; sp.os_w = 1; sp.oa_h = 0; sp.oa_w = 0; sp.ldY = cols; sp.flat = true;
+  sp.slices = slices; sp.slice_len = slice_len;
+  hq_sub_problem sub;
+  std::vector<uint8_t> rc, cc;
+  MaskVec rm, cm;
+  hq_status st = plan_sub_fixed(ctx, sp, sub, rc, cc, rm, cm, d.R * per_row, 0);
+  if (st != HQ_OK) return st;
+  if (sub.p.BN != brows / per_row || sub.p.tiles_col != d.R * per_row || sub.p.b_resident || sub.p.pair)
+    return HQ_OK;   // not the tiling this form needs: the general form takes the layer
+  sub.p.corr = nullptr;       // both zero points are taken out after the slabs are summed
+  sub.p.zc_in_smem = 0;
+  sub.p.zc_elems = 0;
+  sub.p.Cpad = slice_len;
+  sub.p.b_group_tiles = per_row;
+  sub.p.b_k_base = -d.pad_h * P;
+  sub.p.b_k_step = P;
+  CUtensorMap ta, tb;
+  {   // operand A: [rows][Mp] seen as (reduction byte within the slice, row, 1, slice)
+    uint64_t dims[4] = {(uint64_t)slice_len, (uint64_t)rows, 1, (uint64_t)slices};
+    uint64_t strides[3] = {(uint64_t)Mp, (uint64_t)Mp * rows, (uint64_t)slice_len};
+    uint32_t box[4] = {(uint32_t)sub.p.BK, (uint32_t)sub.p.Wt, 1, 1};
+    uint32_t es[4] = {1, 1, 1, 1};
+    st = encode_map(ctx, &ta, At, 4, dims, strides, box, es, sub.p.swizzle64, false);
+    if (st != HQ_OK) return st;
+  }
+  {   // operand B: [brows][Mp]; coordinates left of 0 and right of Mp read as zeros
+    uint64_t dims[2] = {(uint64_t)Mp, (uint64_t)brows};
+    uint64_t strides[1] = {(uint64_t)Mp};
+    uint32_t box[2] = {(uint32_t)sub.p.BK, (uint32_t)sub.p.BN};
+    uint32_t es[2] = {1, 1};
+    st = encode_map(ctx, &tb, Bs, 2, dims, strides, box, es, sub.p.swizzle64, true);
+    if (st != HQ_OK) return st;
+  }
+  const float* x_scale = reinterpret_cast<const float*>(reinterpret_cast<const char*>(xq) + offsetof(hq_range_state, scale));
+  st = launch_sub(ctx, s, sub, ta, tb, dyq, x_scale, nullptr, slabs, tmp, kOutAcc);
+  if (st != HQ_OK) return st;
+  HQ_CUDA(ctx, launch_wgrad_reduce_taps(slabs, slices, rows, rows, cols, d.C, colsum, rowsum, mvalid, dyq, xq, GW, s));
+  ctx->launches += 1;
+  *done = true;
+  return HQ_OK;
+}
+
+extern "C" {
+
 __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc, const int8_t* dY,
                                                                const hq_range_state* dyq, const int8_t* X, const hq_range_state* xq, float* GW) {
   if (!ctx) return HQ_ERR_INVALID_ARG;
@@ -1591,6 +1717,11 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
   }
   const int64_t cols64 = (int64_t)d.R * d.S * d.C;
   if (M64 > (1 << 24) || cols64 > (1 << 20)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels or filter elements");
+  if (ctx->wgrad_windows != 1) {
+    bool done = false;
+    st = conv_wgrad_stride1(ctx, s, d, Ho, Wo, dY, dyq, X, xq, GW, &done);
+    if (st != HQ_OK || done) return st;
+  }
   const int M = (int)M64, rows = d.K, cols = (int)cols64;
   // G_W as one GEMM over the output pixels m: rows k (dY^T [K][M]) x columns (r,s,c) (the filter windows of X,
   // transposed: Bt [(r,s,c)][M]).  The output is as small as the weights while the reduction is long, so the reduction is

@@ -567,6 +567,154 @@ __global__ void wgrad_reduce_kernel(const int32_t* __restrict__ slabs, int nslab
   }
 }
 
+// The same for the stride-1 form, where image padding is left out of the sums instead of being filled with the zero
+// point: per filter tap t = (r, s), with sums over the output pixels whose tap lies inside the image,
+//   sum (dy - z_dy)(x - z_x) = sum dy x - z_dy * colsum[t][c] - z_x * (rowsum[t][k] - z_dy * count[t]).
+// Slabs have slab_rows rows of which the first `rows` are output channels.
+__global__ void __launch_bounds__(256) wgrad_reduce_taps_kernel(const int32_t* __restrict__ slabs, int nslabs, int rows, int slab_rows, int cols,
+                                                                 int C, const int32_t* __restrict__ colsum, const int32_t* __restrict__ rowsum,
+                                                                 TapCounts mvalid, const hq_range_state* __restrict__ dyq,
+                                                                 const hq_range_state* __restrict__ xq, float* __restrict__ G) {
+  // a block: 32 consecutive outputs (lanes) x 8 groups of slabs (warps), joined through shared memory
+  __shared__ uint32_t part_s[8][32];
+  const float sc = __fmul_rn(dyq->scale, xq->scale);
+  const int zdy = dyq->zero_point, zx = xq->zero_point;
+  const int64_t total = (int64_t)rows * cols, slab = (int64_t)slab_rows * cols;
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  for (int64_t base = (int64_t)blockIdx.x * 32; base < total; base += (int64_t)gridDim.x * 32) {
+    const int64_t idx = base + lane;
+    uint32_t g = 0;
+    if (idx < total)
+      for (int sl = grp; sl < nslabs; sl += 8) g += (uint32_t)slabs[(int64_t)sl * slab + idx];
+    part_s[grp][lane] = g;
+    __syncthreads();
+    if (grp == 0 && idx < total) {
+#pragma unroll
+      for (int k = 1; k < 8; ++k) g += part_s[k][lane];
+      const int row = (int)(idx / cols), col = (int)(idx - (int64_t)row * cols);
+      const int tap = col / C;
+      g -= (uint32_t)zdy * (uint32_t)colsum[col];
+      g -= (uint32_t)zx * ((uint32_t)rowsum[tap * rows + row] - (uint32_t)zdy * (uint32_t)mvalid.v[tap]);
+      G[idx] = __fmul_rn(__int2float_rn((int)g), sc);
+    }
+    __syncthreads();
+  }
+}
+
+// Packs one NHWC tensor for the stride-1 weight-gradient GEMM (reduction over pixels): dst[copy][c][m] with
+// m = (n * Hp + row_off + h) * P + w holds src(n, h, w + shift, c), 0 where that column lies outside the source row, in
+// the rows of the padded index space that no source row maps to, and for w >= the source width.  In this index space a
+// vertical filter offset is a shift by a multiple of P (16-byte aligned, which a TMA coordinate needs), the horizontal
+// offsets are the copies, and image padding is real zeros.
+// The kernel forms `ns` shifted views of every source row, shift_j = sign * (j - pad): the input (sign +1) writes all of
+// them (copy j); the output gradient (sign -1) writes only the unshifted one (as copy 0).  The sum of view j over its
+// first `limit` columns is the sum of the source row over the columns that filter column j pairs with a pixel inside
+// the other tensor's row; it is added to sums[(r * ns + j) * Cs + c] (zeroed by the caller) for every filter row r whose
+// row range rg.row_* contains the source row.
+// One block: 32 channels of kPackRows padded rows of one image, all rows at once: the source rows go to shared memory
+// transposed (4x4 byte blocks turned in registers; channel-major words behind 16 zero bytes, zeros after), each view is
+// read from there as aligned words and funnel-shifted, written in 16-byte pieces and summed with dp4a.
+constexpr int kPackRows = 4;
+constexpr int kPackMaxP = 256;
+// words per channel row of the tile: 16 zero bytes, the row, room for the shifted reads past its end; odd, so that the
+// transposing stores spread over the banks
+static int pack_tile_pitch(int P, int Ws, int limit) { return ((std::max(std::max(P, limit), Ws) + 64) / 4) | 1; }
+__global__ void __launch_bounds__(256) wgrad_pack_kernel(const int8_t* __restrict__ src, int8_t* __restrict__ dst, int Hs, int Ws, int Cs, int Hp,
+                                                          int P, int row_off, int sign, int pad, int limit, int64_t pitch, PackRanges rg,
+                                                          int32_t* __restrict__ sums, int tp) {
+  extern __shared__ uint32_t pack_tile[];   // [kPackRows][32][tp]
+  auto tile = [&](int rl, int c) { return pack_tile + (rl * 32 + c) * tp; };
+  __shared__ int acc_s[64][32];    // [filter row * ns + view][channel of the block]
+  const int n = blockIdx.z, c0 = blockIdx.y * 32, pr0 = blockIdx.x * kPackRows;
+  const int tid = threadIdx.x;
+  for (int i = tid; i < rg.nr * rg.ns * 32; i += 256) acc_s[i >> 5][i & 31] = 0;
+  for (int i = tid; i < kPackRows * 32 * tp; i += 256) pack_tile[i] = 0u;   // margins and missing rows stay zero
+  const int wgroups = (Ws + 3) / 4;                // groups of 4 source pixels
+  __syncthreads();
+  for (int i = tid; i < kPackRows * wgroups * 8; i += 256) {   // (row of the block, pixel group, channel word)
+    const int cg = i & 7, wg = (i >> 3) % wgroups, rl = (i >> 3) / wgroups;
+    const int h = pr0 + rl - row_off;
+    if (pr0 + rl >= Hp || h < 0 || h >= Hs || c0 + cg * 4 >= Cs) continue;   // Cs is a multiple of 4
+    const int8_t* row = src + (((int64_t)n * Hs + h) * Ws) * Cs + c0;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (wg * 4 + j < Ws) w[j] = *reinterpret_cast<const uint32_t*>(row + (int64_t)(wg * 4 + j) * Cs + cg * 4);
+    const uint32_t a0 = __byte_perm(w[0], w[1], 0x5140), a1 = __byte_perm(w[0], w[1], 0x7362);
+    const uint32_t b0 = __byte_perm(w[2], w[3], 0x5140), b1 = __byte_perm(w[2], w[3], 0x7362);
+    tile(rl, cg * 4 + 0)[4 + wg] = __byte_perm(a0, b0, 0x5410);
+    tile(rl, cg * 4 + 1)[4 + wg] = __byte_perm(a0, b0, 0x7632);
+    tile(rl, cg * 4 + 2)[4 + wg] = __byte_perm(a1, b1, 0x5410);
+    tile(rl, cg * 4 + 3)[4 + wg] = __byte_perm(a1, b1, 0x7632);
+  }
+  __syncthreads();
+  // One task = one (row of the block, view, channel): its thread walks along the row in 16-byte pieces (the lanes of a warp
+  // are 32 channels: conflict-free shared-memory reads, one sum per task), two pieces per store where rows allow 32 bytes.
+  const int per_row = rg.ns * 32;
+  const bool wide = (P & 31) == 0 && (pitch & 31) == 0 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
+  for (int task = tid; task < kPackRows * per_row; task += 256) {
+    const int rl = task / per_row, t = task - rl * per_row;
+    const int c = t & 31, j = t >> 5;
+    const int pr = pr0 + rl, h = pr - row_off;
+    if (pr >= Hp || c0 + c >= Cs) continue;
+    const int shift = sign * (j - pad);
+    const bool stored = sign > 0 || shift == 0;
+    const uint32_t* trow = tile(rl, c);
+    // sum of the view's first `limit` columns = sum of the whole source row minus what the window [shift, shift + limit)
+    // leaves out at either end (a few bytes)
+    int part = 0;
+    if (h >= 0 && h < Hs) {
+      for (int g = 0; g < wgroups; ++g) part = __dp4a((int)trow[4 + g], 0x01010101, part);
+      const int8_t* bytes = reinterpret_cast<const int8_t*>(trow) + 16;
+      for (int i = 0; i < min(shift, Ws); ++i) part -= bytes[i];
+      for (int i = max(0, shift + limit); i < Ws; ++i) part -= bytes[i];
+    }
+    if (stored) {
+      const int b0 = 16 + shift;                     // first byte of the view in the tile row (>= 0)
+      const uint32_t* wp = trow + (b0 >> 2);
+      const uint32_t sh = (uint32_t)(b0 & 3) * 8u;
+      int8_t* out = dst + ((int64_t)(sign > 0 ? j : 0) * Cs + c0 + c) * pitch + ((int64_t)n * Hp + pr) * P;
+      uint32_t lo = wp[0];
+      uint32_t prev[4];
+      for (int q = 0; q * 16 < P; ++q) {
+        uint32_t w4[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t hi = wp[q * 4 + e + 1];
+          w4[e] = __funnelshift_r(lo, hi, sh);
+          lo = hi;
+        }
+        if (wide) {
+          if (q & 1) {
+            const uint32_t w8[8] = {prev[0], prev[1], prev[2], prev[3], w4[0], w4[1], w4[2], w4[3]};
+            st_global_v8(reinterpret_cast<uint32_t*>(out + (q - 1) * 16), w8);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) prev[e] = w4[e];
+          }
+        } else {
+          *reinterpret_cast<uint4*>(out + q * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+        }
+      }
+    }
+    if (part != 0 && h >= 0 && h < Hs)
+      for (int r = 0; r < rg.nr; ++r)
+        if (h >= rg.row_lo[r] && h < rg.row_hi[r]) atomicAdd(&acc_s[r * rg.ns + j][c], part);
+  }
+  __syncthreads();
+  for (int i = tid; i < rg.nr * rg.ns * 32; i += 256) {
+    const int c = i & 31, t = i >> 5;
+    if (c0 + c < Cs && acc_s[t][c] != 0) atomicAdd(&sums[t * Cs + c0 + c], acc_s[t][c]);
+  }
+}
+__global__ void zero_tail_kernel(int8_t* base, int rows, int64_t pitch, int64_t from) {   // bytes [from, pitch) of every row; both multiples of 16
+  const int64_t per_row = (pitch - from) / 16;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < per_row * rows; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / per_row, q = i - r * per_row;
+    *reinterpret_cast<uint4*>(base + r * pitch + from + q * 16) = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
 // sum_m (dy - z_dy)(x - z_x) = sum_m (dy - z_dy) x  -  z_x * sum_m (dy - z_dy): the second term, one number per output
 // row n, which the layer kernel's epilogue subtracts from every accumulator of that row.
 __global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int N, const hq_range_state* __restrict__ dyq,
@@ -1345,6 +1493,29 @@ cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int 
   const int64_t total = (int64_t)rows * cols;
   const int blocks = (int)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 16));
   wgrad_reduce_kernel<<<blocks, 256, 0, s>>>(slabs, nslabs, rows, cols, colsum, rowsum, M, dyq, xq, G);
+  return cudaGetLastError();
+}
+cudaError_t launch_wgrad_pack(const int8_t* src, int8_t* dst, int N, int Hs, int Ws, int Cs, int Hp, int P, int row_off, int sign, int pad, int limit,
+                              int64_t pitch, const PackRanges& rg, int32_t* sums, cudaStream_t s) {
+  if (P > kPackMaxP || P % 16 != 0 || Ws > kPackMaxP || rg.nr * rg.ns > 64 || rg.ns > 8 || pad > 16 || rg.ns - 1 - pad > 16 || Cs % 4 != 0)
+    return cudaErrorInvalidValue;
+  dim3 grid((unsigned)((Hp + kPackRows - 1) / kPackRows), (unsigned)((Cs + 31) / 32), (unsigned)N);
+  const int tp = pack_tile_pitch(P, Ws, limit);
+  wgrad_pack_kernel<<<grid, 256, (size_t)kPackRows * 32 * tp * sizeof(uint32_t), s>>>(src, dst, Hs, Ws, Cs, Hp, P, row_off, sign, pad, limit, pitch, rg, sums, tp);
+  return cudaGetLastError();
+}
+cudaError_t launch_zero_tail(int8_t* base, int rows, int64_t pitch, int64_t from, cudaStream_t s) {
+  if (from >= pitch) return cudaSuccess;
+  const int64_t total = (pitch - from) / 16 * rows;
+  zero_tail_kernel<<<(int)std::max<int64_t>(1, std::min<int64_t>((total + 255) / 256, 148 * 8)), 256, 0, s>>>(base, rows, pitch, from);
+  return cudaGetLastError();
+}
+cudaError_t launch_wgrad_reduce_taps(const int32_t* slabs, int nslabs, int rows, int slab_rows, int cols, int C, const int32_t* colsum,
+                                     const int32_t* rowsum, const TapCounts& mvalid, const hq_range_state* dyq, const hq_range_state* xq, float* G,
+                                     cudaStream_t s) {
+  const int64_t total = (int64_t)rows * cols;
+  const int blocks = (int)std::max<int64_t>(1, std::min<int64_t>((total + 31) / 32, 148 * 16));
+  wgrad_reduce_taps_kernel<<<blocks, 256, 0, s>>>(slabs, nslabs, rows, slab_rows, cols, C, colsum, rowsum, mvalid, dyq, xq, G);
   return cudaGetLastError();
 }
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,

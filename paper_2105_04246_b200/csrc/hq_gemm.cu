@@ -419,6 +419,14 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
             }
           }
         } else {
+          // rows and reduction offset of operand B: the tile's own columns, or (column tiles that share rows of B, each
+          // group of them at its own shift along the reduction) the group's
+          int b_row = col0, b_k_shift = 0;
+          if (p.b_group_tiles > 0) {
+            const int ct = col0 / p.BN, grp = ct / p.b_group_tiles;
+            b_row = (ct - grp * p.b_group_tiles) * p.BN;
+            b_k_shift = p.b_k_base + grp * p.b_k_step;
+          }
           for (int t = 0; t < p.ntaps && ok; ++t) {
             const int ch = h0 * p.in_mul_h + p.tap_dh[t];
             const int cw = w0 * p.in_mul_w + p.tap_dw[t];
@@ -434,7 +442,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
                 } else {
                   mbar_expect_tx(a_full(stage), a_stride);
                   tma_load_4d(sa, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
-                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK + n0 * p.b_slice, col0, a_full(stage));
+                  if (!p.b_resident) tma_load_2d(sa + p.stage_bytes_a, &tmap_b, t * p.Cpad + cc * p.BK + n0 * p.b_slice + b_k_shift, b_row, a_full(stage));
                 }
               }
               if (++stage == p.stages_a) {

@@ -108,6 +108,9 @@ struct GemmParams {
   int32_t cls_in_smem;                // both tables are non-null and fit the kernel's shared copy (TH, TW <= 512)
   const int32_t* bias;                // [Nout] or null
   int32_t b_slice;                    // kModeTap, streamed weights: image n of the tile space reads operand B at reduction offset n * b_slice
+  // kModeTap, streamed operand B shared by groups of column tiles (weight gradient of a stride-1 convolution): column tile ct
+  // reads rows (ct % b_group_tiles) * BN at reduction offset + b_k_base + (ct / b_group_tiles) * b_k_step; 0 = off
+  int32_t b_group_tiles, b_k_base, b_k_step;
                                       // (the reduction of one GEMM cut into slices that run as "images"; 0 otherwise)
   const int32_t* row_term;            // [output pixels] or null: subtracted from every accumulator of the pixel (weight zero point times
                                       // the pixel's input sum; the weight gradient's input-zero-point term)
@@ -281,6 +284,22 @@ cudaError_t launch_im2col_t(const int8_t* X, int8_t* Bt, const hq_range_state* x
 // depthwise weight gradient, 3x3 or 5x5 filters, C a multiple of 4 and at most 1024; acc: C*R*S zeroed int32
 cudaError_t launch_dw_wgrad(const int8_t* dY, const int8_t* X, const hq_range_state* dyq, const hq_range_state* xq, const hq_conv_desc& d, int Ho,
                             int Wo, int num_sms, FastDiv fd_wo, FastDiv fd_ho, int32_t* acc, float* G, cudaStream_t s);
+// Weight gradient of a stride-1 convolution: packs a [N][Hs][Ws][Cs] tensor into channel-major rows over a padded pixel
+// index ((n * Hp + row_off + h) * P + w) in horizontally shifted views; sums per (filter row, filter column, channel) go to
+// `sums` (see the kernel)
+struct PackRanges {
+  int32_t nr, ns;                      // filter rows, filter columns
+  int16_t row_lo[8], row_hi[8];        // source rows that filter row r pairs with a row inside the other tensor
+};
+struct TapCounts {
+  int32_t v[kMaxTaps + 15];
+};
+cudaError_t launch_wgrad_pack(const int8_t* src, int8_t* dst, int N, int Hs, int Ws, int Cs, int Hp, int P, int row_off, int sign, int pad, int limit,
+                              int64_t pitch, const PackRanges& rg, int32_t* sums, cudaStream_t s);
+cudaError_t launch_zero_tail(int8_t* base, int rows, int64_t pitch, int64_t from, cudaStream_t s);
+cudaError_t launch_wgrad_reduce_taps(const int32_t* slabs, int nslabs, int rows, int slab_rows, int cols, int C, const int32_t* colsum,
+                                     const int32_t* rowsum, const TapCounts& mvalid, const hq_range_state* dyq, const hq_range_state* xq, float* G,
+                                     cudaStream_t s);
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
                                 const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
 cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
@@ -317,6 +336,7 @@ struct hq_ctx {
   int force_epi_groups = -1;          // log2 of the epilogue warp groups: -1 chosen per layer, else min(value, log2 of the accumulator buffers)
   int force_cols = -1;                // column tiles: -1 chosen by estimated duration, 0 as wide as the MMA allows, n > 0 at least n
   int force_pair = -1;                // CTA pairs on 256-row tiles: -1 choose per layer, 0 never, 1 wherever the layer allows
+  int wgrad_windows = -1;             // dense weight gradient: -1 choose, 0 packed tensors wherever the shape allows, 1 always filter-window copies
   int max_issuers = 3;                // upper limit of the warps that issue MMAs in one CTA (1, 2 or 3)
   cudaStream_t side[3] = {nullptr, nullptr, nullptr};   // independent launches of one call run side by side (see run_conv)
   cudaEvent_t ev_fork = nullptr, ev_join[3] = {nullptr, nullptr, nullptr};

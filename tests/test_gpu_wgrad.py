@@ -103,11 +103,25 @@ CONV_WGRAD_CASES = {
     "3x3_c128_k256_big": dict(N=8, H=28, W=28, Cin=128, K=256, R=3, S=3, stride=1, pad=1),
     "7x7_s2_c3_k64_stem": dict(N=2, H=30, W=26, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
     "3x3_nopad": dict(N=1, H=10, W=10, Cin=64, K=64, R=3, S=3, stride=1, pad=0),
+    "5x5_c16_k8_pad1": dict(N=2, H=11, W=13, Cin=16, K=8, R=5, S=5, stride=1, pad=1),
+    "3x3_c32_k20_wide": dict(N=2, H=6, W=70, Cin=32, K=20, R=3, S=3, stride=1, pad=1),
+    "3x3_nopad_wo16": dict(N=2, H=6, W=18, Cin=16, K=16, R=3, S=3, stride=1, pad=0),
 }
 
 
+@pytest.mark.parametrize("windows", [-1, 1])
 @pytest.mark.parametrize("name", list(CONV_WGRAD_CASES))
-def test_conv_wgrad_matches_oracle(ctx, name):
+def test_conv_wgrad_matches_oracle(ctx, name, windows):
+    """Both forms of the dense weight gradient (stride-1 layers: tensors packed over a padded pixel index; any layer: one
+    transposed copy of the input per filter tap) give the oracle's bits."""
+    ctx.set_option("wgrad_windows", windows)
+    try:
+        _conv_wgrad_case(ctx, name)
+    finally:
+        ctx.set_option("wgrad_windows", -1)
+
+
+def _conv_wgrad_case(ctx, name):
     c = CONV_WGRAD_CASES[name]
     dev = torch.device("cuda", ctx.device)
     r = synth.rng(303, len(name), c["H"], c["Cin"])
