@@ -692,7 +692,8 @@ def run_wgrad(args):
         label = (f"{args.workload}: weight gradient of {'depthwise ' if cs.depthwise else ''}conv3x3 {cs.C}->{cs.K} @{cs.H}x{cs.W}, batch {cs.N} "
                  f"-> FP32 G_W{list(gw_shape)}")
         path = ("CUDA-core kernel, integer atomics, conversion" if cs.depthwise else
-                "transposed filter windows, sliced reduction on the tensor-core layer kernel (int32 slabs), slab sum + conversion")
+                "dY and X packed channel-major over a padded pixel index (one copy of X per horizontal filter offset), sliced reduction on the "
+                "tensor-core layer kernel (int32 slabs), slab sum + conversion")
     else:
         M, N, K = WGRAD_SHAPE["M"], WGRAD_SHAPE["N"], WGRAD_SHAPE["K"]
         dy_shape, x_shape, gw_shape = (M, N), (M, K), (N, K)
