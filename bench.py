@@ -718,6 +718,13 @@ def run_wgrad(args):
     call(stream, 0)      # also sizes the context's scratch before any capture
     launches = ctx.launch_count() - l0
     torch.cuda.synchronize()
+    if args.profile:     # eager launches only, for a profiler
+        for k in range(args.steps):
+            call(stream, k % pool)
+        torch.cuda.synchronize()
+        assert ctx.get_async_error() == 0
+        print(json.dumps({"profile": args.workload, "steps": args.steps, "launches_per_call": launches}))
+        return
     g_full = capture(torch, call, pool)
     for _ in range(-(-W // pool)):
         g_full.replay()
@@ -784,7 +791,7 @@ def run_wgrad(args):
 
 
 def run_profile(args):
-    """Eager launches only, for a profiler.  The ranges are initialised by one dynamic step per pool slot; then, for the
+    """Eager launches only, for a profiler.  The ranges are initialised by two dynamic steps; then, for the
     chosen layer (--layer NAME; all layers when absent), --steps in-hindsight launches rotate through the layer's buffer
     pool (more than L2, so that earlier outputs are evicted to DRAM while later launches run), then --steps dynamic ones."""
     import torch
@@ -801,7 +808,7 @@ def run_profile(args):
     sel = [i for i, n in enumerate(names) if args.layer in (None, n)]
     if not sel:
         raise SystemExit(f"no layer named {args.layer} in {args.workload}: {names}")
-    for j in range(max(wk.pool[i] for i in sel) if not wk.chained else 2):
+    for j in range(2):
         wk.step(stream, j, dynamic=True)
     torch.cuda.synchronize()
     for k in range(args.steps):
@@ -864,7 +871,7 @@ def main():
     args = ap.parse_args()
     if args.impl == "hq" and args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.profile:
         sys.exit(spawn_ranks(args))
-    if args.workload in ("wgrad", "wgrad_conv", "wgrad_dw") and args.impl == "hq" and not args.profile:
+    if args.workload in ("wgrad", "wgrad_conv", "wgrad_dw") and args.impl == "hq":
         run_wgrad(args)
     elif args.impl == "reference":
         run_reference(args)

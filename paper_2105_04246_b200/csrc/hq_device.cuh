@@ -68,6 +68,31 @@ __device__ __forceinline__ void st_global_v8(uint32_t* dst, const uint32_t* w) {
                : "memory");
 }
 
+// After a CTA has given up (abort flag set), the thread that issued bulk copies waits, again bounded (about 10 ms), until
+// the copy armed on `bar` for the phase of parity `parity` has delivered its bytes: the CTA does not return with copies
+// into its shared memory in flight.  A stage that was never armed answers at once (parity of the phase before the first).
+constexpr long long kDrainLimitCycles = 20000000ll;
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity, 1000u)) {
+    if (clock64() - t0 > kDrainLimitCycles) break;
+    __nanosleep(200);
+  }
+}
+// the same for a ring of `stages` barriers of which `stage` (in the lap of parity `phase`) would have been armed next
+template <typename BarFn>
+__device__ __forceinline__ void ring_drain(BarFn bar, int stages, int stage, uint32_t phase) {
+  for (int k = 1; k <= stages; ++k) {   // the stages armed last, newest first
+    int s = stage - k;
+    uint32_t ph = phase;
+    if (s < 0) {
+      s += stages;
+      ph ^= 1u;
+    }
+    mbar_drain(bar(s), ph);
+  }
+}
+
 // n / d for 0 <= n < 2^31 with the multiplier and shift prepared on the host (see make_fastdiv)
 __device__ __forceinline__ int fdiv(int n, FastDiv d) { return (int)((__umulhi(d.m, (uint32_t)n) + (uint32_t)n) >> d.l); }
 

@@ -52,10 +52,12 @@ __global__ void __launch_bounds__(kDwColMaxThreads) depthwise3x3_col_kernel(cons
   grid_dependency_wait();   // launched ahead of its predecessor's end: see launch_overlapped
 
   const int total = p.N * p.tiles_h * p.tiles_w;
+  int armed[2] = {0, 0};   // thread 0: copies issued into each buffer (for the drain of a CTA that gave up)
   auto issue = [&](int tile, int buf) {   // one thread: the patch of `tile` into buffer `buf`
     const int tw = tile % p.tiles_w;
     const int th = (tile / p.tiles_w) % p.tiles_h;
     const int n = tile / (p.tiles_w * p.tiles_h);
+    ++armed[buf];
     mbar_expect_tx(bar0 + 8u * buf, p.patch_bytes);
     tma_load_4d(patch0 + buf * p.patch_stride, &tmap, 0, tw * p.TWt - p.pad_w, th * kRows - p.pad_h, n, bar0 + 8u * buf);
   };
@@ -199,6 +201,10 @@ __global__ void __launch_bounds__(kDwColMaxThreads) depthwise3x3_col_kernel(cons
   else run_tiles(std::integral_constant<int, kLeanClamp>{});
 
   grid_launch_dependents();   // the successor may take the SMs that free up from here on
+  if (*abort_flag != 0 && threadIdx.x == 0) {   // gave up: wait, bounded, for the patches still on their way
+    for (int b = 0; b < 2; ++b)
+      if (armed[b] > 0) mbar_drain(bar0 + 8u * b, (uint32_t)(armed[b] - 1) & 1u);
+  }
   if (q.count_sat) {   // clipped outputs: one atomic pair per warp that saw any
     sat_below = __reduce_add_sync(0xffffffffu, sat_below);
     sat_above = __reduce_add_sync(0xffffffffu, sat_above);

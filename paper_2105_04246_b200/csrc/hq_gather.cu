@@ -173,6 +173,8 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
   // first byte (in the image row) of the tile's raw box: the leftmost filter tap of its first pixel, rounded down to 16
   auto box_start = [&](int wo0) { return ((wo0 * p.stride_w - p.pad_w) * p.C) & ~15; };   // arithmetic on negative values: & rounds towards -inf
 
+  int fin_stage = 0;          // the raw-row producer's ring position when it stopped (see the end of the kernel)
+  uint32_t fin_phase = 0;
   if (warp == 0) {
     // ------------------------------ raw rows: one TMA box per tile ------------------------------
     int stage = 0;
@@ -195,6 +197,8 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
         phase ^= 1u;
       }
     }
+    fin_stage = stage;   // where the ring stands, for the drain of a CTA that gave up
+    fin_phase = phase;
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -468,6 +472,10 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
 
   tc_fence_before();
   __syncthreads();
+  if (*abort_flag != 0) {   // gave up: the thread that issued the raw-row copies waits, bounded, for those still in flight
+    if (warp == 0 && lane == 0) ring_drain(raw_full, p.stages_raw, fin_stage, fin_phase);
+    __syncthreads();
+  }
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");

@@ -179,6 +179,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     return mt * p.tiles_col + ct;
   };
   const int my_tiles = own_tile(0) >= 0 ? 1 : 0;   // only "has any" is used
+  int fin_stage = 0;          // the producers' ring position when they stopped (see the end of the kernel)
+  uint32_t fin_phase = 0;
 
   // The three single-issuer roles below are executed by their WHOLE warp with warp-uniform control flow and
   // values; only the copy / MMA / commit instructions themselves sit under a one-lane predicate (elect.sync).
@@ -453,6 +455,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
           }
         }
       }
+      fin_stage = stage;   // where the ring stands, for the drain of a CTA that gave up
+      fin_phase = phase;
     }
     __syncwarp();
   } else if (warp == 2) {
@@ -508,6 +512,8 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
             }
           }
         }
+        fin_stage = stage;
+        fin_phase = phase;
       }
     }
     __syncwarp();
@@ -880,6 +886,21 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   tc_fence_before();
   if constexpr (kPairK) cluster_sync_all();   // neither CTA leaves while the other may still read its operands or arrive on its barriers
   else __syncthreads();
+  if constexpr (!kPairK) {
+    // A CTA that gave up does not leave with bulk copies into its shared memory in flight: the threads that issued them wait,
+    // again bounded, for the stages they armed last.  (A pair's "full" barriers live in rank 0, which rank 1 cannot poll:
+    // pairs rely on the cluster barrier above.)
+    if (abort_flag_s != 0) {   // the same for every thread: read after the barrier
+      if (kiters > 0 && lane == 0) {
+        if (warp == 0) ring_drain(a_full, p.stages_a, fin_stage, fin_phase);
+        if (warp == 2 && my_tiles > 0) {
+          if (p.b_resident) mbar_drain(b_full(0), 0u);
+          else if (halo) ring_drain(b_full, p.stages_b, fin_stage, fin_phase);
+        }
+      }
+      __syncthreads();
+    }
+  }
   if (warp == 1) {
     tc_fence_after();
     if constexpr (kPairK) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
