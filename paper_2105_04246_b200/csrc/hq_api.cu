@@ -1632,8 +1632,23 @@ static hq_status conv_wgrad_stride1(hq_ctx* ctx, cudaStream_t s, const hq_conv_d
     }
   // dY: views shifted by pad_w - s, summed over the first W columns (the pixels of the input row they pair with); X: views
   // shifted by s - pad_w, summed over the first Wo columns
-  HQ_CUDA(ctx, launch_wgrad_pack(dY, At, d.N, Ho, Wo, d.K, Hp, P, d.pad_h, -1, d.pad_w, d.W, Mp, ry, rowsum, s));
-  HQ_CUDA(ctx, launch_wgrad_pack(X, Bs, d.N, d.H, d.W, d.C, Hp, P, d.pad_h, +1, d.pad_w, Wo, Mp, rx, colsum, s));
+  // the two packing kernels are independent: the smaller one (dY) runs on a side stream next to the other, forked from
+  // and joined into the caller's stream with events (as the parity classes of a strided backward pass do)
+  const bool side = ctx->parallel_subs && ctx->side[0] != nullptr;
+  cudaStream_t s_dy = side ? ctx->side[0] : s;
+  if (side) {
+    HQ_CUDA(ctx, cudaEventRecord(ctx->ev_fork, s));
+    HQ_CUDA(ctx, cudaStreamWaitEvent(s_dy, ctx->ev_fork, 0));
+  }
+  cudaError_t pe = launch_wgrad_pack(dY, At, d.N, Ho, Wo, d.K, Hp, P, d.pad_h, -1, d.pad_w, d.W, Mp, ry, rowsum, s_dy);
+  const cudaError_t xe = launch_wgrad_pack(X, Bs, d.N, d.H, d.W, d.C, Hp, P, d.pad_h, +1, d.pad_w, Wo, Mp, rx, colsum, s);
+  if (side) {   // joined whatever happened, so that the side stream never stays forked
+    const cudaError_t re = cudaEventRecord(ctx->ev_join[0], s_dy);
+    const cudaError_t we = re == cudaSuccess ? cudaStreamWaitEvent(s, ctx->ev_join[0], 0) : re;
+    if (pe == cudaSuccess) pe = we;
+  }
+  HQ_CUDA(ctx, pe);
+  HQ_CUDA(ctx, xe);
   HQ_CUDA(ctx, launch_zero_tail(At, rows + brows, Mp, Mv, s));
   ctx->launches += Mp > Mv ? 3 : 2;
   SubSpec sp{};
