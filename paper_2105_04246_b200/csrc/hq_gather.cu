@@ -173,8 +173,7 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
   // first byte (in the image row) of the tile's raw box: the leftmost filter tap of its first pixel, rounded down to 16
   auto box_start = [&](int wo0) { return ((wo0 * p.stride_w - p.pad_w) * p.C) & ~15; };   // arithmetic on negative values: & rounds towards -inf
 
-  int fin_stage = 0;          // the raw-row producer's ring position when it stopped (see the end of the kernel)
-  uint32_t fin_phase = 0;
+  __shared__ int fin_s[2];    // the raw-row producer's ring position when it stopped (see the end of the kernel)
   if (warp == 0) {
     // ------------------------------ raw rows: one TMA box per tile ------------------------------
     int stage = 0;
@@ -197,8 +196,10 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
         phase ^= 1u;
       }
     }
-    fin_stage = stage;   // where the ring stands, for the drain of a CTA that gave up
-    fin_phase = phase;
+    if (lane == 0) {   // where the ring stands, for the drain of a CTA that gave up
+      fin_s[0] = stage;
+      fin_s[1] = (int)phase;
+    }
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -327,9 +328,8 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
     const int c_begin = 0, c_end = p.BN / 16;   // a warp drains all columns of its 32 rows
     const QPacked qk = qpacked(q);
     const bool lean = kOut == kOutInt8 && q.fast && !q.count_sat;
-    // 32-byte stores where every output row starts on a 32-byte boundary (int8 rows of BN bytes; 4-byte rows of 4 BN)
+    // 32-byte stores of the 4-byte output forms where every output row starts on a 32-byte boundary
     const bool base32 = (reinterpret_cast<uintptr_t>(p.out) & 31u) == 0;
-    [[maybe_unused]] const bool wide = base32 && (p.BN & 31) == 0;
     [[maybe_unused]] const bool wide32 = base32 && (p.BN & 7) == 0;
     // The tile loop, instantiated per epilogue variant (kMode >= 0: straight-line int8 pass with that rounding; -1: the
     // general pass), so that the loop a warp actually runs holds one variant's code only.
@@ -387,12 +387,9 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
               pass16(vb, (ch + 1) * 16, wd + 4);
             }
             if (row_valid) {
-              if (!last && wide) {   // 32 columns in one store: a whole 32-byte sector per thread
-                st_global_v8(reinterpret_cast<uint32_t*>(dst_row + ch * 16), wd);
-              } else {
-                *reinterpret_cast<uint4*>(dst_row + ch * 16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-                if (!last) *reinterpret_cast<uint4*>(dst_row + (ch + 1) * 16) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
-              }
+              // 16-byte stores: one 32-byte store per two passes was measured 1 us slower on the stem (register pressure)
+              *reinterpret_cast<uint4*>(dst_row + ch * 16) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+              if (!last) *reinterpret_cast<uint4*>(dst_row + (ch + 1) * 16) = make_uint4(wd[4], wd[5], wd[6], wd[7]);
             }
           }
           if (row_valid) {
@@ -473,7 +470,7 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
   tc_fence_before();
   __syncthreads();
   if (*abort_flag != 0) {   // gave up: the thread that issued the raw-row copies waits, bounded, for those still in flight
-    if (warp == 0 && lane == 0) ring_drain(raw_full, p.stages_raw, fin_stage, fin_phase);
+    if (warp == 0 && lane == 0) ring_drain(raw_full, p.stages_raw, fin_s[0], (uint32_t)fin_s[1]);
     __syncthreads();
   }
   if (warp == 1) {
