@@ -1555,7 +1555,7 @@ __attribute__((visibility("default"))) hq_status hq_linear_wgrad(hq_ctx* ctx, vo
   hq_range_state* tmp = reinterpret_cast<hq_range_state*>(ctx->d_wgrad + a_bytes + b_bytes + t_bytes);
   HQ_CUDA(ctx, launch_transpose_rows(dY, At, M, N, Mp, 0, s));
   HQ_CUDA(ctx, launch_transpose_rows(X, Bt, M, K, Mp, 0, s));
-  HQ_CUDA(ctx, launch_wgrad_row_terms(dY, M, N, dyq, xq, terms, s));
+  HQ_CUDA(ctx, launch_wgrad_row_terms(At, M, Mp, N, dyq, xq, terms, s));   // row sums of dY^T, from the transposed copy
   ctx->launches += 3;
   // GW[n][k] = fl(float(acc) * fl(s_dy * s_x)): the layer kernel's binary32 output mode; its "weight scale" is the scale of X
   const float* x_scale = reinterpret_cast<const float*>(reinterpret_cast<const char*>(xq) + offsetof(hq_range_state, scale));

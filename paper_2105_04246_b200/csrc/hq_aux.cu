@@ -717,13 +717,23 @@ __global__ void zero_tail_kernel(int8_t* base, int rows, int64_t pitch, int64_t 
 
 // sum_m (dy - z_dy)(x - z_x) = sum_m (dy - z_dy) x  -  z_x * sum_m (dy - z_dy): the second term, one number per output
 // row n, which the layer kernel's epilogue subtracts from every accumulator of that row.
-__global__ void wgrad_row_terms_kernel(const int8_t* __restrict__ dY, int M, int N, const hq_range_state* __restrict__ dyq,
-                                       const hq_range_state* __restrict__ xq, int32_t* __restrict__ terms) {
-  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+// Reads the transposed copy dY^T [N][Mp] (rows zero-filled beyond M): one warp per row, 16 bytes per lane and step.
+__global__ void __launch_bounds__(256) wgrad_row_terms_kernel(const int8_t* __restrict__ dYt, int M, int Mp, int N,
+                                                               const hq_range_state* __restrict__ dyq, const hq_range_state* __restrict__ xq,
+                                                               int32_t* __restrict__ terms) {
+  const int n = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (n >= N) return;
+  const uint4* row = reinterpret_cast<const uint4*>(dYt + (int64_t)n * Mp);   // Mp is a multiple of 16
   int sum = 0;
-  for (int m = 0; m < M; ++m) sum += dY[(int64_t)m * N + n];
-  terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
+  for (int i = lane; i < Mp / 16; i += 32) {
+    const uint4 v = row[i];
+    sum = __dp4a((int)v.x, 0x01010101, sum);
+    sum = __dp4a((int)v.y, 0x01010101, sum);
+    sum = __dp4a((int)v.z, 0x01010101, sum);
+    sum = __dp4a((int)v.w, 0x01010101, sum);
+  }
+  sum = __reduce_add_sync(0xffffffffu, sum);
+  if (lane == 0) terms[n] = xq->zero_point * (sum - dyq->zero_point * M);
 }
 
 // ---- weight gradient of a depthwise layer (CUDA cores) -----------------------------------------------------------
@@ -1524,9 +1534,9 @@ cudaError_t launch_wgrad_reduce_taps(const int32_t* slabs, int nslabs, int rows,
   wgrad_reduce_taps_kernel<<<blocks, 256, 0, s>>>(slabs, nslabs, rows, slab_rows, cols, C, colsum, rowsum, mvalid, dyq, xq, G);
   return cudaGetLastError();
 }
-cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
+cudaError_t launch_wgrad_row_terms(const int8_t* dYt, int M, int Mp, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
                                    cudaStream_t s) {
-  wgrad_row_terms_kernel<<<(N + 127) / 128, 128, 0, s>>>(dY, M, N, dyq, xq, terms);
+  wgrad_row_terms_kernel<<<(N + 7) / 8, 256, 0, s>>>(dYt, M, Mp, N, dyq, xq, terms);
   return cudaGetLastError();
 }
 

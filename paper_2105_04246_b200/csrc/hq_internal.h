@@ -302,7 +302,7 @@ cudaError_t launch_wgrad_reduce_taps(const int32_t* slabs, int nslabs, int rows,
                                      cudaStream_t s);
 cudaError_t launch_wgrad_reduce(const int32_t* slabs, int nslabs, int rows, int cols, const int32_t* colsum, const int32_t* rowsum, int M,
                                 const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
-cudaError_t launch_wgrad_row_terms(const int8_t* dY, int M, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
+cudaError_t launch_wgrad_row_terms(const int8_t* dYt, int M, int Mp, int N, const hq_range_state* dyq, const hq_range_state* xq, int32_t* terms,
                                    cudaStream_t s);
 // sum over the in-image taps and the channels of (a - z_a), times zw, per output pixel of the layer (forward: over the
 // input windows; backward data: over the output-gradient pixels that reach the input pixel): the weight-zero-point term
