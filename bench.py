@@ -691,7 +691,7 @@ def run_wgrad(args):
         dy, x = synth.tiled(synth.gradients, g, dy_shape), synth.tiled(synth.relu_activations, g, x_shape)
         label = (f"{args.workload}: weight gradient of {'depthwise ' if cs.depthwise else ''}conv3x3 {cs.C}->{cs.K} @{cs.H}x{cs.W}, batch {cs.N} "
                  f"-> FP32 G_W{list(gw_shape)}")
-        path = ("CUDA-core kernel, integer atomics, conversion" if cs.depthwise else
+        path = ("CUDA-core kernel on transposed words (four pixels per dot-product instruction), border sums for the zero points, conversion" if cs.depthwise else
                 "dY and X packed channel-major over a padded pixel index (one copy of X per horizontal filter offset), sliced reduction on the "
                 "tensor-core layer kernel (int32 slabs), slab sum + conversion")
     else:
@@ -764,7 +764,7 @@ def run_wgrad(args):
         "gpu_launches": int(launches * pool * repeats), "launches_per_step": int(launches),
         "hbm_bytes_per_step": {"algorithmic": int(nbytes)},
         "roofline": {"bound": "hbm", "achieved": round(ach, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                     "kernel": ("dw_wgrad_kernel" if cs.depthwise else "wgrad_pack_kernel x 2 + hq_gemm_kernel (int32 slabs) + wgrad_reduce_taps_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
+                     "kernel": ("dw_wgrad3x3_kernel + dw_wgrad_finish_kernel" if cs.depthwise else "wgrad_pack_kernel x 2 + hq_gemm_kernel (int32 slabs) + wgrad_reduce_taps_kernel") if conv else "hq_gemm_kernel (binary32 output) after transpose_rows_kernel x 2", "launch_us": round(ms_step * 1e3, 3), "traffic": None,
                      "peak_source": peak_kind, "frac_of": f"of {peak_kind}"},
         "e2e": {"value": round(ops / (e2e_ms * 1e-3) / 1e12, 4), "unit": "TOPS", "ms_per_step": round(e2e_ms, 4),
                 "h2d_bytes_per_step": int(M * N + M * K), "d2h_bytes_per_step": int(4 * N * K), "steps": e2e_steps},

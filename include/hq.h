@@ -182,7 +182,8 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              (default), 0 = every CTA works on its own 128-row tile, 1 = pairs of CTAs on neighbouring SMs share
  *              256-row tiles (one tensor-core instruction for both, each CTA holding half of the weight rows)
  *              wherever the layer allows.
- *   "wgrad_windows": weight gradient of dense convolutions (read at every call): -1 = library's choice (default),
+ *   "wgrad_windows": weight gradients of convolutions (read at every call; 1 also selects the general depthwise form
+ *              instead of the transposing one for 3x3 stride-1 pad-1 depthwise layers): -1 = library's choice (default),
  *              0 = stride-1 layers pack both tensors channel-major over a padded pixel index (one copy of dY, one
  *              copy of X per horizontal filter offset) wherever the shape allows, 1 = always the general form
  *              (one transposed copy of X per filter tap).

@@ -948,7 +948,7 @@ __attribute__((visibility("default"))) hq_status hq_create(hq_ctx** out, int dev
   ctx->scratch_elems = 4096;
   if (cudaMalloc((void**)&ctx->d_status, sizeof(int32_t)) != cudaSuccess || cudaMemset(ctx->d_status, 0, sizeof(int32_t)) != cudaSuccess ||
       cudaMalloc((void**)&ctx->d_scratch, ctx->scratch_elems * sizeof(int32_t)) != cudaSuccess ||
-      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess || depthwise_col_set_smem_attr(200u * 1024u) != cudaSuccess ||
+      gemm_set_smem_attr(kSmemBudget + 1024) != cudaSuccess || depthwise_tiled_set_smem_attr(200u * 1024u) != cudaSuccess || depthwise_col_set_smem_attr(200u * 1024u) != cudaSuccess || dw_wgrad3x3_set_smem_attr(200u * 1024u) != cudaSuccess ||
       !make_side_streams(ctx)) {
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_scratch) cudaFree(ctx->d_scratch);
@@ -1716,6 +1716,52 @@ __attribute__((visibility("default"))) hq_status hq_conv_wgrad(hq_ctx* ctx, void
     if (d.C % 4 != 0 || d.C > 1024 || (size_t)d.C * d.R * d.S * sizeof(int32_t) > 48u * 1024u)
       return fail(ctx, HQ_ERR_UNSUPPORTED, "depthwise weight gradient needs C %% 4 == 0, C <= 1024 and C * R * S <= 12288");
     if (M64 > (1 << 30)) return fail(ctx, HQ_ERR_UNSUPPORTED, "weight gradient: too many output pixels");
+    // 3x3, stride 1, padding 1: four pixels per dp4a on transposed words, zero points taken out from border sums
+    if (d.R == 3 && d.S == 3 && d.stride_h == 1 && d.stride_w == 1 && d.pad_h == 1 && d.pad_w == 1 && d.C % 16 == 0 && d.C <= 256 &&
+        d.H >= 2 && d.W >= 2 && ctx->wgrad_windows != 1) {
+      DwWgradParams p{};
+      p.N = d.N; p.H = d.H; p.W = d.W; p.C = d.C;
+      const int cwords = d.C / 4;
+      int cols4 = std::min(std::min(round_up(d.W, 4) / 4, 7), kDwColMaxThreads / cwords);
+      for (;; --cols4) {   // the widest tile whose two buffers and sums fit
+        p.TWt = 4 * std::max(cols4, 1);
+        p.x_bytes = (uint32_t)d.C * (uint32_t)(p.TWt + 2) * (uint32_t)(kDwColRows + 2);
+        p.dy_bytes = (uint32_t)d.C * (uint32_t)p.TWt * (uint32_t)kDwColRows;
+        p.dy_offset = (p.x_bytes + 127u) & ~127u;
+        p.buf_stride = p.dy_offset + ((p.dy_bytes + 127u) & ~127u);
+        if (dw_wgrad3x3_smem_bytes(p) <= 200u * 1024u || cols4 <= 1) break;
+      }
+      p.tiles_h = ceil_div(d.H, kDwColRows);
+      p.tiles_w = ceil_div(d.W, p.TWt);
+      const int64_t n_tiles = (int64_t)d.N * p.tiles_h * p.tiles_w;
+      if (cols4 >= 1 && cwords * (p.TWt / 4) >= 64 && n_tiles <= INT32_MAX && dw_wgrad3x3_smem_bytes(p) <= 200u * 1024u) {
+        const size_t need = (size_t)kDwWgSlots * d.C * sizeof(int32_t) + 256;
+        if (need > ctx->wgrad_bytes) {
+          if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));
+          ctx->d_wgrad = nullptr;
+          ctx->wgrad_bytes = 0;
+          HQ_CUDA(ctx, cudaMalloc((void**)&ctx->d_wgrad, need));
+          ctx->wgrad_bytes = need;
+        }
+        p.sums = reinterpret_cast<int32_t*>(ctx->d_wgrad);
+        p.status = ctx->d_status;
+        HQ_CUDA(ctx, cudaMemsetAsync(p.sums, 0, (size_t)kDwWgSlots * d.C * sizeof(int32_t), s));
+        CUtensorMap tx, ty;
+        uint64_t dims[4] = {(uint64_t)d.C, (uint64_t)d.W, (uint64_t)d.H, (uint64_t)d.N};
+        uint64_t strides[3] = {(uint64_t)d.C, (uint64_t)d.C * d.W, (uint64_t)d.C * d.W * d.H};
+        uint32_t es[4] = {1, 1, 1, 1};
+        uint32_t box_x[4] = {(uint32_t)d.C, (uint32_t)(p.TWt + 2), (uint32_t)(kDwColRows + 2), 1u};
+        uint32_t box_y[4] = {(uint32_t)d.C, (uint32_t)p.TWt, (uint32_t)kDwColRows, 1u};
+        CUresult r1 = ctx->encode(&tx, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(X), dims, strides, box_x, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        CUresult r2 = ctx->encode(&ty, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(dY), dims, strides, box_y, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r1 != CUDA_SUCCESS || r2 != CUDA_SUCCESS) return fail(ctx, HQ_ERR_CUDA, "tensor map encoding failed (CUresult %d, %d)", (int)r1, (int)r2);
+        HQ_CUDA(ctx, launch_dw_wgrad3x3(p, tx, ty, ctx->num_sms, dyq, xq, GW, s));
+        ctx->launches += 3;
+        return HQ_OK;
+      }
+    }
     const size_t need = (size_t)d.C * d.R * d.S * sizeof(int32_t) + 256;
     if (need > ctx->wgrad_bytes) {
       if (ctx->d_wgrad) HQ_CUDA(ctx, cudaFree(ctx->d_wgrad));

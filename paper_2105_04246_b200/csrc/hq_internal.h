@@ -253,6 +253,20 @@ cudaError_t launch_depthwise_tiled(const DwParams& p, const CUtensorMap& tmap, i
 // 3x3 stride-1 depthwise, columns of tiles of kDwColRows x 4 pixels per thread (hq_dw3x3.cu): TR = kDwColRows, TWt a multiple of 4
 constexpr int kDwColRows = 7;
 constexpr int kDwColMaxThreads = 448;
+// weight gradient of a 3x3 stride-1 pad-1 depthwise layer (hq_dw_wgrad.cu)
+constexpr int kDwWgSlots = 27;          // rows of C ints in the sum buffer: 9 taps, 2 totals, 8 border sums per tensor
+struct DwWgradParams {
+  int32_t N, H, W, C;                   // H == Ho, W == Wo
+  int32_t TWt, tiles_h, tiles_w;        // tiles of kDwColRows rows x TWt columns (a multiple of 4)
+  uint32_t x_bytes, dy_bytes;           // bytes the two TMA boxes of a tile deliver
+  uint32_t dy_offset, buf_stride;       // dy tile behind the x patch; distance of the two buffers (multiples of 128)
+  int32_t* sums;                        // [kDwWgSlots][C], zeroed by the caller
+  int32_t* status;
+};
+cudaError_t launch_dw_wgrad3x3(const DwWgradParams& p, const CUtensorMap& tmap_x, const CUtensorMap& tmap_dy, int num_sms,
+                               const hq_range_state* dyq, const hq_range_state* xq, float* G, cudaStream_t s);
+cudaError_t dw_wgrad3x3_set_smem_attr(uint32_t smem_bytes);
+uint32_t dw_wgrad3x3_smem_bytes(const DwWgradParams& p);
 cudaError_t launch_depthwise_col(const DwParams& p, const CUtensorMap& tmap, int out_mode, int num_sms, int ctas_per_sm, cudaStream_t s, bool overlap);
 cudaError_t depthwise_col_set_smem_attr(uint32_t smem_bytes);
 uint32_t depthwise_col_smem_bytes(const DwParams& p);

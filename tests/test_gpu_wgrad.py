@@ -178,11 +178,24 @@ DW_WGRAD_CASES = {
     "dw5x5_c48": dict(N=1, H=13, W=9, C=48, R=5, stride=1, pad=2),
     "dw3x3_c320": dict(N=2, H=7, W=7, C=320, R=3, stride=1, pad=1),
     "dw3x3_c144_56": dict(N=4, H=56, W=56, C=144, R=3, stride=1, pad=1),
+    "dw3x3_c64_ragged": dict(N=3, H=15, W=30, C=64, R=3, stride=1, pad=1),
+    "dw3x3_c256_small": dict(N=2, H=2, W=5, C=256, R=3, stride=1, pad=1),
 }
 
 
+@pytest.mark.parametrize("windows", [-1, 1])
 @pytest.mark.parametrize("name", list(DW_WGRAD_CASES))
-def test_depthwise_wgrad_matches_oracle(ctx, name):
+def test_depthwise_wgrad_matches_oracle(ctx, name, windows):
+    """Both depthwise forms (3x3 stride 1 pad 1: four pixels per dot-product instruction on transposed words with the zero
+    points taken out from border sums; any other shape, and option 1: one product at a time) give the oracle's bits."""
+    ctx.set_option("wgrad_windows", windows)
+    try:
+        _dw_wgrad_case(ctx, name)
+    finally:
+        ctx.set_option("wgrad_windows", -1)
+
+
+def _dw_wgrad_case(ctx, name):
     c = DW_WGRAD_CASES[name]
     dev = torch.device("cuda", ctx.device)
     r = synth.rng(305, len(name), c["H"], c["C"])
