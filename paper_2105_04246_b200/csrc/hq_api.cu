@@ -1591,7 +1591,8 @@ static hq_status conv_wgrad_stride1(hq_ctx* ctx, cudaStream_t s, const hq_conv_d
   const int64_t Mv = (int64_t)d.N * Hp * P;   // padded reduction length
   if (Mv > (1 << 26)) return HQ_OK;
   const int tiles_one = ceil_div(rows, kTileM) * d.R * per_row;
-  const int want_slices = std::max(1, (2 * ctx->num_sms + tiles_one - 1) / tiles_one);
+  // one tile per SM, none left over for a second round: fewer slices also mean fewer slab bytes for the last pass
+  const int want_slices = std::max(1, ctx->num_sms / tiles_one);
   const int slice_len = (int)std::max<int64_t>(128, round_up((int)ceil_div((int)Mv, want_slices), 128));
   const int slices = ceil_div((int)Mv, slice_len);
   const int64_t Mp = (int64_t)slices * slice_len;

@@ -614,7 +614,7 @@ __global__ void __launch_bounds__(256) wgrad_reduce_taps_kernel(const int32_t* _
 // One block: 32 channels of kPackRows padded rows of one image, all rows at once: the source rows go to shared memory
 // transposed (4x4 byte blocks turned in registers; channel-major words behind 16 zero bytes, zeros after), each view is
 // read from there as aligned words and funnel-shifted, written in 16-byte pieces and summed with dp4a.
-constexpr int kPackRows = 4;
+constexpr int kPackRows = 8;   // x 32 channels = the 256 threads of a block
 constexpr int kPackMaxP = 256;
 // words per channel row of the tile: 16 zero bytes, the row, room for the shifted reads past its end; odd, so that the
 // transposing stores spread over the banks
@@ -648,58 +648,59 @@ __global__ void __launch_bounds__(256) wgrad_pack_kernel(const int8_t* __restric
     tile(rl, cg * 4 + 3)[4 + wg] = __byte_perm(a1, b1, 0x7632);
   }
   __syncthreads();
-  // One task = one (row of the block, view, channel): its thread walks along the row in 16-byte pieces (the lanes of a warp
-  // are 32 channels: conflict-free shared-memory reads, one sum per task), two pieces per store where rows allow 32 bytes.
-  const int per_row = rg.ns * 32;
+  // One thread = one (row of the block, channel): the lanes of a warp are 32 channels (conflict-free shared-memory reads).
+  // It sums the row once, then for every view takes out the few bytes the view's window leaves, and, for a stored view,
+  // walks along the row in 16-byte pieces, two pieces per store where rows allow 32 bytes.
   const bool wide = (P & 31) == 0 && (pitch & 31) == 0 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
-  for (int task = tid; task < kPackRows * per_row; task += 256) {
-    const int rl = task / per_row, t = task - rl * per_row;
-    const int c = t & 31, j = t >> 5;
+  {
+    const int rl = tid >> 5, c = tid & 31;   // kPackRows * 32 == 256 threads
     const int pr = pr0 + rl, h = pr - row_off;
-    if (pr >= Hp || c0 + c >= Cs) continue;
-    const int shift = sign * (j - pad);
-    const bool stored = sign > 0 || shift == 0;
-    const uint32_t* trow = tile(rl, c);
-    // sum of the view's first `limit` columns = sum of the whole source row minus what the window [shift, shift + limit)
-    // leaves out at either end (a few bytes)
-    int part = 0;
-    if (h >= 0 && h < Hs) {
-      for (int g = 0; g < wgroups; ++g) part = __dp4a((int)trow[4 + g], 0x01010101, part);
+    if (pr < Hp && c0 + c < Cs) {
+      const uint32_t* trow = tile(rl, c);
+      const bool has = h >= 0 && h < Hs;
+      int total = 0;
+      if (has)
+        for (int g = 0; g < wgroups; ++g) total = __dp4a((int)trow[4 + g], 0x01010101, total);
       const int8_t* bytes = reinterpret_cast<const int8_t*>(trow) + 16;
-      for (int i = 0; i < min(shift, Ws); ++i) part -= bytes[i];
-      for (int i = max(0, shift + limit); i < Ws; ++i) part -= bytes[i];
-    }
-    if (stored) {
-      const int b0 = 16 + shift;                     // first byte of the view in the tile row (>= 0)
-      const uint32_t* wp = trow + (b0 >> 2);
-      const uint32_t sh = (uint32_t)(b0 & 3) * 8u;
-      int8_t* out = dst + ((int64_t)(sign > 0 ? j : 0) * Cs + c0 + c) * pitch + ((int64_t)n * Hp + pr) * P;
-      uint32_t lo = wp[0];
-      uint32_t prev[4];
-      for (int q = 0; q * 16 < P; ++q) {
-        uint32_t w4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t hi = wp[q * 4 + e + 1];
-          w4[e] = __funnelshift_r(lo, hi, sh);
-          lo = hi;
+      for (int j = 0; j < rg.ns; ++j) {
+        const int shift = sign * (j - pad);
+        if (has) {   // sum of the view's first `limit` columns = row total minus what the window [shift, shift + limit) leaves out
+          int part = total;
+          for (int i = 0; i < min(shift, Ws); ++i) part -= bytes[i];
+          for (int i = max(0, shift + limit); i < Ws; ++i) part -= bytes[i];
+          if (part != 0)
+            for (int r = 0; r < rg.nr; ++r)
+              if (h >= rg.row_lo[r] && h < rg.row_hi[r]) atomicAdd(&acc_s[r * rg.ns + j][c], part);
         }
-        if (wide) {
-          if (q & 1) {
-            const uint32_t w8[8] = {prev[0], prev[1], prev[2], prev[3], w4[0], w4[1], w4[2], w4[3]};
-            st_global_v8(reinterpret_cast<uint32_t*>(out + (q - 1) * 16), w8);
-          } else {
+        if (!(sign > 0 || shift == 0)) continue;   // this view is only summed
+        const int b0 = 16 + shift;                 // first byte of the view in the tile row (>= 0)
+        const uint32_t* wp = trow + (b0 >> 2);
+        const uint32_t sh = (uint32_t)(b0 & 3) * 8u;
+        int8_t* out = dst + ((int64_t)(sign > 0 ? j : 0) * Cs + c0 + c) * pitch + ((int64_t)n * Hp + pr) * P;
+        uint32_t lo = wp[0];
+        uint32_t prev[4];
+        for (int q = 0; q * 16 < P; ++q) {
+          uint32_t w4[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) prev[e] = w4[e];
+          for (int e = 0; e < 4; ++e) {
+            const uint32_t hi = wp[q * 4 + e + 1];
+            w4[e] = __funnelshift_r(lo, hi, sh);
+            lo = hi;
           }
-        } else {
-          *reinterpret_cast<uint4*>(out + q * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          if (wide) {
+            if (q & 1) {
+              const uint32_t w8[8] = {prev[0], prev[1], prev[2], prev[3], w4[0], w4[1], w4[2], w4[3]};
+              st_global_v8(reinterpret_cast<uint32_t*>(out + (q - 1) * 16), w8);
+            } else {
+#pragma unroll
+              for (int e = 0; e < 4; ++e) prev[e] = w4[e];
+            }
+          } else {
+            *reinterpret_cast<uint4*>(out + q * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          }
         }
       }
     }
-    if (part != 0 && h >= 0 && h < Hs)
-      for (int r = 0; r < rg.nr; ++r)
-        if (h >= rg.row_lo[r] && h < rg.row_hi[r]) atomicAdd(&acc_s[r * rg.ns + j][c], part);
   }
   __syncthreads();
   for (int i = tid; i < rg.nr * rg.ns * 32; i += 256) {
