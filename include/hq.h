@@ -289,12 +289,16 @@ hq_status hq_linear_wgrad(hq_ctx* ctx, void* stream, int32_t M, int32_t N, int32
  * hi = ho*stride_h - pad_h + r (wi alike), output pixels whose (hi,wi) lies outside the image contributing nothing (padding
  * is zero in the real domain).  dY is N x Ho x Wo x K, X is N x H x W x C, GW has the layout of the weights, binary32.
  * The sum is formed modulo 2^32: exact whenever the true sum fits in int32.  At most 2^24 output pixels.  Depthwise layers
- * (groups == C == K; 3x3 or 5x5 filters, C a multiple of 4, at most 1024): GW is [C][R][S], the sum runs with k == c, on a
- * CUDA-core kernel with integer atomics.
- * How it runs: the filter windows of X and dY are written transposed (pixels innermost) into context-owned scratch (grown
- * with cudaMalloc when a larger layer is first seen: R*S times the size of X; calls on one context must not overlap);
- * the reduction over the pixels is cut into slices that the tensor-core layer kernel multiplies side by side, and a last
- * pass sums the slices, removes both zero points and converts.  No range state is written. */
+ * (groups == C == K; 3x3 or 5x5 filters, C a multiple of 4, at most 1024): GW is [C][R][S], the sum runs with k == c, on
+ * CUDA-core kernels (3x3, stride 1, padding 1, C a multiple of 16 of at most 256: four pixels per 4-way dot product on
+ * words transposed in registers, the zero points taken out from per-channel totals and border sums; else one product at
+ * a time with integer atomics).
+ * How dense layers run: both tensors are written pixels-innermost into context-owned scratch (grown with cudaMalloc when a
+ * larger layer is first seen; calls on one context must not overlap) -- stride-1 layers: dY once and X once per horizontal
+ * filter offset over a padded pixel index in which a vertical filter offset is a shift of the reduction coordinate
+ * (scratch about (S + 1) times the size of X); any other layer: one transposed copy of X per filter tap (R*S times X).
+ * The reduction over the pixels is cut into slices that the tensor-core layer kernel multiplies side by side, and a last
+ * pass sums the slices, removes both zero points and converts.  No range state is written.  (Option "wgrad_windows".) */
 hq_status hq_conv_wgrad(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
                         const int8_t* dY, const hq_range_state* dyq,
                         const int8_t* X, const hq_range_state* xq, float* GW);
