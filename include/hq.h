@@ -173,6 +173,9 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              1 = horizontal filter windows per input row gathered into a library-owned tensor where the
  *              shape allows, 2 = the fused kernel that gathers the filter windows in shared memory (nothing
  *              repacked in global memory) where the shape allows, else as -1.
+ *   "gather_span": the fused few-channel kernel of layers prepared AFTER this call, for output rows shorter than a
+ *              128-pixel tile: 1 (default) = a tile is 128 consecutive pixels of one image in row-major order, across
+ *              row ends (no unused tile rows), 0 = one output row per tile.
  *   "epilogue_groups": layers prepared AFTER this call: -1 = chosen per layer (default); g = 0, 1, 2: the sixteen
  *              epilogue warps form 2^g groups that drain alternate tiles (at most one group per accumulator buffer).
  *   "col_tiles": into how many column tiles (each a multiple of 16 columns, at most 256) the output channels of

@@ -657,7 +657,7 @@ hq_status run_conv(hq_ctx* ctx, cudaStream_t s, const hq_conv_desc* desc, hq_dir
     const uint64_t row_bytes = (uint64_t)desc->W * desc->C;
     uint64_t dims[3] = {row_bytes / 4, (uint64_t)desc->H, (uint64_t)desc->N};
     uint64_t strides[2] = {row_bytes, row_bytes * desc->H};
-    uint32_t box[3] = {g.raw_pitch / 4, (uint32_t)desc->R, 1u};
+    uint32_t box[3] = {g.raw_pitch / 4, (uint32_t)g.box_rows, 1u};
     uint32_t es[3] = {1, 1, 1};
     CUresult r = ctx->encode(&tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<int8_t*>(in), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1003,6 +1003,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
     ctx->force_repack = value;
     return HQ_OK;
   }
+  if (std::string(key) == "gather_span") {
+    if (value < 0 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "gather_span must be 0 or 1");
+    ctx->gather_span = value;
+    return HQ_OK;
+  }
   if (std::string(key) == "epilogue_groups") {
     if (value < -1 || value > 2) return fail(ctx, HQ_ERR_INVALID_ARG, "epilogue_groups must be -1, 0, 1 or 2");
     ctx->force_epi_groups = value;
@@ -1205,11 +1210,32 @@ hq_status prepare_conv_body(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
             g.BN = d.K;
             g.tiles_w = ceil_div(Wo, kTileM);
             g.num_tiles = d.N * Ho * g.tiles_w;
+            g.span = 0;
+            g.tiles_img = Ho * g.tiles_w;
+            g.box_rows = d.R;
+            // Output rows shorter than a tile would leave tile rows unused (Wo = 112: an eighth of every MMA and epilogue
+            // pass).  Tiles then run over the pixels of an image in row-major order, across row ends, and the raw box holds
+            // the input rows under every output row a tile touches (the box is as wide as the image row either way).
+            if (Wo < kTileM && ctx->gather_span != 0) {
+              const int HW = Ho * Wo, tiles_img = ceil_div(HW, kTileM);
+              int rows_max = 1;
+              for (int t = 0; t < tiles_img; ++t) {
+                const int f0 = t * kTileM, f1 = std::min(f0 + kTileM, HW) - 1;
+                rows_max = std::max(rows_max, f1 / Wo - f0 / Wo + 1);
+              }
+              const int box_rows = (rows_max - 1) * d.stride_h + d.R;
+              if (box_rows <= 256 && tiles_img < Ho && (uint64_t)pitch * box_rows <= 32u * 1024u) {
+                g.span = 1;
+                g.tiles_img = tiles_img;
+                g.box_rows = box_rows;
+                g.num_tiles = d.N * tiles_img;
+              }
+            }
             g.raw_pitch = pitch;
-            g.raw_box_bytes = pitch * (uint32_t)d.R;
+            g.raw_box_bytes = pitch * (uint32_t)g.box_rows;
             g.raw_stage_stride = (g.raw_box_bytes + 127u) & ~127u;
             g.a_stage_bytes = (uint32_t)kTileM * (uint32_t)Kp;
-            g.stages_raw = 4;
+            g.stages_raw = g.raw_stage_stride * 4u <= 48u * 1024u ? 4 : 2;
             g.off_w = 0;
             g.off_zc = (uint32_t)round_up(d.K * Kp, 128);
             g.off_raw = (uint32_t)round_up((int)(g.off_zc + zc_bytes), 1024);
@@ -1233,6 +1259,8 @@ hq_status prepare_conv_body(hq_ctx* ctx, void* stream, const hq_conv_desc* desc,
               g.epi_groups_log2 = g.epi_groups == 4 ? 2 : 1;
               g.fd_tiles_w = make_fastdiv(g.tiles_w);
               g.fd_Ho = make_fastdiv(Ho);
+              g.fd_Wo = make_fastdiv(Wo);
+              g.fd_tiles_img = make_fastdiv(g.tiles_img);
               g.status = ctx->d_status;
               g.acc_bound = (float)(d.R * SC) * 255.0f * 128.0f;
               int8_t* wm = nullptr;

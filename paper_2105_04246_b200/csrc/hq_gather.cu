@@ -163,7 +163,17 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
   const uint32_t tmem_base = tmem_base_slot;
 
   // divisions by launch constants: multiplier and shift prepared on the host; the buffer and group counts are powers of two
+  // span = 0: tile -> image n, output row ho, first output column wo0.  span = 1 (tiles run across the ends of short output
+  // rows): image n, wo0 = row-major index of the tile's first pixel in the image, ho = the output row that pixel lies in.
+  const int span = p.span;
+  const int HW = p.Ho * p.Wo;
   auto decode = [&](int tile, int& n, int& ho, int& wo0) {
+    if (span) {
+      n = fdiv(tile, p.fd_tiles_img);
+      wo0 = (tile - n * p.tiles_img) * kTileM;
+      ho = fdiv(wo0, p.fd_Wo);
+      return;
+    }
     const int t2 = fdiv(tile, p.fd_tiles_w);
     wo0 = (tile - t2 * p.tiles_w) * kTileM;
     n = fdiv(t2, p.fd_Ho);
@@ -189,7 +199,7 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
       if (!ok) break;
       if (elect_one()) {
         mbar_expect_tx(raw_full(stage), p.raw_box_bytes);
-        tma_load_3d(raw_s + stage * p.raw_stage_stride, &tmap, box_start(wo0) >> 2, ho * p.stride_h - p.pad_h, n, raw_full(stage));
+        tma_load_3d(raw_s + stage * p.raw_stage_stride, &tmap, box_start(span ? 0 : wo0) >> 2, ho * p.stride_h - p.pad_h, n, raw_full(stage));
       }
       if (++stage == p.stages_raw) {
         stage = 0;
@@ -272,9 +282,16 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
       ok = warp_wait(raw_full(rs), rph, abort_flag, p.status, kAsyncMmaFullWait, 2000u);
       if (!ok) break;
       uint32_t D[KW];
-      const uint32_t src0 = (uint32_t)(((wo0 + gt) * p.stride_w - p.pad_w) * p.C - box_start(wo0));
+      uint32_t src0;
+      if (span) {   // pixels beyond the image's end gather the last pixel's runs, their results are dropped
+        const int f = min(wo0 + gt, HW - 1);
+        const int fh = fdiv(f, p.fd_Wo);
+        src0 = (uint32_t)((fh - ho) * p.stride_h) * p.raw_pitch + (uint32_t)(((f - fh * p.Wo) * p.stride_w - p.pad_w) * p.C - box_start(0));
+      } else {
+        src0 = (uint32_t)(((wo0 + gt) * p.stride_w - p.pad_w) * p.C - box_start(wo0));
+      }
       // pixels beyond the row's end gather from inside the box as well (clamped), their results are dropped
-      const uint32_t src0c = min(src0, p.raw_pitch - (uint32_t)SC - 4u);
+      const uint32_t src0c = span ? src0 : min(src0, p.raw_pitch - (uint32_t)SC - 4u);
       gather_row<R, SC>(raw_s + rs * p.raw_stage_stride, p.raw_pitch, src0c, D);
       ok = warp_wait(a_empty(as), aph ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 4000u);
       if (!ok) break;
@@ -340,8 +357,14 @@ __global__ void __launch_bounds__(kGatherThreads, 1) hq_gather_conv_kernel(const
         if (tile >= p.num_tiles) break;
         int n, ho, wo0;
         decode(tile, n, ho, wo0);
-        const int wo = wo0 + row;
-        const bool row_valid = wo < p.Wo;
+        int wo = wo0 + row;
+        bool row_valid = wo < p.Wo;
+        if (span) {
+          row_valid = wo < HW;
+          const int f = min(wo, HW - 1);
+          ho = fdiv(f, p.fd_Wo);
+          wo = f - ho * p.Wo;
+        }
         const int64_t pix = ((int64_t)n * p.Ho + ho) * p.Wo + wo;
         int zoff = 0;
         if (row_valid) {

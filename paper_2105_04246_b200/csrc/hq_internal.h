@@ -163,8 +163,11 @@ struct GatherParams {
   int32_t N, H, W, C, Ho, Wo, R, S, stride_h, stride_w, pad_h, pad_w;
   int32_t BN;                          // output channels (a multiple of 16, at most 256): one column tile
   int32_t tiles_w, num_tiles;          // tiles of up to 128 output pixels per output row; N * Ho * tiles_w
+  int32_t span, tiles_img, box_rows;   // span = 1 (output rows shorter than a tile): a tile is 128 consecutive pixels of one image in
+                                       // row-major order (tiles_img per image, num_tiles = N * tiles_img) and its raw box holds the
+                                       // box_rows input rows under every output row it touches; span = 0: box_rows = R
   uint32_t raw_pitch;                  // bytes of one raw row in shared memory = width of the TMA box (a multiple of 16, at most 1024)
-  uint32_t raw_box_bytes, raw_stage_stride;   // raw_pitch * R, and that rounded up to 128
+  uint32_t raw_box_bytes, raw_stage_stride;   // raw_pitch * box_rows, and that rounded up to 128
   uint32_t a_stage_bytes;              // 128 * Kp
   int32_t stages_raw, stages_a;
   uint32_t off_w, off_zc, off_raw, off_a;   // byte offsets from the 1024-aligned base of dynamic shared memory
@@ -182,7 +185,7 @@ struct GatherParams {
   uint32_t idesc, tmem_cols, tmem_buf_stride;
   int32_t tmem_bufs, epi_groups;       // powers of two
   int32_t tmem_bufs_log2, epi_groups_log2;
-  FastDiv fd_tiles_w, fd_Ho;
+  FastDiv fd_tiles_w, fd_Ho, fd_Wo, fd_tiles_img;
   int32_t weights_early;
   float acc_bound;
 };
@@ -346,6 +349,7 @@ struct hq_ctx {
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
   int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
+  int gather_span = 1;                // few-channel fused kernel: 1 = tiles may run across the ends of short output rows, 0 = one output row per tile
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
   int force_epi_groups = -1;          // log2 of the epilogue warp groups: -1 chosen per layer, else min(value, log2 of the accumulator buffers)
   int force_cols = -1;                // column tiles: -1 chosen by estimated duration, 0 as wide as the MMA allows, n > 0 at least n

@@ -131,6 +131,7 @@ FWD_CASES = {
     # few channels with image rows a TMA box can address (W * C a multiple of 16): the fused gather kernel
     "7x7_s2_c3_w32_gather": dict(N=2, H=30, W=32, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
     "7x7_s2_c3_w224_gather": dict(N=1, H=12, W=224, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
+    "7x7_s2_c3_w224_h16_gather": dict(N=2, H=16, W=224, Cin=3, K=64, R=7, S=7, stride=2, pad=3),
     "3x3_c3_w320_gather": dict(N=2, H=6, W=320, Cin=3, K=32, R=3, S=3, stride=1, pad=1),
     "5x5_s2_c4_w20_gather": dict(N=1, H=17, W=20, Cin=4, K=16, R=5, S=5, stride=2, pad=1),
     "3x3_c5_w16_gather": dict(N=3, H=9, W=16, Cin=5, K=48, R=3, S=3, stride=1, pad=1),
@@ -205,6 +206,22 @@ def test_conv_fwd_few_channels_repacking(ctx, name, repack):
     in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
     makers = [synth.image_like, synth.signed_activations, synth.relu_activations]
     _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, repack=repack)
+
+
+@pytest.mark.parametrize("name", [n for n in FWD_CASES if n.endswith("_gather")])
+def test_conv_fwd_few_channels_one_row_per_tile(ctx, name):
+    """The fused few-channel kernel with tiles that stay inside one output row (the default lets them run across the ends
+    of rows shorter than a tile): the same bytes."""
+    shape = dict(FWD_CASES[name])
+    r = synth.rng(105, len(name), shape["H"])
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    makers = [synth.image_like, synth.signed_activations, synth.relu_activations]
+    ctx.set_option("gather_span", 0)
+    try:
+        _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, repack=2)
+    finally:
+        ctx.set_option("gather_span", 1)
 
 
 BWD_CASES = {
