@@ -192,6 +192,9 @@ uint64_t hq_pair_launch_count(const hq_ctx* ctx);
  *              (one transposed copy of X per filter tap).
  *   "issuers": upper limit (1, 2 or 3; default 3) of the warps of a CTA that issue tensor-core instructions,
  *              each for every n-th tile, in layers prepared AFTER this call.
+ *   "a_producers": layers prepared AFTER this call that take one copy of the input per filter tap and keep their weights
+ *              in shared memory (1x1 layers): -1 = chosen per layer (default), 1 = one warp copies the input tiles,
+ *              2 = two warps copy them for alternate tiles (with at most two issuing warps) wherever the layer allows.
  *   "overlap_launches": 1 (default) = the layer and range-update kernels are launched so that their
  *              set-up may run while the previous kernel in the stream drains; each waits for that
  *              kernel to finish before it reads memory, so stream order is unchanged.  0 = ordinary

@@ -330,12 +330,23 @@ hq_status plan_sub_fixed(hq_ctx* ctx, const SubSpec& sp, hq_sub_problem& sub, st
     // The kernel gets that from the operand ring (see its issuer loop), provided the ring holds no more than as many tiles
     // as there are buffers: the ring is shortened to that where needed.
     const int ring3 = std::min(p.stages_a, p.tmem_bufs * a_per_tile);
+    p.a_producers = 1;
+    const bool two_prod_ok = p.mode == kModeTap && p.b_resident && !p.pair && p.b_group_tiles == 0 && rings_ok && kiters > 0;
     if (p.mma_issuers == 2 && ctx->max_issuers >= 3 && p.b_resident && p.BN <= 64 && 3 * a_per_tile <= ring3 && ring3 >= 6 &&
         p.num_tiles >= 3 * ctx->num_sms && p.tmem_bufs >= 4) {
-      p.mma_issuers = 3;
-      p.stages_a = ring3;
-      if (p.mode == kModeTap) p.producer_lanes = std::min(p.producer_lanes, p.stages_a);
+      // Such layers (1x1 with few channels on either side) were measured to wait for operand A: one warp gets a copy
+      // under way about every 0.5-0.7 us whatever its size.  Up to 192 input channels a second producer (the weight
+      // producer's warp, with two issuers) beats a third issuer: 64 -> 32 channels 31 -> 25 us, 144 -> 24 44.8 -> 38.6 us,
+      // 192 -> 32 41.7 -> 36.4 us per 800k pixels; at 256 input channels the layer is close to the HBM bound either way.
+      if (two_prod_ok && ctx->a_producers != 1 && sp.Cin <= 192) {
+        p.a_producers = 2;
+      } else {
+        p.mma_issuers = 3;
+        p.stages_a = ring3;
+        if (p.mode == kModeTap) p.producer_lanes = std::min(p.producer_lanes, p.stages_a);
+      }
     }
+    if (two_prod_ok && ctx->a_producers == 2 && p.mma_issuers <= 2) p.a_producers = 2;
     p.mma_issuers = std::min(p.mma_issuers, ctx->max_issuers);
     // Several tiles per CTA: as many epilogue groups as there are accumulator buffers (at most four), so that a warp
     // pays its per-tile set-up once per several column passes; one or two tiles per CTA: all warps on every tile (the
@@ -1026,6 +1037,11 @@ __attribute__((visibility("default"))) hq_status hq_set_option(hq_ctx* ctx, cons
   if (std::string(key) == "wgrad_windows") {
     if (value < -1 || value > 1) return fail(ctx, HQ_ERR_INVALID_ARG, "wgrad_windows must be -1, 0 or 1");
     ctx->wgrad_windows = value;
+    return HQ_OK;
+  }
+  if (std::string(key) == "a_producers") {
+    if (value < -1 || value > 2 || value == 0) return fail(ctx, HQ_ERR_INVALID_ARG, "a_producers must be -1, 1 or 2");
+    ctx->a_producers = value;
     return HQ_OK;
   }
   if (std::string(key) == "issuers") {

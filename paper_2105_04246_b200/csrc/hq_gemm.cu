@@ -181,6 +181,7 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
   const int my_tiles = own_tile(0) >= 0 ? 1 : 0;   // only "has any" is used
   int fin_stage = 0;          // the producers' ring position when they stopped (see the end of the kernel)
   uint32_t fin_phase = 0;
+  int fin_passed = 0;         // two operand producers: how many ring stages this one got through
 
   // The three single-issuer roles below are executed by their WHOLE warp with warp-uniform control flow and
   // values; only the copy / MMA / commit instructions themselves sit under a one-lane predicate (elect.sync).
@@ -388,9 +389,53 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       }
     }
   };
+  // kModeTap, two operand producers (resident weights): producer `first` of `nprod` copies operand A for the CTA's tiles
+  // first, first + nprod, ...  Ring positions are global over the CTA's tiles, so a producer steps over the other's
+  // stages.  A producer never runs more than a lap ahead of the other at any stage: it passed the stages of its own
+  // previous tile, whose release implies that everything one lap before them was consumed, hence filled (the host
+  // allows two producers only where the ring holds at least two tiles).  Returns the number of stages it got through.
+  __shared__ int fin2_s[3];   // the second producer's ring position when it stopped: stages passed, stage, phase
+  auto produce_tap = [&](int first, int nprod, int& stage, uint32_t& phase) -> int {
+    bool ok = true;
+    int passed = 0;
+    auto advance = [&](int n) {
+      passed += n;
+      stage += n;
+      while (stage >= p.stages_a) {
+        stage -= p.stages_a;
+        phase ^= 1u;
+      }
+    };
+    advance(first * kiters);
+    for (int it = first; ok; it += nprod) {
+      const int tile = own_tile(it);
+      if (tile < 0) break;
+      int n0, h0, w0, col0;
+      decode(tile, n0, h0, w0, col0);
+      if (it == first) grid_dependency_wait();   // the first copy reads what the previous kernel may have written
+      for (int t = 0; t < p.ntaps && ok; ++t) {
+        const int ch = h0 * p.in_mul_h + p.tap_dh[t];
+        const int cw = w0 * p.in_mul_w + p.tap_dw[t];
+        for (int cc = 0; cc < p.chunks_per_tap; ++cc) {
+          ok = warp_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status, kAsyncProducerEmptyWait, 1000u);
+          if (!ok) break;
+          if (elect_one()) {
+            mbar_expect_tx(a_full(stage), a_stride);
+            tma_load_4d(ring_a + stage * a_stride, &tmap_a, cc * p.BK, cw, ch, n0, a_full(stage));
+          }
+          advance(1);
+        }
+      }
+      if (ok) advance((nprod - 1) * kiters);
+    }
+    return passed;
+  };
+  const bool two_producers = !kPairK && !halo && p.a_producers == 2 && kiters > 0;
   if (warp == 0) {
     // ------------------------------ operand A producer ------------------------------
-    if (kiters > 0) {
+    if (two_producers) {
+      fin_passed = produce_tap(0, 2, fin_stage, fin_phase);
+    } else if (kiters > 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -517,6 +562,17 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
       }
     }
     __syncwarp();
+    if (two_producers) {   // the weights are on their way: this warp copies operand A for the odd tiles
+      int st2 = 0;
+      uint32_t ph2 = 0;
+      const int passed = produce_tap(1, 2, st2, ph2);
+      if (lane == 0) {
+        fin2_s[0] = passed;
+        fin2_s[1] = st2;
+        fin2_s[2] = (int)ph2;
+      }
+      __syncwarp();
+    }
     if (p.mma_issuers == 3) {   // the weights are on their way and stay: nothing more to copy
       run_issuer(2);
       __syncwarp();
@@ -892,7 +948,13 @@ hq_gemm_kernel(const __grid_constant__ GemmParams p, const __grid_constant__ CUt
     // pairs rely on the cluster barrier above.)
     if (abort_flag_s != 0) {   // the same for every thread: read after the barrier
       if (kiters > 0 && lane == 0) {
-        if (warp == 0) ring_drain(a_full, p.stages_a, fin_stage, fin_phase);
+        if (warp == 0) {
+          if (two_producers && fin2_s[0] > fin_passed) {   // the other producer got further: drain from where it stood (a stage
+            fin_stage = fin2_s[1];                         // the slower one never armed in that lap costs one bounded wait)
+            fin_phase = (uint32_t)fin2_s[2];
+          }
+          ring_drain(a_full, p.stages_a, fin_stage, fin_phase);
+        }
         if (warp == 2 && my_tiles > 0) {
           if (p.b_resident) mbar_drain(b_full(0), 0u);
           else if (halo) ring_drain(b_full, p.stages_b, fin_stage, fin_phase);

@@ -124,6 +124,7 @@ struct GemmParams {
   uint32_t idesc;
   uint32_t tmem_cols, tmem_buf_stride;
   int32_t mma_issuers;                // 1, 2 or 3 warps issuing MMAs (tiles in turn)
+  int32_t a_producers;                // kModeTap with resident weights: 1, or 2 = the weight producer's warp copies operand A for every second tile
   int32_t pair;                       // 1: launched as clusters of two CTAs that share 256-row tiles (tcgen05 cta_group::2);
                                       //    stage_bytes_b and the B tensor map's box then cover BN/2 rows
   int32_t num_pair_tiles;             // pair tiles (two row tiles x one column tile)
@@ -349,6 +350,7 @@ struct hq_ctx {
   int force_mode = -1;                // -1: choose per layer; else hq::GemmMode where the layer allows it
   int force_dw_tiled = -1;            // depthwise 3x3 stride 1 on CUDA cores: -1 choose, 0 direct loads, 1 patches staged by TMA
   int force_depthwise = -1;           // depthwise layers: -1 choose, 0 CUDA-core kernel, 1 dense expansion on the tensor cores
+  int a_producers = -1;               // warps copying operand A in 1x1 layers with resident weights: -1 choose, 1, 2 where the layer allows
   int gather_span = 1;                // few-channel fused kernel: 1 = tiles may run across the ends of short output rows, 0 = one output row per tile
   int force_repack = -1;              // small-C spatial filters: -1 choose, 0 patch rows, 1 window rows where possible
   int force_epi_groups = -1;          // log2 of the epilogue warp groups: -1 chosen per layer, else min(value, log2 of the accumulator buffers)

@@ -116,6 +116,7 @@ FWD_CASES = {
     "1x1_s2": dict(N=2, H=14, W=14, Cin=64, K=128, R=1, S=1, stride=2, pad=0),
     "1x1_c24_k144_fold": dict(N=2, H=10, W=13, Cin=24, K=144, R=1, S=1),
     "1x1_c144_k24": dict(N=2, H=10, W=13, Cin=144, K=24, R=1, S=1),
+    "1x1_c64_k32_many_tiles": dict(N=4, H=112, W=112, Cin=64, K=32, R=1, S=1),   # several tiles per CTA
     "3x3_c64_56x56": dict(N=2, H=56, W=56, Cin=64, K=64, R=3, S=3, stride=1, pad=1),
     "3x3_c128_28x28": dict(N=3, H=28, W=28, Cin=128, K=128, R=3, S=3, stride=1, pad=1),
     "3x3_c512_k512_7x7": dict(N=4, H=7, W=7, Cin=512, K=512, R=3, S=3, stride=1, pad=1),
@@ -222,6 +223,22 @@ def test_conv_fwd_few_channels_one_row_per_tile(ctx, name):
         _run_iterations(ctx, "conv_fwd", W, shape, lambda t: makers[t % 3](r, in_shape), 3, repack=2)
     finally:
         ctx.set_option("gather_span", 1)
+
+
+@pytest.mark.parametrize("producers", [1, 2])
+@pytest.mark.parametrize("name", [n for n, c in FWD_CASES.items() if c.get("R", 1) == 1] + ["3x3_s2_odd", "3x3_c512_k512_7x7"])
+def test_conv_fwd_operand_producers(ctx, name, producers):
+    """Layers that take one input copy per filter tap, with one warp copying the input tiles or two warps copying them for
+    alternate tiles (where the layer keeps its weights in shared memory; elsewhere the option changes nothing): same bytes."""
+    shape = dict(FWD_CASES[name])
+    r = synth.rng(106, len(name), shape["H"], producers)
+    W = _weights(r, shape)
+    in_shape = (shape["N"], shape["H"], shape["W"], shape["Cin"])
+    ctx.set_option("a_producers", producers)
+    try:
+        _run_iterations(ctx, "conv_fwd", W, shape, lambda t: synth.relu_activations(r, in_shape), 3, staging=0)
+    finally:
+        ctx.set_option("a_producers", -1)
 
 
 BWD_CASES = {
