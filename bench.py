@@ -42,9 +42,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # earlier launches is written back to DRAM while later ones run (ncu captures summarised under profiles/, taken with
 # the kernels as committed; set an entry to None when its kernel changes).
 NCU_TRAFFIC = {
-    "stem7x7": 122247216, "layer1.0": 51061200, "layer2.1": 25371120, "layer3.1": 12623376, "layer4.1": 6624832,
-    "resnet_conv3x3_64": 25354048, "resnet_conv3x3_256_bwd": 25547600,
-    "mbv2_expand": 134998432, "mbv2_dw3x3": 231814896, "mbv2_project": 135030400,
+    "stem7x7": 122226672, "layer1.0": 50976208, "layer2.1": 25329152, "layer3.1": 12603200, "layer4.1": 6623488,
+    "resnet_conv3x3_64": 25385552, "resnet_conv3x3_256_bwd": 25491936,
+    "mbv2_expand": 135021248, "mbv2_dw3x3": 231826688, "mbv2_project": 135043808,
 }
 # kernels other than the tensor-core layer kernel, by layer name
 KERNEL_OF = {"mbv2_dw3x3": "depthwise3x3_col_kernel", "stem7x7": "hq_gather_conv_kernel"}
